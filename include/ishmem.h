@@ -1,0 +1,362 @@
+/*
+ * ishmem.h -- C ABI of libishmem.so: GPU-initiated OpenSHMEM-style communication on a
+ * symmetric heap, after Intel SHMEM (arXiv 2409.20476), for one NVIDIA B200 (sm_100a).
+ *
+ * Execution model.  One process hosts `npes` logical processing elements (PEs).  Each
+ * PE owns one slice of `heap_bytes` of a single device allocation: its symmetric heap
+ * (Section 2.3: PEs 0..npes-1, identical layout on every PE, different contents;
+ * Section 3.5: the heap lives in GPU memory).  Because every PE lives in this process,
+ * host calls that OpenSHMEM makes "as a PE" carry the calling PE as their first
+ * argument `my_pe`; collectives are called once for the whole team.
+ *
+ * Addresses.  A *symmetric address* is the device address of the object in PE 0's
+ * slice, as returned by ishmem_malloc; the library translates it to the addressed PE
+ * with `addr - heap_base[0] + heap_base[pe]` (Section 3.7.1, the ishmem_long_p
+ * walk-through).  Unless stated otherwise: the `dest` of a put, the `src` of a get,
+ * atomic targets, signal words and all collective buffers must be symmetric; the
+ * other side may be a symmetric address (meaning my_pe's copy) or any other device
+ * pointer.  All data pointers are DEVICE pointers unless the parameter is documented
+ * as host memory.  The library never takes ownership of caller memory; memory from
+ * ishmem_malloc belongs to the library until ishmem_free / ishmem_finalize.
+ *
+ * Ordering.  Host-initiated operations of PE p are enqueued on PE p's CUDA stream and
+ * return at once (stream-ordered); team collectives and SPMD launches run on the
+ * team stream, after everything already enqueued on the member PEs' streams.
+ * ishmem_quiet / ishmem_barrier_all are the completion points (Section 3.7.2: barrier
+ * = quiet + sync).  Overlapping src/dest ranges on one PE are undefined.
+ *
+ * Errors.  Functions returning int give ISHMEM_OK (0) or a negative ishmem_status;
+ * nothing is enqueued when an argument check fails.  Pointer-returning functions
+ * give NULL on failure.  Device-side waits are bounded: when a wait gives up it
+ * latches ISHMEM_ERR_TIMEOUT in a device status word that ishmemx_status() reads.
+ * There is no CPU fallback anywhere: without a CUDA device ishmem_init fails.
+ */
+#ifndef ISHMEM_H
+#define ISHMEM_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define ISHMEM_MAX_PES 64
+
+typedef enum ishmem_status {
+    ISHMEM_OK = 0,
+    ISHMEM_ERR_INVALID_PE = -1,     /* PE outside 0..npes-1, or outside the team */
+    ISHMEM_ERR_NOT_SYMMETRIC = -2,  /* address range is not inside the symmetric heap */
+    ISHMEM_ERR_ALIGN = -3,          /* address not aligned for the element type */
+    ISHMEM_ERR_OOM = -4,            /* symmetric heap or device memory exhausted */
+    ISHMEM_ERR_TIMEOUT = -5,        /* a bounded device-side wait gave up */
+    ISHMEM_ERR_NOT_CORESIDENT = -6, /* a launch whose blocks wait on one another does not fit */
+    ISHMEM_ERR_CUDA = -7,           /* a CUDA runtime call failed (see ishmemx_last_cuda_error) */
+    ISHMEM_ERR_ARG = -8,            /* other invalid argument */
+    ISHMEM_ERR_NOT_INITIALIZED = -9
+} ishmem_status;
+
+/* Teams (Section 3.7.2 uses ISHMEM_TEAM_SHARED; OpenSHMEM 1.5 teams API).  A team is the
+ * PE set {start + i*stride}.  WORLD and SHARED both name all PEs here: every PE is
+ * reachable by load/store from every other. */
+typedef int ishmem_team_t;
+#define ISHMEM_TEAM_WORLD 0
+#define ISHMEM_TEAM_SHARED 1
+#define ISHMEM_TEAM_INVALID (-1)
+#define ISHMEM_MAX_TEAMS 16
+
+/* signal operators of put_signal, comparisons of wait_until */
+#define ISHMEM_SIGNAL_SET 0
+#define ISHMEM_SIGNAL_ADD 1
+#define ISHMEM_CMP_EQ 0
+#define ISHMEM_CMP_NE 1
+#define ISHMEM_CMP_GT 2
+#define ISHMEM_CMP_GE 3
+#define ISHMEM_CMP_LT 4
+#define ISHMEM_CMP_LE 5
+
+/* thread-collaboration level of the device-side copy routines (Section 3.6: work-item =
+ * one thread, sub-group = one warp of 32 lanes, work-group = one thread block). */
+#define ISHMEMX_WORK_ITEM 0
+#define ISHMEMX_SUB_GROUP 1
+#define ISHMEMX_WORK_GROUP 2       /* 16-byte vector loads/stores by all threads */
+#define ISHMEMX_WORK_GROUP_BULK 3  /* work-group; large aligned blocks go through TMA bulk copies */
+
+/* reduction operators and element types of the generic reduce entry point */
+#define ISHMEM_OP_SUM 0
+#define ISHMEM_OP_MAX 1
+#define ISHMEM_OP_MIN 2
+#define ISHMEM_OP_PROD 3
+#define ISHMEM_OP_AND 4
+#define ISHMEM_OP_OR 5
+#define ISHMEM_OP_XOR 6
+#define ISHMEM_T_INT32 0
+#define ISHMEM_T_INT64 1
+#define ISHMEM_T_FLOAT 2
+#define ISHMEM_T_DOUBLE 3
+#define ISHMEM_T_UINT32 4
+#define ISHMEM_T_UINT64 5
+
+/* reduce algorithms (Section 3.7.2, "Reduction") */
+#define ISHMEMX_REDUCE_AUTO 0
+#define ISHMEMX_REDUCE_DUPLICATED 1 /* every PE folds all sources itself, no inter-PE sync */
+#define ISHMEMX_REDUCE_SPLIT 2      /* addresses split across PEs; the owner folds and pushes */
+
+/* ------------------------------------------------------------------ lifecycle --- */
+
+/* Host-only (Section 3.6).  Creates `npes` PEs (1..ISHMEM_MAX_PES) on the current CUDA
+ * device, each with `heap_bytes` of symmetric heap (rounded up to 256 B), zero-filled.
+ * ishmem_init allocates the heap with cudaMalloc; ishmemx_init_external uses
+ * npes*heap_bytes bytes at `base` (device memory, 256-byte aligned, owned by the caller,
+ * e.g. a torch tensor; cf. the external-heap registration of Section 3.5) and does
+ * not clear it.  ISHMEM_ERR_ARG if already initialised. */
+int ishmem_init(int npes, size_t heap_bytes);
+int ishmemx_init_external(int npes, size_t heap_bytes, void *base);
+/* Waits for all streams, frees everything the library allocated. */
+int ishmem_finalize(void);
+int ishmem_n_pes(void);                /* 0 when not initialised */
+size_t ishmemx_heap_bytes(void);
+/* Device pointer to PE `pe`'s context (ishmem_ctx_t, see ishmem_device.cuh), to hand to
+ * user kernels; the array of all contexts starts at ishmemx_ctx(0).  NULL on error. */
+void *ishmemx_ctx(int pe);
+/* Replace PE `pe`'s stream (pe = -1: the team stream) by a caller-owned cudaStream_t. */
+int ishmemx_set_stream(int pe, void *cuda_stream);
+void *ishmemx_get_stream(int pe);
+const char *ishmem_strerror(int status);
+const char *ishmemx_last_cuda_error(void);
+/* Reads (and with clear != 0 resets) the device status word latched by bounded waits.
+ * Blocks until all library streams are idle. */
+int ishmemx_status(int clear);
+/* Number of kernels the library has launched since ishmem_init. */
+unsigned long long ishmemx_launch_count(void);
+/* Time bound, in nanoseconds, of every device-side wait (default 2e9 = two seconds). */
+int ishmemx_set_wait_limit_ns(uint64_t ns);
+
+/* --------------------------------------------------- symmetric memory (host only) --- */
+
+/* Collective allocation: the same offset on every PE (Section 2.3).  256-byte aligned
+ * (ishmem_align: `alignment` a power of two).  Returns the symmetric address (PE 0's
+ * copy) or NULL when the heap is exhausted.  ishmem_calloc zero-fills every PE's copy.
+ * ishmem_free(NULL) is a no-op; freeing a pointer not returned by these is an error. */
+void *ishmem_malloc(size_t size);
+void *ishmem_calloc(size_t count, size_t size);
+void *ishmem_align(size_t alignment, size_t size);
+int ishmem_free(void *ptr);
+/* PE `pe`'s copy of the symmetric object (device pointer usable by loads and stores from
+ * any kernel: Section 3.3, every peer heap is mapped).  NULL if not symmetric. */
+void *ishmem_ptr(const void *sym, int pe);
+/* Staging helpers (host <-> one PE's copy), enqueued on that PE's stream.  `host` is HOST
+ * memory; pinned memory makes the copy asynchronous. */
+int ishmemx_heap_write(int pe, void *sym_dest, const void *host, size_t nbytes);
+int ishmemx_heap_read(int pe, void *host, const void *sym_src, size_t nbytes);
+
+/* ----------------------------------------------------------- RMA (Section 3.7.1) --- */
+
+/* Host-initiated put/get of `nbytes`: PE my_pe copies src -> dest@pe (put) or src@pe ->
+ * dest (get).  Subject to the cutover (Sections 3.2, 4): below the tuned size a kernel of
+ * cooperating threads does loads/stores, above it the copy engine (cudaMemcpyAsync on a
+ * side stream) is started.  The blocking forms order later work of my_pe's stream after
+ * the transfer; the _nbi forms only guarantee completion after ishmem_quiet(my_pe). */
+int ishmem_putmem(int my_pe, void *dest, const void *src, size_t nbytes, int pe);
+int ishmem_getmem(int my_pe, void *dest, const void *src, size_t nbytes, int pe);
+int ishmem_putmem_nbi(int my_pe, void *dest, const void *src, size_t nbytes, int pe);
+int ishmem_getmem_nbi(int my_pe, void *dest, const void *src, size_t nbytes, int pe);
+
+/* Typed forms: `nelems` elements; addresses must be aligned to the element size. */
+#define ISHMEM_DECL_RMA(NAME, T)                                                              \
+    int ishmem_##NAME##_put(int my_pe, T *dest, const T *src, size_t nelems, int pe);         \
+    int ishmem_##NAME##_get(int my_pe, T *dest, const T *src, size_t nelems, int pe);         \
+    int ishmem_##NAME##_put_nbi(int my_pe, T *dest, const T *src, size_t nelems, int pe);     \
+    int ishmem_##NAME##_get_nbi(int my_pe, T *dest, const T *src, size_t nelems, int pe);     \
+    /* scalar store / load of one element at a symmetric address (the ishmem_long_p example \
+     * of Section 3.7.1).  g blocks the host and writes the value to HOST memory. */         \
+    int ishmem_##NAME##_p(int my_pe, T *dest, T value, int pe);                               \
+    int ishmem_##NAME##_g(int my_pe, T *value_out_host, const T *src, int pe);
+ISHMEM_DECL_RMA(float, float)
+ISHMEM_DECL_RMA(double, double)
+ISHMEM_DECL_RMA(int, int)
+ISHMEM_DECL_RMA(long, long)
+ISHMEM_DECL_RMA(int32, int32_t)
+ISHMEM_DECL_RMA(int64, int64_t)
+ISHMEM_DECL_RMA(uint8, uint8_t)
+ISHMEM_DECL_RMA(uint32, uint32_t)
+ISHMEM_DECL_RMA(uint64, uint64_t)
+#undef ISHMEM_DECL_RMA
+
+/* Explicit thread-collaborative variants (Section 3.6; experiments of Section 4): a
+ * kernel of `groups` blocks x `threads` threads is launched on my_pe's stream; the message
+ * is cut into one contiguous slice per collaboration unit (thread / warp / block,
+ * `level` = ISHMEMX_WORK_ITEM..ISHMEMX_WORK_GROUP_BULK) and every unit calls the device
+ * routine ishmem_putmem / ishmemx_putmem_sub_group / ishmemx_putmem_work_group once on its
+ * slice.  threads in 1..1024, groups >= 1.  No cutover. */
+int ishmemx_putmem_on_device(int my_pe, void *dest, const void *src, size_t nbytes, int pe,
+                             int level, int threads, int groups);
+int ishmemx_getmem_on_device(int my_pe, void *dest, const void *src, size_t nbytes, int pe,
+                             int level, int threads, int groups);
+/* The copy-engine path alone (cudaMemcpyAsync on the side stream, joined back into
+ * my_pe's stream). */
+int ishmemx_putmem_copy_engine(int my_pe, void *dest, const void *src, size_t nbytes, int pe);
+int ishmemx_getmem_copy_engine(int my_pe, void *dest, const void *src, size_t nbytes, int pe);
+/* SPMD form: ONE launch on the team stream in which every PE p runs the same device call
+ * with target (p + shift) mod npes -- shift 1 is the ring pattern, shifts 1..npes-1 in turn
+ * the all-pairs pattern.  `groups` blocks per PE.  dest and src are symmetric. */
+int ishmemx_putmem_spmd(void *dest, const void *src, size_t nbytes, int shift, int level,
+                        int threads, int groups);
+int ishmemx_getmem_spmd(void *dest, const void *src, size_t nbytes, int shift, int level,
+                        int threads, int groups);
+/* Same pattern through the copy engine: npes cudaMemcpyAsync calls on the side stream. */
+int ishmemx_putmem_spmd_copy_engine(void *dest, const void *src, size_t nbytes, int shift);
+
+/* Cutover sizes in bytes (Section 4: tuned from measurement; for the collaborative calls
+ * it depends on the number of threads).  which: 0 = put/get, 1 = broadcast, 2 = fcollect.
+ * SIZE_MAX = never use the copy engine, 0 = always. */
+int ishmemx_set_cutover(int which, size_t nbytes);
+size_t ishmemx_get_cutover(int which);
+
+/* ------------------------------------------- signalling, ordering, synchronisation --- */
+
+/* put, then update the 64-bit signal word `sig_addr`@pe (symmetric) with `signal`
+ * (ISHMEM_SIGNAL_SET / _ADD); the update becomes visible only after the payload. */
+int ishmem_putmem_signal(int my_pe, void *dest, const void *src, size_t nbytes,
+                         uint64_t *sig_addr, uint64_t signal, int sig_op, int pe);
+/* Enqueues a bounded device-side wait on my_pe's stream until `*ivar`@my_pe cmp value.
+ * On expiry the status word latches ISHMEM_ERR_TIMEOUT and the stream continues. */
+int ishmem_uint64_wait_until(int my_pe, uint64_t *ivar, int cmp, uint64_t value);
+/* fence: orders my_pe's earlier puts before its later ones per target (stream order
+ * already gives this; kept for API parity).  quiet: completes all outstanding operations
+ * of my_pe, including _nbi transfers on the copy engine, in stream order. */
+int ishmem_fence(int my_pe);
+int ishmem_quiet(int my_pe);
+/* sync: team members wait for one another (Section 3.7.2: each PE sends an atomic
+ * increment to every other member's counter and waits on its own).  Runs the push
+ * algorithm in one co-resident launch.  barrier_all = quiet on every PE + sync, and blocks
+ * the host until done.  sync_all = team_sync(WORLD), stream-ordered. */
+int ishmem_team_sync(ishmem_team_t team);
+int ishmem_sync_all(void);
+int ishmem_barrier_all(void);
+/* Strided sub-team of a parent team; returns the new team or ISHMEM_TEAM_INVALID. */
+ishmem_team_t ishmem_team_split_strided(ishmem_team_t parent, int start, int stride, int size);
+int ishmem_team_destroy(ishmem_team_t team);
+int ishmem_team_n_pes(ishmem_team_t team);
+
+/* --------------------------------------------------------------- remote atomics --- */
+
+/* One atomic on the integer at symmetric address `target` on PE `pe`, issued by my_pe.
+ * Non-fetching forms are stream-ordered; fetching forms block the host and write the old
+ * value to HOST memory `fetched_host`. */
+#define ISHMEM_DECL_AMO(NAME, T)                                                               \
+    int ishmem_##NAME##_atomic_add(int my_pe, T *target, T value, int pe);                     \
+    int ishmem_##NAME##_atomic_inc(int my_pe, T *target, int pe);                              \
+    int ishmem_##NAME##_atomic_set(int my_pe, T *target, T value, int pe);                     \
+    int ishmem_##NAME##_atomic_fetch(int my_pe, T *fetched_host, const T *target, int pe);     \
+    int ishmem_##NAME##_atomic_fetch_add(int my_pe, T *fetched_host, T *target, T value, int pe); \
+    int ishmem_##NAME##_atomic_fetch_inc(int my_pe, T *fetched_host, T *target, int pe);       \
+    int ishmem_##NAME##_atomic_swap(int my_pe, T *fetched_host, T *target, T value, int pe);   \
+    int ishmem_##NAME##_atomic_compare_swap(int my_pe, T *fetched_host, T *target, T cond,     \
+                                            T value, int pe);                                  \
+    int ishmem_##NAME##_atomic_fetch_and(int my_pe, T *fetched_host, T *target, T value, int pe); \
+    int ishmem_##NAME##_atomic_fetch_or(int my_pe, T *fetched_host, T *target, T value, int pe);  \
+    int ishmem_##NAME##_atomic_fetch_xor(int my_pe, T *fetched_host, T *target, T value, int pe);
+ISHMEM_DECL_AMO(int32, int32_t)
+ISHMEM_DECL_AMO(int64, int64_t)
+ISHMEM_DECL_AMO(uint32, uint32_t)
+ISHMEM_DECL_AMO(uint64, uint64_t)
+#undef ISHMEM_DECL_AMO
+
+/* Device-initiated batches (one op per GPU thread, "issued from all threads"): op i is
+ * issued by PE (i mod npes); word w of the table lives on PE (w mod npes) at
+ * table + 8*(w div npes).  word_idx/inc/cond/value/fetched are device arrays of `nops`
+ * entries (fetched may be NULL).  aggregate != 0 lets the lanes of a warp that hit the same
+ * word combine into one atomic and rebuild their fetched values (still one valid
+ * serialisation).  One launch on the team stream. */
+int ishmemx_int64_atomic_fetch_add_batch(int64_t *table, const int32_t *word_idx,
+                                         const int64_t *inc, int64_t *fetched, size_t nops,
+                                         int threads, int aggregate);
+int ishmemx_int64_atomic_compare_swap_batch(int64_t *table, const int32_t *word_idx,
+                                            const int64_t *cond, const int64_t *value,
+                                            int64_t *fetched, size_t nops, int threads);
+
+/* ------------------------------------------------- collectives (Section 3.7.2) --- */
+
+/* broadcast: dest@q[0:nbytes] = src@root for every team member q ("push": the root stores
+ * into every destination, destinations in the inner loop).  `root` is the index inside
+ * the team.  The root's own dest is written too unless ishmemx_set_bcast_root_dest(0). */
+int ishmem_broadcastmem(ishmem_team_t team, void *dest, const void *src, size_t nbytes, int root);
+int ishmemx_set_bcast_root_dest(int enable);
+/* fcollect: dest@q[i*nbytes:(i+1)*nbytes] = src@member_i for every member q (allgather
+ * with equal contributions; push). */
+int ishmem_fcollectmem(ishmem_team_t team, void *dest, const void *src, size_t nbytes);
+/* reduce: dest@q[j] = ((src@m0[j] op src@m1[j]) op ...) op src@m_{P-1}[j], folded in team
+ * order (floating point bit-exact in that order), for every member q.  dest and src may
+ * not overlap unless identical, which is handled with snapshot semantics only by the
+ * SPLIT algorithm.  Integer sum/prod wrap. */
+int ishmemx_reduce(ishmem_team_t team, void *dest, const void *src, size_t nreduce, int op,
+                   int dtype, int algorithm);
+#define ISHMEM_DECL_REDUCE(NAME, T, OP)                                                        \
+    int ishmem_##NAME##_##OP##_reduce(ishmem_team_t team, T *dest, const T *src, size_t nreduce);
+#define ISHMEM_DECL_REDUCE_ARITH(NAME, T)                                                      \
+    ISHMEM_DECL_REDUCE(NAME, T, sum) ISHMEM_DECL_REDUCE(NAME, T, max)                          \
+    ISHMEM_DECL_REDUCE(NAME, T, min) ISHMEM_DECL_REDUCE(NAME, T, prod)
+#define ISHMEM_DECL_REDUCE_BITS(NAME, T)                                                       \
+    ISHMEM_DECL_REDUCE(NAME, T, and) ISHMEM_DECL_REDUCE(NAME, T, or) ISHMEM_DECL_REDUCE(NAME, T, xor)
+ISHMEM_DECL_REDUCE_ARITH(int32, int32_t)
+ISHMEM_DECL_REDUCE_ARITH(int64, int64_t)
+ISHMEM_DECL_REDUCE_ARITH(uint32, uint32_t)
+ISHMEM_DECL_REDUCE_ARITH(uint64, uint64_t)
+ISHMEM_DECL_REDUCE_ARITH(float, float)
+ISHMEM_DECL_REDUCE_ARITH(double, double)
+ISHMEM_DECL_REDUCE_BITS(int32, int32_t)
+ISHMEM_DECL_REDUCE_BITS(int64, int64_t)
+ISHMEM_DECL_REDUCE_BITS(uint32, uint32_t)
+ISHMEM_DECL_REDUCE_BITS(uint64, uint64_t)
+#undef ISHMEM_DECL_REDUCE
+#undef ISHMEM_DECL_REDUCE_ARITH
+#undef ISHMEM_DECL_REDUCE_BITS
+/* Launch geometry of collective kernels: blocks per PE (0 = automatic) and threads. */
+int ishmemx_set_collective_geometry(int groups_per_pe, int threads);
+
+/* Device-resident collectives: ONE co-resident launch in which one work-group per PE calls
+ * the device routine ishmemx_{broadcastmem,fcollectmem,reduce,sync_all}_work_group of
+ * ishmem_device.cuh, with in-kernel push synchronisation (for tests and latency
+ * measurements of the device API itself).  which: 0 broadcast, 1 fcollect, 2 reduce
+ * (op/dtype as above), 3 sync_all repeated `repeat` times. */
+int ishmemx_collective_on_device(int which, ishmem_team_t team, void *dest, const void *src,
+                                 size_t n, int root, int op, int dtype, int threads, int repeat);
+
+/* ----------------------------------------------- device-initiated test programs --- */
+
+/* put_signal / wait_until ping-pong between PE a and PE b, entirely inside one
+ * co-resident launch: `rounds` round trips of `nbytes` (work-group put_signal with
+ * `threads` threads, SIGNAL_SET to the round number, wait_until GE).  data: symmetric,
+ * >= nbytes; sig: symmetric 64-bit word, zero on entry.  Writes the mean half round trip
+ * in nanoseconds (measured in-kernel with the global timer) to HOST memory `half_rtt_ns`.
+ * Each round stamps the round number into the first and last 8 bytes of the payload; the
+ * receiver counts stamps that do not match the signalled round into HOST `mismatches`
+ * (a non-zero count means a signal overtook its payload).  Blocks the host. */
+int ishmemx_pingpong(int pe_a, int pe_b, void *data, uint64_t *sig, size_t nbytes, int rounds,
+                     int threads, double *half_rtt_ns, uint64_t *mismatches);
+
+/* Overlap workload: `iters` sweeps of the 5-point Jacobi update on an ny x nx float64
+ * grid cut into npes row strips (the first ny mod npes strips have one more row), in one
+ * persistent co-resident launch: each sweep every PE sends its first and last rows to the
+ * neighbours' halo rows with in-kernel work-group put_signal, updates its interior rows
+ * meanwhile, waits for its own halos, then updates its edge rows.  buf0/buf1: symmetric,
+ * (ceil(ny/npes)+2)*nx doubles each, strip row r at local row r+1 of buf0 on entry (buf1
+ * is overwritten); sig: symmetric, 2 words, zero on entry.  overlap = 0 disables the
+ * interior-first ordering (exchange, wait, then compute).  The final strips are in buf0
+ * if iters is even, else buf1.  residual_sq_host (HOST, may be NULL) receives
+ * ||u_iters - u_(iters-1)||_2^2 over the interior.  Blocks the host. */
+int ishmemx_jacobi(double *buf0, double *buf1, uint64_t *sig, size_t ny, size_t nx, int iters,
+                   int overlap, int groups_per_pe, int threads, double *residual_sq_host);
+
+/* Host-buffer convenience for end-to-end measurements: copy `nbytes` from HOST `src_host`
+ * into src@p for every PE p (per-PE stride `nbytes` in the host buffer), run
+ * ishmemx_putmem_spmd(dest, src, nbytes, shift, level, threads, groups), and copy every
+ * dest@p back to HOST `dest_host`.  Blocks the host. */
+int ishmemx_host_put_ring(void *dest_host, const void *src_host, void *dest, void *src,
+                          size_t nbytes, int shift, int level, int threads, int groups);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ISHMEM_H */

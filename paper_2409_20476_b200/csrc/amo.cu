@@ -1,0 +1,240 @@
+/* Remote atomic memory operations: host-initiated single operations and the device-initiated
+ * batches ("one op per GPU thread").  All atomics go through the device API of
+ * ishmem_device.cuh (address translation + .gpu-scope atomic). */
+#include "internal.h"
+
+enum { AMO_ADD, AMO_INC, AMO_SET, AMO_FETCH, AMO_FETCH_ADD, AMO_FETCH_INC, AMO_SWAP, AMO_CAS, AMO_FETCH_AND,
+       AMO_FETCH_OR, AMO_FETCH_XOR };
+
+template <typename T>
+__global__ void k_amo(const ishmem_ctx_t *ctxs, int my_pe, int op, T *target_local, T value, T cond, int pe,
+                      T *out_host_mapped)
+{
+    const ishmem_ctx_t *ctx = ctxs + my_pe;
+    T old = T();
+    switch (op) {
+    case AMO_ADD: ishmem_atomic_add<T>(ctx, target_local, value, pe); break;
+    case AMO_INC: ishmem_atomic_inc<T>(ctx, target_local, pe); break;
+    case AMO_SET: ishmem_atomic_set<T>(ctx, target_local, value, pe); break;
+    case AMO_FETCH: old = ishmem_atomic_fetch<T>(ctx, target_local, pe); break;
+    case AMO_FETCH_ADD: old = ishmem_atomic_fetch_add<T>(ctx, target_local, value, pe); break;
+    case AMO_FETCH_INC: old = ishmem_atomic_fetch_inc<T>(ctx, target_local, pe); break;
+    case AMO_SWAP: old = ishmem_atomic_swap<T>(ctx, target_local, value, pe); break;
+    case AMO_CAS: old = ishmem_atomic_compare_swap<T>(ctx, target_local, cond, value, pe); break;
+    case AMO_FETCH_AND: old = ishmem_atomic_fetch_and<T>(ctx, target_local, value, pe); break;
+    case AMO_FETCH_OR: old = ishmem_atomic_fetch_or<T>(ctx, target_local, value, pe); break;
+    default: old = ishmem_atomic_fetch_xor<T>(ctx, target_local, value, pe); break;
+    }
+    if (out_host_mapped) *out_host_mapped = old;
+}
+
+/* D = the device-side type with the same size as the ABI type T */
+template <typename T, typename D>
+static int host_amo(int my_pe, int op, T *fetched_host, const T *target, T value, T cond, int pe, bool fetching)
+{
+    ISHMEMI_REQUIRE_INIT();
+    auto &g = g_ishmem;
+    if (ishmemi_check_pe(my_pe) || ishmemi_check_pe(pe)) return ISHMEM_ERR_INVALID_PE;
+    if ((uintptr_t)target % sizeof(T)) return ISHMEM_ERR_ALIGN;
+    if (ishmemi_sym_offset(target, sizeof(T)) < 0) return ISHMEM_ERR_NOT_SYMMETRIC;
+    if (fetching && !fetched_host) return ISHMEM_ERR_ARG;
+    D *tl = (D *)ishmemi_localise(target, sizeof(T), my_pe);
+    cudaStream_t s = ishmemi_pe_stream_for_op(my_pe);
+    k_amo<D><<<1, 1, 0, s>>>(g.d_ctx, my_pe, op, tl, (D)value, (D)cond, pe, fetching ? (D *)g.h_pinned : nullptr);
+    ishmemi_count_launch();
+    int rc = ishmemi_check_launch("k_amo");
+    if (rc || !fetching) return rc;
+    ISHMEMI_CUDA(cudaStreamSynchronize(s));
+    *fetched_host = (T)(*(D *)g.h_pinned);
+    return ISHMEM_OK;
+}
+
+#define ISHMEMI_DEF_AMO(NAME, T, D)                                                                               \
+    extern "C" int ishmem_##NAME##_atomic_add(int my_pe, T *target, T value, int pe)                              \
+    {                                                                                                             \
+        return host_amo<T, D>(my_pe, AMO_ADD, nullptr, target, value, 0, pe, false);                              \
+    }                                                                                                             \
+    extern "C" int ishmem_##NAME##_atomic_inc(int my_pe, T *target, int pe)                                       \
+    {                                                                                                             \
+        return host_amo<T, D>(my_pe, AMO_INC, nullptr, target, 0, 0, pe, false);                                  \
+    }                                                                                                             \
+    extern "C" int ishmem_##NAME##_atomic_set(int my_pe, T *target, T value, int pe)                              \
+    {                                                                                                             \
+        return host_amo<T, D>(my_pe, AMO_SET, nullptr, target, value, 0, pe, false);                              \
+    }                                                                                                             \
+    extern "C" int ishmem_##NAME##_atomic_fetch(int my_pe, T *fetched_host, const T *target, int pe)              \
+    {                                                                                                             \
+        return host_amo<T, D>(my_pe, AMO_FETCH, fetched_host, target, 0, 0, pe, true);                            \
+    }                                                                                                             \
+    extern "C" int ishmem_##NAME##_atomic_fetch_add(int my_pe, T *fetched_host, T *target, T value, int pe)       \
+    {                                                                                                             \
+        return host_amo<T, D>(my_pe, AMO_FETCH_ADD, fetched_host, target, value, 0, pe, true);                    \
+    }                                                                                                             \
+    extern "C" int ishmem_##NAME##_atomic_fetch_inc(int my_pe, T *fetched_host, T *target, int pe)                \
+    {                                                                                                             \
+        return host_amo<T, D>(my_pe, AMO_FETCH_INC, fetched_host, target, 0, 0, pe, true);                        \
+    }                                                                                                             \
+    extern "C" int ishmem_##NAME##_atomic_swap(int my_pe, T *fetched_host, T *target, T value, int pe)            \
+    {                                                                                                             \
+        return host_amo<T, D>(my_pe, AMO_SWAP, fetched_host, target, value, 0, pe, true);                         \
+    }                                                                                                             \
+    extern "C" int ishmem_##NAME##_atomic_compare_swap(int my_pe, T *fetched_host, T *target, T cond, T value,    \
+                                                       int pe)                                                    \
+    {                                                                                                             \
+        return host_amo<T, D>(my_pe, AMO_CAS, fetched_host, target, value, cond, pe, true);                       \
+    }                                                                                                             \
+    extern "C" int ishmem_##NAME##_atomic_fetch_and(int my_pe, T *fetched_host, T *target, T value, int pe)       \
+    {                                                                                                             \
+        return host_amo<T, D>(my_pe, AMO_FETCH_AND, fetched_host, target, value, 0, pe, true);                    \
+    }                                                                                                             \
+    extern "C" int ishmem_##NAME##_atomic_fetch_or(int my_pe, T *fetched_host, T *target, T value, int pe)        \
+    {                                                                                                             \
+        return host_amo<T, D>(my_pe, AMO_FETCH_OR, fetched_host, target, value, 0, pe, true);                     \
+    }                                                                                                             \
+    extern "C" int ishmem_##NAME##_atomic_fetch_xor(int my_pe, T *fetched_host, T *target, T value, int pe)       \
+    {                                                                                                             \
+        return host_amo<T, D>(my_pe, AMO_FETCH_XOR, fetched_host, target, value, 0, pe, true);                    \
+    }
+ISHMEMI_DEF_AMO(int32, int32_t, int)
+ISHMEMI_DEF_AMO(int64, int64_t, long long)
+ISHMEMI_DEF_AMO(uint32, uint32_t, unsigned)
+ISHMEMI_DEF_AMO(uint64, uint64_t, unsigned long long)
+
+/* ---- device-initiated batches ---------------------------------------------------------- */
+/* Block b belongs to PE (b mod npes); its threads issue that PE's ops i = k*npes + pe in
+ * order, one per thread.  Word w lives on PE (w mod npes), slot (w div npes). */
+
+template <bool AGGREGATE>
+__global__ void __launch_bounds__(1024) k_fetch_add_batch(const ishmem_ctx_t *ctxs, long long *table0,
+                                                          const int *word_idx, const long long *inc,
+                                                          long long *fetched, size_t nops)
+{
+    const int npes = ctxs[0].npes;
+    const int my = (int)(blockIdx.x % (unsigned)npes);
+    const ishmem_ctx_t *ctx = ctxs + my;
+    const size_t k = (size_t)(blockIdx.x / (unsigned)npes) * blockDim.x + threadIdx.x;
+    const size_t i = k * (size_t)npes + (size_t)my;
+    const bool active = i < nops;
+    long long *table = (long long *)((char *)table0 + (ctx->heap_base - ctxs[0].heap_base));
+    int w = 0;
+    long long v = 0;
+    if (active) {
+        w = word_idx[i];
+        v = inc[i];
+    }
+    if (!AGGREGATE) {
+        if (active) {
+            long long old = ishmem_atomic_fetch_add<long long>(ctx, table + w / npes, v, w % npes);
+            if (fetched) fetched[i] = old;
+        }
+        return;
+    }
+    /* Lanes of the warp that hit the same word combine: the lowest such lane issues one
+     * atomic with the sum and every lane rebuilds the value it would have fetched had the
+     * group's ops been applied back to back in lane order. */
+    const unsigned lane = threadIdx.x & 31u;
+    const unsigned act = __ballot_sync(0xffffffffu, active);
+    if (!active) return;
+    const unsigned peers = __match_any_sync(act, w);
+    const unsigned leader = __ffs(peers) - 1;
+    long long before = 0, total = 0; /* sum over peers in lower lanes; sum over all peers */
+    unsigned rest = peers;
+    /* round r: every lane reads the increment of its r-th peer; the number of rounds is the
+     * largest group in the warp, so the shuffles stay converged */
+    const unsigned rounds = __reduce_max_sync(act, (unsigned)__popc(peers));
+#pragma unroll 1
+    for (unsigned r = 0; r < rounds; ++r) {
+        const unsigned src = rest ? (unsigned)(__ffs(rest) - 1) : lane;
+        const long long x = __shfl_sync(act, v, src);
+        if (rest) {
+            total += x;
+            if (src < lane) before += x;
+            rest &= rest - 1;
+        }
+    }
+    long long base = 0;
+    if (lane == leader) base = ishmem_atomic_fetch_add<long long>(ctx, table + w / npes, total, w % npes);
+    base = __shfl_sync(act, base, leader);
+    if (fetched) fetched[i] = base + before;
+}
+
+__global__ void __launch_bounds__(1024) k_compare_swap_batch(const ishmem_ctx_t *ctxs, long long *table0,
+                                                             const int *word_idx, const long long *cond,
+                                                             const long long *value, long long *fetched,
+                                                             size_t nops)
+{
+    const int npes = ctxs[0].npes;
+    const int my = (int)(blockIdx.x % (unsigned)npes);
+    const ishmem_ctx_t *ctx = ctxs + my;
+    const size_t k = (size_t)(blockIdx.x / (unsigned)npes) * blockDim.x + threadIdx.x;
+    const size_t i = k * (size_t)npes + (size_t)my;
+    if (i >= nops) return;
+    long long *table = (long long *)((char *)table0 + (ctx->heap_base - ctxs[0].heap_base));
+    const int w = word_idx[i];
+    long long old = ishmem_atomic_compare_swap<long long>(ctx, table + w / npes, cond[i], value[i], w % npes);
+    if (fetched) fetched[i] = old;
+}
+
+static int batch_geometry(size_t nops, int threads, unsigned *blocks)
+{
+    auto &g = g_ishmem;
+    if (threads < 32 || threads > 1024 || threads % 32) return ISHMEM_ERR_ARG;
+    size_t per_pe = (nops + g.npes - 1) / g.npes;
+    size_t bpp = (per_pe + threads - 1) / threads;
+    if (bpp == 0) bpp = 1;
+    if (bpp * g.npes > 0x7fffffffull) return ISHMEM_ERR_ARG;
+    *blocks = (unsigned)(bpp * g.npes);
+    return ISHMEM_OK;
+}
+
+extern "C" int ishmemx_int64_atomic_fetch_add_batch(int64_t *table, const int32_t *word_idx, const int64_t *inc,
+                                                    int64_t *fetched, size_t nops, int threads, int aggregate)
+{
+    ISHMEMI_REQUIRE_INIT();
+    auto &g = g_ishmem;
+    if (!word_idx || !inc) return ISHMEM_ERR_ARG;
+    if ((uintptr_t)table % 8) return ISHMEM_ERR_ALIGN;
+    if (ishmemi_sym_offset(table, 8) < 0) return ISHMEM_ERR_NOT_SYMMETRIC;
+    unsigned blocks;
+    int rc = batch_geometry(nops, threads, &blocks);
+    if (rc) return rc;
+    cudaStream_t s;
+    if ((rc = ishmemi_team_stream_begin(ISHMEM_TEAM_WORLD, &s))) return rc;
+    if (nops) {
+        if (aggregate)
+            k_fetch_add_batch<true><<<blocks, threads, 0, s>>>(g.d_ctx, (long long *)table, word_idx,
+                                                               (const long long *)inc, (long long *)fetched, nops);
+        else
+            k_fetch_add_batch<false><<<blocks, threads, 0, s>>>(g.d_ctx, (long long *)table, word_idx,
+                                                                (const long long *)inc, (long long *)fetched, nops);
+        ishmemi_count_launch();
+        rc = ishmemi_check_launch("k_fetch_add_batch");
+    }
+    ishmemi_team_stream_end();
+    return rc;
+}
+
+extern "C" int ishmemx_int64_atomic_compare_swap_batch(int64_t *table, const int32_t *word_idx,
+                                                       const int64_t *cond, const int64_t *value,
+                                                       int64_t *fetched, size_t nops, int threads)
+{
+    ISHMEMI_REQUIRE_INIT();
+    auto &g = g_ishmem;
+    if (!word_idx || !cond || !value) return ISHMEM_ERR_ARG;
+    if ((uintptr_t)table % 8) return ISHMEM_ERR_ALIGN;
+    if (ishmemi_sym_offset(table, 8) < 0) return ISHMEM_ERR_NOT_SYMMETRIC;
+    unsigned blocks;
+    int rc = batch_geometry(nops, threads, &blocks);
+    if (rc) return rc;
+    cudaStream_t s;
+    if ((rc = ishmemi_team_stream_begin(ISHMEM_TEAM_WORLD, &s))) return rc;
+    if (nops) {
+        k_compare_swap_batch<<<blocks, threads, 0, s>>>(g.d_ctx, (long long *)table, word_idx,
+                                                        (const long long *)cond, (const long long *)value,
+                                                        (long long *)fetched, nops);
+        ishmemi_count_launch();
+        rc = ishmemi_check_launch("k_compare_swap_batch");
+    }
+    ishmemi_team_stream_end();
+    return rc;
+}

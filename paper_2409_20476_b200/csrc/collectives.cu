@@ -1,0 +1,449 @@
+/* Team synchronisation and collectives (Section 3.7.2 of the paper): push sync, push
+ * broadcast / fcollect, reduce in its duplicated and split-by-address forms.
+ *
+ * Host-called collectives run as ONE launch for the whole team on the team stream; the
+ * launch boundary is their synchronisation.  The device-resident forms (one work-group
+ * per PE with in-kernel push sync) are exercised by ishmemx_collective_on_device, a
+ * co-resident (cooperative) launch. */
+#include "internal.h"
+
+struct coll_args {
+    ishmem_team_t team;
+    char *dest;       /* PE 0's copy (symmetric address) */
+    const char *src;
+    size_t n;         /* bytes (broadcast, fcollect) or elements (reduce) */
+    int root;
+    int groups;       /* blocks per member */
+    int duplicated;   /* reduce: every member folds everything into its own dest */
+    int repeat;
+};
+
+/* local address on `ctx`'s PE of a symmetric address given as PE 0's copy */
+__device__ __forceinline__ char *local_of(const ishmem_ctx_t *ctxs, const ishmem_ctx_t *ctx, const char *sym0)
+{
+    return (char *)sym0 + (ctx->heap_base - ctxs[0].heap_base);
+}
+
+/* vector-slot range [lo, hi) of part `k` of `parts` over `n` slots */
+__device__ __forceinline__ void part_of(size_t n, unsigned k, unsigned parts, size_t *lo, size_t *hi)
+{
+    *lo = (size_t)(((unsigned __int128)n * k) / parts);
+    *hi = (size_t)(((unsigned __int128)n * (k + 1)) / parts);
+}
+
+/* ---- broadcast: the root's blocks push slices of the source to every member ------------- */
+__global__ void __launch_bounds__(1024) k_broadcast(const ishmem_ctx_t *ctxs, coll_args a)
+{
+    __shared__ long long delta[ISHMEM_MAX_PES];
+    const ishmemi_team t = ctxs[0].teams[a.team];
+    const ishmem_ctx_t *ctx = ctxs + (t.start + a.root * t.stride);
+    if (!ishmemi::team_deltas(ctx, t, delta)) return;
+    size_t lo, hi;
+    part_of((a.n + 15) / 16, blockIdx.x, gridDim.x, &lo, &hi);
+    lo *= 16;
+    hi = hi * 16 < a.n ? hi * 16 : a.n;
+    if (lo >= hi) return;
+    ishmemi::push_bytes(local_of(ctxs, ctx, a.dest) + lo, delta, t.size, ctx->bcast_root_dest ? -1 : a.root,
+                        local_of(ctxs, ctx, a.src) + lo, hi - lo, threadIdx.x, blockDim.x);
+}
+
+/* ---- fcollect: member i's blocks push slices of its source into block i of every dest ---- */
+__global__ void __launch_bounds__(1024) k_fcollect(const ishmem_ctx_t *ctxs, coll_args a)
+{
+    __shared__ long long delta[ISHMEM_MAX_PES];
+    const ishmemi_team t = ctxs[0].teams[a.team];
+    const unsigned me = blockIdx.x % (unsigned)t.size, g = blockIdx.x / (unsigned)t.size;
+    const ishmem_ctx_t *ctx = ctxs + (t.start + (int)me * t.stride);
+    if (!ishmemi::team_deltas(ctx, t, delta)) return;
+    size_t lo, hi;
+    part_of((a.n + 15) / 16, g, (unsigned)a.groups, &lo, &hi);
+    lo *= 16;
+    hi = hi * 16 < a.n ? hi * 16 : a.n;
+    if (lo >= hi) return;
+    ishmemi::push_bytes(local_of(ctxs, ctx, a.dest) + (size_t)me * a.n + lo, delta, t.size, -1,
+                        local_of(ctxs, ctx, a.src) + lo, hi - lo, threadIdx.x, blockDim.x);
+}
+
+/* ---- reduce ------------------------------------------------------------------------------- */
+/* split: member q owns a contiguous address range, folds it from all sources in team order
+ * and stores the result into every member's dest (traffic: each source and each dest once).
+ * duplicated: member q folds the whole range and stores into its own dest only. */
+template <typename T, int OP>
+__global__ void __launch_bounds__(1024) k_reduce(const ishmem_ctx_t *ctxs, coll_args a)
+{
+    __shared__ long long delta[ISHMEM_MAX_PES];
+    const ishmemi_team t = ctxs[0].teams[a.team];
+    const unsigned me = blockIdx.x % (unsigned)t.size, g = blockIdx.x / (unsigned)t.size;
+    const ishmem_ctx_t *ctx = ctxs + (t.start + (int)me * t.stride);
+    if (!ishmemi::team_deltas(ctx, t, delta)) return;
+    constexpr size_t EPV = 16 / sizeof(T);
+    const size_t nslots = (a.n + EPV - 1) / EPV;
+    size_t lo = 0, hi = nslots;
+    if (!a.duplicated) part_of(nslots, me, (unsigned)t.size, &lo, &hi);
+    size_t glo, ghi;
+    part_of(hi - lo, g, (unsigned)a.groups, &glo, &ghi);
+    size_t begin = (lo + glo) * EPV, end = (lo + ghi) * EPV;
+    if (end > a.n) end = a.n;
+    if (begin >= end) return;
+    ishmemi::fold_range<T, OP>(local_of(ctxs, ctx, a.src), local_of(ctxs, ctx, a.dest), delta, t.size,
+                               a.duplicated ? (int)me : 0, a.duplicated ? 1 : t.size, begin, end,
+                               threadIdx.x, blockDim.x);
+}
+
+typedef void (*reduce_kernel_t)(const ishmem_ctx_t *, coll_args);
+
+template <typename T>
+static reduce_kernel_t pick_arith(int op)
+{
+    switch (op) {
+    case ISHMEM_OP_SUM: return k_reduce<T, ISHMEM_OP_SUM>;
+    case ISHMEM_OP_MAX: return k_reduce<T, ISHMEM_OP_MAX>;
+    case ISHMEM_OP_MIN: return k_reduce<T, ISHMEM_OP_MIN>;
+    case ISHMEM_OP_PROD: return k_reduce<T, ISHMEM_OP_PROD>;
+    default: return nullptr;
+    }
+}
+template <typename T>
+static reduce_kernel_t pick_int(int op)
+{
+    switch (op) {
+    case ISHMEM_OP_AND: return k_reduce<T, ISHMEM_OP_AND>;
+    case ISHMEM_OP_OR: return k_reduce<T, ISHMEM_OP_OR>;
+    case ISHMEM_OP_XOR: return k_reduce<T, ISHMEM_OP_XOR>;
+    default: return pick_arith<T>(op);
+    }
+}
+static reduce_kernel_t pick_reduce(int op, int dtype)
+{
+    switch (dtype) {
+    case ISHMEM_T_INT32: return pick_int<int>(op);
+    case ISHMEM_T_INT64: return pick_int<long long>(op);
+    case ISHMEM_T_UINT32: return pick_int<unsigned>(op);
+    case ISHMEM_T_UINT64: return pick_int<unsigned long long>(op);
+    case ISHMEM_T_FLOAT: return pick_arith<float>(op);
+    case ISHMEM_T_DOUBLE: return pick_arith<double>(op);
+    default: return nullptr;
+    }
+}
+static size_t dtype_size(int dtype)
+{
+    switch (dtype) {
+    case ISHMEM_T_INT32: case ISHMEM_T_UINT32: case ISHMEM_T_FLOAT: return 4;
+    case ISHMEM_T_INT64: case ISHMEM_T_UINT64: case ISHMEM_T_DOUBLE: return 8;
+    default: return 0;
+    }
+}
+
+/* ---- device-resident forms: one work-group per member, in-kernel push sync ---------------- */
+/* WHICH: 0 broadcast, 1 fcollect, 2 reduce<T, OP>, 3 sync */
+template <int WHICH, typename T, int OP>
+__global__ void __launch_bounds__(1024) k_collective_on_device(const ishmem_ctx_t *ctxs, coll_args a)
+{
+    const ishmemi_team t = ctxs[0].teams[a.team];
+    const ishmem_ctx_t *ctx = ctxs + (t.start + (int)blockIdx.x * t.stride);
+    char *d = a.dest ? local_of(ctxs, ctx, a.dest) : nullptr;
+    const char *s = a.src ? local_of(ctxs, ctx, a.src) : nullptr;
+    for (int r = 0; r < a.repeat; ++r) {
+        int rc;
+        if (WHICH == 0) rc = ishmemx_broadcastmem_work_group(ctx, a.team, d, s, a.n, a.root);
+        else if (WHICH == 1) rc = ishmemx_fcollectmem_work_group(ctx, a.team, d, s, a.n);
+        else if (WHICH == 2) rc = ishmemx_reduce_work_group<T, OP>(ctx, a.team, (T *)d, (const T *)s, a.n);
+        else rc = ishmemx_team_sync_work_group(ctx, a.team);
+        if (rc) return; /* the error is latched; every member gives up the same way */
+    }
+}
+
+template <typename T>
+static reduce_kernel_t pick_dev_arith(int op)
+{
+    switch (op) {
+    case ISHMEM_OP_SUM: return k_collective_on_device<2, T, ISHMEM_OP_SUM>;
+    case ISHMEM_OP_MAX: return k_collective_on_device<2, T, ISHMEM_OP_MAX>;
+    case ISHMEM_OP_MIN: return k_collective_on_device<2, T, ISHMEM_OP_MIN>;
+    case ISHMEM_OP_PROD: return k_collective_on_device<2, T, ISHMEM_OP_PROD>;
+    default: return nullptr;
+    }
+}
+template <typename T>
+static reduce_kernel_t pick_dev_int(int op)
+{
+    switch (op) {
+    case ISHMEM_OP_AND: return k_collective_on_device<2, T, ISHMEM_OP_AND>;
+    case ISHMEM_OP_OR: return k_collective_on_device<2, T, ISHMEM_OP_OR>;
+    case ISHMEM_OP_XOR: return k_collective_on_device<2, T, ISHMEM_OP_XOR>;
+    default: return pick_dev_arith<T>(op);
+    }
+}
+static reduce_kernel_t pick_dev(int which, int op, int dtype)
+{
+    if (which == 0) return k_collective_on_device<0, int, 0>;
+    if (which == 1) return k_collective_on_device<1, int, 0>;
+    if (which == 3) return k_collective_on_device<3, int, 0>;
+    switch (dtype) {
+    case ISHMEM_T_INT32: return pick_dev_int<int>(op);
+    case ISHMEM_T_INT64: return pick_dev_int<long long>(op);
+    case ISHMEM_T_UINT32: return pick_dev_int<unsigned>(op);
+    case ISHMEM_T_UINT64: return pick_dev_int<unsigned long long>(op);
+    case ISHMEM_T_FLOAT: return pick_dev_arith<float>(op);
+    case ISHMEM_T_DOUBLE: return pick_dev_arith<double>(op);
+    default: return nullptr;
+    }
+}
+
+/* ---- host side ---------------------------------------------------------------------------- */
+
+static int team_of(ishmem_team_t team, ishmemi_team *out)
+{
+    auto &g = g_ishmem;
+    if (team < 0 || team >= ISHMEM_MAX_TEAMS || !g.teams[team].valid) return ISHMEM_ERR_ARG;
+    *out = g.teams[team];
+    return ISHMEM_OK;
+}
+
+/* blocks per member for `bytes` of work per member */
+static int auto_groups(size_t bytes_per_member, int members)
+{
+    auto &g = g_ishmem;
+    if (g.coll_groups > 0) return g.coll_groups;
+    size_t want = (bytes_per_member + 32767) / 32768;
+    size_t cap = ((size_t)g.sm_count * 4 + members - 1) / members;
+    if (want < 1) want = 1;
+    return (int)(want < cap ? want : cap);
+}
+
+static int launch_sync_kernel(ishmem_team_t team, int repeat)
+{
+    auto &g = g_ishmem;
+    ishmemi_team t;
+    int rc = team_of(team, &t);
+    if (rc) return rc;
+    cudaStream_t s;
+    if ((rc = ishmemi_team_stream_begin(team, &s))) return rc;
+    coll_args a = {};
+    a.team = team;
+    a.repeat = repeat;
+    const ishmem_ctx_t *ctxs = g.d_ctx;
+    void *params[] = {(void *)&ctxs, (void *)&a};
+    rc = ishmemi_cuda(cudaLaunchCooperativeKernel((void *)pick_dev(3, 0, 0), dim3(t.size), dim3(64),
+                                                  params, 0, s),
+                      "cudaLaunchCooperativeKernel(sync)");
+    ishmemi_count_launch();
+    ishmemi_team_stream_end();
+    return rc;
+}
+
+extern "C" int ishmem_team_sync(ishmem_team_t team)
+{
+    ISHMEMI_REQUIRE_INIT();
+    return launch_sync_kernel(team, 1);
+}
+extern "C" int ishmem_sync_all(void)
+{
+    ISHMEMI_REQUIRE_INIT();
+    return launch_sync_kernel(ISHMEM_TEAM_WORLD, 1);
+}
+extern "C" int ishmem_barrier_all(void)
+{
+    auto &g = g_ishmem;
+    ISHMEMI_REQUIRE_INIT();
+    int rc;
+    for (int p = 0; p < g.npes; ++p)
+        if ((rc = ishmem_quiet(p))) return rc;
+    if ((rc = launch_sync_kernel(ISHMEM_TEAM_WORLD, 1))) return rc;
+    ISHMEMI_CUDA(cudaStreamSynchronize(g.team_stream));
+    return ISHMEM_OK;
+}
+
+static int check_sym2(const void *dest, size_t dbytes, const void *src, size_t sbytes)
+{
+    if (ishmemi_sym_offset(dest, dbytes) < 0 || ishmemi_sym_offset(src, sbytes) < 0)
+        return ISHMEM_ERR_NOT_SYMMETRIC;
+    return ISHMEM_OK;
+}
+
+extern "C" int ishmem_broadcastmem(ishmem_team_t team, void *dest, const void *src, size_t nbytes, int root)
+{
+    auto &g = g_ishmem;
+    ISHMEMI_REQUIRE_INIT();
+    ishmemi_team t;
+    int rc = team_of(team, &t);
+    if (rc) return rc;
+    if (root < 0 || root >= t.size) return ISHMEM_ERR_INVALID_PE;
+    if ((rc = check_sym2(dest, nbytes, src, nbytes))) return rc;
+    cudaStream_t s;
+    if ((rc = ishmemi_team_stream_begin(team, &s))) return rc;
+    if (nbytes == 0) {
+        ishmemi_team_stream_end();
+        return ISHMEM_OK;
+    }
+    if (nbytes >= g.cutover[1]) {
+        /* copy engine: one transfer per destination */
+        size_t doff = (size_t)ishmemi_sym_offset(dest, nbytes), soff = (size_t)ishmemi_sym_offset(src, nbytes);
+        int root_pe = t.start + root * t.stride;
+        for (int i = 0; i < t.size && !rc; ++i) {
+            if (i == root && !g.bcast_root_dest) continue;
+            int q = t.start + i * t.stride;
+            rc = ishmemi_cuda(cudaMemcpyAsync(g.base + (size_t)q * g.heap_bytes + doff,
+                                              g.base + (size_t)root_pe * g.heap_bytes + soff, nbytes,
+                                              cudaMemcpyDeviceToDevice, s),
+                              "cudaMemcpyAsync(broadcast)");
+        }
+    } else {
+        coll_args a = {};
+        a.team = team;
+        a.dest = (char *)dest;
+        a.src = (const char *)src;
+        a.n = nbytes;
+        a.root = root;
+        int blocks = auto_groups(nbytes, 1);
+        k_broadcast<<<blocks, g.coll_threads, 0, s>>>(g.d_ctx, a);
+        ishmemi_count_launch();
+        rc = ishmemi_check_launch("k_broadcast");
+    }
+    ishmemi_team_stream_end();
+    return rc;
+}
+
+extern "C" int ishmem_fcollectmem(ishmem_team_t team, void *dest, const void *src, size_t nbytes)
+{
+    auto &g = g_ishmem;
+    ISHMEMI_REQUIRE_INIT();
+    ishmemi_team t;
+    int rc = team_of(team, &t);
+    if (rc) return rc;
+    if (nbytes && (size_t)t.size > (size_t)-1 / nbytes) return ISHMEM_ERR_ARG;
+    if ((rc = check_sym2(dest, nbytes * t.size, src, nbytes))) return rc;
+    cudaStream_t s;
+    if ((rc = ishmemi_team_stream_begin(team, &s))) return rc;
+    if (nbytes == 0) {
+        ishmemi_team_stream_end();
+        return ISHMEM_OK;
+    }
+    if (nbytes >= g.cutover[2]) {
+        size_t doff = (size_t)ishmemi_sym_offset(dest, nbytes), soff = (size_t)ishmemi_sym_offset(src, nbytes);
+        for (int i = 0; i < t.size && !rc; ++i)
+            for (int j = 0; j < t.size && !rc; ++j) {
+                int from = t.start + i * t.stride, to = t.start + j * t.stride;
+                rc = ishmemi_cuda(cudaMemcpyAsync(g.base + (size_t)to * g.heap_bytes + doff + (size_t)i * nbytes,
+                                                  g.base + (size_t)from * g.heap_bytes + soff, nbytes,
+                                                  cudaMemcpyDeviceToDevice, s),
+                                  "cudaMemcpyAsync(fcollect)");
+            }
+    } else {
+        coll_args a = {};
+        a.team = team;
+        a.dest = (char *)dest;
+        a.src = (const char *)src;
+        a.n = nbytes;
+        a.groups = auto_groups(nbytes, t.size);
+        k_fcollect<<<a.groups * t.size, g.coll_threads, 0, s>>>(g.d_ctx, a);
+        ishmemi_count_launch();
+        rc = ishmemi_check_launch("k_fcollect");
+    }
+    ishmemi_team_stream_end();
+    return rc;
+}
+
+extern "C" int ishmemx_reduce(ishmem_team_t team, void *dest, const void *src, size_t nreduce, int op, int dtype,
+                              int algorithm)
+{
+    auto &g = g_ishmem;
+    ISHMEMI_REQUIRE_INIT();
+    ishmemi_team t;
+    int rc = team_of(team, &t);
+    if (rc) return rc;
+    const size_t es = dtype_size(dtype);
+    reduce_kernel_t k = pick_reduce(op, dtype);
+    if (!es || !k) return ISHMEM_ERR_ARG;
+    if (algorithm < ISHMEMX_REDUCE_AUTO || algorithm > ISHMEMX_REDUCE_SPLIT) return ISHMEM_ERR_ARG;
+    if (((uintptr_t)dest | (uintptr_t)src) % es) return ISHMEM_ERR_ALIGN;
+    if (nreduce > (size_t)-1 / es) return ISHMEM_ERR_ARG;
+    const size_t bytes = nreduce * es;
+    if ((rc = check_sym2(dest, bytes, src, bytes))) return rc;
+    const char *d = (const char *)dest, *sp = (const char *)src;
+    const bool overlap = d < sp + bytes && sp < d + bytes;
+    if (algorithm == ISHMEMX_REDUCE_AUTO) algorithm = ISHMEMX_REDUCE_SPLIT;
+    /* in place is fine when each element is read from all sources and written to all dests by
+     * one thread (split); any other overlap would mix old and new values */
+    if (overlap && !(d == sp && algorithm == ISHMEMX_REDUCE_SPLIT)) return ISHMEM_ERR_ARG;
+    cudaStream_t s;
+    if ((rc = ishmemi_team_stream_begin(team, &s))) return rc;
+    if (nreduce) {
+        coll_args a = {};
+        a.team = team;
+        a.dest = (char *)dest;
+        a.src = sp;
+        a.n = nreduce;
+        a.duplicated = (algorithm == ISHMEMX_REDUCE_DUPLICATED);
+        a.groups = auto_groups(a.duplicated ? bytes : bytes / t.size + 1, t.size);
+        k<<<a.groups * t.size, g.coll_threads, 0, s>>>(g.d_ctx, a);
+        ishmemi_count_launch();
+        rc = ishmemi_check_launch("k_reduce");
+    }
+    ishmemi_team_stream_end();
+    return rc;
+}
+
+#define ISHMEMI_DEF_REDUCE(NAME, T, OPNAME, OP, DT)                                                          \
+    extern "C" int ishmem_##NAME##_##OPNAME##_reduce(ishmem_team_t team, T *dest, const T *src, size_t nreduce) \
+    {                                                                                                        \
+        return ishmemx_reduce(team, dest, src, nreduce, OP, DT, ISHMEMX_REDUCE_AUTO);                        \
+    }
+#define ISHMEMI_DEF_REDUCE_ARITH(NAME, T, DT)                                                 \
+    ISHMEMI_DEF_REDUCE(NAME, T, sum, ISHMEM_OP_SUM, DT) ISHMEMI_DEF_REDUCE(NAME, T, max, ISHMEM_OP_MAX, DT) \
+    ISHMEMI_DEF_REDUCE(NAME, T, min, ISHMEM_OP_MIN, DT) ISHMEMI_DEF_REDUCE(NAME, T, prod, ISHMEM_OP_PROD, DT)
+#define ISHMEMI_DEF_REDUCE_BITS(NAME, T, DT)                                                  \
+    ISHMEMI_DEF_REDUCE(NAME, T, and, ISHMEM_OP_AND, DT) ISHMEMI_DEF_REDUCE(NAME, T, or, ISHMEM_OP_OR, DT) \
+    ISHMEMI_DEF_REDUCE(NAME, T, xor, ISHMEM_OP_XOR, DT)
+ISHMEMI_DEF_REDUCE_ARITH(int32, int32_t, ISHMEM_T_INT32)
+ISHMEMI_DEF_REDUCE_ARITH(int64, int64_t, ISHMEM_T_INT64)
+ISHMEMI_DEF_REDUCE_ARITH(uint32, uint32_t, ISHMEM_T_UINT32)
+ISHMEMI_DEF_REDUCE_ARITH(uint64, uint64_t, ISHMEM_T_UINT64)
+ISHMEMI_DEF_REDUCE_ARITH(float, float, ISHMEM_T_FLOAT)
+ISHMEMI_DEF_REDUCE_ARITH(double, double, ISHMEM_T_DOUBLE)
+ISHMEMI_DEF_REDUCE_BITS(int32, int32_t, ISHMEM_T_INT32)
+ISHMEMI_DEF_REDUCE_BITS(int64, int64_t, ISHMEM_T_INT64)
+ISHMEMI_DEF_REDUCE_BITS(uint32, uint32_t, ISHMEM_T_UINT32)
+ISHMEMI_DEF_REDUCE_BITS(uint64, uint64_t, ISHMEM_T_UINT64)
+
+extern "C" int ishmemx_collective_on_device(int which, ishmem_team_t team, void *dest, const void *src, size_t n,
+                                            int root, int op, int dtype, int threads, int repeat)
+{
+    auto &g = g_ishmem;
+    ISHMEMI_REQUIRE_INIT();
+    ishmemi_team t;
+    int rc = team_of(team, &t);
+    if (rc) return rc;
+    if (which < 0 || which > 3 || threads < 32 || threads > 1024 || repeat < 1) return ISHMEM_ERR_ARG;
+    if (which != 3) {
+        size_t es = 1;
+        if (which == 2) {
+            es = dtype_size(dtype);
+            if (!es || !pick_reduce(op, dtype)) return ISHMEM_ERR_ARG;
+            if (((uintptr_t)dest | (uintptr_t)src) % es) return ISHMEM_ERR_ALIGN;
+        }
+        if (which == 0 && (root < 0 || root >= t.size)) return ISHMEM_ERR_INVALID_PE;
+        if (n > (size_t)-1 / (es * t.size)) return ISHMEM_ERR_ARG;
+        size_t sbytes = n * es, dbytes = which == 1 ? sbytes * t.size : sbytes;
+        if ((rc = check_sym2(dest, dbytes, src, sbytes))) return rc;
+        const char *d = (const char *)dest, *sp = (const char *)src;
+        if (d < sp + sbytes && sp < d + dbytes) return ISHMEM_ERR_ARG;
+    }
+    cudaStream_t s;
+    if ((rc = ishmemi_team_stream_begin(team, &s))) return rc;
+    coll_args a = {};
+    a.team = team;
+    a.dest = (char *)dest;
+    a.src = (const char *)src;
+    a.n = n;
+    a.root = root;
+    a.repeat = repeat;
+    const ishmem_ctx_t *ctxs = g.d_ctx;
+    void *params[] = {(void *)&ctxs, (void *)&a};
+    rc = ishmemi_cuda(cudaLaunchCooperativeKernel((void *)pick_dev(which, op, dtype), dim3(t.size), dim3(threads),
+                                                  params, 0, s),
+                      "cudaLaunchCooperativeKernel(collective)");
+    ishmemi_count_launch();
+    ishmemi_team_stream_end();
+    return rc;
+}

@@ -1,0 +1,310 @@
+/* Device-initiated programs built on the device API: the put_signal / wait_until ping-pong
+ * and the Jacobi overlap workload.  Both are co-resident (cooperative) launches in which
+ * blocks of different PEs wait on one another with bounded waits. */
+#include <vector>
+
+#include "internal.h"
+
+__device__ __forceinline__ char *local_of(const ishmem_ctx_t *ctxs, const ishmem_ctx_t *ctx, const void *sym0)
+{
+    return (char *)sym0 + (ctx->heap_base - ctxs[0].heap_base);
+}
+
+/* ---- ping-pong ------------------------------------------------------------------------- */
+
+struct pingpong_out {
+    unsigned long long elapsed_ns;
+    unsigned long long mismatches;
+};
+
+__global__ void __launch_bounds__(1024) k_pingpong(const ishmem_ctx_t *ctxs, int pe_a, int pe_b, char *data0,
+                                                   unsigned long long *sig0, size_t nbytes, int rounds,
+                                                   pingpong_out *out)
+{
+    const bool is_a = (blockIdx.x == 0);
+    const ishmem_ctx_t *ctx = ctxs + (is_a ? pe_a : pe_b);
+    const int other = is_a ? pe_b : pe_a;
+    char *data = local_of(ctxs, ctx, data0);
+    unsigned long long *sig = (unsigned long long *)local_of(ctxs, ctx, sig0);
+    /* round stamps in the first and last 8 bytes of the payload catch a signal that
+     * overtakes its data */
+    volatile unsigned long long *w0 = (nbytes >= 8) ? (volatile unsigned long long *)data : nullptr;
+    volatile unsigned long long *w1 =
+        (nbytes >= 16 && nbytes % 8 == 0) ? (volatile unsigned long long *)(data + nbytes - 8) : nullptr;
+    unsigned long long bad = 0, t0 = 0;
+    if (is_a && threadIdx.x == 0) t0 = ishmemi::globaltimer_ns();
+    for (int r = 1; r <= rounds; ++r) {
+        if (is_a) {
+            if (threadIdx.x == 0) {
+                if (w0) *w0 = (unsigned long long)r;
+                if (w1) *w1 = (unsigned long long)r;
+            }
+            __syncthreads();
+            ishmemx_putmem_signal_work_group(ctx, data, data, nbytes, sig, (unsigned long long)r,
+                                             ISHMEM_SIGNAL_SET, other);
+            if (ishmemx_uint64_wait_until_work_group(ctx, sig, ISHMEM_CMP_GE, (unsigned long long)r)) break;
+        } else {
+            if (ishmemx_uint64_wait_until_work_group(ctx, sig, ISHMEM_CMP_GE, (unsigned long long)r)) break;
+            if (threadIdx.x == 0) {
+                if (w0 && *w0 != (unsigned long long)r) ++bad;
+                if (w1 && *w1 != (unsigned long long)r) ++bad;
+            }
+            __syncthreads();
+            ishmemx_putmem_signal_work_group(ctx, data, data, nbytes, sig, (unsigned long long)r,
+                                             ISHMEM_SIGNAL_SET, other);
+        }
+    }
+    if (threadIdx.x == 0) {
+        if (is_a) out->elapsed_ns = ishmemi::globaltimer_ns() - t0;
+        if (bad) atomicAdd(&out->mismatches, bad);
+    }
+}
+
+extern "C" int ishmemx_pingpong(int pe_a, int pe_b, void *data, uint64_t *sig, size_t nbytes, int rounds,
+                                int threads, double *half_rtt_ns, uint64_t *mismatches)
+{
+    ISHMEMI_REQUIRE_INIT();
+    auto &g = g_ishmem;
+    if (ishmemi_check_pe(pe_a) || ishmemi_check_pe(pe_b) || pe_a == pe_b) return ISHMEM_ERR_INVALID_PE;
+    if (rounds < 1 || threads < 32 || threads > 1024) return ISHMEM_ERR_ARG;
+    if ((uintptr_t)sig % 8 || (uintptr_t)data % 8) return ISHMEM_ERR_ALIGN;
+    if (ishmemi_sym_offset(data, nbytes) < 0 || ishmemi_sym_offset(sig, 8) < 0) return ISHMEM_ERR_NOT_SYMMETRIC;
+    cudaStream_t s;
+    int rc = ishmemi_team_stream_begin(ISHMEM_TEAM_WORLD, &s);
+    if (rc) return rc;
+    pingpong_out *out = (pingpong_out *)g.h_pinned;
+    out->elapsed_ns = 0;
+    out->mismatches = 0;
+    const ishmem_ctx_t *ctxs = g.d_ctx;
+    char *d0 = (char *)data;
+    unsigned long long *s0 = (unsigned long long *)sig;
+    void *params[] = {(void *)&ctxs, (void *)&pe_a, (void *)&pe_b, (void *)&d0, (void *)&s0,
+                      (void *)&nbytes, (void *)&rounds, (void *)&out};
+    rc = ishmemi_cuda(cudaLaunchCooperativeKernel((void *)k_pingpong, dim3(2), dim3(threads), params, 0, s),
+                      "cudaLaunchCooperativeKernel(pingpong)");
+    ishmemi_count_launch();
+    ishmemi_team_stream_end();
+    if (rc) return rc;
+    ISHMEMI_CUDA(cudaStreamSynchronize(s));
+    if (half_rtt_ns) *half_rtt_ns = (double)out->elapsed_ns / (2.0 * rounds);
+    if (mismatches) *mismatches = out->mismatches;
+    return ISHMEM_OK;
+}
+
+/* ---- Jacobi overlap workload -------------------------------------------------------------- */
+
+struct jacobi_args {
+    double *buf0, *buf1;          /* PE 0's copies */
+    unsigned long long *sig;      /* [0]: halo from the PE above arrived, [1]: from below */
+    size_t ny, nx;
+    int iters, overlap, groups;
+    unsigned long long *done;     /* scratch [npes*groups]: sweeps completed by each block */
+    double *partial;              /* scratch [npes*groups]: residual partial sums */
+};
+
+__device__ __forceinline__ void strip_of(size_t ny, int npes, int pe, size_t *first, size_t *rows)
+{
+    const size_t base = ny / (size_t)npes, extra = ny % (size_t)npes;
+    *rows = base + ((size_t)pe < extra ? 1 : 0);
+    *first = (size_t)pe * base + ((size_t)pe < extra ? (size_t)pe : extra);
+}
+
+/* One local row r of the strip: nxt[r] = sweep(cur[r-1..r+1]); boundary cells are copied.
+ * Adds the squared update to *acc when want_res. */
+__device__ __forceinline__ void jacobi_row(const double *cur, double *nxt, size_t r, size_t nx, bool fixed_row,
+                                           unsigned tid, unsigned nthr, bool want_res, double *acc)
+{
+    const double *up = cur + (r - 1) * nx, *mid = cur + r * nx, *dn = cur + (r + 1) * nx;
+    double *out = nxt + r * nx;
+    if (fixed_row) {
+        for (size_t j = tid; j < nx; j += nthr) out[j] = mid[j];
+        return;
+    }
+    if ((nx & 1) == 0) {
+        const size_t half = nx >> 1;
+        for (size_t c = tid; c < half; c += nthr) {
+            const size_t j = c << 1;
+            const double2 u = *(const double2 *)(up + j);
+            const double2 d = *(const double2 *)(dn + j);
+            const double2 m = *(const double2 *)(mid + j);
+            const double left = (j > 0) ? mid[j - 1] : 0.0;
+            const double right = (j + 2 < nx) ? mid[j + 2] : 0.0;
+            double2 v;
+            v.x = (j == 0) ? m.x : 0.25 * ((u.x + d.x) + (left + m.y));
+            v.y = (j + 2 == nx) ? m.y : 0.25 * ((u.y + d.y) + (m.x + right));
+            *(double2 *)(out + j) = v;
+            if (want_res) {
+                const double dx = v.x - m.x, dy = v.y - m.y;
+                *acc += dx * dx;
+                *acc += dy * dy;
+            }
+        }
+        return;
+    }
+    for (size_t j = tid; j < nx; j += nthr) {
+        double v = mid[j];
+        if (j > 0 && j + 1 < nx) v = 0.25 * ((up[j] + dn[j]) + (mid[j - 1] + mid[j + 1]));
+        out[j] = v;
+        if (want_res) {
+            const double dd = v - mid[j];
+            *acc += dd * dd;
+        }
+    }
+}
+
+__global__ void __launch_bounds__(1024) k_jacobi(const ishmem_ctx_t *ctxs, jacobi_args a)
+{
+    const int P = ctxs[0].npes, G = a.groups;
+    const int p = (int)blockIdx.x / G, g = (int)blockIdx.x % G;
+    const ishmem_ctx_t *ctx = ctxs + p;
+    const unsigned tid = threadIdx.x, nthr = blockDim.x;
+    size_t first, rows, rows_above = 0, f2;
+    strip_of(a.ny, P, p, &first, &rows);
+    if (p > 0) strip_of(a.ny, P, p - 1, &f2, &rows_above);
+    double *b[2] = {(double *)local_of(ctxs, ctx, a.buf0), (double *)local_of(ctxs, ctx, a.buf1)};
+    unsigned long long *sig = (unsigned long long *)local_of(ctxs, ctx, a.sig);
+    const size_t nx = a.nx;
+    /* this block's local rows [r0, r1) out of 1..rows */
+    const size_t r0 = 1 + rows * (size_t)g / (size_t)G, r1 = 1 + rows * (size_t)(g + 1) / (size_t)G;
+    unsigned long long *done = a.done + (size_t)p * G;
+    double acc = 0.0;
+    __shared__ int give_up;
+    if (tid == 0) give_up = 0;
+    __syncthreads();
+
+    for (int it = 0; it < a.iters; ++it) {
+        const double *cur = b[it & 1];
+        double *nxt = b[(it + 1) & 1];
+        const unsigned long long round = (unsigned long long)it + 1;
+        const bool want_res = (it == a.iters - 1);
+        /* (a) halo rows of the current sweep go out first: my first row to the bottom halo of
+         * the PE above, my last row to the top halo of the PE below */
+        if (g == 0 && p > 0)
+            ishmemx_putmem_signal_work_group(ctx, (void *)(cur + (rows_above + 1) * nx), cur + nx, nx * 8,
+                                             sig + 1, round, ISHMEM_SIGNAL_SET, p - 1);
+        if (g == G - 1 && p + 1 < P)
+            ishmemx_putmem_signal_work_group(ctx, (void *)cur, cur + rows * nx, nx * 8, sig + 0, round,
+                                             ISHMEM_SIGNAL_SET, p + 1);
+        /* (b) rows that need nobody else's data of this sweep */
+        if (a.overlap)
+            for (size_t r = r0 + 1; r + 1 < r1; ++r) {
+                const size_t gi = first + r - 1;
+                jacobi_row(cur, nxt, r, nx, gi == 0 || gi == a.ny - 1, tid, nthr, want_res, &acc);
+            }
+        /* (c) wait for the rows above and below this block's range: neighbouring blocks of
+         * the same PE publish a sweep counter, neighbouring PEs signal their halo */
+        if (tid == 0) {
+            int rc = 0;
+            ishmemi::deadline dl(ctx->wait_limit_ns);
+            if (g > 0) {
+                while (ishmemi::ld_acquire(done + g - 1) < (unsigned long long)it)
+                    if (dl.expired()) { rc = ISHMEM_ERR_TIMEOUT; break; }
+            } else if (p > 0) {
+                rc = ishmem_uint64_wait_until(ctx, sig + 0, ISHMEM_CMP_GE, round);
+            }
+            if (!rc) {
+                if (g < G - 1) {
+                    while (ishmemi::ld_acquire(done + g + 1) < (unsigned long long)it)
+                        if (dl.expired()) { rc = ISHMEM_ERR_TIMEOUT; break; }
+                } else if (p + 1 < P) {
+                    rc = ishmem_uint64_wait_until(ctx, sig + 1, ISHMEM_CMP_GE, round);
+                }
+            }
+            if (rc) {
+                ishmemi::latch_error(ctx, rc);
+                give_up = 1;
+            }
+        }
+        __syncthreads();
+        if (give_up) break;
+        /* (d) the remaining rows */
+        if (a.overlap) {
+            if (r1 > r0) {
+                size_t gi = first + r0 - 1;
+                jacobi_row(cur, nxt, r0, nx, gi == 0 || gi == a.ny - 1, tid, nthr, want_res, &acc);
+                if (r1 - 1 > r0) {
+                    gi = first + (r1 - 1) - 1;
+                    jacobi_row(cur, nxt, r1 - 1, nx, gi == 0 || gi == a.ny - 1, tid, nthr, want_res, &acc);
+                }
+            }
+        } else {
+            for (size_t r = r0; r < r1; ++r) {
+                const size_t gi = first + r - 1;
+                jacobi_row(cur, nxt, r, nx, gi == 0 || gi == a.ny - 1, tid, nthr, want_res, &acc);
+            }
+        }
+        /* (e) publish this sweep */
+        __syncthreads();
+        if (tid == 0) {
+            ishmemi::fence_acq_rel_gpu();
+            ishmemi::st_release(done + g, (unsigned long long)it + 1);
+        }
+    }
+    /* residual partial of this block, summed in a fixed order */
+    __shared__ double red[32];
+    for (int o = 16; o > 0; o >>= 1) acc += __shfl_down_sync(0xffffffffu, acc, o);
+    if ((tid & 31u) == 0) red[tid >> 5] = acc;
+    __syncthreads();
+    if (tid == 0) {
+        double s = 0.0;
+        for (unsigned w = 0; w < (nthr + 31) / 32; ++w) s += red[w];
+        a.partial[blockIdx.x] = s;
+    }
+}
+
+extern "C" int ishmemx_jacobi(double *buf0, double *buf1, uint64_t *sig, size_t ny, size_t nx, int iters,
+                              int overlap, int groups_per_pe, int threads, double *residual_sq_host)
+{
+    ISHMEMI_REQUIRE_INIT();
+    auto &g = g_ishmem;
+    const int P = g.npes;
+    if (ny < 3 || nx < 3 || iters < 0 || (size_t)P > ny) return ISHMEM_ERR_ARG;
+    if (threads < 32 || threads > 1024 || threads % 32 || groups_per_pe < 1) return ISHMEM_ERR_ARG;
+    const size_t rows_min = ny / P, rows_max = (ny + P - 1) / P;
+    if ((size_t)groups_per_pe > rows_min) groups_per_pe = (int)rows_min;
+    const size_t bytes = (rows_max + 2) * nx * 8;
+    if ((uintptr_t)buf0 % 16 || (uintptr_t)buf1 % 16 || (uintptr_t)sig % 8) return ISHMEM_ERR_ALIGN;
+    if (ishmemi_sym_offset(buf0, bytes) < 0 || ishmemi_sym_offset(buf1, bytes) < 0 ||
+        ishmemi_sym_offset(sig, 16) < 0)
+        return ISHMEM_ERR_NOT_SYMMETRIC;
+    const size_t nblocks = (size_t)P * groups_per_pe;
+    /* scratch: per-block sweep counters and residual partials */
+    char *scratch = nullptr;
+    ISHMEMI_CUDA(cudaMalloc((void **)&scratch, nblocks * 16));
+    cudaStream_t s;
+    int rc = ishmemi_team_stream_begin(ISHMEM_TEAM_WORLD, &s);
+    if (rc) {
+        cudaFree(scratch);
+        return rc;
+    }
+    rc = ishmemi_cuda(cudaMemsetAsync(scratch, 0, nblocks * 16, s), "cudaMemsetAsync");
+    jacobi_args a = {};
+    a.buf0 = buf0;
+    a.buf1 = buf1;
+    a.sig = (unsigned long long *)sig;
+    a.ny = ny;
+    a.nx = nx;
+    a.iters = iters;
+    a.overlap = overlap;
+    a.groups = groups_per_pe;
+    a.done = (unsigned long long *)scratch;
+    a.partial = (double *)(scratch + nblocks * 8);
+    const ishmem_ctx_t *ctxs = g.d_ctx;
+    void *params[] = {(void *)&ctxs, (void *)&a};
+    if (!rc)
+        rc = ishmemi_cuda(cudaLaunchCooperativeKernel((void *)k_jacobi, dim3((unsigned)nblocks), dim3(threads),
+                                                      params, 0, s),
+                          "cudaLaunchCooperativeKernel(jacobi)");
+    ishmemi_count_launch();
+    ishmemi_team_stream_end();
+    if (!rc) rc = ishmemi_cuda(cudaStreamSynchronize(s), "cudaStreamSynchronize");
+    if (!rc && residual_sq_host) {
+        std::vector<double> part(nblocks);
+        rc = ishmemi_cuda(cudaMemcpy(part.data(), a.partial, nblocks * 8, cudaMemcpyDeviceToHost), "cudaMemcpy");
+        double sum = 0.0;
+        for (size_t i = 0; i < nblocks; ++i) sum += part[i];
+        *residual_sq_host = sum;
+    }
+    cudaFree(scratch);
+    return rc;
+}

@@ -1,0 +1,506 @@
+/* Host runtime of libishmem.so: PE contexts, symmetric heap and allocator, streams, teams,
+ * status.  Host-only work (Section 3.6 of the paper: initialisation and all memory
+ * management are host calls). */
+#include <cstdlib>
+#include <cstring>
+
+#include "internal.h"
+
+ishmemi_state g_ishmem;
+
+int ishmemi_cuda(cudaError_t e, const char *what)
+{
+    if (e == cudaSuccess) return ISHMEM_OK;
+    g_ishmem.last_cuda_error = std::string(what) + ": " + cudaGetErrorString(e);
+    if (e == cudaErrorCooperativeLaunchTooLarge) return ISHMEM_ERR_NOT_CORESIDENT;
+    if (e == cudaErrorMemoryAllocation) return ISHMEM_ERR_OOM;
+    return ISHMEM_ERR_CUDA;
+}
+
+int ishmemi_check_launch(const char *what) { return ishmemi_cuda(cudaGetLastError(), what); }
+void ishmemi_count_launch(unsigned n) { g_ishmem.launches += n; }
+
+int ishmemi_check_pe(int pe)
+{
+    return (pe >= 0 && pe < g_ishmem.npes) ? ISHMEM_OK : ISHMEM_ERR_INVALID_PE;
+}
+
+long long ishmemi_sym_offset(const void *p, size_t n)
+{
+    const char *c = (const char *)p;
+    if (c < g_ishmem.base) return -1;
+    size_t off = (size_t)(c - g_ishmem.base);
+    if (off > g_ishmem.heap_bytes || n > g_ishmem.heap_bytes - off) return -1;
+    return (long long)off;
+}
+
+char *ishmemi_localise(const void *p, size_t n, int my_pe)
+{
+    long long off = ishmemi_sym_offset(p, n);
+    if (off < 0) return (char *)p;
+    return g_ishmem.base + (size_t)my_pe * g_ishmem.heap_bytes + (size_t)off;
+}
+
+void ishmemi_push_ctx()
+{
+    auto &g = g_ishmem;
+    for (int p = 0; p < g.npes; ++p) {
+        memcpy(g.h_ctx[p].teams, g.teams, sizeof(g.teams));
+        g.h_ctx[p].wait_limit_ns = g.wait_limit_ns;
+        g.h_ctx[p].bcast_root_dest = g.bcast_root_dest;
+    }
+    cudaMemcpy(g.d_ctx, g.h_ctx, sizeof(ishmem_ctx_t) * g.npes, cudaMemcpyHostToDevice);
+}
+
+/* ---- stream ordering ---------------------------------------------------------------- */
+
+cudaStream_t ishmemi_pe_stream_for_op(int pe)
+{
+    auto &g = g_ishmem;
+    if (g.pe_seen_team[pe] != g.team_seq) {
+        cudaStreamWaitEvent(g.pe_stream[pe], g.ev_team, 0);
+        g.pe_seen_team[pe] = g.team_seq;
+    }
+    g.pe_dirty[pe] = true;
+    return g.pe_stream[pe];
+}
+
+static void join_engine(int pe)
+{
+    auto &g = g_ishmem;
+    if (g.nbi_pending[pe]) {
+        cudaEventRecord(g.ev_engine[pe], g.engine_stream[pe]);
+        cudaStreamWaitEvent(g.pe_stream[pe], g.ev_engine[pe], 0);
+        g.nbi_pending[pe] = false;
+        g.pe_dirty[pe] = true;
+    }
+}
+
+int ishmemi_team_stream_begin(ishmem_team_t team, cudaStream_t *out)
+{
+    auto &g = g_ishmem;
+    if (team < 0 || team >= ISHMEM_MAX_TEAMS || !g.teams[team].valid) return ISHMEM_ERR_ARG;
+    const ishmemi_team &t = g.teams[team];
+    for (int i = 0; i < t.size; ++i) {
+        int p = t.start + i * t.stride;
+        join_engine(p);
+        if (g.pe_dirty[p]) {
+            cudaEventRecord(g.ev_pe[p], g.pe_stream[p]);
+            cudaStreamWaitEvent(g.team_stream, g.ev_pe[p], 0);
+            g.pe_dirty[p] = false;
+        }
+    }
+    *out = g.team_stream;
+    return ISHMEM_OK;
+}
+
+void ishmemi_team_stream_end()
+{
+    auto &g = g_ishmem;
+    cudaEventRecord(g.ev_team, g.team_stream);
+    ++g.team_seq;
+}
+
+int ishmemi_engine_copy(int my_pe, void *dst, const void *src, size_t n, bool blocking)
+{
+    auto &g = g_ishmem;
+    cudaStream_t ps = ishmemi_pe_stream_for_op(my_pe);
+    /* the engine starts after everything already enqueued by this PE */
+    ISHMEMI_CUDA(cudaEventRecord(g.ev_pe[my_pe], ps));
+    ISHMEMI_CUDA(cudaStreamWaitEvent(g.engine_stream[my_pe], g.ev_pe[my_pe], 0));
+    ISHMEMI_CUDA(cudaMemcpyAsync(dst, src, n, cudaMemcpyDeviceToDevice, g.engine_stream[my_pe]));
+    if (blocking) {
+        ISHMEMI_CUDA(cudaEventRecord(g.ev_engine[my_pe], g.engine_stream[my_pe]));
+        ISHMEMI_CUDA(cudaStreamWaitEvent(ps, g.ev_engine[my_pe], 0));
+    } else {
+        g.nbi_pending[my_pe] = true;
+    }
+    return ISHMEM_OK;
+}
+
+/* ---- lifecycle -------------------------------------------------------------------------- */
+
+static int init_common(int npes, size_t heap_bytes, void *external)
+{
+    auto &g = g_ishmem;
+    if (g.initialised) return ISHMEM_ERR_ARG;
+    if (npes < 1 || npes > ISHMEM_MAX_PES || heap_bytes == 0) return ISHMEM_ERR_ARG;
+    int ndev = 0;
+    if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev == 0) {
+        g.last_cuda_error = "no CUDA device: this library has no CPU path";
+        return ISHMEM_ERR_CUDA;
+    }
+    ISHMEMI_CUDA(cudaGetDevice(&g.device));
+    cudaDeviceProp prop;
+    ISHMEMI_CUDA(cudaGetDeviceProperties(&prop, g.device));
+    g.sm_count = prop.multiProcessorCount;
+    g.max_dyn_smem = prop.sharedMemPerBlockOptin;
+    heap_bytes = (heap_bytes + ISHMEMI_ALIGN - 1) / ISHMEMI_ALIGN * ISHMEMI_ALIGN;
+    if (external) {
+        if (((uintptr_t)external) % ISHMEMI_ALIGN) return ISHMEM_ERR_ALIGN;
+        g.base = (char *)external;
+        g.owns_heap = false;
+    } else {
+        void *p = nullptr;
+        ISHMEMI_CUDA(cudaMalloc(&p, heap_bytes * (size_t)npes));
+        ISHMEMI_CUDA(cudaMemset(p, 0, heap_bytes * (size_t)npes));
+        g.base = (char *)p;
+        g.owns_heap = true;
+    }
+    g.npes = npes;
+    g.heap_bytes = heap_bytes;
+    size_t internal = (size_t)npes * ISHMEMI_INTERNAL_BYTES + 256;
+    ISHMEMI_CUDA(cudaMalloc((void **)&g.d_internal, internal));
+    ISHMEMI_CUDA(cudaMemset(g.d_internal, 0, internal));
+    g.d_status = (int *)(g.d_internal + (size_t)npes * ISHMEMI_INTERNAL_BYTES);
+    ISHMEMI_CUDA(cudaMalloc((void **)&g.d_ctx, sizeof(ishmem_ctx_t) * npes));
+    ISHMEMI_CUDA(cudaHostAlloc(&g.h_pinned, 4096, cudaHostAllocDefault));
+
+    memset(g.teams, 0, sizeof(g.teams));
+    g.teams[ISHMEM_TEAM_WORLD] = {0, 1, npes, 1};
+    g.teams[ISHMEM_TEAM_SHARED] = {0, 1, npes, 1};
+    for (int p = 0; p < npes; ++p) {
+        ishmem_ctx_t &c = g.h_ctx[p];
+        memset(&c, 0, sizeof(c));
+        c.my_pe = p;
+        c.npes = npes;
+        c.heap_bytes = heap_bytes;
+        c.heap_base = g.base + (size_t)p * heap_bytes;
+        for (int q = 0; q < npes; ++q) {
+            /* every PE is reachable by load/store; entry q+1 of the table names the slot of
+             * the offset array that holds heap_base[q] - heap_base[p] */
+            c.reach[q] = (unsigned char)(q + 1);
+            c.heap_delta[q] = ((long long)q - (long long)p) * (long long)heap_bytes;
+        }
+        char *mine = g.d_internal + (size_t)p * ISHMEMI_INTERNAL_BYTES;
+        c.sync_arrive = (unsigned long long *)mine;
+        c.sync_epoch = (unsigned long long *)(mine + 8 * ISHMEM_MAX_TEAMS);
+        c.internal_stride = ISHMEMI_INTERNAL_BYTES;
+        c.status = g.d_status;
+    }
+    for (int p = 0; p < npes; ++p) {
+        ISHMEMI_CUDA(cudaStreamCreateWithFlags(&g.pe_stream[p], cudaStreamNonBlocking));
+        g.owns_pe_stream[p] = true;
+        ISHMEMI_CUDA(cudaStreamCreateWithFlags(&g.engine_stream[p], cudaStreamNonBlocking));
+        ISHMEMI_CUDA(cudaEventCreateWithFlags(&g.ev_pe[p], cudaEventDisableTiming));
+        ISHMEMI_CUDA(cudaEventCreateWithFlags(&g.ev_engine[p], cudaEventDisableTiming));
+        g.pe_dirty[p] = false;
+        g.nbi_pending[p] = false;
+        g.pe_seen_team[p] = 0;
+    }
+    ISHMEMI_CUDA(cudaStreamCreateWithFlags(&g.team_stream, cudaStreamNonBlocking));
+    g.owns_team_stream = true;
+    ISHMEMI_CUDA(cudaEventCreateWithFlags(&g.ev_team, cudaEventDisableTiming));
+    g.team_seq = 0;
+    g.free_blocks.clear();
+    g.used_blocks.clear();
+    g.free_blocks[0] = heap_bytes;
+    /* default cutovers: see ishmemx_set_cutover; tuned from the committed size sweep */
+    const char *env;
+    g.cutover[0] = (env = getenv("ISHMEM_CUTOVER_PUT")) ? strtoull(env, nullptr, 0) : (size_t)-1;
+    g.cutover[1] = (env = getenv("ISHMEM_CUTOVER_BCAST")) ? strtoull(env, nullptr, 0) : (size_t)-1;
+    g.cutover[2] = (env = getenv("ISHMEM_CUTOVER_FCOLLECT")) ? strtoull(env, nullptr, 0) : (size_t)-1;
+    if ((env = getenv("ISHMEM_WAIT_TIMEOUT_NS"))) g.wait_limit_ns = strtoull(env, nullptr, 0);
+    g.launches = 0;
+    g.initialised = true;
+    ishmemi_push_ctx();
+    ISHMEMI_CUDA(cudaDeviceSynchronize());
+    return ISHMEM_OK;
+}
+
+extern "C" int ishmem_init(int npes, size_t heap_bytes) { return init_common(npes, heap_bytes, nullptr); }
+
+extern "C" int ishmemx_init_external(int npes, size_t heap_bytes, void *base)
+{
+    if (!base) return ISHMEM_ERR_ARG;
+    if (heap_bytes % ISHMEMI_ALIGN) return ISHMEM_ERR_ALIGN;
+    return init_common(npes, heap_bytes, base);
+}
+
+extern "C" int ishmem_finalize(void)
+{
+    auto &g = g_ishmem;
+    ISHMEMI_REQUIRE_INIT();
+    cudaDeviceSynchronize();
+    for (int p = 0; p < g.npes; ++p) {
+        if (g.owns_pe_stream[p]) cudaStreamDestroy(g.pe_stream[p]);
+        cudaStreamDestroy(g.engine_stream[p]);
+        cudaEventDestroy(g.ev_pe[p]);
+        cudaEventDestroy(g.ev_engine[p]);
+    }
+    if (g.owns_team_stream) cudaStreamDestroy(g.team_stream);
+    cudaEventDestroy(g.ev_team);
+    if (g.owns_heap) cudaFree(g.base);
+    cudaFree(g.d_internal);
+    cudaFree(g.d_ctx);
+    cudaFreeHost(g.h_pinned);
+    g.base = nullptr;
+    g.d_internal = nullptr;
+    g.d_ctx = nullptr;
+    g.h_pinned = nullptr;
+    g.free_blocks.clear();
+    g.used_blocks.clear();
+    g.npes = 0;
+    g.initialised = false;
+    return ISHMEM_OK;
+}
+
+extern "C" int ishmem_n_pes(void) { return g_ishmem.initialised ? g_ishmem.npes : 0; }
+extern "C" size_t ishmemx_heap_bytes(void) { return g_ishmem.initialised ? g_ishmem.heap_bytes : 0; }
+
+extern "C" void *ishmemx_ctx(int pe)
+{
+    if (!g_ishmem.initialised || ishmemi_check_pe(pe)) return nullptr;
+    return g_ishmem.d_ctx + pe;
+}
+
+extern "C" int ishmemx_set_stream(int pe, void *cuda_stream)
+{
+    auto &g = g_ishmem;
+    ISHMEMI_REQUIRE_INIT();
+    if (pe == -1) {
+        ISHMEMI_CUDA(cudaStreamSynchronize(g.team_stream));
+        if (g.owns_team_stream) cudaStreamDestroy(g.team_stream);
+        g.team_stream = (cudaStream_t)cuda_stream;
+        g.owns_team_stream = false;
+        return ISHMEM_OK;
+    }
+    if (ishmemi_check_pe(pe)) return ISHMEM_ERR_INVALID_PE;
+    ISHMEMI_CUDA(cudaStreamSynchronize(g.pe_stream[pe]));
+    if (g.owns_pe_stream[pe]) cudaStreamDestroy(g.pe_stream[pe]);
+    g.pe_stream[pe] = (cudaStream_t)cuda_stream;
+    g.owns_pe_stream[pe] = false;
+    return ISHMEM_OK;
+}
+
+extern "C" void *ishmemx_get_stream(int pe)
+{
+    auto &g = g_ishmem;
+    if (!g.initialised) return nullptr;
+    if (pe == -1) return (void *)g.team_stream;
+    if (ishmemi_check_pe(pe)) return nullptr;
+    return (void *)g.pe_stream[pe];
+}
+
+extern "C" const char *ishmem_strerror(int status)
+{
+    switch (status) {
+    case ISHMEM_OK: return "success";
+    case ISHMEM_ERR_INVALID_PE: return "invalid PE";
+    case ISHMEM_ERR_NOT_SYMMETRIC: return "address range is not in the symmetric heap";
+    case ISHMEM_ERR_ALIGN: return "misaligned address";
+    case ISHMEM_ERR_OOM: return "out of memory";
+    case ISHMEM_ERR_TIMEOUT: return "a bounded device-side wait timed out";
+    case ISHMEM_ERR_NOT_CORESIDENT: return "launch does not fit co-resident on the device";
+    case ISHMEM_ERR_CUDA: return "CUDA runtime error";
+    case ISHMEM_ERR_ARG: return "invalid argument";
+    case ISHMEM_ERR_NOT_INITIALIZED: return "library not initialised";
+    default: return "unknown status";
+    }
+}
+
+extern "C" const char *ishmemx_last_cuda_error(void) { return g_ishmem.last_cuda_error.c_str(); }
+
+extern "C" int ishmemx_status(int clear)
+{
+    auto &g = g_ishmem;
+    ISHMEMI_REQUIRE_INIT();
+    ISHMEMI_CUDA(cudaDeviceSynchronize());
+    int st = 0;
+    ISHMEMI_CUDA(cudaMemcpy(&st, g.d_status, sizeof(int), cudaMemcpyDeviceToHost));
+    if (clear && st) ISHMEMI_CUDA(cudaMemset(g.d_status, 0, sizeof(int)));
+    return st;
+}
+
+extern "C" int ishmemx_set_wait_limit_ns(uint64_t ns)
+{
+    ISHMEMI_REQUIRE_INIT();
+    if (ns == 0) return ISHMEM_ERR_ARG;
+    ISHMEMI_CUDA(cudaDeviceSynchronize());
+    g_ishmem.wait_limit_ns = ns;
+    ishmemi_push_ctx();
+    return ISHMEM_OK;
+}
+
+extern "C" unsigned long long ishmemx_launch_count(void) { return g_ishmem.launches; }
+
+/* ---- symmetric allocator: first fit over a sorted free list, coalescing on free ----------- */
+
+static void *sym_alloc(size_t alignment, size_t size)
+{
+    auto &g = g_ishmem;
+    if (!g.initialised || size == 0) return nullptr;
+    if (alignment < ISHMEMI_ALIGN) alignment = ISHMEMI_ALIGN;
+    if (alignment & (alignment - 1)) return nullptr;
+    size_t need = (size + ISHMEMI_ALIGN - 1) / ISHMEMI_ALIGN * ISHMEMI_ALIGN;
+    if (need < size) return nullptr;
+    std::lock_guard<std::mutex> lk(g.mu);
+    for (auto it = g.free_blocks.begin(); it != g.free_blocks.end(); ++it) {
+        size_t off = it->first, len = it->second;
+        /* alignment is relative to the device address; heap bases are 256-byte aligned */
+        uintptr_t addr = (uintptr_t)g.base + off;
+        size_t pad = (size_t)((alignment - addr % alignment) % alignment);
+        if (pad > len || need > len - pad) continue;
+        size_t start = off + pad;
+        g.free_blocks.erase(it);
+        if (pad) g.free_blocks[off] = pad;
+        if (len - pad - need) g.free_blocks[start + need] = len - pad - need;
+        g.used_blocks[start] = need;
+        return g.base + start;
+    }
+    return nullptr;
+}
+
+extern "C" void *ishmem_malloc(size_t size) { return sym_alloc(ISHMEMI_ALIGN, size); }
+extern "C" void *ishmem_align(size_t alignment, size_t size) { return sym_alloc(alignment, size); }
+
+extern "C" void *ishmem_calloc(size_t count, size_t size)
+{
+    auto &g = g_ishmem;
+    if (size && count > (size_t)-1 / size) return nullptr;
+    void *p = sym_alloc(ISHMEMI_ALIGN, count * size);
+    if (!p) return nullptr;
+    size_t off = (size_t)((char *)p - g.base);
+    for (int pe = 0; pe < g.npes; ++pe) {
+        cudaStream_t s = ishmemi_pe_stream_for_op(pe);
+        if (cudaMemsetAsync(g.base + (size_t)pe * g.heap_bytes + off, 0, count * size, s) != cudaSuccess) {
+            ishmem_free(p);
+            return nullptr;
+        }
+    }
+    return p;
+}
+
+extern "C" int ishmem_free(void *ptr)
+{
+    auto &g = g_ishmem;
+    ISHMEMI_REQUIRE_INIT();
+    if (!ptr) return ISHMEM_OK;
+    std::lock_guard<std::mutex> lk(g.mu);
+    long long off = ishmemi_sym_offset(ptr, 0);
+    if (off < 0) return ISHMEM_ERR_NOT_SYMMETRIC;
+    auto it = g.used_blocks.find((size_t)off);
+    if (it == g.used_blocks.end()) return ISHMEM_ERR_ARG;
+    size_t start = it->first, len = it->second;
+    g.used_blocks.erase(it);
+    auto next = g.free_blocks.lower_bound(start);
+    if (next != g.free_blocks.end() && next->first == start + len) {
+        len += next->second;
+        next = g.free_blocks.erase(next);
+    }
+    if (next != g.free_blocks.begin()) {
+        auto prev = std::prev(next);
+        if (prev->first + prev->second == start) {
+            prev->second += len;
+            return ISHMEM_OK;
+        }
+    }
+    g.free_blocks[start] = len;
+    return ISHMEM_OK;
+}
+
+extern "C" void *ishmem_ptr(const void *sym, int pe)
+{
+    auto &g = g_ishmem;
+    if (!g.initialised || ishmemi_check_pe(pe)) return nullptr;
+    long long off = ishmemi_sym_offset(sym, 0);
+    if (off < 0) return nullptr;
+    return g.base + (size_t)pe * g.heap_bytes + (size_t)off;
+}
+
+extern "C" int ishmemx_heap_write(int pe, void *sym_dest, const void *host, size_t nbytes)
+{
+    auto &g = g_ishmem;
+    ISHMEMI_REQUIRE_INIT();
+    if (ishmemi_check_pe(pe)) return ISHMEM_ERR_INVALID_PE;
+    long long off = ishmemi_sym_offset(sym_dest, nbytes);
+    if (off < 0) return ISHMEM_ERR_NOT_SYMMETRIC;
+    cudaStream_t s = ishmemi_pe_stream_for_op(pe);
+    ISHMEMI_CUDA(cudaMemcpyAsync(g.base + (size_t)pe * g.heap_bytes + (size_t)off, host, nbytes,
+                                 cudaMemcpyHostToDevice, s));
+    return ISHMEM_OK;
+}
+
+extern "C" int ishmemx_heap_read(int pe, void *host, const void *sym_src, size_t nbytes)
+{
+    auto &g = g_ishmem;
+    ISHMEMI_REQUIRE_INIT();
+    if (ishmemi_check_pe(pe)) return ISHMEM_ERR_INVALID_PE;
+    long long off = ishmemi_sym_offset(sym_src, nbytes);
+    if (off < 0) return ISHMEM_ERR_NOT_SYMMETRIC;
+    cudaStream_t s = ishmemi_pe_stream_for_op(pe);
+    ISHMEMI_CUDA(cudaMemcpyAsync(host, g.base + (size_t)pe * g.heap_bytes + (size_t)off, nbytes,
+                                 cudaMemcpyDeviceToHost, s));
+    return ISHMEM_OK;
+}
+
+/* ---- teams ---------------------------------------------------------------------------------- */
+
+extern "C" ishmem_team_t ishmem_team_split_strided(ishmem_team_t parent, int start, int stride, int size)
+{
+    auto &g = g_ishmem;
+    if (!g.initialised || parent < 0 || parent >= ISHMEM_MAX_TEAMS || !g.teams[parent].valid)
+        return ISHMEM_TEAM_INVALID;
+    const ishmemi_team pt = g.teams[parent];
+    if (size < 1 || stride < 1 || start < 0 || start + (size - 1) * stride >= pt.size)
+        return ISHMEM_TEAM_INVALID;
+    for (int t = 2; t < ISHMEM_MAX_TEAMS; ++t)
+        if (!g.teams[t].valid) {
+            cudaDeviceSynchronize();
+            g.teams[t] = {pt.start + start * pt.stride, stride * pt.stride, size, 1};
+            /* a recycled slot starts from fresh counters on every PE */
+            for (int p = 0; p < g.npes; ++p) {
+                cudaMemset(g.h_ctx[p].sync_arrive + t, 0, 8);
+                cudaMemset(g.h_ctx[p].sync_epoch + t, 0, 8);
+            }
+            ishmemi_push_ctx();
+            return t;
+        }
+    return ISHMEM_TEAM_INVALID;
+}
+
+extern "C" int ishmem_team_destroy(ishmem_team_t team)
+{
+    auto &g = g_ishmem;
+    ISHMEMI_REQUIRE_INIT();
+    if (team < 2 || team >= ISHMEM_MAX_TEAMS || !g.teams[team].valid) return ISHMEM_ERR_ARG;
+    cudaDeviceSynchronize();
+    g.teams[team].valid = 0;
+    ishmemi_push_ctx();
+    return ISHMEM_OK;
+}
+
+extern "C" int ishmem_team_n_pes(ishmem_team_t team)
+{
+    auto &g = g_ishmem;
+    if (!g.initialised || team < 0 || team >= ISHMEM_MAX_TEAMS || !g.teams[team].valid) return -1;
+    return g.teams[team].size;
+}
+
+extern "C" int ishmemx_set_cutover(int which, size_t nbytes)
+{
+    ISHMEMI_REQUIRE_INIT();
+    if (which < 0 || which > 2) return ISHMEM_ERR_ARG;
+    g_ishmem.cutover[which] = nbytes;
+    return ISHMEM_OK;
+}
+extern "C" size_t ishmemx_get_cutover(int which)
+{
+    return (which < 0 || which > 2) ? 0 : g_ishmem.cutover[which];
+}
+extern "C" int ishmemx_set_bcast_root_dest(int enable)
+{
+    ISHMEMI_REQUIRE_INIT();
+    cudaDeviceSynchronize();
+    g_ishmem.bcast_root_dest = enable ? 1 : 0;
+    ishmemi_push_ctx();
+    return ISHMEM_OK;
+}
+extern "C" int ishmemx_set_collective_geometry(int groups_per_pe, int threads)
+{
+    ISHMEMI_REQUIRE_INIT();
+    if (groups_per_pe < 0 || threads < 32 || threads > 1024 || threads % 32) return ISHMEM_ERR_ARG;
+    g_ishmem.coll_groups = groups_per_pe;
+    g_ishmem.coll_threads = threads;
+    return ISHMEM_OK;
+}
