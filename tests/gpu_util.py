@@ -15,6 +15,7 @@ class Session:
 
     def __init__(self, npes: int, heap_bytes: int, with_oracle: bool = True):
         assert torch.cuda.is_available()
+        heap_bytes = (heap_bytes + 255) // 256 * 256
         self.npes, self.heap_bytes = npes, heap_bytes
         self.heap = torch.zeros(npes * heap_bytes, dtype=torch.uint8, device="cuda")
         torch.cuda.synchronize()
