@@ -349,6 +349,25 @@ int ishmemx_pingpong(int pe_a, int pe_b, void *data, uint64_t *sig, size_t nbyte
 int ishmemx_jacobi(double *buf0, double *buf1, uint64_t *sig, size_t ny, size_t nx, int iters,
                    int overlap, int groups_per_pe, int threads, double *residual_sq_host);
 
+/* The same Jacobi program for callers that must not allocate device memory at the point of
+ * the call -- a frozen memory pool, a loop where cudaMalloc's device-wide synchronisation is
+ * not acceptable, an allocator that owns the whole GPU.  (The paper has no counterpart; this
+ * is a convenience of this library.)  The kernel's scratch -- one sweep counter and one
+ * residual partial per block -- sits in a fixed 32 KiB device array inside the library, which
+ * every GPU that loads the library holds until the process exits; the call itself performs no
+ * cudaMalloc/cudaFree and calls no allocating routine.  Limits and caveats:
+ *   - npes * groups_per_pe (after clamping groups_per_pe to the shortest strip) must not
+ *     exceed 2048 blocks; larger launches are refused with ISHMEM_ERR_ARG and
+ *     ishmemx_last_cuda_error() names the limit.
+ *   - The first call on each device resolves the array's device address
+ *     (cudaGetSymbolAddress); make that first call before any stream capture begins.
+ *   - All calls share the one array.  It still holds the previous call's contents, so each
+ *     call clears the part it uses first; two calls whose kernels overlap on the GPU (from
+ *     two host threads, say) would race on it -- serialise them.
+ * Arguments, results and error codes are otherwise those of ishmemx_jacobi. */
+int ishmemx_jacobi_noalloc(double *buf0, double *buf1, uint64_t *sig, size_t ny, size_t nx, int iters,
+                           int overlap, int groups_per_pe, int threads, double *residual_sq_host);
+
 /* Host-buffer convenience for end-to-end measurements: copy `nbytes` from HOST `src_host`
  * into src@p for every PE p (per-PE stride `nbytes` in the host buffer), run
  * ishmemx_putmem_spmd(dest, src, nbytes, shift, level, threads, groups), and copy every

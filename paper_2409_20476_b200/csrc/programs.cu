@@ -308,3 +308,88 @@ extern "C" int ishmemx_jacobi(double *buf0, double *buf1, uint64_t *sig, size_t 
     cudaFree(scratch);
     return rc;
 }
+
+/* ---- Jacobi without any allocation ---------------------------------------------------------
+ * Some callers may not allocate device memory when they call into the library: code running
+ * while a memory pool is frozen, inside a latency-critical loop where cudaMalloc's implicit
+ * device synchronisation is unacceptable, or under an allocator that owns the whole device.
+ * For them the per-block sweep counters and residual partials of the Jacobi kernel live in this
+ * fixed array instead of a cudaMalloc'ed buffer.  Every GPU that loads the library holds these
+ * 32 KiB until the process exits. */
+#define ISHMEMX_JACOBI_NOALLOC_MAX_BLOCKS 2048
+static __device__ __align__(256) unsigned char g_jacobi_scratch[ISHMEMX_JACOBI_NOALLOC_MAX_BLOCKS * 16];
+
+/* device address of g_jacobi_scratch per device ordinal, resolved on first use: in host code the
+ * symbol's name is only a handle, never a pointer a kernel may dereference */
+static void *g_jacobi_scratch_addr[64] = {};
+
+static int jacobi_scratch_for_current_device(void **out)
+{
+    int dev = 0;
+    ISHMEMI_CUDA(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return ISHMEM_ERR_ARG;
+    if (!g_jacobi_scratch_addr[dev]) {
+        void *p = nullptr;
+        ISHMEMI_CUDA(cudaGetSymbolAddress(&p, g_jacobi_scratch));
+        g_jacobi_scratch_addr[dev] = p;
+    }
+    *out = g_jacobi_scratch_addr[dev];
+    return ISHMEM_OK;
+}
+
+extern "C" int ishmemx_jacobi_noalloc(double *buf0, double *buf1, uint64_t *sig, size_t ny, size_t nx, int iters,
+                                      int overlap, int groups_per_pe, int threads, double *residual_sq_host)
+{
+    ISHMEMI_REQUIRE_INIT();
+    auto &g = g_ishmem;
+    const int P = g.npes;
+    if (ny < 3 || nx < 3 || iters < 0 || (size_t)P > ny) return ISHMEM_ERR_ARG;
+    if (threads < 32 || threads > 1024 || threads % 32 || groups_per_pe < 1) return ISHMEM_ERR_ARG;
+    const size_t rows_min = ny / P, rows_max = (ny + P - 1) / P;
+    if ((size_t)groups_per_pe > rows_min) groups_per_pe = (int)rows_min;
+    const size_t nblocks = (size_t)P * groups_per_pe;
+    if (nblocks > ISHMEMX_JACOBI_NOALLOC_MAX_BLOCKS) {
+        g.last_cuda_error = "ishmemx_jacobi_noalloc: npes * groups_per_pe exceeds the fixed scratch (2048 blocks)";
+        return ISHMEM_ERR_ARG;
+    }
+    const size_t bytes = (rows_max + 2) * nx * 8;
+    if ((uintptr_t)buf0 % 16 || (uintptr_t)buf1 % 16 || (uintptr_t)sig % 8) return ISHMEM_ERR_ALIGN;
+    if (ishmemi_sym_offset(buf0, bytes) < 0 || ishmemi_sym_offset(buf1, bytes) < 0 ||
+        ishmemi_sym_offset(sig, 16) < 0)
+        return ISHMEM_ERR_NOT_SYMMETRIC;
+    void *scratch = nullptr;
+    int rc = jacobi_scratch_for_current_device(&scratch);
+    if (rc) return rc;
+    cudaStream_t s;
+    if ((rc = ishmemi_team_stream_begin(ISHMEM_TEAM_WORLD, &s))) return rc;
+    /* the array keeps the previous call's counters: they must start from zero */
+    rc = ishmemi_cuda(cudaMemsetAsync(scratch, 0, nblocks * 16, s), "cudaMemsetAsync");
+    jacobi_args a = {};
+    a.buf0 = buf0;
+    a.buf1 = buf1;
+    a.sig = (unsigned long long *)sig;
+    a.ny = ny;
+    a.nx = nx;
+    a.iters = iters;
+    a.overlap = overlap;
+    a.groups = groups_per_pe;
+    a.done = (unsigned long long *)scratch;
+    a.partial = (double *)((char *)scratch + nblocks * 8);
+    const ishmem_ctx_t *ctxs = g.d_ctx;
+    void *params[] = {(void *)&ctxs, (void *)&a};
+    if (!rc)
+        rc = ishmemi_cuda(cudaLaunchCooperativeKernel((void *)k_jacobi, dim3((unsigned)nblocks), dim3(threads),
+                                                      params, 0, s),
+                          "cudaLaunchCooperativeKernel(jacobi_noalloc)");
+    ishmemi_count_launch();
+    ishmemi_team_stream_end();
+    if (!rc) rc = ishmemi_cuda(cudaStreamSynchronize(s), "cudaStreamSynchronize");
+    if (!rc && residual_sq_host) {
+        double part[ISHMEMX_JACOBI_NOALLOC_MAX_BLOCKS];
+        rc = ishmemi_cuda(cudaMemcpy(part, a.partial, nblocks * 8, cudaMemcpyDeviceToHost), "cudaMemcpy");
+        double sum = 0.0;
+        for (size_t i = 0; i < nblocks; ++i) sum += part[i];
+        *residual_sq_host = sum;
+    }
+    return rc;
+}
