@@ -268,7 +268,7 @@ def run_ours(args) -> dict:
     if not args.no_e2e:
         out["e2e"] = e2e(B, torch, replicas, dst, src, level, args, world)
     if rank == 0 and world == 1 and not args.no_cpu:
-        out["cpu_baseline"] = cpu_baseline(args.cpu_scale, reps=3)
+        out["cpu_baseline"] = cpu_baseline(args.cpu_scale, reps=5)
     B.ishmem_finalize()
     replicas.finalize()
     return out if rank == 0 else {}
@@ -500,11 +500,11 @@ def main():
     ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--level", default="ldst", choices=["bulk", "ldst"])
-    ap.add_argument("--threads", type=int, default=512)
-    ap.add_argument("--groups", type=int, default=74, help="work-groups per PE in the put/get launch")
+    ap.add_argument("--level", default="bulk", choices=["bulk", "ldst"])
+    ap.add_argument("--threads", type=int, default=256)
+    ap.add_argument("--groups", type=int, default=37, help="work-groups per PE in the put/get launch")
     ap.add_argument("--jacobi-groups", type=int, default=18)
-    ap.add_argument("--cpu-scale", type=int, default=2)
+    ap.add_argument("--cpu-scale", type=int, default=1)
     ap.add_argument("--e2e-bytes", type=int, default=64 * MiB, help="payload per PE of the end-to-end leg")
     ap.add_argument("--no-breakdown", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")

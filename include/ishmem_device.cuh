@@ -341,10 +341,13 @@ __device__ __forceinline__ void bulk_wait()
  * shared -> global by cp.async.bulk in bulk groups.  nstages-1 loads are kept in flight.
  * When `complete` is false the last stores may still be in flight on return (the _nbi
  * forms; ishmem_quiet by the same thread completes them) -- their shared-memory reads
- * are finished either way, so the staging may be reused.  Returns 0 or
- * ISHMEM_ERR_TIMEOUT. */
+ * are finished either way, so the staging may be reused.  With `delta` every staged chunk is
+ * stored to the ndst destinations d + delta[q] (q != skip): the push form used by broadcast
+ * and fcollect, one load and ndst stores per chunk.  Returns 0 or ISHMEM_ERR_TIMEOUT. */
 static __device__ __noinline__ int bulk_copy_ring(const ishmem_ctx_t *ctx, char *d, const char *s,
-                                           size_t n, ishmemx_staging_t st, bool complete)
+                                                  size_t n, ishmemx_staging_t st, bool complete,
+                                                  const long long *delta = nullptr, int ndst = 1,
+                                                  int skip = -1, size_t first = 0, size_t stride = 1)
 {
     /* layout: [0,64) mbarriers, [128, ...) stages */
     unsigned long long *bars = (unsigned long long *)st.smem;
@@ -357,22 +360,26 @@ static __device__ __noinline__ int bulk_copy_ring(const ishmem_ctx_t *ctx, char 
         stage_bytes = (avail / nstages) & ~1023u;
     }
     if (stage_bytes > 65536u) stage_bytes = 65536u;
-    const size_t nchunks = (n + stage_bytes - 1) / stage_bytes;
+    /* chunks first, first + stride, ... of the range belong to this caller (blocks of one
+     * launch take chunks round-robin so that together they sweep one contiguous window) */
+    const size_t total = (n + stage_bytes - 1) / stage_bytes;
+    const size_t nchunks = total > first ? (total - first + stride - 1) / stride : 0;
     const unsigned bar0 = smem_u32(bars);
     const unsigned sm0 = smem_u32(stage0);
     for (unsigned k = 0; k < nstages; ++k) mbar_init(bar0 + 8 * k, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     fence_proxy_async();
 
+    auto chunk_off = [&](size_t c) -> size_t { return (first + c * stride) * stage_bytes; };
     auto chunk_bytes = [&](size_t c) -> unsigned {
-        size_t left = n - c * stage_bytes;
+        size_t left = n - chunk_off(c);
         return left < stage_bytes ? (unsigned)left : stage_bytes;
     };
     auto issue_load = [&](size_t c) {
         unsigned sidx = (unsigned)(c % nstages);
         unsigned b = chunk_bytes(c);
         mbar_expect_tx(bar0 + 8 * sidx, b);
-        bulk_g2s(sm0 + sidx * stage_bytes, s + c * stage_bytes, b, bar0 + 8 * sidx);
+        bulk_g2s(sm0 + sidx * stage_bytes, s + chunk_off(c), b, bar0 + 8 * sidx);
     };
 
     int rc = 0;
@@ -386,7 +393,12 @@ static __device__ __noinline__ int bulk_copy_ring(const ishmem_ctx_t *ctx, char 
             rc = ISHMEM_ERR_TIMEOUT;
             break;
         }
-        bulk_s2g(d + c * stage_bytes, sm0 + sidx * stage_bytes, chunk_bytes(c));
+        if (delta == nullptr) {
+            bulk_s2g(d + chunk_off(c), sm0 + sidx * stage_bytes, chunk_bytes(c));
+        } else {
+            for (int q = 0; q < ndst; ++q)
+                if (q != skip) bulk_s2g(d + delta[q] + chunk_off(c), sm0 + sidx * stage_bytes, chunk_bytes(c));
+        }
         bulk_commit();
         if (issued < nchunks) {
             /* the stage of chunk c-1 is the one chunk `issued` will land in: its store
@@ -430,15 +442,16 @@ __device__ __forceinline__ int wg_copy(const ishmem_ctx_t *ctx, char *d, const c
         size_t body = (n - head) & ~(size_t)15;
         size_t tail = n - head - body;
         /* edges by loads/stores */
-        if (tid < head) stv<unsigned char>(d + tid, ldv<unsigned char>(s + tid));
-        if (tid < tail)
-            stv<unsigned char>(d + head + body + tid, ldv<unsigned char>(s + head + body + tid));
+        for (size_t i = tid; i < head; i += nthr) stv<unsigned char>(d + i, ldv<unsigned char>(s + i));
+        for (size_t i = tid; i < tail; i += nthr)
+            stv<unsigned char>(d + head + body + i, ldv<unsigned char>(s + head + body + i));
         /* the source may have been written by this block's threads: make those writes
          * visible to the async proxy before the leader starts the bulk loads */
         fence_proxy_async();
         __syncthreads();
         __shared__ int rc_sh;
-        if (tid == 0) rc_sh = bulk_copy_ring(ctx, d + head, s + head, body, st, complete);
+        if (tid == 0)
+            rc_sh = bulk_copy_ring(ctx, d + head, s + head, body, st, complete);
         __syncthreads();
         return rc_sh;
     }
@@ -917,49 +930,44 @@ __device__ __forceinline__ bool team_deltas(const ishmem_ctx_t *ctx, const ishme
     return ok;
 }
 
-/* Fold elements [begin, end) of the team's sources in team order and store the result in
- * the `ndst` destinations starting at team index dst0 (ndst = 1, dst0 = my index: the
- * duplicated algorithm; ndst = team size, dst0 = 0: the owner pushes to everybody).  src and
- * dest are the calling PE's local addresses; member i's copy is delta[i] bytes further.
- * 16-byte vectors when both buffers are 16-byte aligned, else element by element. */
-template <typename T, int OP>
-__device__ __forceinline__ void fold_range(const char *src, char *dest, const long long *delta,
-                                           int tsize, int dst0, int ndst, size_t begin, size_t end,
-                                           unsigned tid, unsigned nthr)
+/* Vector body of a fold: 16-byte vectors [v0, v1) of the team's sources, combined in team
+ * order, stored to ndst destinations.  VPT vectors per thread and iteration, B sources per
+ * batch: VPT*B independent 16-byte loads are in flight before the first combine. */
+template <typename T, int OP, int VPT, int B>
+__device__ __forceinline__ void fold_vectors(const char *src, char *dest, const long long *delta, int tsize,
+                                             int dst0, int ndst, size_t v0, size_t v1, unsigned tid,
+                                             unsigned nthr)
 {
     constexpr int EPV = 16 / sizeof(T);
-    const bool vec_ok = ((((uintptr_t)src | (uintptr_t)dest) & 15u) == 0);
-    size_t vbeg = begin, vend = begin;
-    if (vec_ok) {
-        vbeg = (begin + EPV - 1) / EPV * EPV;
-        vend = end / EPV * EPV;
-        if (vbeg > vend) vbeg = vend = begin;
-    }
-    /* scalar edges: [begin, vbeg) and [vend, end) */
-    for (size_t j = begin + tid; j < end; j += nthr) {
-        if (j >= vbeg && j < vend) continue;
-        T acc = ldv<T>(src + delta[0] + j * sizeof(T));
-        for (int i = 1; i < tsize; ++i)
-            acc = folder<T, OP>::f(acc, ldv<T>(src + delta[i] + j * sizeof(T)));
-        for (int q = 0; q < ndst; ++q) stv<T>(dest + delta[dst0 + q] + j * sizeof(T), acc);
-    }
-    for (size_t v = vbeg / EPV + tid; v < vend / EPV; v += nthr) {
-        vec16<T> acc;
-        acc.v = ld16(src + delta[0] + v * 16);
-        constexpr int B = 4; /* sources loaded per batch: B independent loads in flight */
+    for (size_t v = v0 + tid; v < v1; v += (size_t)nthr * VPT) {
+        vec16<T> acc[VPT];
+#pragma unroll
+        for (int u = 0; u < VPT; ++u)
+            if (v + (size_t)u * nthr < v1) acc[u].v = ld16(src + delta[0] + (v + (size_t)u * nthr) * 16);
         for (int i = 1; i < tsize; i += B) {
-            vec16<T> x[B];
+            vec16<T> x[VPT][B];
 #pragma unroll
-            for (int k = 0; k < B; ++k)
-                if (i + k < tsize) x[k].v = ld16(src + delta[i + k] + v * 16);
+            for (int u = 0; u < VPT; ++u)
 #pragma unroll
-            for (int k = 0; k < B; ++k)
-                if (i + k < tsize) {
+                for (int k = 0; k < B; ++k)
+                    if (i + k < tsize && v + (size_t)u * nthr < v1)
+                        x[u][k].v = ld16(src + delta[i + k] + (v + (size_t)u * nthr) * 16);
 #pragma unroll
-                    for (int e = 0; e < EPV; ++e) acc.e[e] = folder<T, OP>::f(acc.e[e], x[k].e[e]);
-                }
+            for (int u = 0; u < VPT; ++u)
+#pragma unroll
+                for (int k = 0; k < B; ++k)
+                    if (i + k < tsize && v + (size_t)u * nthr < v1) {
+#pragma unroll
+                        for (int e = 0; e < EPV; ++e)
+                            acc[u].e[e] = folder<T, OP>::f(acc[u].e[e], x[u][k].e[e]);
+                    }
         }
-        for (int q = 0; q < ndst; ++q) st16(dest + delta[dst0 + q] + v * 16, acc.v);
+        for (int q = 0; q < ndst; ++q) {
+#pragma unroll
+            for (int u = 0; u < VPT; ++u)
+                if (v + (size_t)u * nthr < v1)
+                    st16(dest + delta[dst0 + q] + (v + (size_t)u * nthr) * 16, acc[u].v);
+        }
     }
 }
 
@@ -990,6 +998,169 @@ __device__ __forceinline__ void push_bytes(char *dest, const long long *delta, i
         for (int q = 0; q < ndst; ++q)
             if (q != skip) stv<unsigned char>(dest + delta[q] + j, c);
     }
+}
+
+/* Fold elements [begin, end) of the team's sources in team order and store the result in
+ * the `ndst` destinations starting at team index dst0 (ndst = 1, dst0 = my index: the
+ * duplicated algorithm; ndst = team size, dst0 = 0: the owner pushes to everybody).  src and
+ * dest are the calling PE's local addresses; member i's copy is delta[i] bytes further.
+ * 16-byte vectors when both buffers are 16-byte aligned, else element by element. */
+template <typename T, int OP, int VPT = 1, int B = 4>
+__device__ __forceinline__ void fold_range(const char *src, char *dest, const long long *delta,
+                                           int tsize, int dst0, int ndst, size_t begin, size_t end,
+                                           unsigned tid, unsigned nthr)
+{
+    constexpr int EPV = 16 / sizeof(T);
+    const bool vec_ok = ((((uintptr_t)src | (uintptr_t)dest) & 15u) == 0);
+    size_t vbeg = begin, vend = begin;
+    if (vec_ok) {
+        vbeg = (begin + EPV - 1) / EPV * EPV;
+        vend = end / EPV * EPV;
+        if (vbeg > vend) vbeg = vend = begin;
+    }
+    /* scalar edges: [begin, vbeg) and [vend, end) */
+    for (size_t j = begin + tid; j < end; j += nthr) {
+        if (j >= vbeg && j < vend) continue;
+        T acc = ldv<T>(src + delta[0] + j * sizeof(T));
+        for (int i = 1; i < tsize; ++i)
+            acc = folder<T, OP>::f(acc, ldv<T>(src + delta[i] + j * sizeof(T)));
+        for (int q = 0; q < ndst; ++q) stv<T>(dest + delta[dst0 + q] + j * sizeof(T), acc);
+    }
+    fold_vectors<T, OP, VPT, B>(src, dest, delta, tsize, dst0, ndst, vbeg / EPV, vend / EPV, tid, nthr);
+}
+
+/* Reduce through shared memory with TMA on both sides, called by every thread of the block:
+ * for each chunk one elected thread bulk-loads the chunk of all `tsize` sources into one
+ * stage (completing on one mbarrier), all threads fold the stage in team order into its
+ * first tile, and the elected thread bulk-stores that tile to the `ndst` destinations
+ * dest + delta[dst0 + q].  `nbytes` is a multiple of 16, src/dest 16-byte aligned, the ring
+ * has 3 stages of tsize tiles.  The block handles chunks first, first+stride, ... of the range.
+ * Returns 0, ISHMEM_ERR_TIMEOUT, or 1 when the staging is too small for this team (nothing
+ * done). */
+template <typename T, int OP>
+__device__ __forceinline__ int bulk_fold_ring(const ishmem_ctx_t *ctx, const char *src, char *dest,
+                                              const long long *delta, int tsize, int dst0, int ndst,
+                                              size_t nbytes, ishmemx_staging_t st, size_t first = 0,
+                                              size_t stride = 1)
+{
+    constexpr int EPV = 16 / sizeof(T);
+    constexpr unsigned NST = 3;
+    const unsigned tid = block_tid(), nthr = block_nthr();
+    if (st.smem == nullptr || st.bytes < 128u + NST * 1024u * (unsigned)tsize) return 1;
+    unsigned C = ((st.bytes - 128u) / (NST * (unsigned)tsize)) & ~1023u;
+    if (C > 16384u) C = 16384u;
+    const unsigned stage_bytes = C * (unsigned)tsize;
+    /* this block takes chunks first, first + stride, ... of the range (round-robin with the
+     * other blocks of the launch) */
+    const size_t total = (nbytes + C - 1) / C;
+    const size_t nchunks = total > first ? (total - first + stride - 1) / stride : 0;
+    char *stage0 = (char *)st.smem + 128;
+    const unsigned bar0 = smem_u32(st.smem), sm0 = smem_u32(stage0);
+    __shared__ int fail;
+    if (tid == 0) {
+        fail = 0;
+        for (unsigned k = 0; k < NST; ++k) mbar_init(bar0 + 8 * k, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        fence_proxy_async();
+    }
+    __syncthreads();
+    auto chunk_off = [&](size_t c) -> size_t { return (first + c * stride) * C; };
+    auto chunk_bytes = [&](size_t c) -> unsigned {
+        size_t left = nbytes - chunk_off(c);
+        return left < C ? (unsigned)left : C;
+    };
+    auto issue_load = [&](size_t c) {
+        const unsigned sidx = (unsigned)(c % NST), b = chunk_bytes(c);
+        mbar_expect_tx(bar0 + 8 * sidx, b * (unsigned)tsize);
+        for (int i = 0; i < tsize; ++i)
+            bulk_g2s(sm0 + sidx * stage_bytes + (unsigned)i * C, src + delta[i] + chunk_off(c), b,
+                     bar0 + 8 * sidx);
+    };
+    size_t issued = 0;
+    if (tid == 0)
+        for (; issued < nchunks && issued + 1 < NST; ++issued) issue_load(issued);
+    size_t c = 0;
+    for (; c < nchunks; ++c) {
+        const unsigned sidx = (unsigned)(c % NST);
+        const bool ok = mbar_wait(bar0 + 8 * sidx, (unsigned)((c / NST) & 1), ctx->wait_limit_ns);
+        if (!ok) fail = 1;
+        const unsigned b = chunk_bytes(c);
+        char *tile = stage0 + (size_t)sidx * stage_bytes;
+        if (ok)
+            for (unsigned v = tid; v < (b >> 4); v += nthr) {
+                vec16<T> acc;
+                acc.v = *(const uint4 *)(tile + (size_t)v * 16);
+                for (int i = 1; i < tsize; ++i) {
+                    vec16<T> x;
+                    x.v = *(const uint4 *)(tile + (size_t)i * C + (size_t)v * 16);
+#pragma unroll
+                    for (int e = 0; e < EPV; ++e) acc.e[e] = folder<T, OP>::f(acc.e[e], x.e[e]);
+                }
+                *(uint4 *)(tile + (size_t)v * 16) = acc.v;
+            }
+        fence_proxy_async(); /* the folded tile is read by the bulk stores below */
+        __syncthreads();
+        if (fail) break;
+        if (tid == 0) {
+            for (int q = 0; q < ndst; ++q)
+                bulk_s2g(dest + delta[dst0 + q] + chunk_off(c), sm0 + sidx * stage_bytes, b);
+            bulk_commit();
+            if (issued < nchunks) {
+                bulk_wait_read<1>(); /* the stores of chunk c-1 have read their stage: refill it */
+                issue_load(issued);
+                ++issued;
+            }
+        }
+    }
+    if (tid == 0) {
+        if (fail) {
+            latch_error(ctx, ISHMEM_ERR_TIMEOUT);
+            for (size_t k = c; k < issued; ++k)
+                mbar_wait(bar0 + 8 * (unsigned)(k % NST), (unsigned)((k / NST) & 1), ctx->wait_limit_ns);
+        }
+        bulk_wait<0>();
+        fence_proxy_async();
+        for (unsigned k = 0; k < NST; ++k) mbar_inval(bar0 + 8 * k);
+    }
+    __syncthreads();
+    return fail ? ISHMEM_ERR_TIMEOUT : 0;
+}
+
+/* work-group push of n bytes to ndst destinations dest + delta[q] (q != skip); delta lives in
+ * shared memory.  TMA ring for the aligned body when staging is given, else loads/stores with
+ * the destinations in the inner loop (see push_bytes). */
+__device__ __forceinline__ int wg_push(const ishmem_ctx_t *ctx, char *dest, const long long *delta, int ndst,
+                                       int skip, const char *src, size_t n, ishmemx_staging_t st,
+                                       size_t first = 0, size_t stride = 1)
+{
+    const unsigned tid = threadIdx.x + blockDim.x * (threadIdx.y + blockDim.y * threadIdx.z);
+    const unsigned nthr = blockDim.x * blockDim.y * blockDim.z;
+    const bool congruent = ((((uintptr_t)dest - (uintptr_t)src) & 15u) == 0);
+    if (st.smem != nullptr && st.bytes >= 128u + 2048u && congruent && n >= ISHMEMI_BULK_MIN_BYTES) {
+        size_t head = (size_t)((16u - ((unsigned)(uintptr_t)dest & 15u)) & 15u);
+        size_t body = (n - head) & ~(size_t)15;
+        size_t tail = n - head - body;
+        if (first == 0) {
+            push_bytes(dest, delta, ndst, skip, src, head, tid, nthr);
+            push_bytes(dest + head + body, delta, ndst, skip, src + head + body, tail, tid, nthr);
+        }
+        fence_proxy_async();
+        __syncthreads();
+        __shared__ int rc_sh;
+        if (tid == 0)
+            rc_sh = bulk_copy_ring(ctx, dest + head, src + head, body, st, true, delta, ndst, skip, first, stride);
+        __syncthreads();
+        return rc_sh;
+    }
+    /* loads/stores: tiles of 16 KiB dealt round-robin (the whole range when stride is 1) */
+    if (stride == 1) {
+        push_bytes(dest, delta, ndst, skip, src, n, tid, nthr);
+    } else {
+        const size_t tile = 16384;
+        for (size_t o = first * tile; o < n; o += stride * tile)
+            push_bytes(dest + o, delta, ndst, skip, src + o, (n - o < tile) ? n - o : tile, tid, nthr);
+    }
+    return 0;
 }
 
 } /* namespace ishmemi */

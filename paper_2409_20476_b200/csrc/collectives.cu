@@ -16,6 +16,8 @@ struct coll_args {
     int groups;       /* blocks per member */
     int duplicated;   /* reduce: every member folds everything into its own dest */
     int repeat;
+    unsigned staging_bytes; /* dynamic shared memory for the TMA push ring (0: loads/stores) */
+    unsigned tile_vpt;      /* reduce: 16-byte vectors per thread in one tile */
 };
 
 /* local address on `ctx`'s PE of a symmetric address given as PE 0's copy */
@@ -34,34 +36,29 @@ __device__ __forceinline__ void part_of(size_t n, unsigned k, unsigned parts, si
 /* ---- broadcast: the root's blocks push slices of the source to every member ------------- */
 __global__ void __launch_bounds__(1024) k_broadcast(const ishmem_ctx_t *ctxs, coll_args a)
 {
+    extern __shared__ __align__(128) unsigned char dyn_smem[];
     __shared__ long long delta[ISHMEM_MAX_PES];
     const ishmemi_team t = ctxs[0].teams[a.team];
     const ishmem_ctx_t *ctx = ctxs + (t.start + a.root * t.stride);
     if (!ishmemi::team_deltas(ctx, t, delta)) return;
-    size_t lo, hi;
-    part_of((a.n + 15) / 16, blockIdx.x, gridDim.x, &lo, &hi);
-    lo *= 16;
-    hi = hi * 16 < a.n ? hi * 16 : a.n;
-    if (lo >= hi) return;
-    ishmemi::push_bytes(local_of(ctxs, ctx, a.dest) + lo, delta, t.size, ctx->bcast_root_dest ? -1 : a.root,
-                        local_of(ctxs, ctx, a.src) + lo, hi - lo, threadIdx.x, blockDim.x);
+    /* the root's blocks take chunks of the message round-robin */
+    ishmemx_staging_t st = {a.staging_bytes ? dyn_smem : nullptr, a.staging_bytes};
+    ishmemi::wg_push(ctx, local_of(ctxs, ctx, a.dest), delta, t.size, ctx->bcast_root_dest ? -1 : a.root,
+                     local_of(ctxs, ctx, a.src), a.n, st, blockIdx.x, gridDim.x);
 }
 
 /* ---- fcollect: member i's blocks push slices of its source into block i of every dest ---- */
 __global__ void __launch_bounds__(1024) k_fcollect(const ishmem_ctx_t *ctxs, coll_args a)
 {
+    extern __shared__ __align__(128) unsigned char dyn_smem[];
     __shared__ long long delta[ISHMEM_MAX_PES];
     const ishmemi_team t = ctxs[0].teams[a.team];
     const unsigned me = blockIdx.x % (unsigned)t.size, g = blockIdx.x / (unsigned)t.size;
     const ishmem_ctx_t *ctx = ctxs + (t.start + (int)me * t.stride);
     if (!ishmemi::team_deltas(ctx, t, delta)) return;
-    size_t lo, hi;
-    part_of((a.n + 15) / 16, g, (unsigned)a.groups, &lo, &hi);
-    lo *= 16;
-    hi = hi * 16 < a.n ? hi * 16 : a.n;
-    if (lo >= hi) return;
-    ishmemi::push_bytes(local_of(ctxs, ctx, a.dest) + (size_t)me * a.n + lo, delta, t.size, -1,
-                        local_of(ctxs, ctx, a.src) + lo, hi - lo, threadIdx.x, blockDim.x);
+    ishmemx_staging_t st = {a.staging_bytes ? dyn_smem : nullptr, a.staging_bytes};
+    ishmemi::wg_push(ctx, local_of(ctxs, ctx, a.dest) + (size_t)me * a.n, delta, t.size, -1,
+                     local_of(ctxs, ctx, a.src), a.n, st, g, (size_t)a.groups);
 }
 
 /* ---- reduce ------------------------------------------------------------------------------- */
@@ -69,25 +66,48 @@ __global__ void __launch_bounds__(1024) k_fcollect(const ishmem_ctx_t *ctxs, col
  * and stores the result into every member's dest (traffic: each source and each dest once).
  * duplicated: member q folds the whole range and stores into its own dest only. */
 template <typename T, int OP>
-__global__ void __launch_bounds__(1024) k_reduce(const ishmem_ctx_t *ctxs, coll_args a)
+__global__ void __launch_bounds__(512, 2) k_reduce(const ishmem_ctx_t *ctxs, coll_args a)
 {
+    extern __shared__ __align__(128) unsigned char dyn_smem[];
     __shared__ long long delta[ISHMEM_MAX_PES];
     const ishmemi_team t = ctxs[0].teams[a.team];
     const unsigned me = blockIdx.x % (unsigned)t.size, g = blockIdx.x / (unsigned)t.size;
     const ishmem_ctx_t *ctx = ctxs + (t.start + (int)me * t.stride);
     if (!ishmemi::team_deltas(ctx, t, delta)) return;
     constexpr size_t EPV = 16 / sizeof(T);
-    const size_t nslots = (a.n + EPV - 1) / EPV;
-    size_t lo = 0, hi = nslots;
-    if (!a.duplicated) part_of(nslots, me, (unsigned)t.size, &lo, &hi);
-    size_t glo, ghi;
-    part_of(hi - lo, g, (unsigned)a.groups, &glo, &ghi);
-    size_t begin = (lo + glo) * EPV, end = (lo + ghi) * EPV;
-    if (end > a.n) end = a.n;
-    if (begin >= end) return;
-    ishmemi::fold_range<T, OP>(local_of(ctxs, ctx, a.src), local_of(ctxs, ctx, a.dest), delta, t.size,
-                               a.duplicated ? (int)me : 0, a.duplicated ? 1 : t.size, begin, end,
-                               threadIdx.x, blockDim.x);
+    const char *src = local_of(ctxs, ctx, a.src);
+    char *dest = local_of(ctxs, ctx, a.dest);
+    const int dst0 = a.duplicated ? (int)me : 0, ndst = a.duplicated ? 1 : t.size;
+    const unsigned tid = threadIdx.x, nthr = blockDim.x;
+    if ((((uintptr_t)src | (uintptr_t)dest) & 15u) != 0) {
+        /* buffers aligned to the element only: contiguous element ranges, element by element */
+        size_t lo = 0, hi = a.n, glo, ghi;
+        if (!a.duplicated) part_of(a.n, me, (unsigned)t.size, &lo, &hi);
+        part_of(hi - lo, g, (unsigned)a.groups, &glo, &ghi);
+        ishmemi::fold_range<T, OP, 1, 4>(src, dest, delta, t.size, dst0, ndst, lo + glo, lo + ghi, tid, nthr);
+        return;
+    }
+    /* The address range is cut into tiles that the blocks take round-robin, so that at any
+     * moment the running blocks cover one contiguous window of every source and destination
+     * (whole DRAM rows, all channels).  Split form: tile k belongs to member k mod P -- still
+     * a split of the work by address across PEs; duplicated form: each member's blocks sweep
+     * all tiles. */
+    const size_t nv = a.n / EPV;
+    const size_t tile = (size_t)nthr * a.tile_vpt;
+    const size_t ntiles = (nv + tile - 1) / tile;
+    const size_t first = a.duplicated ? g : blockIdx.x, stride = a.duplicated ? (size_t)a.groups : gridDim.x;
+    if (a.staging_bytes) {
+        ishmemx_staging_t st = {dyn_smem, a.staging_bytes};
+        ishmemi::bulk_fold_ring<T, OP>(ctx, src, dest, delta, t.size, dst0, ndst, nv * 16, st, first, stride);
+    } else {
+        for (size_t k = first; k < ntiles; k += stride) {
+            const size_t v0 = k * tile, v1 = (v0 + tile < nv) ? v0 + tile : nv;
+            ishmemi::fold_vectors<T, OP, 1, 4>(src, dest, delta, t.size, dst0, ndst, v0, v1, tid, nthr);
+        }
+    }
+    /* elements past the last whole vector */
+    if (first == 0)
+        ishmemi::fold_range<T, OP, 1, 4>(src, dest, delta, t.size, dst0, ndst, nv * EPV, a.n, tid, nthr);
 }
 
 typedef void (*reduce_kernel_t)(const ishmem_ctx_t *, coll_args);
@@ -211,6 +231,28 @@ static int auto_groups(size_t bytes_per_member, int members)
     return (int)(want < cap ? want : cap);
 }
 
+/* Dynamic shared memory of the push kernels' TMA ring; 0 (loads/stores) for small messages.
+ * With the ring one elected thread per block moves the data, so about one block per SM with
+ * a deep ring is the right shape: `*blocks` is set accordingly. */
+static unsigned push_staging(size_t bytes_per_member, int members, int *blocks_per_member)
+{
+    auto &g = g_ishmem;
+    static unsigned smem = 0;
+    if (!smem) {
+        unsigned want = 192 * 1024 + 128;
+        if (want > g.max_dyn_smem) want = (unsigned)g.max_dyn_smem;
+        cudaFuncSetAttribute(k_broadcast, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)want);
+        cudaFuncSetAttribute(k_fcollect, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)want);
+        smem = want;
+    }
+    if (g.coll_groups > 0 || bytes_per_member < (1u << 20)) return 0; /* caller-shaped or small */
+    size_t want_blocks = (bytes_per_member + (256u << 10) - 1) / (256u << 10);
+    size_t cap = (size_t)g.sm_count / members;
+    if (cap < 1) cap = 1;
+    *blocks_per_member = (int)(want_blocks < cap ? want_blocks : cap);
+    return smem;
+}
+
 static int launch_sync_kernel(ishmem_team_t team, int repeat)
 {
     auto &g = g_ishmem;
@@ -296,7 +338,8 @@ extern "C" int ishmem_broadcastmem(ishmem_team_t team, void *dest, const void *s
         a.n = nbytes;
         a.root = root;
         int blocks = auto_groups(nbytes, 1);
-        k_broadcast<<<blocks, g.coll_threads, 0, s>>>(g.d_ctx, a);
+        a.staging_bytes = push_staging(nbytes, 1, &blocks);
+        k_broadcast<<<blocks, a.staging_bytes ? 128 : g.coll_threads, a.staging_bytes, s>>>(g.d_ctx, a);
         ishmemi_count_launch();
         rc = ishmemi_check_launch("k_broadcast");
     }
@@ -336,7 +379,8 @@ extern "C" int ishmem_fcollectmem(ishmem_team_t team, void *dest, const void *sr
         a.src = (const char *)src;
         a.n = nbytes;
         a.groups = auto_groups(nbytes, t.size);
-        k_fcollect<<<a.groups * t.size, g.coll_threads, 0, s>>>(g.d_ctx, a);
+        a.staging_bytes = push_staging(nbytes, t.size, &a.groups);
+        k_fcollect<<<a.groups * t.size, a.staging_bytes ? 128 : g.coll_threads, a.staging_bytes, s>>>(g.d_ctx, a);
         ishmemi_count_launch();
         rc = ishmemi_check_launch("k_fcollect");
     }
@@ -375,8 +419,28 @@ extern "C" int ishmemx_reduce(ishmem_team_t team, void *dest, const void *src, s
         a.src = sp;
         a.n = nreduce;
         a.duplicated = (algorithm == ISHMEMX_REDUCE_DUPLICATED);
-        a.groups = auto_groups(a.duplicated ? bytes : bytes / t.size + 1, t.size);
-        k<<<a.groups * t.size, g.coll_threads, 0, s>>>(g.d_ctx, a);
+        a.tile_vpt = 2;
+        const size_t per_member = a.duplicated ? bytes : bytes / t.size + 1;
+        a.groups = auto_groups(per_member, t.size);
+        int threads = g.coll_threads > 512 ? 512 : g.coll_threads;
+        /* Loads/stores over round-robin tiles are the default; from 64 MiB per member on the
+         * TMA fold ring (one block per SM) is at least as fast.  ISHMEM_REDUCE_BULK=0/1 forces. */
+        static const char *env_bulk = getenv("ISHMEM_REDUCE_BULK");
+        const bool use_bulk = env_bulk ? atoi(env_bulk) != 0 : per_member >= ((size_t)64 << 20);
+        if (use_bulk && g.coll_groups == 0 && per_member >= (1u << 20) && t.size <= 48) {
+            /* large: TMA ring, one block per SM */
+            unsigned want = 192 * 1024 + 128;
+            if (want > g.max_dyn_smem) want = (unsigned)g.max_dyn_smem;
+            if (cudaFuncSetAttribute((const void *)k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)want) ==
+                cudaSuccess) {
+                a.staging_bytes = want;
+                size_t cap = (size_t)g.sm_count / t.size, need = (per_member + (256u << 10) - 1) / (256u << 10);
+                if (cap < 1) cap = 1;
+                a.groups = (int)(need < cap ? need : cap);
+                threads = 512;
+            }
+        }
+        k<<<a.groups * t.size, threads, a.staging_bytes, s>>>(g.d_ctx, a);
         ishmemi_count_launch();
         rc = ishmemi_check_launch("k_reduce");
     }
