@@ -336,6 +336,16 @@ int ishmemx_collective_on_device(int which, ishmem_team_t team, void *dest, cons
 int ishmemx_pingpong(int pe_a, int pe_b, void *data, uint64_t *sig, size_t nbytes, int rounds,
                      int threads, double *half_rtt_ns, uint64_t *mismatches);
 
+/* Device-initiated latency of one collaboration level (the measurement method of Section 4:
+ * many back-to-back operations inside one kernel, timed on the device).  ONE work-group of
+ * `threads` threads runs as PE my_pe and issues `iters` puts (is_get = 0) or gets of `nbytes`
+ * to/from PE `pe`, each followed by quiet: by its first thread alone (ISHMEMX_WORK_ITEM), by
+ * its first warp (ISHMEMX_SUB_GROUP), or by all threads (ISHMEMX_WORK_GROUP, _BULK).  dest/src
+ * as for ishmem_putmem / ishmem_getmem.  Writes the mean time per operation in nanoseconds
+ * (global timer, read inside the kernel) to HOST memory `ns_per_op`.  Blocks the host. */
+int ishmemx_rma_latency(int my_pe, void *dest, const void *src, size_t nbytes, int pe, int is_get,
+                        int level, int threads, int iters, double *ns_per_op);
+
 /* Overlap workload: `iters` sweeps of the 5-point Jacobi update on an ny x nx float64
  * grid cut into npes row strips (the first ny mod npes strips have one more row), in one
  * persistent co-resident launch: each sweep every PE sends its first and last rows to the

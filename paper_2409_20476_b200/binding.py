@@ -130,6 +130,7 @@ def _signatures() -> dict[str, tuple[str, list[str]]]:
         "ishmemx_set_collective_geometry": ("status", ["i", "i"]),
         "ishmemx_collective_on_device": ("status", ["i", "i", "p", "p", "z", "i", "i", "i", "i", "i"]),
         "ishmemx_pingpong": ("status", ["i", "i", "p", "p", "z", "i", "i", "p", "p"]),
+        "ishmemx_rma_latency": ("status", ["i", "p", "p", "z", "i", "i", "i", "i", "i", "p"]),
         "ishmemx_jacobi": ("status", ["p", "p", "p", "z", "z", "i", "i", "i", "i", "p"]),
         "ishmemx_jacobi_noalloc": ("status", ["p", "p", "p", "z", "z", "i", "i", "i", "i", "p"]),
         "ishmemx_host_put_ring": ("status", ["p", "p", "p", "p", "z", "i", "i", "i", "i"]),

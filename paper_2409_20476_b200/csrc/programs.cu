@@ -91,6 +91,97 @@ extern "C" int ishmemx_pingpong(int pe_a, int pe_b, void *data, uint64_t *sig, s
     return ISHMEM_OK;
 }
 
+/* ---- device-timed put/get latency --------------------------------------------------------- */
+
+template <int LEVEL>
+__global__ void __launch_bounds__(1024) k_rma_latency(const ishmem_ctx_t *ctxs, int my_pe, char *dest,
+                                                      const char *src, size_t nbytes, int pe, int is_get,
+                                                      int iters, unsigned staging_bytes, unsigned long long *elapsed_ns)
+{
+    extern __shared__ __align__(128) unsigned char dyn_smem[];
+    const ishmem_ctx_t *ctx = ctxs + my_pe;
+    ishmemx_staging_t st = {nullptr, 0};
+    if (LEVEL == ISHMEMX_WORK_GROUP_BULK) {
+        st.smem = dyn_smem;
+        st.bytes = staging_bytes;
+    }
+    __syncthreads();
+    unsigned long long t0 = 0;
+    if (threadIdx.x == 0) t0 = ishmemi::globaltimer_ns();
+    for (int it = 0; it < iters; ++it) {
+        if (LEVEL == ISHMEMX_WORK_ITEM) {
+            if (threadIdx.x == 0) {
+                if (is_get) ishmem_getmem(ctx, dest, src, nbytes, pe);
+                else ishmem_putmem(ctx, dest, src, nbytes, pe);
+                ishmem_quiet(ctx);
+            }
+        } else if (LEVEL == ISHMEMX_SUB_GROUP) {
+            if (threadIdx.x < 32u) {
+                if (is_get) ishmemx_getmem_sub_group(ctx, dest, src, nbytes, pe);
+                else ishmemx_putmem_sub_group(ctx, dest, src, nbytes, pe);
+                ishmem_quiet(ctx);
+            }
+        } else {
+            int rc = is_get ? ishmemx_getmem_work_group(ctx, dest, src, nbytes, pe, st)
+                            : ishmemx_putmem_work_group(ctx, dest, src, nbytes, pe, st);
+            ishmemx_quiet_work_group(ctx);
+            if (rc) break; /* latched; same value in every thread */
+        }
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) *elapsed_ns = ishmemi::globaltimer_ns() - t0;
+}
+
+extern "C" int ishmemx_rma_latency(int my_pe, void *dest, const void *src, size_t nbytes, int pe, int is_get,
+                                   int level, int threads, int iters, double *ns_per_op)
+{
+    ISHMEMI_REQUIRE_INIT();
+    auto &g = g_ishmem;
+    if (ishmemi_check_pe(my_pe) || ishmemi_check_pe(pe)) return ISHMEM_ERR_INVALID_PE;
+    if (iters < 1 || threads < 1 || threads > 1024 || !ns_per_op) return ISHMEM_ERR_ARG;
+    if (level < ISHMEMX_WORK_ITEM || level > ISHMEMX_WORK_GROUP_BULK) return ISHMEM_ERR_ARG;
+    if (level == ISHMEMX_SUB_GROUP && threads < 32) return ISHMEM_ERR_ARG;
+    if (nbytes && (!dest || !src)) return ISHMEM_ERR_ARG;
+    if (ishmemi_sym_offset(is_get ? src : (const void *)dest, nbytes) < 0) return ISHMEM_ERR_NOT_SYMMETRIC;
+    char *dl = ishmemi_localise(dest, nbytes, my_pe);
+    const char *sl = ishmemi_localise(src, nbytes, my_pe);
+    unsigned long long *out = (unsigned long long *)g.h_pinned;
+    *out = 0;
+    unsigned staging = 0;
+    cudaStream_t s = ishmemi_pe_stream_for_op(my_pe);
+    const ishmem_ctx_t *ctxs = g.d_ctx;
+    switch (level) {
+    case ISHMEMX_WORK_ITEM:
+        k_rma_latency<ISHMEMX_WORK_ITEM><<<1, threads, 0, s>>>(ctxs, my_pe, dl, sl, nbytes, pe, is_get, iters, 0, out);
+        break;
+    case ISHMEMX_SUB_GROUP:
+        k_rma_latency<ISHMEMX_SUB_GROUP><<<1, threads, 0, s>>>(ctxs, my_pe, dl, sl, nbytes, pe, is_get, iters, 0, out);
+        break;
+    case ISHMEMX_WORK_GROUP:
+        k_rma_latency<ISHMEMX_WORK_GROUP><<<1, threads, 0, s>>>(ctxs, my_pe, dl, sl, nbytes, pe, is_get, iters, 0, out);
+        break;
+    default: {
+        static unsigned smem = 0;
+        if (!smem) {
+            unsigned want = 192 * 1024 + 128;
+            if (want > g.max_dyn_smem) want = (unsigned)g.max_dyn_smem;
+            ISHMEMI_CUDA(cudaFuncSetAttribute(k_rma_latency<ISHMEMX_WORK_GROUP_BULK>,
+                                              cudaFuncAttributeMaxDynamicSharedMemorySize, (int)want));
+            smem = want;
+        }
+        staging = smem;
+        k_rma_latency<ISHMEMX_WORK_GROUP_BULK><<<1, threads, staging, s>>>(ctxs, my_pe, dl, sl, nbytes, pe, is_get,
+                                                                          iters, staging, out);
+    }
+    }
+    ishmemi_count_launch();
+    int rc = ishmemi_check_launch("k_rma_latency");
+    if (rc) return rc;
+    ISHMEMI_CUDA(cudaStreamSynchronize(s));
+    *ns_per_op = (double)*out / (double)iters;
+    return ISHMEM_OK;
+}
+
 /* ---- Jacobi overlap workload -------------------------------------------------------------- */
 
 struct jacobi_args {

@@ -12,6 +12,7 @@ int ishmemi_cuda(cudaError_t e, const char *what)
 {
     if (e == cudaSuccess) return ISHMEM_OK;
     g_ishmem.last_cuda_error = std::string(what) + ": " + cudaGetErrorString(e);
+    (void)cudaGetLastError(); /* a refused launch must not show up again in the next call's check */
     if (e == cudaErrorCooperativeLaunchTooLarge) return ISHMEM_ERR_NOT_CORESIDENT;
     if (e == cudaErrorMemoryAllocation) return ISHMEM_ERR_OOM;
     return ISHMEM_ERR_CUDA;

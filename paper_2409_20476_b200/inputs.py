@@ -111,3 +111,40 @@ def jacobi_grid_block(seed: int, ny: int, nx: int, block: int,
 def message_sizes(lo_log2: int, hi_log2: int) -> list[int]:
     """Powers of two from 2**lo_log2 to 2**hi_log2 bytes inclusive."""
     return [1 << k for k in range(lo_log2, hi_log2 + 1)]
+
+
+# ---- full-size inputs, drawn block by block so that any window can be regenerated ---------
+
+BLOCK_ELEMS = 1 << 20
+
+
+def _block(kind: str, seed: int, pe: int, block: int, count: int) -> np.ndarray:
+    r = rng_for(seed, 60, pe, block)
+    if kind == "u8":
+        return r.integers(0, 256, size=count, dtype=np.uint8)
+    if kind == "f32":
+        return r.standard_normal(count, dtype=np.float32)
+    if kind == "f64":
+        return r.standard_normal(count)
+    if kind == "i64":
+        return r.integers(-2**20, 2**20 + 1, size=count, dtype=np.int64)
+    raise ValueError(kind)
+
+
+def block_values(kind: str, seed: int, pe: int, start: int, count: int) -> np.ndarray:
+    """Elements [start, start+count) of PE ``pe``'s full-size source of the given kind
+    ('u8' uniform bytes, 'f32'/'f64' N(0,1), 'i64' uniform in [-2^20, 2^20]).  The stream is
+    defined in blocks of 2^20 elements, each with its own generator, so a window costs only
+    the blocks it touches and is identical to the same range of the whole array."""
+    out = []
+    b = start // BLOCK_ELEMS
+    pos = start
+    end = start + count
+    while pos < end:
+        blk = _block(kind, seed, pe, b, BLOCK_ELEMS)
+        lo = pos - b * BLOCK_ELEMS
+        hi = min(end - b * BLOCK_ELEMS, BLOCK_ELEMS)
+        out.append(blk[lo:hi])
+        pos += hi - lo
+        b += 1
+    return np.concatenate(out) if len(out) != 1 else out[0]

@@ -1,0 +1,474 @@
+"""Message-size sweeps of the library on one B200, one sub-command per benchmark configuration.
+
+    python -m paper_2409_20476_b200.sweeps --config 2 --out sweep_c2.csv
+
+Timing follows the method of the paper's Section 4: the iteration count is doubled until
+one batch of back-to-back operations lasts longer than 2 ms, then 10 batches are timed and
+the best is kept.  Host-launched operations are timed with CUDA events on the stream they
+are launched on; the in-kernel latencies come from ``ishmemx_rma_latency`` and
+``ishmemx_pingpong`` (device global timer).  Bandwidth is *algorithmic* bytes (read plus
+written, summed over the PEs that run concurrently) over time; ``frac_hbm`` divides by the
+measured copy peak given with ``--peak-gbs`` and ``frac_8tbs`` by the nominal 8 TB/s.
+
+``l2 = hot`` rows reuse one pair of buffers, so everything up to a few MiB per PE is served
+by the 126 MB L2 and can exceed the HBM line; ``l2 = cold`` rows rotate through the whole
+256 MiB buffers so that consecutive operations touch memory that has left L2.
+"""
+from __future__ import annotations
+
+import argparse
+import csv
+import sys
+from pathlib import Path
+
+import numpy as np
+
+MiB = 1 << 20
+FIELDS = ["config", "op", "pattern", "variant", "level", "threads", "groups", "npes", "dtype", "nbytes",
+          "l2", "iters", "us_per_op", "gbps", "frac_hbm", "frac_8tbs", "mops", "note"]
+
+
+class Timer:
+    def __init__(self, torch, stream, min_ms=2.0, trials=10, max_iters=1 << 13):
+        self.torch, self.stream = torch, stream
+        self.min_ms, self.trials, self.max_iters = min_ms, trials, max_iters
+
+    def batch(self, fn, iters) -> float:
+        t = self.torch
+        a, b = t.cuda.Event(enable_timing=True), t.cuda.Event(enable_timing=True)
+        t.cuda.synchronize()
+        a.record(self.stream)
+        for i in range(iters):
+            fn(i)
+        b.record(self.stream)
+        t.cuda.synchronize()
+        return a.elapsed_time(b)
+
+    def __call__(self, fn):
+        """-> (microseconds per call, iterations per batch)."""
+        iters = 1
+        self.batch(fn, 1)
+        while True:
+            ms = self.batch(fn, iters)
+            if ms >= self.min_ms or iters >= self.max_iters:
+                break
+            iters *= 2
+        trials = self.trials if ms < 50 else 3
+        best = min([ms] + [self.batch(fn, iters) for _ in range(trials)])
+        return best / iters * 1e3, iters
+
+
+class Out:
+    def __init__(self, path, peak_gbs):
+        self.rows, self.path, self.peak = [], path, peak_gbs
+
+    def add(self, **kw):
+        us, nb = kw.get("us_per_op"), kw.pop("alg_bytes", None)
+        if nb is not None and us:
+            g = nb / us / 1e3
+            kw["gbps"] = round(g, 2)
+            kw["frac_hbm"] = round(g / self.peak, 4)
+            kw["frac_8tbs"] = round(g / 8000.0, 4)
+        if us is not None:
+            kw["us_per_op"] = round(us, 3)
+        self.rows.append({k: kw.get(k, "") for k in FIELDS})
+        r = self.rows[-1]
+        print(",".join(str(r[k]) for k in FIELDS), file=sys.stderr, flush=True)
+
+    def write(self):
+        Path(self.path).parent.mkdir(parents=True, exist_ok=True)
+        with open(self.path, "w", newline="") as f:
+            w = csv.DictWriter(f, fieldnames=FIELDS)
+            w.writeheader()
+            w.writerows(self.rows)
+
+
+def _session(torch, B, npes, heap_bytes):
+    heap = torch.empty(npes * heap_bytes, dtype=torch.uint8, device="cuda")
+    B.ishmemx_init_external(npes, heap_bytes, heap.data_ptr())
+    stream = torch.cuda.Stream()
+    B.ishmemx_set_stream(-1, stream.cuda_stream)
+    return heap, stream
+
+
+def _fill_bytes(torch, heap, npes, heap_bytes, off, nbytes, seed, inputs):
+    """uniform random bytes, one seeded 16 MiB block per PE tiled over [off, off+nbytes)"""
+    for p in range(npes):
+        blk = torch.from_numpy(inputs.byte_payload(seed, p, min(nbytes, 16 * MiB))).cuda()
+        view = heap[p * heap_bytes + off:p * heap_bytes + off + nbytes]
+        if nbytes > blk.numel():
+            view.view(-1, blk.numel())[:] = blk
+        else:
+            view.copy_(blk)
+
+
+# ------------------------------------------------------------------------------ config 2 ---
+
+def sweep_c2(args, out):
+    """8 PEs x 512 MiB: put/get, 8 B..256 MiB, every collaboration level and the copy engine,
+    ring and all-pairs, plus the host API's adaptive path on one PE."""
+    import torch
+    from . import binding as B
+    from . import inputs
+
+    npes, heap_bytes, big = 8, 512 * MiB, 256 * MiB
+    heap, stream = _session(torch, B, npes, heap_bytes)
+    src, dst = B.ishmem_malloc(big), B.ishmem_malloc(big)
+    _fill_bytes(torch, heap, npes, heap_bytes, src - heap.data_ptr(), big, inputs.SEED_C2, inputs)
+    T = Timer(torch, stream)
+    sizes = inputs.message_sizes(3, 28)
+    if args.quick:
+        sizes = sizes[::5]
+    WI, SG, WG, BK = B.ISHMEMX_WORK_ITEM, B.ISHMEMX_SUB_GROUP, B.ISHMEMX_WORK_GROUP, B.ISHMEMX_WORK_GROUP_BULK
+    variants = [("work_item", WI, 1, 1, 4 * MiB), ("sub_group", SG, 32, 1, 64 * MiB)]
+    variants += [(f"work_group_{t}x1", WG, t, 1, big) for t in (16, 128, 256, 1024)]
+    variants += [(f"work_group_256x{g}", WG, 256, g, big) for g in (4, 18, 37, 74)]
+    variants += [(f"work_group_512x{g}", WG, 512, g, big) for g in (37, 74)]
+    variants += [(f"work_group_bulk_256x{g}", BK, 256, g, big) for g in (1, 4, 18, 37)]
+
+    def slots(n):
+        stride = max((n + 255) // 256 * 256, big // 1024)
+        return max(1, big // stride), stride
+
+    for op in ("put", "get"):
+        spmd = B.ishmemx_putmem_spmd if op == "put" else B.ishmemx_getmem_spmd
+        for name, level, threads, groups, cap in variants:
+            for n in sizes:
+                if n > cap:
+                    continue
+                us, it = T(lambda i: spmd(dst, src, n, 1, level, threads, groups))
+                out.add(config=2, op=op, pattern="ring", variant=name, level=level, threads=threads, groups=groups,
+                        npes=npes, dtype="u8", nbytes=n, l2="hot", iters=it, us_per_op=us, alg_bytes=2 * n * npes)
+                if groups >= 18 and n < big:
+                    nsl, stride = slots(n)
+                    us, it = T(lambda i: spmd(dst + (i % nsl) * stride, src + (i % nsl) * stride, n, 1, level,
+                                              threads, groups))
+                    out.add(config=2, op=op, pattern="ring", variant=name, level=level, threads=threads,
+                            groups=groups, npes=npes, dtype="u8", nbytes=n, l2="cold", iters=it, us_per_op=us,
+                            alg_bytes=2 * n * npes)
+    # copy engine, same pattern (8 cudaMemcpyAsync per operation)
+    for n in sizes:
+        us, it = T(lambda i: B.ishmemx_putmem_spmd_copy_engine(dst, src, n, 1))
+        out.add(config=2, op="put", pattern="ring", variant="copy_engine", npes=npes, dtype="u8", nbytes=n, l2="hot",
+                iters=it, us_per_op=us, alg_bytes=2 * n * npes)
+        if n < big:
+            nsl, stride = slots(n)
+            us, it = T(lambda i: B.ishmemx_putmem_spmd_copy_engine(dst + (i % nsl) * stride, src + (i % nsl) * stride,
+                                                                  n, 1))
+            out.add(config=2, op="put", pattern="ring", variant="copy_engine", npes=npes, dtype="u8", nbytes=n,
+                    l2="cold", iters=it, us_per_op=us, alg_bytes=2 * n * npes)
+    # all-pairs: 7 permutation rounds p -> (p+r) mod 8 per operation
+    for name, level, threads, groups in (("work_group_bulk_256x37", BK, 256, 37), ("work_group_512x74", WG, 512, 74),
+                                          ("copy_engine", None, 0, 0)):
+        for n in sizes:
+            def rounds(i, n=n):
+                for r in range(1, npes):
+                    if level is None:
+                        B.ishmemx_putmem_spmd_copy_engine(dst, src, n, r)
+                    else:
+                        B.ishmemx_putmem_spmd(dst, src, n, r, level, threads, groups)
+            us, it = T(rounds)
+            out.add(config=2, op="put", pattern="all_pairs", variant=name, level=level if level is not None else "",
+                    threads=threads, groups=groups, npes=npes, dtype="u8", nbytes=n, l2="hot", iters=it,
+                    us_per_op=us / (npes - 1), alg_bytes=2 * n * npes, note="mean of the 7 rounds")
+    # host API on ONE PE (PE 0 -> PE 1): the load/store kernel against the copy engine -- the cutover
+    s0 = torch.cuda.Stream()
+    B.ishmemx_set_stream(0, s0.cuda_stream)
+    T0 = Timer(torch, s0)
+    for n in sizes:
+        B.ishmemx_set_cutover(0, B.SIZE_MAX)
+        us, it = T0(lambda i: B.ishmem_putmem(0, dst, src, n, 1))
+        out.add(config=2, op="put", pattern="one_pe", variant="host_api_kernel", npes=1, dtype="u8", nbytes=n,
+                l2="hot", iters=it, us_per_op=us, alg_bytes=2 * n)
+        B.ishmemx_set_cutover(0, 0)
+        us, it = T0(lambda i: B.ishmem_putmem(0, dst, src, n, 1))
+        out.add(config=2, op="put", pattern="one_pe", variant="host_api_copy_engine", npes=1, dtype="u8", nbytes=n,
+                l2="hot", iters=it, us_per_op=us, alg_bytes=2 * n)
+    B.ishmemx_set_cutover(0, B.SIZE_MAX)
+    # device-timed latency of one collaboration unit (in-kernel loop, PE 0 -> PE 1)
+    ns = np.zeros(1)
+    for op, is_get in (("put", 0), ("get", 1)):
+        for name, level, threads, cap in (("work_item", WI, 32, 1 * MiB), ("sub_group", SG, 32, 16 * MiB),
+                                          ("work_group_16", WG, 16, 16 * MiB), ("work_group_128", WG, 128, 64 * MiB),
+                                          ("work_group_256", WG, 256, 64 * MiB),
+                                          ("work_group_1024", WG, 1024, 64 * MiB),
+                                          ("work_group_bulk_256", BK, 256, 64 * MiB)):
+            for n in sizes:
+                if n > cap:
+                    continue
+                iters = int(max(4, min(2000, (64 * MiB) // max(n, 4096))))
+                B.ishmemx_rma_latency(0, dst, src, n, 1, is_get, level, threads, iters, ns)
+                B.ishmemx_rma_latency(0, dst, src, n, 1, is_get, level, threads, iters, ns)
+                out.add(config=2, op=op, pattern="one_pe", variant="in_kernel_" + name, level=level, threads=threads,
+                        groups=1, npes=1, dtype="u8", nbytes=n, l2="hot", iters=iters, us_per_op=float(ns[0]) / 1e3,
+                        alg_bytes=2 * n, note="device global timer, op + quiet")
+    assert B.ishmemx_status(1) == 0
+    B.ishmem_finalize()
+
+
+# ------------------------------------------------------------------------------ config 1 ---
+
+def sweep_c1(args, out):
+    """4 PEs x 16 MiB: work-group put/get of int32 messages 4 B..1 MiB on the ring, then the
+    int32 sum_reduce of 262144 elements."""
+    import torch
+    from . import binding as B
+    from . import inputs
+
+    npes, heap_bytes = 4, 16 * MiB
+    heap, stream = _session(torch, B, npes, heap_bytes)
+    src, dst = B.ishmem_malloc(MiB), B.ishmem_malloc(MiB)
+    for p in range(npes):
+        v = torch.from_numpy(inputs.int32_payload(inputs.SEED_C1, p, MiB // 4)).cuda().view(torch.uint8)
+        o = p * heap_bytes + src - heap.data_ptr()
+        heap[o:o + MiB].copy_(v)
+    T = Timer(torch, stream)
+    ns = np.zeros(1)
+    for n in inputs.message_sizes(2, 20):
+        groups = max(1, min(37, n // 16384))
+        for op, fn in (("put", B.ishmemx_putmem_spmd), ("get", B.ishmemx_getmem_spmd)):
+            us, it = T(lambda i: fn(dst, src, n, 1, B.ISHMEMX_WORK_GROUP, 256, groups))
+            out.add(config=1, op=op, pattern="ring", variant=f"work_group_256x{groups}", level=B.ISHMEMX_WORK_GROUP,
+                    threads=256, groups=groups, npes=npes, dtype="i32", nbytes=n, l2="hot", iters=it, us_per_op=us,
+                    alg_bytes=2 * n * npes, note="host-launched, all 4 PEs in one launch")
+            iters = int(max(4, min(2000, (16 * MiB) // max(n, 4096))))
+            B.ishmemx_rma_latency(0, dst, src, n, 1, int(op == "get"), B.ISHMEMX_WORK_GROUP, 256, iters, ns)
+            out.add(config=1, op=op, pattern="one_pe", variant="in_kernel_work_group_256", level=B.ISHMEMX_WORK_GROUP,
+                    threads=256, groups=1, npes=1, dtype="i32", nbytes=n, l2="hot", iters=iters,
+                    us_per_op=float(ns[0]) / 1e3, alg_bytes=2 * n, note="device global timer, op + quiet")
+    n = 262144
+    for p in range(npes):
+        v = torch.from_numpy(inputs.int32_reduce_values(inputs.SEED_C1, p, n)).cuda().view(torch.uint8)
+        o = p * heap_bytes + src - heap.data_ptr()
+        heap[o:o + 4 * n].copy_(v)
+    for alg, name in ((B.ISHMEMX_REDUCE_SPLIT, "split"), (B.ISHMEMX_REDUCE_DUPLICATED, "duplicated")):
+        us, it = T(lambda i: B.ishmemx_reduce(B.ISHMEM_TEAM_WORLD, dst, src, n, B.ISHMEM_OP_SUM, B.ISHMEM_T_INT32, alg))
+        out.add(config=1, op="sum_reduce", pattern="team", variant=name, npes=npes, dtype="i32", nbytes=4 * n,
+                l2="hot", iters=it, us_per_op=us, alg_bytes=2 * npes * 4 * n)
+    assert B.ishmemx_status(1) == 0
+    B.ishmem_finalize()
+
+
+# ------------------------------------------------------------------------------ config 3 ---
+
+def sweep_c3(args, out):
+    """12 PEs: sum/max/min/prod reduce on float32, float64, int64; broadcast from root 0;
+    fcollect; 1..64 Mi elements in powers of 4; stores against the copy engine for the push
+    collectives; device-resident forms (one work-group per PE, in-kernel sync) for small sizes."""
+    import torch
+    from . import binding as B
+    from . import inputs
+
+    npes = 12
+    max_el = (4 ** 13) if not args.quick else (4 ** 11)
+    fc_el = min(max_el, args.fcollect_max_elems)
+    heap_bytes = 8 * max_el + 8 * fc_el * npes + 4 * MiB
+    heap, stream = _session(torch, B, npes, heap_bytes)
+    src = B.ishmem_malloc(8 * max_el)
+    dst = B.ishmem_malloc(max(8 * max_el, 8 * fc_el * npes))
+    T = Timer(torch, stream)
+    W = B.ISHMEM_TEAM_WORLD
+    counts = [4 ** k for k in range(0, 14) if 4 ** k <= max_el]
+    types = [("f32", np.float32, B.ISHMEM_T_FLOAT, 4), ("f64", np.float64, B.ISHMEM_T_DOUBLE, 8),
+             ("i64", np.int64, B.ISHMEM_T_INT64, 8)]
+    ops = [("sum", B.ISHMEM_OP_SUM), ("max", B.ISHMEM_OP_MAX), ("min", B.ISHMEM_OP_MIN), ("prod", B.ISHMEM_OP_PROD)]
+    blk_el = MiB
+    for tname, npdt, dt, es in types:
+        for p in range(npes):
+            if tname == "i64":
+                v = inputs.int64_values(inputs.SEED_C3, p, blk_el)
+            else:
+                v = inputs.normal_values(inputs.SEED_C3, p, blk_el, npdt)
+            blk = torch.from_numpy(v).cuda().view(torch.uint8)
+            o = p * heap_bytes + src - heap.data_ptr()
+            heap[o:o + es * max_el].view(-1, blk.numel())[:] = blk
+        for n in counts:
+            for oname, op in ops:
+                us, it = T(lambda i: B.ishmemx_reduce(W, dst, src, n, op, dt, B.ISHMEMX_REDUCE_AUTO))
+                out.add(config=3, op=oname + "_reduce", pattern="team", variant="auto", npes=npes, dtype=tname,
+                        nbytes=n * es, l2="hot", iters=it, us_per_op=us, alg_bytes=2 * npes * n * es)
+            if n * es <= 4 * MiB:
+                us, it = T(lambda i: B.ishmemx_reduce(W, dst, src, n, B.ISHMEM_OP_SUM, dt, B.ISHMEMX_REDUCE_DUPLICATED))
+                out.add(config=3, op="sum_reduce", pattern="team", variant="duplicated", npes=npes, dtype=tname,
+                        nbytes=n * es, l2="hot", iters=it, us_per_op=us, alg_bytes=2 * npes * n * es)
+            B.ishmemx_set_cutover(1, B.SIZE_MAX)
+            us, it = T(lambda i: B.ishmem_broadcastmem(W, dst, src, n * es, 0))
+            out.add(config=3, op="broadcast", pattern="team", variant="stores", npes=npes, dtype=tname, nbytes=n * es,
+                    l2="hot", iters=it, us_per_op=us, alg_bytes=n * es * (1 + npes))
+            if n <= fc_el:
+                B.ishmemx_set_cutover(2, B.SIZE_MAX)
+                us, it = T(lambda i: B.ishmem_fcollectmem(W, dst, src, n * es))
+                out.add(config=3, op="fcollect", pattern="team", variant="stores", npes=npes, dtype=tname,
+                        nbytes=n * es, l2="hot", iters=it, us_per_op=us, alg_bytes=n * es * (npes + npes * npes))
+    # push collectives: stores against the copy engine, team sizes 2..12 (bytes; type-agnostic)
+    for P in (2, 4, 8, 12):
+        team = W if P == npes else B.ishmem_team_split_strided(W, 0, 1, P)
+        for n in [4 ** k for k in range(1, 14) if 4 ** k <= 4 * fc_el]:
+            for which, opname, fn, nb in ((1, "broadcast", lambda i: B.ishmem_broadcastmem(team, dst, src, n, 0),
+                                          n * (1 + P)),
+                                         (2, "fcollect", lambda i: B.ishmem_fcollectmem(team, dst, src, n),
+                                          n * (P + P * P))):
+                for variant, cut in (("stores", B.SIZE_MAX), ("copy_engine", 0)):
+                    B.ishmemx_set_cutover(which, cut)
+                    us, it = T(fn)
+                    out.add(config=3, op=opname, pattern="team", variant=variant, npes=P, dtype="u8", nbytes=n,
+                            l2="hot", iters=it, us_per_op=us, alg_bytes=nb)
+        B.ishmemx_set_cutover(1, B.SIZE_MAX)
+        B.ishmemx_set_cutover(2, B.SIZE_MAX)
+        # device-resident forms: one work-group per PE, push sync inside the kernel, `rep` calls per launch
+        rep = 50
+        for threads in (128, 256, 1024):
+            for n in [4 ** k for k in range(0, 10)]:
+                for which, opname, nb in ((0, "broadcast", n * (1 + P)), (1, "fcollect", n * (P + P * P)),
+                                          (2, "sum_reduce_f32", 2 * P * n)):
+                    if which == 2 and n < 4:
+                        continue
+                    cnt = n // 4 if which == 2 else n
+                    us, it = T(lambda i: B.ishmemx_collective_on_device(which, team, dst, src, cnt, 0, B.ISHMEM_OP_SUM,
+                                                                       B.ISHMEM_T_FLOAT, threads, rep))
+                    out.add(config=3, op=opname, pattern="team", variant="device_resident", threads=threads, groups=1,
+                            npes=P, dtype="u8", nbytes=n, l2="hot", iters=it * rep, us_per_op=us / rep, alg_bytes=nb,
+                            note="one work-group per PE, in-kernel push sync")
+            us, it = T(lambda i: B.ishmemx_collective_on_device(3, team, None, None, 0, 0, 0, 0, threads, rep))
+            out.add(config=3, op="sync", pattern="team", variant="device_resident", threads=threads, groups=1, npes=P,
+                    dtype="", nbytes=0, l2="hot", iters=it * rep, us_per_op=us / rep)
+        if team != W:
+            B.ishmem_team_destroy(team)
+    assert B.ishmemx_status(1) == 0
+    B.ishmem_finalize()
+
+
+# ------------------------------------------------------------------------------ config 4 ---
+
+def sweep_c4(args, out):
+    """16 PEs: 2^22 fetch_add on 4096 words (Zipf 1.1) and on a uniform index stream, 2^20
+    compare_swap on 1024 words, put_signal / wait_until ping-pong 8 B..64 KiB."""
+    import torch
+    from . import binding as B
+    from . import inputs
+
+    npes, heap_bytes = 16, 4 * MiB
+    heap, stream = _session(torch, B, npes, heap_bytes)
+    table = B.ishmem_calloc(4096, 8)
+    data, sig = B.ishmem_malloc(64 << 10), B.ishmem_calloc(8, 8)
+    T = Timer(torch, stream)
+    nops, nwords = 1 << 22, 4096
+    inc = torch.from_numpy(inputs.increments(inputs.SEED_C4, 0, nops)).cuda()
+    fetched = torch.empty(nops, dtype=torch.int64, device="cuda")
+    streams = {"zipf1.1": inputs.zipf_indices(inputs.SEED_C4, 0, nops, nwords),
+               "uniform": inputs.rng_for(inputs.SEED_C4, 42).integers(0, nwords, nops).astype(np.int32),
+               "one_word": np.zeros(nops, dtype=np.int32)}
+    for sname, idx in streams.items():
+        word = torch.from_numpy(idx).cuda()
+        for agg in (1, 0):
+            for fet, fname in ((fetched, "fetch_add"), (None, "add")):
+                for threads in (256, 1024):
+                    us, it = T(lambda i: B.ishmemx_int64_atomic_fetch_add_batch(table, word, inc, fet, nops, threads, agg))
+                    out.add(config=4, op=fname, pattern=sname, variant="aggregate" if agg else "plain",
+                            threads=threads, npes=npes, dtype="i64", nbytes=8, l2="hot", iters=it, us_per_op=us,
+                            mops=round(nops / us, 1), note=f"{nops} ops on {nwords} words")
+    nops_c, nwords_c = 1 << 20, 1024
+    cword = torch.from_numpy(inputs.zipf_indices(inputs.SEED_C4, 1, nops_c, nwords_c)).cuda()
+    cval = torch.arange(1, nops_c + 1, dtype=torch.int64, device="cuda")
+    for cname, ccond in (("claim_cond_0", torch.zeros(nops_c, dtype=torch.int64, device="cuda")),
+                         ("never_matches", torch.full((nops_c,), -7, dtype=torch.int64, device="cuda"))):
+        us, it = T(lambda i: B.ishmemx_int64_atomic_compare_swap_batch(table, cword, ccond, cval, fetched, nops_c, 256))
+        out.add(config=4, op="compare_swap", pattern="zipf1.1", variant=cname, threads=256, npes=npes, dtype="i64",
+                nbytes=8, l2="hot", iters=it, us_per_op=us, mops=round(nops_c / us, 1),
+                note=f"{nops_c} ops on {nwords_c} words")
+    rtt, bad = np.zeros(1), np.zeros(1, dtype=np.uint64)
+    rounds = 1000
+    for threads in (32, 256, 1024):
+        for n in inputs.message_sizes(3, 16):
+            for a, b in ((0, 1),):
+                B.ishmem_uint64_p(a, sig, 0, a)
+                B.ishmem_uint64_p(b, sig, 0, b)
+                B.ishmemx_pingpong(a, b, data, sig, n, rounds, threads, rtt, bad)
+                out.add(config=4, op="put_signal_pingpong", pattern="pe0<->pe1", variant="in_kernel", threads=threads,
+                        groups=1, npes=2, dtype="u8", nbytes=n, l2="hot", iters=rounds, us_per_op=float(rtt[0]) / 1e3,
+                        alg_bytes=2 * n + 8, note=f"half round trip; stamp mismatches {int(bad[0])}")
+    assert B.ishmemx_status(1) == 0
+    B.ishmem_finalize()
+
+
+# ------------------------------------------------------------------------------ config 5 ---
+
+def sweep_c5(args, out):
+    """12 PEs: float64 5-point Jacobi on 16384 x 16384, 200 sweeps, halo rows by in-kernel
+    work-group put_signal; with and without the interior-first overlap."""
+    import torch
+    from . import binding as B
+    from . import inputs
+
+    npes, n, iters = 12, (16384 if not args.quick else 4096), 200
+    rows_max = -(-n // npes)
+    nbytes = (rows_max + 2) * n * 8
+    heap_bytes = 2 * nbytes + MiB
+    heap, stream = _session(torch, B, npes, heap_bytes)
+    b0, b1, sig = B.ishmem_malloc(nbytes), B.ishmem_malloc(nbytes), B.ishmem_calloc(2, 8)
+    base, extra = divmod(n, npes)
+    res = np.zeros(1)
+
+    def load():
+        first = 0
+        heap.zero_()
+        for p in range(npes):
+            rows = base + (1 if p < extra else 0)
+            win = inputs.jacobi_cell_init(inputs.SEED_C5, n, n, first, first + rows, 0, n)
+            o = p * heap_bytes + (b0 - heap.data_ptr()) + n * 8
+            heap[o:o + rows * n * 8].copy_(torch.from_numpy(win.view(np.uint8).ravel()))
+            first += rows
+
+    load()
+    for overlap in (1, 0):
+        for groups in (6, 12, 24):
+            for threads in (256, 512, 1024):
+                if npes * groups * threads > 148 * 2048:
+                    continue
+                for p in range(npes):
+                    B.ishmem_uint64_p(p, sig, 0, p)
+                    B.ishmem_uint64_p(p, sig + 8, 0, p)
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                torch.cuda.synchronize()
+                a.record(stream)
+                try:
+                    B.ishmemx_jacobi(b0, b1, sig, n, n, iters, overlap, groups, threads, res)
+                except B.IshmemError as e:
+                    out.add(config=5, op="jacobi", variant=f"overlap={overlap}", threads=threads, groups=groups,
+                            npes=npes, dtype="f64", nbytes=n * n * 8, note=str(e))
+                    continue
+                b.record(stream)
+                torch.cuda.synchronize()
+                us = a.elapsed_time(b) * 1e3 / iters
+                out.add(config=5, op="jacobi", pattern=f"{n}x{n}", variant=f"overlap={overlap}", threads=threads,
+                        groups=groups, npes=npes, dtype="f64", nbytes=n * n * 8, l2="cold", iters=iters, us_per_op=us,
+                        alg_bytes=16 * n * n, note=f"per sweep; residual_sq {res[0]:.6e} (grid keeps evolving)")
+    assert B.ishmemx_status(1) == 0
+    B.ishmem_finalize()
+
+
+def main(argv=None):
+    ap = argparse.ArgumentParser(description=__doc__, formatter_class=argparse.RawDescriptionHelpFormatter)
+    ap.add_argument("--config", type=int, required=True, choices=[1, 2, 3, 4, 5])
+    ap.add_argument("--out", required=True, help="CSV file to write")
+    ap.add_argument("--peak-gbs", type=float, default=None,
+                    help="measured HBM copy peak in GB/s (default: MEASURED_PEAKS.json beside the package, else 6650)")
+    ap.add_argument("--quick", action="store_true", help="fewer sizes (smoke run)")
+    ap.add_argument("--fcollect-max-elems", type=int, default=4 ** 12,
+                    help="largest per-PE element count of the 8-byte fcollect rows")
+    args = ap.parse_args(argv)
+    peak = args.peak_gbs
+    if peak is None:
+        import json
+        f = Path(__file__).resolve().parent.parent / "MEASURED_PEAKS.json"
+        peak = float(json.loads(f.read_text())["hbm_gbs"]) if f.exists() else 6650.0
+    out = Out(args.out, peak)
+    try:
+        {1: sweep_c1, 2: sweep_c2, 3: sweep_c3, 4: sweep_c4, 5: sweep_c5}[args.config](args, out)
+    finally:
+        out.write()
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -57,3 +57,19 @@ def test_jacobi_even_iterations_and_zero():
         exp, _ = orc.jacobi(grid, iters)
         got, _ = run_gpu(grid, 12, iters, 1, 2, 64)
         assert got.tobytes() == exp.tobytes(), iters
+
+
+def test_refused_coresident_launch_leaves_the_library_usable():
+    """A persistent launch that cannot be co-resident is refused with NOT_CORESIDENT; the
+    refusal must not leak into the next call."""
+    npes, ny, nx = 12, 4800, 16
+    nbytes = (ny // npes + 2) * nx * 8
+    with Session(npes, 2 * nbytes + (1 << 16), with_oracle=False) as s:
+        b0, b1, sig = s.malloc(nbytes), s.malloc(nbytes), s.malloc(64)
+        with pytest.raises(B.IshmemError) as e:
+            B.ishmemx_jacobi(b0.addr, b1.addr, sig.addr, ny, nx, 2, 1, 400, 1024, None)
+        assert e.value.code == B.ISHMEM_ERR_NOT_CORESIDENT
+        B.ishmem_uint64_p(0, sig.addr, 5, 1)
+        B.ishmem_barrier_all()
+        assert sig.read(1, np.uint64)[0] == 5
+        assert s.status() == 0

@@ -263,3 +263,28 @@ def test_put_signal_wait_until_and_bounded_timeout():
         B.ishmem_putmem(0, data.addr, data.addr, 16, 1)
         B.ishmem_barrier_all()
         assert s.status() == 0
+
+
+@pytest.mark.parametrize("level", list(LEVELS))
+def test_device_timed_latency_program_moves_the_data(level):
+    """ishmemx_rma_latency: repeated in-kernel put/get + quiet by one collaboration unit; the
+    payload must arrive exactly as the oracle's put/get says and the time must be positive."""
+    npes, heap = 3, 1 << 20
+    with Session(npes, heap) as s:
+        src, dst = s.malloc(200_000), s.malloc(200_000)
+        for p in range(npes):
+            src.fill(p, inputs.byte_payload(inputs.SEED_C2, p, 200_000))
+        ns = np.zeros(1)
+        for n, is_get in ((8, 0), (4099, 0), (150_001, 0), (65_536, 1), (33, 1)):
+            threads = {"work_item": 32, "sub_group": 64, "work_group": 128, "work_group_bulk": 256}[level]
+            B.ishmemx_rma_latency(1, dst.addr + 5, src.addr + 5, n, 2, is_get, LEVELS[level], threads, 3, ns)
+            assert ns[0] > 0
+            if is_get:
+                s.oracle.getmem(1, s.oracle.ptr(dst.ooff + 5, n, 1), src.ooff + 5, n, 2)
+            else:
+                s.oracle.putmem(1, dst.ooff + 5, s.oracle.ptr(src.ooff + 5, n, 1), n, 2)
+            heaps_equal(s, f"{level} n={n} get={is_get}")
+        with pytest.raises(B.IshmemError) as e:
+            B.ishmemx_rma_latency(1, dst.addr, src.addr, 8, 7, 0, LEVELS[level], 64, 1, ns)
+        assert e.value.code == B.ISHMEM_ERR_INVALID_PE
+        assert s.status() == 0
