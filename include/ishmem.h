@@ -81,6 +81,7 @@ typedef int ishmem_team_t;
 #define ISHMEMX_SUB_GROUP 1
 #define ISHMEMX_WORK_GROUP 2       /* 16-byte vector loads/stores by all threads */
 #define ISHMEMX_WORK_GROUP_BULK 3  /* work-group; large aligned blocks go through TMA bulk copies */
+#define ISHMEMX_WORK_GROUP_ENGINE 4 /* work-group; the leader asks the host proxy to start the copy engine */
 
 /* reduction operators and element types of the generic reduce entry point */
 #define ISHMEM_OP_SUM 0
@@ -186,9 +187,10 @@ ISHMEM_DECL_RMA(uint64, uint64_t)
 /* Explicit thread-collaborative variants (Section 3.6; experiments of Section 4): a
  * kernel of `groups` blocks x `threads` threads is launched on my_pe's stream; the message
  * is cut into one contiguous slice per collaboration unit (thread / warp / block,
- * `level` = ISHMEMX_WORK_ITEM..ISHMEMX_WORK_GROUP_BULK) and every unit calls the device
- * routine ishmem_putmem / ishmemx_putmem_sub_group / ishmemx_putmem_work_group once on its
- * slice.  threads in 1..1024, groups >= 1.  No cutover. */
+ * `level` = ISHMEMX_WORK_ITEM..ISHMEMX_WORK_GROUP_ENGINE) and every unit calls the device
+ * routine ishmem_putmem / ishmemx_putmem_sub_group / ishmemx_putmem_work_group /
+ * ishmemx_putmem_engine_work_group once on its slice.  threads in 1..1024, groups >= 1.
+ * ISHMEMX_WORK_GROUP_ENGINE needs a running proxy (ISHMEM_ERR_ARG otherwise). */
 int ishmemx_putmem_on_device(int my_pe, void *dest, const void *src, size_t nbytes, int pe,
                              int level, int threads, int groups);
 int ishmemx_getmem_on_device(int my_pe, void *dest, const void *src, size_t nbytes, int pe,
@@ -208,10 +210,35 @@ int ishmemx_getmem_spmd(void *dest, const void *src, size_t nbytes, int shift, i
 int ishmemx_putmem_spmd_copy_engine(void *dest, const void *src, size_t nbytes, int shift);
 
 /* Cutover sizes in bytes (Section 4: tuned from measurement; for the collaborative calls
- * it depends on the number of threads).  which: 0 = put/get, 1 = broadcast, 2 = fcollect.
- * SIZE_MAX = never use the copy engine, 0 = always. */
+ * it depends on the number of threads).  which: 0 = host-initiated put/get, 1 = broadcast,
+ * 2 = fcollect, 3 = device-initiated work-group put/get (takes effect while the host proxy of
+ * ishmemx_proxy_start runs).  SIZE_MAX = never use the copy engine (the default), 0 = always. */
 int ishmemx_set_cutover(int which, size_t nbytes);
 size_t ishmemx_get_cutover(int which);
+
+/* ------------------------------------- reverse offload: GPU -> host requests (Section 3.4) --- */
+
+/* Starts / stops the host proxy thread and its request ring.  While it runs, device code can
+ * hand copies to the copy engine (ishmemx_putmem_engine_work_group and the cutover of
+ * ishmemx_putmem_work_group, see ishmem_device.cuh): a GPU thread writes one 64-byte request
+ * into a ring in pinned host memory (one fetch-and-increment to allocate the slot, stores
+ * only), the proxy issues cudaMemcpyAsync on the issuing PE's copy-engine stream, and the reply
+ * is written behind the copy in stream order into a word the GPU thread polls.  Both calls
+ * block until the device is idle; ishmem_finalize stops a running proxy.  Allocates pinned host
+ * memory (ring of 1024 requests, 65536 reply words). */
+int ishmemx_proxy_start(void);
+int ishmemx_proxy_stop(void);
+/* Requests served and copies started since ishmemx_proxy_start (HOST pointers, may be NULL);
+ * *uses_stream_memops = 1 when replies are written by stream memory operations, 0 when by
+ * 8-byte copies.  ISHMEM_ERR_ARG when no proxy runs. */
+int ishmemx_proxy_stats(uint64_t *requests_served, uint64_t *copies_started, int *uses_stream_memops);
+/* Ring measurement: `blocks` x `threads` GPU threads each post `iters` no-op requests.
+ * mode 0: each request waits for its reply -> *mean_rtt_ns = mean GPU -> host -> GPU round trip
+ * (device global timer).  mode 1: no replies except for each thread's last request ->
+ * *requests_per_second = requests / time as seen from the GPU (HOST pointers, may be NULL).
+ * Needs a running proxy.  Blocks the host. */
+int ishmemx_ring_benchmark(int mode, int blocks, int threads, int iters, double *mean_rtt_ns,
+                           double *requests_per_second);
 
 /* ------------------------------------------- signalling, ordering, synchronisation --- */
 
@@ -340,7 +367,7 @@ int ishmemx_pingpong(int pe_a, int pe_b, void *data, uint64_t *sig, size_t nbyte
  * many back-to-back operations inside one kernel, timed on the device).  ONE work-group of
  * `threads` threads runs as PE my_pe and issues `iters` puts (is_get = 0) or gets of `nbytes`
  * to/from PE `pe`, each followed by quiet: by its first thread alone (ISHMEMX_WORK_ITEM), by
- * its first warp (ISHMEMX_SUB_GROUP), or by all threads (ISHMEMX_WORK_GROUP, _BULK).  dest/src
+ * its first warp (ISHMEMX_SUB_GROUP), or by all threads (ISHMEMX_WORK_GROUP, _BULK, _ENGINE).  dest/src
  * as for ishmem_putmem / ishmem_getmem.  Writes the mean time per operation in nanoseconds
  * (global timer, read inside the kernel) to HOST memory `ns_per_op`.  Blocks the host. */
 int ishmemx_rma_latency(int my_pe, void *dest, const void *src, size_t nbytes, int pe, int is_get,

@@ -31,6 +31,43 @@ struct ishmemi_team {
     int start, stride, size, valid;
 };
 
+/* Reverse-offload request (Section 3.4 of the paper, "Synchronization with Host"): a fixed
+ * 64-byte message that a GPU thread composes in a ring in host memory for the host proxy
+ * thread.  `seq` (ticket + 1) is stored last, with release semantics at system scope: a slot
+ * whose seq matches the host's expectation is complete. */
+struct __align__(64) ishmemi_request {
+    unsigned long long dest;       /* device address on the target PE (already translated) */
+    unsigned long long src;        /* device address of the source */
+    unsigned long long nbytes;
+    unsigned long long sig_addr;   /* translated signal word, or 0 */
+    unsigned long long sig_value;
+    unsigned op;                   /* ISHMEMI_REQ_* */
+    unsigned pe;                   /* issuing PE: selects the copy-engine stream */
+    unsigned long long completion; /* completion ticket + 1, or 0: counted in nbi_done[pe] instead */
+    unsigned long long seq;
+};
+#define ISHMEMI_REQ_NOP 0u        /* reply only (round-trip measurement) */
+#define ISHMEMI_REQ_COPY 1u       /* cudaMemcpyAsync dest <- src on the issuing PE's engine stream */
+#define ISHMEMI_REQ_COPY_SIGNAL 2u /* copy, then set the signal word, in stream order */
+
+/* Device-side view of the ring.  The ring, the published tail and the completion words live in
+ * pinned host memory mapped into the device's address space; the ticket counters live in device
+ * memory.  Both directions use stores only; the GPU end needs no progress thread. */
+struct ishmemi_proxy_t {
+    ishmemi_request *ring;                 /* host memory, ring_slots entries */
+    unsigned ring_slots;                   /* power of two */
+    unsigned comp_slots;                   /* power of two */
+    unsigned long long *head;              /* device: next ticket (one fetch-and-increment per message) */
+    unsigned long long *tail_cache;        /* device: last value of *tail_pub any thread has seen */
+    const unsigned long long *tail_pub;    /* host: messages consumed, published by the proxy now and then */
+    unsigned long long *comp_alloc;        /* device: next completion ticket */
+    const unsigned long long *comp;        /* host: slot c % comp_slots holds c + 1 once ticket c is complete */
+    unsigned long long *nbi_issued;        /* device [npes]: non-blocking requests posted by each PE */
+    unsigned long long *nbi_seen;          /* device [npes]: last value of nbi_done[pe] any thread has seen */
+    const unsigned long long *nbi_done;    /* host [npes]: non-blocking requests of each PE completed */
+    unsigned long long wg_cutover;         /* work-group put/get of at least this size use the engine */
+};
+
 /* Per-PE context, resident in device memory (Section 3.7.1: a separate GPU-side copy of
  * the runtime state, so that device calls never touch host memory). */
 struct ishmem_ctx_t {
@@ -51,6 +88,7 @@ struct ishmem_ctx_t {
     int *status;                       /* one word shared by all PEs; first error wins */
     unsigned long long wait_limit_ns;  /* time bound of every device-side wait */
     int bcast_root_dest;               /* broadcast writes the root's own dest */
+    const ishmemi_proxy_t *proxy;      /* reverse-offload ring, or nullptr while no host proxy runs */
 };
 
 /* shared-memory staging handed to the *_work_group copy routines to enable the TMA bulk
@@ -426,6 +464,109 @@ static __device__ __noinline__ int bulk_copy_ring(const ishmem_ctx_t *ctx, char 
     return rc;
 }
 
+/* ---- reverse offload: requests to the host proxy ------------------------------------------- */
+
+__device__ __forceinline__ unsigned long long ld_acquire_sys(const unsigned long long *p)
+{
+    unsigned long long v;
+    asm volatile("ld.acquire.sys.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_release_sys(unsigned long long *p, unsigned long long v)
+{
+    asm volatile("st.release.sys.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
+}
+
+/* Posts one request: one fetch-and-increment allocates the slot, the message is written with
+ * plain stores and published by the release store of its sequence number.  Flow control (the
+ * host must have consumed the slot's previous message) is checked against a cached copy of the
+ * host's tail in device memory; host memory is only read when the ring looks full.  One thread
+ * calls.  Returns 0 or ISHMEM_ERR_TIMEOUT. */
+__device__ __forceinline__ int proxy_post(const ishmem_ctx_t *ctx, unsigned op, void *dest, const void *src,
+                                          unsigned long long nbytes, unsigned long long *sig_addr,
+                                          unsigned long long sig_value, unsigned long long completion)
+{
+    const ishmemi_proxy_t *px = ctx->proxy;
+    const unsigned long long t = atomicAdd(px->head, 1ull);
+    if (t - ld_relaxed(px->tail_cache) >= px->ring_slots) {
+        deadline dl(ctx->wait_limit_ns);
+        for (;;) {
+            const unsigned long long tail = ld_acquire_sys(px->tail_pub);
+            if (t - tail < px->ring_slots) {
+                atomicMax(px->tail_cache, tail);
+                break;
+            }
+            if (dl.expired()) {
+                latch_error(ctx, ISHMEM_ERR_TIMEOUT);
+                return ISHMEM_ERR_TIMEOUT; /* the slot stays unwritten: the proxy stops at it */
+            }
+            __nanosleep(500);
+        }
+    }
+    ishmemi_request *slot = px->ring + (t & (px->ring_slots - 1));
+    uint4 *w = (uint4 *)slot;
+    const unsigned long long d = (unsigned long long)dest, sa = (unsigned long long)src, sg = (unsigned long long)sig_addr;
+    w[0] = make_uint4((unsigned)d, (unsigned)(d >> 32), (unsigned)sa, (unsigned)(sa >> 32));
+    w[1] = make_uint4((unsigned)nbytes, (unsigned)(nbytes >> 32), (unsigned)sg, (unsigned)(sg >> 32));
+    w[2] = make_uint4((unsigned)sig_value, (unsigned)(sig_value >> 32), op, (unsigned)ctx->my_pe);
+    slot->completion = completion;
+    st_release_sys(&slot->seq, t + 1);
+    return 0;
+}
+
+/* Waits (bounded) until completion ticket c has been answered; acquires at system scope, so
+ * data the copy engine wrote before the reply is visible afterwards. */
+__device__ __forceinline__ int proxy_wait(const ishmem_ctx_t *ctx, unsigned long long c)
+{
+    const ishmemi_proxy_t *px = ctx->proxy;
+    const unsigned long long *word = px->comp + (c & (px->comp_slots - 1));
+    deadline dl(ctx->wait_limit_ns);
+    for (;;) {
+        if (ld_acquire_sys(word) >= c + 1) return 0;
+        if (dl.expired()) break;
+        __nanosleep(200);
+    }
+    latch_error(ctx, ISHMEM_ERR_TIMEOUT);
+    return ISHMEM_ERR_TIMEOUT;
+}
+
+/* All non-blocking engine requests posted so far by the calling PE are complete. */
+__device__ __forceinline__ int proxy_quiet(const ishmem_ctx_t *ctx)
+{
+    const ishmemi_proxy_t *px = ctx->proxy;
+    if (px == nullptr) return 0;
+    const unsigned long long want = ld_relaxed(px->nbi_issued + ctx->my_pe);
+    if (ld_relaxed(px->nbi_seen + ctx->my_pe) >= want) return 0;
+    deadline dl(ctx->wait_limit_ns);
+    for (;;) {
+        const unsigned long long done = ld_acquire_sys(px->nbi_done + ctx->my_pe);
+        if (done >= want) {
+            atomicMax(px->nbi_seen + ctx->my_pe, done);
+            return 0;
+        }
+        if (dl.expired()) break;
+        __nanosleep(200);
+    }
+    latch_error(ctx, ISHMEM_ERR_TIMEOUT);
+    return ISHMEM_ERR_TIMEOUT;
+}
+
+/* One thread hands a copy to the copy engine through the host proxy.  blocking: waits for the
+ * reply.  Otherwise the request is counted for the PE and ishmem_quiet completes it. */
+__device__ __forceinline__ int proxy_copy(const ishmem_ctx_t *ctx, char *d, const char *s, size_t n, bool blocking,
+                                          unsigned long long *sig = nullptr, unsigned long long sig_value = 0)
+{
+    const ishmemi_proxy_t *px = ctx->proxy;
+    const unsigned op = sig ? ISHMEMI_REQ_COPY_SIGNAL : ISHMEMI_REQ_COPY;
+    if (blocking) {
+        const unsigned long long c = atomicAdd(px->comp_alloc, 1ull);
+        int rc = proxy_post(ctx, op, d, s, n, sig, sig_value, c + 1);
+        return rc ? rc : proxy_wait(ctx, c);
+    }
+    atomicAdd(px->nbi_issued + ctx->my_pe, 1ull);
+    return proxy_post(ctx, op, d, s, n, sig, sig_value, 0);
+}
+
 /* smallest aligned body worth starting the TMA ring for */
 #define ISHMEMI_BULK_MIN_BYTES 16384u
 
@@ -436,6 +577,15 @@ __device__ __forceinline__ int wg_copy(const ishmem_ctx_t *ctx, char *d, const c
 {
     const unsigned tid = threadIdx.x + blockDim.x * (threadIdx.y + blockDim.y * threadIdx.z);
     const unsigned nthr = blockDim.x * blockDim.y * blockDim.z;
+    if (ctx->proxy != nullptr && n >= ctx->proxy->wg_cutover) {
+        /* cutover (Sections 3.2 and 3.7.1): above the tuned size the group leader asks the host
+         * to start the copy engine, after a group barrier that makes the source valid */
+        __shared__ int rc_engine;
+        __syncthreads();
+        if (tid == 0) rc_engine = proxy_copy(ctx, d, s, n, complete);
+        __syncthreads();
+        return rc_engine;
+    }
     const bool congruent = ((((uintptr_t)d - (uintptr_t)s) & 15u) == 0);
     if (st.smem != nullptr && st.bytes >= 128u + 2048u && congruent && n >= ISHMEMI_BULK_MIN_BYTES) {
         size_t head = (size_t)((16u - ((unsigned)(uintptr_t)d & 15u)) & 15u);
@@ -621,17 +771,72 @@ __device__ __forceinline__ int ishmemx_getmem_nbi_work_group(const ishmem_ctx_t 
     return rc;
 }
 
+/* Explicit copy-engine forms (device-initiated reverse offload, Sections 3.4 and 3.7.1): after a
+ * group barrier the leader posts one request to the host proxy, which starts the engine; the
+ * other threads are free until the closing barrier.  Need a running proxy (ishmemx_proxy_start),
+ * else ISHMEM_ERR_ARG.  The blocking form returns when the data has arrived; the _nbi form when
+ * the request is posted (ishmem_quiet / ishmemx_quiet_work_group complete it). */
+__device__ __forceinline__ int ishmemx_putmem_engine_work_group(const ishmem_ctx_t *ctx, void *dest,
+                                                                const void *src, size_t nbytes, int pe,
+                                                                bool blocking = true)
+{
+    char *r = ishmemi::translate(ctx, (char *)dest, pe);
+    __shared__ int rc_sh;
+    __syncthreads();
+    if (ishmemi::block_tid() == 0)
+        rc_sh = !r ? ISHMEM_ERR_INVALID_PE
+                   : (ctx->proxy == nullptr ? ISHMEM_ERR_ARG
+                                            : (nbytes ? ishmemi::proxy_copy(ctx, r, (const char *)src, nbytes, blocking) : 0));
+    __syncthreads();
+    return rc_sh;
+}
+__device__ __forceinline__ int ishmemx_getmem_engine_work_group(const ishmem_ctx_t *ctx, void *dest,
+                                                                const void *src, size_t nbytes, int pe,
+                                                                bool blocking = true)
+{
+    const char *r = ishmemi::translate(ctx, (const char *)src, pe);
+    __shared__ int rc_sh;
+    __syncthreads();
+    if (ishmemi::block_tid() == 0)
+        rc_sh = !r ? ISHMEM_ERR_INVALID_PE
+                   : (ctx->proxy == nullptr ? ISHMEM_ERR_ARG
+                                            : (nbytes ? ishmemi::proxy_copy(ctx, (char *)dest, r, nbytes, blocking) : 0));
+    __syncthreads();
+    return rc_sh;
+}
+/* put through the engine followed by SIGNAL_SET of the signal word, both in the engine's stream
+ * order; non-blocking (the waiter's wait_until on the signal is the completion). */
+__device__ __forceinline__ int ishmemx_putmem_signal_engine_work_group(const ishmem_ctx_t *ctx, void *dest,
+                                                                       const void *src, size_t nbytes,
+                                                                       unsigned long long *sig_addr,
+                                                                       unsigned long long signal, int pe)
+{
+    char *r = ishmemi::translate(ctx, (char *)dest, pe);
+    unsigned long long *rs = ishmemi::translate(ctx, sig_addr, pe);
+    __shared__ int rc_sh;
+    __syncthreads();
+    if (ishmemi::block_tid() == 0)
+        rc_sh = (!r || !rs) ? ISHMEM_ERR_INVALID_PE
+                            : (ctx->proxy == nullptr ? ISHMEM_ERR_ARG
+                                                     : ishmemi::proxy_copy(ctx, r, (const char *)src, nbytes, false, rs, signal));
+    __syncthreads();
+    return rc_sh;
+}
+
 /* ---- ordering --------------------------------------------------------------------------- */
 
 /* fence: this thread's earlier puts are ordered before its later puts and signals. */
 __device__ __forceinline__ void ishmem_fence(const ishmem_ctx_t *) { ishmemi::fence_acq_rel_gpu(); }
 /* quiet: all operations issued by this thread are complete and visible device-wide,
- * including bulk stores left in flight by _nbi calls. */
-__device__ __forceinline__ void ishmem_quiet(const ishmem_ctx_t *)
+ * including bulk stores left in flight by _nbi calls and, for the calling PE, copies handed to
+ * the copy engine by _nbi calls above the cutover (a timeout there is latched in the status
+ * word). */
+__device__ __forceinline__ void ishmem_quiet(const ishmem_ctx_t *ctx)
 {
     ishmemi::bulk_wait<0>();
     ishmemi::fence_proxy_async();
     ishmemi::fence_acq_rel_gpu();
+    if (ctx->proxy != nullptr) (void)ishmemi::proxy_quiet(ctx); /* requests left with the copy engine */
 }
 __device__ __forceinline__ void ishmemx_quiet_work_group(const ishmem_ctx_t *ctx)
 {
@@ -1128,10 +1333,11 @@ __device__ __forceinline__ int bulk_fold_ring(const ishmem_ctx_t *ctx, const cha
 
 /* work-group push of n bytes to ndst destinations dest + delta[q] (q != skip); delta lives in
  * shared memory.  TMA ring for the aligned body when staging is given, else loads/stores with
- * the destinations in the inner loop (see push_bytes). */
+ * the destinations in the inner loop (see push_bytes).  With stride > 1 the caller is block
+ * `first` of `stride` blocks that share the range chunk by chunk. */
 __device__ __forceinline__ int wg_push(const ishmem_ctx_t *ctx, char *dest, const long long *delta, int ndst,
                                        int skip, const char *src, size_t n, ishmemx_staging_t st,
-                                       size_t first = 0, size_t stride = 1)
+                                       size_t first = 0, size_t stride = 1, size_t tile = 16384)
 {
     const unsigned tid = threadIdx.x + blockDim.x * (threadIdx.y + blockDim.y * threadIdx.z);
     const unsigned nthr = blockDim.x * blockDim.y * blockDim.z;
@@ -1152,11 +1358,11 @@ __device__ __forceinline__ int wg_push(const ishmem_ctx_t *ctx, char *dest, cons
         __syncthreads();
         return rc_sh;
     }
-    /* loads/stores: tiles of 16 KiB dealt round-robin (the whole range when stride is 1) */
+    /* loads/stores: tiles of `tile` bytes (a multiple of 16) dealt round-robin (the whole range
+     * when stride is 1) */
     if (stride == 1) {
         push_bytes(dest, delta, ndst, skip, src, n, tid, nthr);
     } else {
-        const size_t tile = 16384;
         for (size_t o = first * tile; o < n; o += stride * tile)
             push_bytes(dest + o, delta, ndst, skip, src + o, (n - o < tile) ? n - o : tile, tid, nthr);
     }

@@ -26,7 +26,8 @@ ISHMEM_MAX_PES = 64
 ISHMEM_TEAM_WORLD, ISHMEM_TEAM_SHARED, ISHMEM_TEAM_INVALID = 0, 1, -1
 ISHMEM_SIGNAL_SET, ISHMEM_SIGNAL_ADD = 0, 1
 ISHMEM_CMP_EQ, ISHMEM_CMP_NE, ISHMEM_CMP_GT, ISHMEM_CMP_GE, ISHMEM_CMP_LT, ISHMEM_CMP_LE = range(6)
-ISHMEMX_WORK_ITEM, ISHMEMX_SUB_GROUP, ISHMEMX_WORK_GROUP, ISHMEMX_WORK_GROUP_BULK = range(4)
+(ISHMEMX_WORK_ITEM, ISHMEMX_SUB_GROUP, ISHMEMX_WORK_GROUP, ISHMEMX_WORK_GROUP_BULK,
+ ISHMEMX_WORK_GROUP_ENGINE) = range(5)
 (ISHMEM_OP_SUM, ISHMEM_OP_MAX, ISHMEM_OP_MIN, ISHMEM_OP_PROD, ISHMEM_OP_AND, ISHMEM_OP_OR,
  ISHMEM_OP_XOR) = range(7)
 (ISHMEM_T_INT32, ISHMEM_T_INT64, ISHMEM_T_FLOAT, ISHMEM_T_DOUBLE, ISHMEM_T_UINT32,
@@ -130,6 +131,10 @@ def _signatures() -> dict[str, tuple[str, list[str]]]:
         "ishmemx_set_collective_geometry": ("status", ["i", "i"]),
         "ishmemx_collective_on_device": ("status", ["i", "i", "p", "p", "z", "i", "i", "i", "i", "i"]),
         "ishmemx_pingpong": ("status", ["i", "i", "p", "p", "z", "i", "i", "p", "p"]),
+        "ishmemx_proxy_start": ("status", []),
+        "ishmemx_proxy_stop": ("status", []),
+        "ishmemx_proxy_stats": ("status", ["p", "p", "p"]),
+        "ishmemx_ring_benchmark": ("status", ["i", "i", "i", "i", "p", "p"]),
         "ishmemx_rma_latency": ("status", ["i", "p", "p", "z", "i", "i", "i", "i", "i", "p"]),
         "ishmemx_jacobi": ("status", ["p", "p", "p", "z", "z", "i", "i", "i", "i", "p"]),
         "ishmemx_jacobi_noalloc": ("status", ["p", "p", "p", "z", "z", "i", "i", "i", "i", "p"]),

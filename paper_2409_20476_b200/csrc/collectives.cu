@@ -18,6 +18,7 @@ struct coll_args {
     int repeat;
     unsigned staging_bytes; /* dynamic shared memory for the TMA push ring (0: loads/stores) */
     unsigned tile_vpt;      /* reduce: 16-byte vectors per thread in one tile */
+    unsigned push_tile;     /* broadcast / fcollect by loads and stores: bytes per tile */
 };
 
 /* local address on `ctx`'s PE of a symmetric address given as PE 0's copy */
@@ -44,7 +45,7 @@ __global__ void __launch_bounds__(1024) k_broadcast(const ishmem_ctx_t *ctxs, co
     /* the root's blocks take chunks of the message round-robin */
     ishmemx_staging_t st = {a.staging_bytes ? dyn_smem : nullptr, a.staging_bytes};
     ishmemi::wg_push(ctx, local_of(ctxs, ctx, a.dest), delta, t.size, ctx->bcast_root_dest ? -1 : a.root,
-                     local_of(ctxs, ctx, a.src), a.n, st, blockIdx.x, gridDim.x);
+                     local_of(ctxs, ctx, a.src), a.n, st, blockIdx.x, gridDim.x, a.push_tile);
 }
 
 /* ---- fcollect: member i's blocks push slices of its source into block i of every dest ---- */
@@ -58,7 +59,7 @@ __global__ void __launch_bounds__(1024) k_fcollect(const ishmem_ctx_t *ctxs, col
     if (!ishmemi::team_deltas(ctx, t, delta)) return;
     ishmemx_staging_t st = {a.staging_bytes ? dyn_smem : nullptr, a.staging_bytes};
     ishmemi::wg_push(ctx, local_of(ctxs, ctx, a.dest) + (size_t)me * a.n, delta, t.size, -1,
-                     local_of(ctxs, ctx, a.src), a.n, st, g, (size_t)a.groups);
+                     local_of(ctxs, ctx, a.src), a.n, st, g, (size_t)a.groups, a.push_tile);
 }
 
 /* ---- reduce ------------------------------------------------------------------------------- */
@@ -220,37 +221,50 @@ static int team_of(ishmem_team_t team, ishmemi_team *out)
     return ISHMEM_OK;
 }
 
-/* blocks per member for `bytes` of work per member */
-static int auto_groups(size_t bytes_per_member, int members)
+/* Launch shape of a push collective (broadcast: 1 pushing member; fcollect: `members`), each
+ * pushing `bytes` to `ndst` destinations.
+ *  - loads/stores (small and medium messages): tiles dealt round-robin to the blocks; the tile
+ *    shrinks from 16 KiB down to 2 KiB so that a medium message still reaches every SM;
+ *  - TMA push ring (one elected thread per block moves the data): only when every block of a
+ *    full grid (one per SM) gets at least 1 MiB of loads plus stores. */
+struct push_shape {
+    int blocks_per_member, threads;
+    unsigned staging, tile;
+};
+static push_shape push_geometry(size_t bytes, int members, int ndst, const void *kernel)
 {
     auto &g = g_ishmem;
-    if (g.coll_groups > 0) return g.coll_groups;
-    size_t want = (bytes_per_member + 32767) / 32768;
-    size_t cap = ((size_t)g.sm_count * 4 + members - 1) / members;
-    if (want < 1) want = 1;
-    return (int)(want < cap ? want : cap);
-}
-
-/* Dynamic shared memory of the push kernels' TMA ring; 0 (loads/stores) for small messages.
- * With the ring one elected thread per block moves the data, so about one block per SM with
- * a deep ring is the right shape: `*blocks` is set accordingly. */
-static unsigned push_staging(size_t bytes_per_member, int members, int *blocks_per_member)
-{
-    auto &g = g_ishmem;
+    push_shape sh = {1, g.coll_threads, 0, 16384};
     static unsigned smem = 0;
     if (!smem) {
         unsigned want = 192 * 1024 + 128;
         if (want > g.max_dyn_smem) want = (unsigned)g.max_dyn_smem;
-        cudaFuncSetAttribute(k_broadcast, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)want);
-        cudaFuncSetAttribute(k_fcollect, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)want);
         smem = want;
     }
-    if (g.coll_groups > 0 || bytes_per_member < (1u << 20)) return 0; /* caller-shaped or small */
-    size_t want_blocks = (bytes_per_member + (256u << 10) - 1) / (256u << 10);
+    if (g.coll_groups > 0) { /* caller-shaped */
+        sh.blocks_per_member = g.coll_groups;
+        return sh;
+    }
+    const size_t work = bytes * (size_t)(1 + ndst) * (size_t)members;
     size_t cap = (size_t)g.sm_count / members;
     if (cap < 1) cap = 1;
-    *blocks_per_member = (int)(want_blocks < cap ? want_blocks : cap);
-    return smem;
+    if (work >= (size_t)g.sm_count << 20 &&
+        cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) == cudaSuccess) {
+        sh.staging = smem;
+        sh.threads = 128;
+        sh.blocks_per_member = (int)cap;
+        return sh;
+    }
+    /* loads/stores: aim at two blocks per SM, at least one tile each */
+    cap = ((size_t)g.sm_count * 2 + members - 1) / members;
+    size_t tile = (bytes / cap + 2047) & ~(size_t)2047;
+    if (tile < 2048) tile = 2048;
+    if (tile > 16384) tile = 16384;
+    size_t want = (bytes + tile - 1) / tile;
+    sh.tile = (unsigned)tile;
+    sh.blocks_per_member = (int)(want < 1 ? 1 : (want < cap * 2 ? want : cap * 2));
+    if (bytes <= 4096 * (size_t)ndst && sh.threads > 256) sh.threads = 256;
+    return sh;
 }
 
 static int launch_sync_kernel(ishmem_team_t team, int repeat)
@@ -337,9 +351,10 @@ extern "C" int ishmem_broadcastmem(ishmem_team_t team, void *dest, const void *s
         a.src = (const char *)src;
         a.n = nbytes;
         a.root = root;
-        int blocks = auto_groups(nbytes, 1);
-        a.staging_bytes = push_staging(nbytes, 1, &blocks);
-        k_broadcast<<<blocks, a.staging_bytes ? 128 : g.coll_threads, a.staging_bytes, s>>>(g.d_ctx, a);
+        const push_shape sh = push_geometry(nbytes, 1, t.size, (const void *)k_broadcast);
+        a.staging_bytes = sh.staging;
+        a.push_tile = sh.tile;
+        k_broadcast<<<sh.blocks_per_member, sh.threads, sh.staging, s>>>(g.d_ctx, a);
         ishmemi_count_launch();
         rc = ishmemi_check_launch("k_broadcast");
     }
@@ -378,9 +393,11 @@ extern "C" int ishmem_fcollectmem(ishmem_team_t team, void *dest, const void *sr
         a.dest = (char *)dest;
         a.src = (const char *)src;
         a.n = nbytes;
-        a.groups = auto_groups(nbytes, t.size);
-        a.staging_bytes = push_staging(nbytes, t.size, &a.groups);
-        k_fcollect<<<a.groups * t.size, a.staging_bytes ? 128 : g.coll_threads, a.staging_bytes, s>>>(g.d_ctx, a);
+        const push_shape sh = push_geometry(nbytes, t.size, t.size, (const void *)k_fcollect);
+        a.groups = sh.blocks_per_member;
+        a.staging_bytes = sh.staging;
+        a.push_tile = sh.tile;
+        k_fcollect<<<a.groups * t.size, sh.threads, sh.staging, s>>>(g.d_ctx, a);
         ishmemi_count_launch();
         rc = ishmemi_check_launch("k_fcollect");
     }
@@ -419,10 +436,30 @@ extern "C" int ishmemx_reduce(ishmem_team_t team, void *dest, const void *src, s
         a.src = sp;
         a.n = nreduce;
         a.duplicated = (algorithm == ISHMEMX_REDUCE_DUPLICATED);
-        a.tile_vpt = 2;
         const size_t per_member = a.duplicated ? bytes : bytes / t.size + 1;
-        a.groups = auto_groups(per_member, t.size);
+        /* loads/stores: tiles of threads x tile_vpt vectors dealt round-robin over all blocks.
+         * Small inputs take one vector per thread in 256-thread blocks, so that a few hundred
+         * KiB already occupy every SM; large ones 512 threads x 2 vectors, 4 blocks per SM. */
         int threads = g.coll_threads > 512 ? 512 : g.coll_threads;
+        a.tile_vpt = 2;
+        const size_t nvec = (bytes + 15) / 16;
+        if (g.coll_groups > 0) {
+            a.groups = g.coll_groups;
+        } else {
+            size_t blocks;
+            if (nvec <= (size_t)g.sm_count * 2 * 256 * (a.duplicated ? t.size : 1)) {
+                threads = threads > 256 ? 256 : threads;
+                a.tile_vpt = 1;
+                blocks = (nvec + threads - 1) / threads;
+            } else {
+                blocks = (nvec + (size_t)threads * 2 - 1) / ((size_t)threads * 2);
+                if (blocks > (size_t)g.sm_count * 4) blocks = (size_t)g.sm_count * 4;
+            }
+            /* the grid is groups x members blocks (in the duplicated form each member's `groups`
+             * blocks sweep all tiles, so the tiles per block come out the same) */
+            blocks = (blocks + t.size - 1) / t.size;
+            a.groups = (int)(blocks < 1 ? 1 : blocks);
+        }
         /* Loads/stores over round-robin tiles are the default; from 64 MiB per member on the
          * TMA fold ring (one block per SM) is at least as fast.  ISHMEM_REDUCE_BULK=0/1 forces. */
         static const char *env_bulk = getenv("ISHMEM_REDUCE_BULK");

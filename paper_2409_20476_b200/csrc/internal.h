@@ -48,6 +48,7 @@ struct ishmemi_state {
 
     ishmemi_team teams[ISHMEM_MAX_TEAMS] = {};
     size_t cutover[3] = {0, 0, 0};
+    size_t wg_cutover = (size_t)-1; /* device-initiated work-group put/get: bytes from which the engine is used */
     int coll_groups = 0, coll_threads = 512;
     int bcast_root_dest = 1;
     unsigned long long wait_limit_ns = 2000000000ull;
@@ -85,5 +86,8 @@ void ishmemi_push_ctx();                         /* re-upload host contexts to t
 void ishmemi_count_launch(unsigned n = 1);
 int ishmemi_check_launch(const char *what);      /* cudaGetLastError -> status */
 int ishmemi_engine_copy(int my_pe, void *dst, const void *src, size_t n, bool blocking);
+/* reverse-offload proxy (proxy.cu) */
+void ishmemi_proxy_finalize();
+void ishmemi_proxy_set_cutover(size_t nbytes);
 
 #endif

@@ -121,6 +121,10 @@ __global__ void __launch_bounds__(1024) k_rma_latency(const ishmem_ctx_t *ctxs, 
                 else ishmemx_putmem_sub_group(ctx, dest, src, nbytes, pe);
                 ishmem_quiet(ctx);
             }
+        } else if (LEVEL == ISHMEMX_WORK_GROUP_ENGINE) {
+            int rc = is_get ? ishmemx_getmem_engine_work_group(ctx, dest, src, nbytes, pe)
+                            : ishmemx_putmem_engine_work_group(ctx, dest, src, nbytes, pe);
+            if (rc) break;
         } else {
             int rc = is_get ? ishmemx_getmem_work_group(ctx, dest, src, nbytes, pe, st)
                             : ishmemx_putmem_work_group(ctx, dest, src, nbytes, pe, st);
@@ -139,8 +143,9 @@ extern "C" int ishmemx_rma_latency(int my_pe, void *dest, const void *src, size_
     auto &g = g_ishmem;
     if (ishmemi_check_pe(my_pe) || ishmemi_check_pe(pe)) return ISHMEM_ERR_INVALID_PE;
     if (iters < 1 || threads < 1 || threads > 1024 || !ns_per_op) return ISHMEM_ERR_ARG;
-    if (level < ISHMEMX_WORK_ITEM || level > ISHMEMX_WORK_GROUP_BULK) return ISHMEM_ERR_ARG;
+    if (level < ISHMEMX_WORK_ITEM || level > ISHMEMX_WORK_GROUP_ENGINE) return ISHMEM_ERR_ARG;
     if (level == ISHMEMX_SUB_GROUP && threads < 32) return ISHMEM_ERR_ARG;
+    if (level == ISHMEMX_WORK_GROUP_ENGINE && g.h_ctx[0].proxy == nullptr) return ISHMEM_ERR_ARG;
     if (nbytes && (!dest || !src)) return ISHMEM_ERR_ARG;
     if (ishmemi_sym_offset(is_get ? src : (const void *)dest, nbytes) < 0) return ISHMEM_ERR_NOT_SYMMETRIC;
     char *dl = ishmemi_localise(dest, nbytes, my_pe);
@@ -159,6 +164,10 @@ extern "C" int ishmemx_rma_latency(int my_pe, void *dest, const void *src, size_
         break;
     case ISHMEMX_WORK_GROUP:
         k_rma_latency<ISHMEMX_WORK_GROUP><<<1, threads, 0, s>>>(ctxs, my_pe, dl, sl, nbytes, pe, is_get, iters, 0, out);
+        break;
+    case ISHMEMX_WORK_GROUP_ENGINE:
+        k_rma_latency<ISHMEMX_WORK_GROUP_ENGINE><<<1, threads, 0, s>>>(ctxs, my_pe, dl, sl, nbytes, pe, is_get, iters, 0,
+                                                                        out);
         break;
     default: {
         static unsigned smem = 0;
@@ -191,6 +200,7 @@ struct jacobi_args {
     int iters, overlap, groups;
     unsigned long long *done;     /* scratch [npes*groups]: sweeps completed by each block */
     double *partial;              /* scratch [npes*groups]: residual partial sums */
+    int sliding;                  /* even nx: interior rows by the register sliding window */
 };
 
 __device__ __forceinline__ void strip_of(size_t ny, int npes, int pe, size_t *first, size_t *rows)
@@ -243,7 +253,146 @@ __device__ __forceinline__ void jacobi_row(const double *cur, double *nxt, size_
     }
 }
 
-__global__ void __launch_bounds__(1024) k_jacobi(const ishmem_ctx_t *ctxs, jacobi_args a)
+
+/* ---- register sliding window ------------------------------------------------------------------
+ * Rows [ra, rb) of the strip (local row numbers) for even nx.  Each warp takes tiles of 60 output
+ * columns: its 32 lanes load the 64 columns around them (one aligned double2 per lane, so the
+ * tile's left and right neighbour columns are lanes 0 and 31) and walk down the rows.  The rows
+ * above and at the current position stay in registers, DEPTH further rows are already on their
+ * way (independent 16-byte loads, refilled one per step), and the left/right neighbours of a
+ * lane's pair come from the adjacent lanes by shuffle; lanes 1..30 store.  Every element of `cur`
+ * is loaded once per sweep (plus 4 of every 64 a second time, from cache), every element of `nxt`
+ * stored once, and there is no block-wide barrier inside.  The arithmetic is the same expression,
+ * in the same order, as jacobi_row.  fixed0 / fixed1: local numbers of the rows that are the
+ * grid's first and last row (kept as they are), or ~0u when they lie outside this strip.
+ * Returns this thread's share of the squared update when want_res. */
+template <int DEPTH>
+static __device__ __noinline__ double jacobi_march(const double *cur, double *nxt, unsigned ra, unsigned rb,
+                                                   unsigned fixed0, unsigned fixed1, unsigned nx, bool want_res)
+{
+    double acc = 0.0;
+    if (rb <= ra) return acc;
+    const unsigned lane = threadIdx.x & 31u, nwarps = blockDim.x >> 5;
+    const unsigned ntiles = (nx + 59u) / 60u;
+    const unsigned full = 0xffffffffu;
+    const double2 zero = make_double2(0.0, 0.0);
+    for (unsigned t = threadIdx.x >> 5; t < ntiles; t += nwarps) {
+        const int jl = (int)(t * 60u) - 2 + 2 * (int)lane; /* first column of this lane's pair */
+        const bool ld_ok = jl >= 0 && jl < (int)nx;
+        const bool st_ok = ld_ok && lane >= 1 && lane <= 30;
+        const unsigned j = ld_ok ? (unsigned)jl : 0u;
+        const double *pl = cur + (size_t)(ra - 1) * nx + j; /* next row to load */
+        double2 up = ld_ok ? *(const double2 *)pl : zero;
+        pl += nx;
+        double2 mid = ld_ok ? *(const double2 *)pl : zero;
+        pl += nx;
+        double2 f[DEPTH];
+        unsigned loaded = ra + 1; /* local row number pl points at */
+#pragma unroll
+        for (int s = 0; s < DEPTH; ++s) {
+            f[s] = zero;
+            if (loaded <= rb) {
+                if (ld_ok) f[s] = *(const double2 *)pl;
+                pl += nx;
+                ++loaded;
+            }
+        }
+        double ml = __shfl_up_sync(full, mid.y, 1), mr = __shfl_down_sync(full, mid.x, 1);
+        double *po = nxt + (size_t)ra * nx + j;
+        for (unsigned r = ra; r < rb; r += DEPTH) {
+#pragma unroll
+            for (int s = 0; s < DEPTH; ++s) {
+                if (r + s < rb) { /* uniform over the warp */
+                    const double2 dn = f[s];
+                    if (loaded <= rb) { /* refill this slot with the row DEPTH further down */
+                        if (ld_ok) f[s] = *(const double2 *)pl;
+                        pl += nx;
+                        ++loaded;
+                    }
+                    double2 o = mid;
+                    if (r + s != fixed0 && r + s != fixed1) {
+                        if (j != 0) o.x = 0.25 * ((up.x + dn.x) + (ml + mid.y));
+                        if (j + 2 != nx) o.y = 0.25 * ((up.y + dn.y) + (mid.x + mr));
+                        if (want_res && st_ok) {
+                            const double dx = o.x - mid.x, dy = o.y - mid.y;
+                            acc += dx * dx;
+                            acc += dy * dy;
+                        }
+                    }
+                    if (st_ok) *(double2 *)po = o;
+                    po += nx;
+                    up = mid;
+                    mid = dn;
+                    ml = __shfl_up_sync(full, dn.y, 1);
+                    mr = __shfl_down_sync(full, dn.x, 1);
+                }
+            }
+        }
+    }
+    return acc;
+}
+
+/* The first and the last row of a block's range (local rows rA and rB; rB == ~0u: only rA), which
+ * are computed after the neighbours' rows have arrived.  Same 60-column tiles and shuffles as
+ * jacobi_march; the loads of U tiles x 2 rows x 3 source rows are all issued before the first
+ * use, since there is nothing to slide along. */
+template <int U>
+__device__ __forceinline__ double jacobi_edge_rows(const double *cur, double *nxt, unsigned rA, unsigned rB,
+                                                   unsigned fixed0, unsigned fixed1, unsigned nx, bool want_res)
+{
+    double acc = 0.0;
+    const unsigned lane = threadIdx.x & 31u, nwarps = blockDim.x >> 5;
+    const unsigned ntiles = (nx + 59u) / 60u;
+    const unsigned full = 0xffffffffu;
+    const double2 zero = make_double2(0.0, 0.0);
+    const unsigned rows[2] = {rA, rB};
+    for (unsigned t0 = (threadIdx.x >> 5) * U; t0 < ntiles; t0 += nwarps * U) {
+        double2 up[U][2], mid[U][2], dn[U][2];
+#pragma unroll
+        for (int k = 0; k < U; ++k) {
+            const int jl = (int)((t0 + k) * 60u) - 2 + 2 * (int)lane;
+            const bool ld_ok = t0 + k < ntiles && jl >= 0 && jl < (int)nx;
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+                up[k][e] = mid[k][e] = dn[k][e] = zero;
+                if (ld_ok && rows[e] != ~0u) {
+                    const double *pm = cur + (size_t)rows[e] * nx + jl;
+                    up[k][e] = *(const double2 *)(pm - nx);
+                    mid[k][e] = *(const double2 *)pm;
+                    dn[k][e] = *(const double2 *)(pm + nx);
+                }
+            }
+        }
+#pragma unroll
+        for (int k = 0; k < U; ++k) {
+            const int jl = (int)((t0 + k) * 60u) - 2 + 2 * (int)lane;
+            const bool st_ok = t0 + k < ntiles && jl >= 0 && jl < (int)nx && lane >= 1 && lane <= 30;
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+                const double2 m = mid[k][e];
+                const double ml = __shfl_up_sync(full, m.y, 1), mr = __shfl_down_sync(full, m.x, 1);
+                if (!st_ok || rows[e] == ~0u) continue;
+                double2 o = m;
+                if (rows[e] != fixed0 && rows[e] != fixed1) {
+                    if (jl != 0) o.x = 0.25 * ((up[k][e].x + dn[k][e].x) + (ml + m.y));
+                    if (jl + 2 != (int)nx) o.y = 0.25 * ((up[k][e].y + dn[k][e].y) + (m.x + mr));
+                    if (want_res) {
+                        const double dx = o.x - m.x, dy = o.y - m.y;
+                        acc += dx * dx;
+                        acc += dy * dy;
+                    }
+                }
+                *(double2 *)(nxt + (size_t)rows[e] * nx + jl) = o;
+            }
+        }
+    }
+    return acc;
+}
+
+/* MAXT: largest block the instance may be launched with (it fixes the registers per thread);
+ * DEPTH: rows in flight per lane in the sliding window */
+template <int MAXT, int DEPTH>
+__global__ void __launch_bounds__(MAXT) k_jacobi(const ishmem_ctx_t *ctxs, jacobi_args a)
 {
     const int P = ctxs[0].npes, G = a.groups;
     const int p = (int)blockIdx.x / G, g = (int)blockIdx.x % G;
@@ -260,6 +409,11 @@ __global__ void __launch_bounds__(1024) k_jacobi(const ishmem_ctx_t *ctxs, jacob
     unsigned long long *done = a.done + (size_t)p * G;
     double acc = 0.0;
     __shared__ int give_up;
+    /* even nx: register sliding window; odd nx: row by row with scalar accesses */
+    const bool slide = a.sliding != 0;
+    /* local numbers of the grid's first and last row when they belong to this strip */
+    const unsigned fixed0 = (first == 0) ? 1u : ~0u;
+    const unsigned fixed1 = (first + rows == a.ny) ? (unsigned)rows : ~0u;
     if (tid == 0) give_up = 0;
     __syncthreads();
 
@@ -277,11 +431,18 @@ __global__ void __launch_bounds__(1024) k_jacobi(const ishmem_ctx_t *ctxs, jacob
             ishmemx_putmem_signal_work_group(ctx, (void *)cur, cur + rows * nx, nx * 8, sig + 0, round,
                                              ISHMEM_SIGNAL_SET, p + 1);
         /* (b) rows that need nobody else's data of this sweep */
-        if (a.overlap)
-            for (size_t r = r0 + 1; r + 1 < r1; ++r) {
-                const size_t gi = first + r - 1;
-                jacobi_row(cur, nxt, r, nx, gi == 0 || gi == a.ny - 1, tid, nthr, want_res, &acc);
+        if (a.overlap) {
+            if (slide) {
+                if (r1 > r0 + 2)
+                    acc += jacobi_march<DEPTH>(cur, nxt, (unsigned)r0 + 1, (unsigned)r1 - 1, fixed0, fixed1, (unsigned)nx,
+                                           want_res);
+            } else {
+                for (size_t r = r0 + 1; r + 1 < r1; ++r) {
+                    const size_t gi = first + r - 1;
+                    jacobi_row(cur, nxt, r, nx, gi == 0 || gi == a.ny - 1, tid, nthr, want_res, &acc);
+                }
             }
+        }
         /* (c) wait for the rows above and below this block's range: neighbouring blocks of
          * the same PE publish a sweep counter, neighbouring PEs signal their halo */
         if (tid == 0) {
@@ -309,7 +470,14 @@ __global__ void __launch_bounds__(1024) k_jacobi(const ishmem_ctx_t *ctxs, jacob
         __syncthreads();
         if (give_up) break;
         /* (d) the remaining rows */
-        if (a.overlap) {
+        if (slide && !a.overlap) {
+            acc += jacobi_march<DEPTH>(cur, nxt, (unsigned)r0, (unsigned)r1, fixed0, fixed1, (unsigned)nx, want_res);
+        } else if (slide) {
+            if (r1 > r0)
+                acc += jacobi_edge_rows<(MAXT <= 512) ? 2 : 1>(cur, nxt, (unsigned)r0,
+                                                               (r1 - 1 > r0) ? (unsigned)r1 - 1 : ~0u, fixed0, fixed1,
+                                                               (unsigned)nx, want_res);
+        } else if (a.overlap) {
             if (r1 > r0) {
                 size_t gi = first + r0 - 1;
                 jacobi_row(cur, nxt, r0, nx, gi == 0 || gi == a.ny - 1, tid, nthr, want_res, &acc);
@@ -343,31 +511,35 @@ __global__ void __launch_bounds__(1024) k_jacobi(const ishmem_ctx_t *ctxs, jacob
     }
 }
 
-extern "C" int ishmemx_jacobi(double *buf0, double *buf1, uint64_t *sig, size_t ny, size_t nx, int iters,
-                              int overlap, int groups_per_pe, int threads, double *residual_sq_host)
+/* argument checks shared by the two entry points; *groups_per_pe is clamped to the shortest strip */
+static int jacobi_check(double *buf0, double *buf1, uint64_t *sig, size_t ny, size_t nx, int iters,
+                        int *groups_per_pe, int threads)
 {
-    ISHMEMI_REQUIRE_INIT();
     auto &g = g_ishmem;
     const int P = g.npes;
     if (ny < 3 || nx < 3 || iters < 0 || (size_t)P > ny) return ISHMEM_ERR_ARG;
-    if (threads < 32 || threads > 1024 || threads % 32 || groups_per_pe < 1) return ISHMEM_ERR_ARG;
+    if (threads < 32 || threads > 1024 || threads % 32 || *groups_per_pe < 1) return ISHMEM_ERR_ARG;
     const size_t rows_min = ny / P, rows_max = (ny + P - 1) / P;
-    if ((size_t)groups_per_pe > rows_min) groups_per_pe = (int)rows_min;
+    if ((size_t)*groups_per_pe > rows_min) *groups_per_pe = (int)rows_min;
     const size_t bytes = (rows_max + 2) * nx * 8;
     if ((uintptr_t)buf0 % 16 || (uintptr_t)buf1 % 16 || (uintptr_t)sig % 8) return ISHMEM_ERR_ALIGN;
     if (ishmemi_sym_offset(buf0, bytes) < 0 || ishmemi_sym_offset(buf1, bytes) < 0 ||
         ishmemi_sym_offset(sig, 16) < 0)
         return ISHMEM_ERR_NOT_SYMMETRIC;
-    const size_t nblocks = (size_t)P * groups_per_pe;
-    /* scratch: per-block sweep counters and residual partials */
-    char *scratch = nullptr;
-    ISHMEMI_CUDA(cudaMalloc((void **)&scratch, nblocks * 16));
+    return ISHMEM_OK;
+}
+
+/* clears the scratch, launches the persistent kernel on the team stream and waits for it;
+ * `scratch` holds nblocks sweep counters followed by nblocks residual partials */
+static int jacobi_launch(double *buf0, double *buf1, uint64_t *sig, size_t ny, size_t nx, int iters, int overlap,
+                         int groups_per_pe, int threads, void *scratch, jacobi_args *out_args)
+{
+    auto &g = g_ishmem;
+    const size_t nblocks = (size_t)g.npes * groups_per_pe;
     cudaStream_t s;
     int rc = ishmemi_team_stream_begin(ISHMEM_TEAM_WORLD, &s);
-    if (rc) {
-        cudaFree(scratch);
-        return rc;
-    }
+    if (rc) return rc;
+    /* the counters must start from zero */
     rc = ishmemi_cuda(cudaMemsetAsync(scratch, 0, nblocks * 16, s), "cudaMemsetAsync");
     jacobi_args a = {};
     a.buf0 = buf0;
@@ -379,16 +551,39 @@ extern "C" int ishmemx_jacobi(double *buf0, double *buf1, uint64_t *sig, size_t 
     a.overlap = overlap;
     a.groups = groups_per_pe;
     a.done = (unsigned long long *)scratch;
-    a.partial = (double *)(scratch + nblocks * 8);
+    a.partial = (double *)((char *)scratch + nblocks * 8);
+    a.sliding = (nx % 2 == 0 && nx < 0x7fffffffu && ny < 0x7fffffffu);
     const ishmem_ctx_t *ctxs = g.d_ctx;
     void *params[] = {(void *)&ctxs, (void *)&a};
     if (!rc)
-        rc = ishmemi_cuda(cudaLaunchCooperativeKernel((void *)k_jacobi, dim3((unsigned)nblocks), dim3(threads),
-                                                      params, 0, s),
+    {
+        /* blocks of at most 512 threads that have an SM to themselves get 128 registers per thread
+         * and a deeper window; everything else the 1024-thread instance */
+        const bool wide = threads <= 512 && nblocks <= (size_t)g.sm_count;
+        void *kernel = wide ? (void *)k_jacobi<512, 8> : (void *)k_jacobi<1024, 4>;
+        rc = ishmemi_cuda(cudaLaunchCooperativeKernel(kernel, dim3((unsigned)nblocks), dim3(threads), params, 0, s),
                           "cudaLaunchCooperativeKernel(jacobi)");
+    }
     ishmemi_count_launch();
     ishmemi_team_stream_end();
     if (!rc) rc = ishmemi_cuda(cudaStreamSynchronize(s), "cudaStreamSynchronize");
+    *out_args = a;
+    return rc;
+}
+
+extern "C" int ishmemx_jacobi(double *buf0, double *buf1, uint64_t *sig, size_t ny, size_t nx, int iters,
+                              int overlap, int groups_per_pe, int threads, double *residual_sq_host)
+{
+    ISHMEMI_REQUIRE_INIT();
+    auto &g = g_ishmem;
+    int rc = jacobi_check(buf0, buf1, sig, ny, nx, iters, &groups_per_pe, threads);
+    if (rc) return rc;
+    const size_t nblocks = (size_t)g.npes * groups_per_pe;
+    /* scratch: per-block sweep counters and residual partials */
+    char *scratch = nullptr;
+    ISHMEMI_CUDA(cudaMalloc((void **)&scratch, nblocks * 16));
+    jacobi_args a;
+    rc = jacobi_launch(buf0, buf1, sig, ny, nx, iters, overlap, groups_per_pe, threads, scratch, &a);
     if (!rc && residual_sq_host) {
         std::vector<double> part(nblocks);
         rc = ishmemi_cuda(cudaMemcpy(part.data(), a.partial, nblocks * 8, cudaMemcpyDeviceToHost), "cudaMemcpy");
@@ -433,48 +628,19 @@ extern "C" int ishmemx_jacobi_noalloc(double *buf0, double *buf1, uint64_t *sig,
 {
     ISHMEMI_REQUIRE_INIT();
     auto &g = g_ishmem;
-    const int P = g.npes;
-    if (ny < 3 || nx < 3 || iters < 0 || (size_t)P > ny) return ISHMEM_ERR_ARG;
-    if (threads < 32 || threads > 1024 || threads % 32 || groups_per_pe < 1) return ISHMEM_ERR_ARG;
-    const size_t rows_min = ny / P, rows_max = (ny + P - 1) / P;
-    if ((size_t)groups_per_pe > rows_min) groups_per_pe = (int)rows_min;
-    const size_t nblocks = (size_t)P * groups_per_pe;
+    int rc = jacobi_check(buf0, buf1, sig, ny, nx, iters, &groups_per_pe, threads);
+    if (rc == ISHMEM_ERR_ARG) return rc;
+    const size_t nblocks = (size_t)g.npes * groups_per_pe;
     if (nblocks > ISHMEMX_JACOBI_NOALLOC_MAX_BLOCKS) {
         g.last_cuda_error = "ishmemx_jacobi_noalloc: npes * groups_per_pe exceeds the fixed scratch (2048 blocks)";
         return ISHMEM_ERR_ARG;
     }
-    const size_t bytes = (rows_max + 2) * nx * 8;
-    if ((uintptr_t)buf0 % 16 || (uintptr_t)buf1 % 16 || (uintptr_t)sig % 8) return ISHMEM_ERR_ALIGN;
-    if (ishmemi_sym_offset(buf0, bytes) < 0 || ishmemi_sym_offset(buf1, bytes) < 0 ||
-        ishmemi_sym_offset(sig, 16) < 0)
-        return ISHMEM_ERR_NOT_SYMMETRIC;
-    void *scratch = nullptr;
-    int rc = jacobi_scratch_for_current_device(&scratch);
     if (rc) return rc;
-    cudaStream_t s;
-    if ((rc = ishmemi_team_stream_begin(ISHMEM_TEAM_WORLD, &s))) return rc;
-    /* the array keeps the previous call's counters: they must start from zero */
-    rc = ishmemi_cuda(cudaMemsetAsync(scratch, 0, nblocks * 16, s), "cudaMemsetAsync");
-    jacobi_args a = {};
-    a.buf0 = buf0;
-    a.buf1 = buf1;
-    a.sig = (unsigned long long *)sig;
-    a.ny = ny;
-    a.nx = nx;
-    a.iters = iters;
-    a.overlap = overlap;
-    a.groups = groups_per_pe;
-    a.done = (unsigned long long *)scratch;
-    a.partial = (double *)((char *)scratch + nblocks * 8);
-    const ishmem_ctx_t *ctxs = g.d_ctx;
-    void *params[] = {(void *)&ctxs, (void *)&a};
-    if (!rc)
-        rc = ishmemi_cuda(cudaLaunchCooperativeKernel((void *)k_jacobi, dim3((unsigned)nblocks), dim3(threads),
-                                                      params, 0, s),
-                          "cudaLaunchCooperativeKernel(jacobi_noalloc)");
-    ishmemi_count_launch();
-    ishmemi_team_stream_end();
-    if (!rc) rc = ishmemi_cuda(cudaStreamSynchronize(s), "cudaStreamSynchronize");
+    void *scratch = nullptr;
+    if ((rc = jacobi_scratch_for_current_device(&scratch))) return rc;
+    /* the array keeps the previous call's counters; jacobi_launch clears the part this call uses */
+    jacobi_args a;
+    rc = jacobi_launch(buf0, buf1, sig, ny, nx, iters, overlap, groups_per_pe, threads, scratch, &a);
     if (!rc && residual_sq_host) {
         double part[ISHMEMX_JACOBI_NOALLOC_MAX_BLOCKS];
         rc = ishmemi_cuda(cudaMemcpy(part, a.partial, nblocks * 8, cudaMemcpyDeviceToHost), "cudaMemcpy");

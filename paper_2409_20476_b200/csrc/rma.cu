@@ -74,6 +74,10 @@ __global__ void __launch_bounds__(1024) k_rma(const ishmem_ctx_t *ctxs, rma_args
                  (unsigned long long)a.groups * wpb, &begin, &len);
         if (a.is_get) ishmemx_getmem_sub_group(ctx, dest + begin, src + begin, len, target);
         else ishmemx_putmem_sub_group(ctx, dest + begin, src + begin, len, target);
+    } else if (LEVEL == ISHMEMX_WORK_GROUP_ENGINE) {
+        slice_of(a.nbytes, (unsigned long long)g, (unsigned long long)a.groups, &begin, &len);
+        if (a.is_get) ishmemx_getmem_engine_work_group(ctx, dest + begin, src + begin, len, target);
+        else ishmemx_putmem_engine_work_group(ctx, dest + begin, src + begin, len, target);
     } else {
         ishmemx_staging_t st = {nullptr, 0};
         if (LEVEL == ISHMEMX_WORK_GROUP_BULK) {
@@ -147,6 +151,10 @@ static int launch_rma(cudaStream_t s, rma_args a, int level, int threads, unsign
     case ISHMEMX_WORK_GROUP_BULK:
         a.staging_bytes = bulk_staging_bytes();
         k_rma<ISHMEMX_WORK_GROUP_BULK><<<blocks, threads, a.staging_bytes, s>>>(ctxs, a);
+        break;
+    case ISHMEMX_WORK_GROUP_ENGINE:
+        if (g_ishmem.h_ctx[0].proxy == nullptr) return ISHMEM_ERR_ARG; /* no host proxy running */
+        k_rma<ISHMEMX_WORK_GROUP_ENGINE><<<blocks, threads, 0, s>>>(ctxs, a);
         break;
     default: return ISHMEM_ERR_ARG;
     }

@@ -40,13 +40,15 @@ def run_gpu(grid, npes, iters, overlap, groups, threads):
 
 
 @pytest.mark.parametrize("overlap", [1, 0])
-@pytest.mark.parametrize("ny,nx,npes,groups", [(64, 48, 12, 1), (200, 130, 12, 3), (257, 33, 5, 4),
-                                               (40, 40, 1, 2), (1000, 512, 12, 8)])
-def test_jacobi_matches_oracle(ny, nx, npes, groups, overlap):
+@pytest.mark.parametrize("ny,nx,npes,groups,threads", [
+    (64, 48, 12, 1, 128), (200, 130, 12, 3, 128), (257, 33, 5, 4, 128),       # odd nx: row-by-row path
+    (40, 40, 1, 2, 128), (1000, 512, 12, 8, 128), (301, 1234, 7, 3, 256),      # sliding window, 128 registers
+    (600, 256, 12, 13, 128), (300, 4096, 4, 2, 1024), (97, 62, 3, 5, 1024)])   # sliding window, 64 registers
+def test_jacobi_matches_oracle(ny, nx, npes, groups, threads, overlap):
     grid = inputs.jacobi_grid(inputs.SEED_C5, ny, nx)
     iters = 21
     exp, exp_res = orc.jacobi(grid, iters)
-    got, res = run_gpu(grid, npes, iters, overlap, groups, 128)
+    got, res = run_gpu(grid, npes, iters, overlap, groups, threads)
     assert got.tobytes() == exp.tobytes()
     assert abs(res - exp_res) <= 1e-6 * exp_res
 
