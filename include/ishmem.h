@@ -225,7 +225,14 @@ size_t ishmemx_get_cutover(int which);
  * only), the proxy issues cudaMemcpyAsync on the issuing PE's copy-engine stream, and the reply
  * is written behind the copy in stream order into a word the GPU thread polls.  Both calls
  * block until the device is idle; ishmem_finalize stops a running proxy.  Allocates pinned host
- * memory (ring of 1024 requests, 65536 reply words). */
+ * memory (ring of 8192 requests, 65536 reply words).
+ * Progress: a kernel that waits for the proxy depends on the proxy's streams being served while
+ * it runs.  CUDA multiplexes streams onto a few hardware queues (8 by default); work already
+ * queued BEHIND the waiting kernel, on a stream that shares a queue with a proxy stream, blocks
+ * the proxy's copy, and the wait then ends only by its time limit (ISHMEM_ERR_TIMEOUT latched,
+ * nothing hangs).  Either queue nothing behind such a kernel, or start the process with
+ * CUDA_DEVICE_MAX_CONNECTIONS=32 (read when the CUDA context is created; measured on B200:
+ * 32 launches queued back to back, no time-outs with 32 queues, sporadic ones with 8). */
 int ishmemx_proxy_start(void);
 int ishmemx_proxy_stop(void);
 /* Requests served and copies started since ishmemx_proxy_start (HOST pointers, may be NULL);

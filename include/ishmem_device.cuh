@@ -477,6 +477,18 @@ __device__ __forceinline__ void st_release_sys(unsigned long long *p, unsigned l
     asm volatile("st.release.sys.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
 }
 
+/* Polls of host memory cross the bus: every waiter backs off from 200 ns to 6.4 us between
+ * polls, so that many waiters cannot crowd out the requests themselves. */
+struct host_poll_backoff {
+    unsigned ns;
+    __device__ __forceinline__ host_poll_backoff() : ns(200u) {}
+    __device__ __forceinline__ void pause()
+    {
+        __nanosleep(ns);
+        if (ns < 6400u) ns <<= 1;
+    }
+};
+
 /* Posts one request: one fetch-and-increment allocates the slot, the message is written with
  * plain stores and published by the release store of its sequence number.  Flow control (the
  * host must have consumed the slot's previous message) is checked against a cached copy of the
@@ -490,7 +502,10 @@ __device__ __forceinline__ int proxy_post(const ishmem_ctx_t *ctx, unsigned op, 
     const unsigned long long t = atomicAdd(px->head, 1ull);
     if (t - ld_relaxed(px->tail_cache) >= px->ring_slots) {
         deadline dl(ctx->wait_limit_ns);
+        host_poll_backoff bo;
         for (;;) {
+            /* somebody else may have refreshed the cached tail meanwhile */
+            if (t - ld_relaxed(px->tail_cache) < px->ring_slots) break;
             const unsigned long long tail = ld_acquire_sys(px->tail_pub);
             if (t - tail < px->ring_slots) {
                 atomicMax(px->tail_cache, tail);
@@ -500,7 +515,7 @@ __device__ __forceinline__ int proxy_post(const ishmem_ctx_t *ctx, unsigned op, 
                 latch_error(ctx, ISHMEM_ERR_TIMEOUT);
                 return ISHMEM_ERR_TIMEOUT; /* the slot stays unwritten: the proxy stops at it */
             }
-            __nanosleep(500);
+            bo.pause();
         }
     }
     ishmemi_request *slot = px->ring + (t & (px->ring_slots - 1));
@@ -521,10 +536,11 @@ __device__ __forceinline__ int proxy_wait(const ishmem_ctx_t *ctx, unsigned long
     const ishmemi_proxy_t *px = ctx->proxy;
     const unsigned long long *word = px->comp + (c & (px->comp_slots - 1));
     deadline dl(ctx->wait_limit_ns);
+    host_poll_backoff bo;
     for (;;) {
         if (ld_acquire_sys(word) >= c + 1) return 0;
         if (dl.expired()) break;
-        __nanosleep(200);
+        bo.pause();
     }
     latch_error(ctx, ISHMEM_ERR_TIMEOUT);
     return ISHMEM_ERR_TIMEOUT;
@@ -538,6 +554,7 @@ __device__ __forceinline__ int proxy_quiet(const ishmem_ctx_t *ctx)
     const unsigned long long want = ld_relaxed(px->nbi_issued + ctx->my_pe);
     if (ld_relaxed(px->nbi_seen + ctx->my_pe) >= want) return 0;
     deadline dl(ctx->wait_limit_ns);
+    host_poll_backoff bo;
     for (;;) {
         const unsigned long long done = ld_acquire_sys(px->nbi_done + ctx->my_pe);
         if (done >= want) {
@@ -545,7 +562,7 @@ __device__ __forceinline__ int proxy_quiet(const ishmem_ctx_t *ctx)
             return 0;
         }
         if (dl.expired()) break;
-        __nanosleep(200);
+        bo.pause();
     }
     latch_error(ctx, ISHMEM_ERR_TIMEOUT);
     return ISHMEM_ERR_TIMEOUT;
@@ -840,7 +857,11 @@ __device__ __forceinline__ void ishmem_quiet(const ishmem_ctx_t *ctx)
 }
 __device__ __forceinline__ void ishmemx_quiet_work_group(const ishmem_ctx_t *ctx)
 {
-    ishmem_quiet(ctx);
+    ishmemi::bulk_wait<0>();
+    ishmemi::fence_proxy_async();
+    ishmemi::fence_acq_rel_gpu();
+    /* one thread waits for the copy engine on behalf of the group */
+    if (ctx->proxy != nullptr && ishmemi::block_tid() == 0) (void)ishmemi::proxy_quiet(ctx);
     __syncthreads();
 }
 
@@ -858,12 +879,16 @@ __device__ __forceinline__ void ishmem_putmem_signal(const ishmem_ctx_t *ctx, vo
     ishmemi::signal_update(rs, signal, sig_op); /* release: payload first */
 }
 /* All threads copy; after a block barrier the leader releases the signal word, so the
- * waiter that acquires it sees the whole payload. */
+ * waiter that acquires it sees the whole payload.  Above the work-group cutover (host proxy
+ * running, SIGNAL_SET) payload and signal go through the copy engine instead, in its stream
+ * order, and the call returns once the request is posted. */
 __device__ __forceinline__ int ishmemx_putmem_signal_work_group(
     const ishmem_ctx_t *ctx, void *dest, const void *src, size_t nbytes,
     unsigned long long *sig_addr, unsigned long long signal, int sig_op, int pe,
     ishmemx_staging_t staging = {nullptr, 0})
 {
+    if (ctx->proxy != nullptr && nbytes >= ctx->proxy->wg_cutover && sig_op == ISHMEM_SIGNAL_SET)
+        return ishmemx_putmem_signal_engine_work_group(ctx, dest, src, nbytes, sig_addr, signal, pe);
     char *r = ishmemi::translate(ctx, (char *)dest, pe);
     unsigned long long *rs = ishmemi::translate(ctx, sig_addr, pe);
     int rc = ISHMEM_ERR_INVALID_PE;

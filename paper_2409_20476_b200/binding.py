@@ -11,7 +11,17 @@ the first call raises.
 from __future__ import annotations
 
 import ctypes as C
+import os
 from pathlib import Path
+
+# Device code that waits for the host proxy (ishmemx_proxy_start) needs the proxy's copy-engine
+# streams to make progress while the waiting kernel runs.  CUDA maps streams onto a small number
+# of hardware queues (8 unless told otherwise); work queued behind the waiting kernel on a stream
+# that shares a queue with a proxy stream then sits in front of the proxy's copy and the wait
+# can only end by its time limit.  32 queues give every stream of this library its own.  The
+# variable is read when the CUDA context is created, so it only helps if this module is
+# imported before the first CUDA call of the process; a value set by the user is kept.
+os.environ.setdefault("CUDA_DEVICE_MAX_CONNECTIONS", "32")
 
 import numpy as np
 

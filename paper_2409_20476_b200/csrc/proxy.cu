@@ -18,7 +18,7 @@
 
 #include "internal.h"
 
-#define PROXY_RING_SLOTS 1024u
+#define PROXY_RING_SLOTS 8192u
 #define PROXY_COMP_SLOTS 65536u
 
 typedef CUresult (*write_value64_fn)(CUstream, CUdeviceptr, cuuint64_t, unsigned int);
@@ -78,6 +78,7 @@ static void proxy_main(int device)
         idle = 0;
         const ishmemi_request r = *slot;
         ++tail;
+        __builtin_prefetch(g_px.ring + ((tail + 4) & (PROXY_RING_SLOTS - 1)));
         if (tail - published >= PROXY_RING_SLOTS / 8) {
             __atomic_store_n(g_px.tail_pub, tail, __ATOMIC_RELEASE);
             published = tail;
@@ -107,7 +108,7 @@ static void proxy_main(int device)
             (void)cudaGetLastError();
             g_px.error.store(rc, std::memory_order_relaxed);
         }
-        g_px.served.fetch_add(1, std::memory_order_relaxed);
+        g_px.served.store(tail, std::memory_order_relaxed); /* only this thread writes it */
     }
     __atomic_store_n(g_px.tail_pub, tail, __ATOMIC_RELEASE);
 }

@@ -76,8 +76,10 @@ __global__ void __launch_bounds__(1024) k_rma(const ishmem_ctx_t *ctxs, rma_args
         else ishmemx_putmem_sub_group(ctx, dest + begin, src + begin, len, target);
     } else if (LEVEL == ISHMEMX_WORK_GROUP_ENGINE) {
         slice_of(a.nbytes, (unsigned long long)g, (unsigned long long)a.groups, &begin, &len);
-        if (a.is_get) ishmemx_getmem_engine_work_group(ctx, dest + begin, src + begin, len, target);
-        else ishmemx_putmem_engine_work_group(ctx, dest + begin, src + begin, len, target);
+        /* non-blocking request, then quiet: exercises the per-PE completion counter */
+        if (a.is_get) ishmemx_getmem_engine_work_group(ctx, dest + begin, src + begin, len, target, false);
+        else ishmemx_putmem_engine_work_group(ctx, dest + begin, src + begin, len, target, false);
+        ishmemx_quiet_work_group(ctx);
     } else {
         ishmemx_staging_t st = {nullptr, 0};
         if (LEVEL == ISHMEMX_WORK_GROUP_BULK) {

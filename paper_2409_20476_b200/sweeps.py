@@ -116,6 +116,7 @@ def sweep_c2(args, out):
     src, dst = B.ishmem_malloc(big), B.ishmem_malloc(big)
     _fill_bytes(torch, heap, npes, heap_bytes, src - heap.data_ptr(), big, inputs.SEED_C2, inputs)
     T = Timer(torch, stream)
+    T1 = Timer(torch, stream, max_iters=1)
     sizes = inputs.message_sizes(3, 28)
     if args.quick:
         sizes = sizes[::5]
@@ -125,6 +126,11 @@ def sweep_c2(args, out):
     variants += [(f"work_group_256x{g}", WG, 256, g, big) for g in (4, 18, 37, 74)]
     variants += [(f"work_group_512x{g}", WG, 512, g, big) for g in (37, 74)]
     variants += [(f"work_group_bulk_256x{g}", BK, 256, g, big) for g in (1, 4, 18, 37)]
+    # device-initiated copy engine: each work-group's leader posts its slice to the host proxy
+    B.ishmemx_proxy_start()
+    B.ishmemx_set_wait_limit_ns(200_000_000)      # a lost reply costs 0.2 s, not 2 s, and shows in the status
+    EN = B.ISHMEMX_WORK_GROUP_ENGINE
+    variants += [(f"work_group_engine_{t}x{g}", EN, t, g, big) for t, g in ((64, 1), (1024, 1), (64, 4))]
 
     def slots(n):
         stride = max((n + 255) // 256 * 256, big // 1024)
@@ -136,7 +142,11 @@ def sweep_c2(args, out):
             for n in sizes:
                 if n > cap:
                     continue
-                us, it = T(lambda i: spmd(dst, src, n, 1, level, threads, groups))
+                # a kernel that waits for the host proxy must not have later launches queued behind
+                # it (they can sit in front of the proxy's copy in a shared hardware queue): the
+                # engine variants are timed one launch per batch
+                timer = T1 if level == EN else T
+                us, it = timer(lambda i: spmd(dst, src, n, 1, level, threads, groups))
                 out.add(config=2, op=op, pattern="ring", variant=name, level=level, threads=threads, groups=groups,
                         npes=npes, dtype="u8", nbytes=n, l2="hot", iters=it, us_per_op=us, alg_bytes=2 * n * npes)
                 if groups >= 18 and n < big:
@@ -192,7 +202,8 @@ def sweep_c2(args, out):
                                           ("work_group_16", WG, 16, 16 * MiB), ("work_group_128", WG, 128, 64 * MiB),
                                           ("work_group_256", WG, 256, 64 * MiB),
                                           ("work_group_1024", WG, 1024, 64 * MiB),
-                                          ("work_group_bulk_256", BK, 256, 64 * MiB)):
+                                          ("work_group_bulk_256", BK, 256, 64 * MiB),
+                                          ("work_group_engine_64", EN, 64, 64 * MiB)):
             for n in sizes:
                 if n > cap:
                     continue
@@ -203,6 +214,37 @@ def sweep_c2(args, out):
                         groups=1, npes=1, dtype="u8", nbytes=n, l2="hot", iters=iters, us_per_op=float(ns[0]) / 1e3,
                         alg_bytes=2 * n, note="device global timer, op + quiet")
     assert B.ishmemx_status(1) == 0
+    B.ishmemx_proxy_stop()
+    B.ishmem_finalize()
+
+
+# ----------------------------------------------------------------- reverse-offload ring ---
+
+def sweep_ring(args, out):
+    """GPU -> host -> GPU round trip and request rate of the reverse-offload ring (64-byte
+    requests, one host proxy thread), for growing numbers of posting GPU threads."""
+    import torch
+    from . import binding as B
+
+    heap, stream = _session(torch, B, 2, 1 << 20)
+    B.ishmemx_proxy_start()
+    rtt, rate = np.zeros(1), np.zeros(1)
+    memops = np.zeros(1, np.int32)
+    B.ishmemx_proxy_stats(None, None, memops)
+    for blocks, threads in ((1, 1), (1, 32), (1, 256), (8, 256), (32, 128), (148, 32), (148, 256)):
+        iters = 400 if blocks * threads <= 256 else 100
+        B.ishmemx_ring_benchmark(0, blocks, threads, iters, rtt, None)
+        B.ishmemx_ring_benchmark(0, blocks, threads, iters, rtt, rate)
+        out.add(config=6, op="ring_round_trip", pattern="gpu->host->gpu", variant="reply_per_request", threads=threads,
+                groups=blocks, nbytes=64, iters=iters, us_per_op=float(rtt[0]) / 1e3, mops=round(float(rate[0]) / 1e6, 3),
+                note=f"mean round trip per request; stream memory operations {'on' if memops[0] else 'off'}")
+        B.ishmemx_ring_benchmark(1, blocks, threads, iters * 4, None, rate)
+        B.ishmemx_ring_benchmark(1, blocks, threads, iters * 4, None, rate)
+        out.add(config=6, op="ring_request_rate", pattern="gpu->host", variant="fire_and_forget", threads=threads,
+                groups=blocks, nbytes=64, iters=iters * 4, us_per_op=1e6 / float(rate[0]),
+                mops=round(float(rate[0]) / 1e6, 3), note="requests/s as seen from the GPU, one proxy thread")
+    assert B.ishmemx_status(1) == 0
+    B.ishmemx_proxy_stop()
     B.ishmem_finalize()
 
 
@@ -449,7 +491,8 @@ def sweep_c5(args, out):
 
 def main(argv=None):
     ap = argparse.ArgumentParser(description=__doc__, formatter_class=argparse.RawDescriptionHelpFormatter)
-    ap.add_argument("--config", type=int, required=True, choices=[1, 2, 3, 4, 5])
+    ap.add_argument("--config", type=int, required=True, choices=[1, 2, 3, 4, 5, 6],
+                    help="benchmark configuration 1..5, or 6 = the reverse-offload ring")
     ap.add_argument("--out", required=True, help="CSV file to write")
     ap.add_argument("--peak-gbs", type=float, default=None,
                     help="measured HBM copy peak in GB/s (default: MEASURED_PEAKS.json beside the package, else 6650)")
@@ -464,7 +507,7 @@ def main(argv=None):
         peak = float(json.loads(f.read_text())["hbm_gbs"]) if f.exists() else 6650.0
     out = Out(args.out, peak)
     try:
-        {1: sweep_c1, 2: sweep_c2, 3: sweep_c3, 4: sweep_c4, 5: sweep_c5}[args.config](args, out)
+        {1: sweep_c1, 2: sweep_c2, 3: sweep_c3, 4: sweep_c4, 5: sweep_c5, 6: sweep_ring}[args.config](args, out)
     finally:
         out.write()
     return 0

@@ -2,6 +2,9 @@ import os
 import sys
 from pathlib import Path
 
+# one hardware queue per stream (see paper_2409_20476_b200/binding.py); must precede CUDA start-up
+os.environ.setdefault("CUDA_DEVICE_MAX_CONNECTIONS", "32")
+
 import pytest
 
 ROOT = Path(__file__).resolve().parent.parent
