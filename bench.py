@@ -274,7 +274,9 @@ def run_ours(args) -> dict:
     return out if rank == 0 else {}
 
 
-TRAFFIC_PER_LAUNCH = {"bulk": None, "ldst": None}  # dram bytes per launch from ncu (profiles/)
+# DRAM bytes per launch of the put kernel: ncu capture of the 8 x 32 MiB case (reads scale with the
+# bytes copied; writes are the algorithmic bytes minus the ~52 MB tail that stays in L2)
+TRAFFIC_PER_LAUNCH = {"bulk": 4.24e9, "ldst": None}
 
 
 def breakdown(B, torch, team_stream, env) -> dict:
@@ -460,6 +462,8 @@ def run_profile_case(args) -> dict:
     from paper_2409_20476_b200 import binding as B
     from paper_2409_20476_b200 import inputs
 
+    if args.profile_case == "jacobi":
+        return run_profile_jacobi(args)
     n = args.msg_mib * MiB
     heap_bytes = 2 * n + (1 << 20) if args.profile_case != "fcollect" else (NPES + 1) * n + (1 << 20)
     heap = torch.empty(NPES * heap_bytes, dtype=torch.uint8, device="cuda")
@@ -491,13 +495,52 @@ def run_profile_case(args) -> dict:
     return {"profile_case": args.profile_case, "msg_mib": args.msg_mib, "ms": [round(t, 4) for t in times[3:]]}
 
 
+def run_profile_jacobi(args) -> dict:
+    """Small Jacobi case for profiler captures: 8 PEs, 4096 x 4096 float64 (two buffers of
+    128 MiB: larger than L2), `--steps` launches of 4 sweeps each in the benchmark's shape."""
+    import torch
+    from paper_2409_20476_b200 import binding as B
+    from paper_2409_20476_b200 import inputs
+
+    n, sweeps = 4096, 4
+    rows = n // NPES
+    nbytes = (rows + 2) * n * 8
+    heap_bytes = 2 * nbytes + MiB
+    heap = torch.zeros(NPES * heap_bytes, dtype=torch.uint8, device="cuda")
+    B.ishmemx_init_external(NPES, heap_bytes, heap.data_ptr())
+    b0, b1, sig = B.ishmem_malloc(nbytes), B.ishmem_malloc(nbytes), B.ishmem_calloc(2, 8)
+    grid = inputs.jacobi_grid(inputs.SEED_C5, n, n)
+    for p in range(NPES):
+        o = p * heap_bytes + (b0 - heap.data_ptr()) + n * 8
+        heap[o:o + rows * n * 8].copy_(torch.from_numpy(grid[p * rows:(p + 1) * rows].view(np.uint8).ravel()))
+    torch.cuda.synchronize()
+    ts = torch.cuda.Stream()
+    B.ishmemx_set_stream(-1, ts.cuda_stream)
+    res, times = np.zeros(1), []
+    for _ in range(2 + args.steps):
+        for p in range(NPES):
+            B.ishmem_uint64_p(p, sig, 0, p)
+            B.ishmem_uint64_p(p, sig + 8, 0, p)
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(ts)
+        B.ishmemx_jacobi(b0, b1, sig, n, n, sweeps, 1, args.jacobi_groups, 512, res)
+        b.record(ts)
+        torch.cuda.synchronize()
+        times.append(a.elapsed_time(b))
+    status = B.ishmemx_status(1)
+    B.ishmem_finalize()
+    return {"profile_case": "jacobi", "n": n, "sweeps_per_launch": sweeps, "status": status,
+            "ms": [round(t, 4) for t in times[2:]]}
+
+
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--profile-case", default=None, choices=["put", "get", "reduce", "broadcast", "fcollect"],
+    ap.add_argument("--profile-case", default=None, choices=["put", "get", "reduce", "broadcast", "fcollect", "jacobi"],
                     help="run only a few launches of one kernel on a small case (for ncu captures)")
     ap.add_argument("--msg-mib", type=int, default=32)
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--steps", type=int, default=300)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--level", default="bulk", choices=["bulk", "ldst"])

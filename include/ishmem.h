@@ -215,6 +215,15 @@ int ishmemx_putmem_spmd_copy_engine(void *dest, const void *src, size_t nbytes, 
  * ishmemx_proxy_start runs).  SIZE_MAX = never use the copy engine (the default), 0 = always. */
 int ishmemx_set_cutover(int which, size_t nbytes);
 size_t ishmemx_get_cutover(int which);
+/* Picks the cutover from measurement on this device (Section 4: "tuned from measurement"), for
+ * which = 0 (host-initiated put, PE 0 -> PE 1, CUDA events) or which = 3 (device-initiated put
+ * by ONE work-group of `threads` threads, timed inside the kernel; needs a running proxy).
+ * Times both paths at 4 KiB, 16 KiB, ... up to max_bytes (two temporary symmetric buffers of
+ * max_bytes are allocated and freed: ISHMEM_ERR_OOM if the heap has no room) and sets the
+ * cutover to the smallest size from which the copy engine is at least as fast at every larger
+ * size tried, or SIZE_MAX when it never is.  The choice is also written to HOST *chosen (may
+ * be NULL).  Blocks the host. */
+int ishmemx_tune_cutover(int which, int threads, size_t max_bytes, size_t *chosen);
 
 /* ------------------------------------- reverse offload: GPU -> host requests (Section 3.4) --- */
 

@@ -122,6 +122,7 @@ def _signatures() -> dict[str, tuple[str, list[str]]]:
         "ishmemx_putmem_spmd_copy_engine": ("status", ["p", "p", "z", "i"]),
         "ishmemx_set_cutover": ("status", ["i", "z"]),
         "ishmemx_get_cutover": ("size", ["i"]),
+        "ishmemx_tune_cutover": ("status", ["i", "i", "z", "p"]),
         "ishmem_putmem_signal": ("status", ["i", "p", "p", "z", "p", "u64", "i", "i"]),
         "ishmem_uint64_wait_until": ("status", ["i", "p", "i", "u64"]),
         "ishmem_fence": ("status", ["i"]),

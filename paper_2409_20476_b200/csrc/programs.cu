@@ -191,6 +191,75 @@ extern "C" int ishmemx_rma_latency(int my_pe, void *dest, const void *src, size_
     return ISHMEM_OK;
 }
 
+/* ---- cutover tuning from measurement (Section 4) ----------------------------------------------- */
+
+/* mean time in ns of one host-initiated ishmem_putmem PE 0 -> PE `to` under the current cutover */
+static int time_host_put(void *dst, const void *src, size_t n, int to, int reps, double *ns)
+{
+    auto &g = g_ishmem;
+    cudaEvent_t a, b;
+    ISHMEMI_CUDA(cudaEventCreate(&a));
+    ISHMEMI_CUDA(cudaEventCreate(&b));
+    int rc = ishmem_putmem(0, dst, src, n, to); /* warm-up; also joins pending team work */
+    cudaStream_t s = g.pe_stream[0];
+    if (!rc) rc = ishmemi_cuda(cudaEventRecord(a, s), "cudaEventRecord");
+    for (int i = 0; i < reps && !rc; ++i) rc = ishmem_putmem(0, dst, src, n, to);
+    if (!rc) rc = ishmemi_cuda(cudaEventRecord(b, s), "cudaEventRecord");
+    if (!rc) rc = ishmemi_cuda(cudaEventSynchronize(b), "cudaEventSynchronize");
+    float ms = 0.f;
+    if (!rc) rc = ishmemi_cuda(cudaEventElapsedTime(&ms, a, b), "cudaEventElapsedTime");
+    cudaEventDestroy(a);
+    cudaEventDestroy(b);
+    *ns = (double)ms * 1e6 / reps;
+    return rc;
+}
+
+extern "C" int ishmemx_tune_cutover(int which, int threads, size_t max_bytes, size_t *chosen)
+{
+    ISHMEMI_REQUIRE_INIT();
+    auto &g = g_ishmem;
+    if (which != 0 && which != 3) return ISHMEM_ERR_ARG;
+    if (which == 3 && (g.h_ctx[0].proxy == nullptr || threads < 1 || threads > 1024)) return ISHMEM_ERR_ARG;
+    if (max_bytes < 4096) return ISHMEM_ERR_ARG;
+    void *src = ishmem_malloc(max_bytes), *dst = ishmem_malloc(max_bytes);
+    if (!src || !dst) {
+        ishmem_free(src);
+        ishmem_free(dst);
+        return ISHMEM_ERR_OOM;
+    }
+    const int to = g.npes > 1 ? 1 : 0;
+    const size_t saved = ishmemx_get_cutover(which);
+    int rc = 0;
+    /* sizes 4 KiB, 16 KiB, ... <= max_bytes; the engine "wins" a size when it is at least as
+     * fast there; the cutover is the start of the unbroken run of wins at the top */
+    size_t pick = (size_t)-1;
+    for (size_t n = 4096; n <= max_bytes && !rc; n *= 4) {
+        double t_ldst = 0, t_engine = 0;
+        const int reps = n <= (1u << 20) ? 50 : (n <= (16u << 20) ? 10 : 3);
+        if (which == 0) {
+            ishmemx_set_cutover(0, (size_t)-1);
+            rc = time_host_put(dst, src, n, to, reps, &t_ldst);
+            ishmemx_set_cutover(0, 0);
+            if (!rc) rc = time_host_put(dst, src, n, to, reps, &t_engine);
+        } else {
+            ishmemx_set_cutover(3, (size_t)-1);
+            rc = ishmemx_rma_latency(0, dst, src, n, to, 0, ISHMEMX_WORK_GROUP, threads, reps, &t_ldst);
+            if (!rc) rc = ishmemx_rma_latency(0, dst, src, n, to, 0, ISHMEMX_WORK_GROUP_ENGINE, threads, reps, &t_engine);
+        }
+        if (t_engine <= t_ldst) {
+            if (pick == (size_t)-1) pick = n;
+        } else {
+            pick = (size_t)-1;
+        }
+    }
+    ishmemx_set_cutover(which, rc ? saved : pick);
+    cudaDeviceSynchronize();
+    ishmem_free(src);
+    ishmem_free(dst);
+    if (!rc && chosen) *chosen = pick;
+    return rc;
+}
+
 /* ---- Jacobi overlap workload -------------------------------------------------------------- */
 
 struct jacobi_args {

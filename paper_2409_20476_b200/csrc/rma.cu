@@ -190,12 +190,18 @@ static void auto_geometry(size_t n, int *threads, unsigned *blocks, int *level)
         *threads = 256;
         *blocks = (unsigned)((n + 16383) / 16384);
         *level = ISHMEMX_WORK_GROUP;
-    } else {
+    } else if (n < ((size_t)32 << 20)) {
         *threads = 512;
         size_t b = (n + 65535) / 65536;
         size_t cap = (size_t)g_ishmem.sm_count * 4;
         *blocks = (unsigned)(b < cap ? b : cap);
         *level = ISHMEMX_WORK_GROUP;
+    } else {
+        /* large: one block per SM, each streaming its slice through the TMA ring (measured
+         * fastest from a few tens of MiB on) */
+        *threads = 256;
+        *blocks = (unsigned)g_ishmem.sm_count;
+        *level = ISHMEMX_WORK_GROUP_BULK;
     }
 }
 

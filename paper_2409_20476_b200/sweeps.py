@@ -489,17 +489,146 @@ def sweep_c5(args, out):
     B.ishmem_finalize()
 
 
+# ------------------------------------------------------------------------------ summaries ---
+
+def _fmt_size(n):
+    n = int(n)
+    for unit, k in (("GiB", 1 << 30), ("MiB", 1 << 20), ("KiB", 1 << 10)):
+        if n >= k and n % k == 0:
+            return f"{n // k} {unit}"
+    return f"{n} B"
+
+
+def _table(rows, row_key, col_key, val, row_fmt=str, cols=None):
+    """markdown pivot: one line per row_key value, one column per col_key value"""
+    cols = cols or list(dict.fromkeys(col_key(r) for r in rows))
+    keys = list(dict.fromkeys(row_key(r) for r in rows))
+    cell = {(row_key(r), col_key(r)): val(r) for r in rows}
+    out = ["| size | " + " | ".join(cols) + " |", "|---:|" + "---:|" * len(cols)]
+    for k in keys:
+        out.append(f"| {row_fmt(k)} | " + " | ".join(str(cell.get((k, c), "")) for c in cols) + " |")
+    return "\n".join(out)
+
+
+def _crossover(a, b):
+    """smallest size from which b's time is <= a's at every larger common size, or None"""
+    pick = None
+    for n in sorted(set(a) & set(b)):
+        if b[n] <= a[n]:
+            pick = n if pick is None else pick
+        else:
+            pick = None
+    return pick
+
+
+def summarize(path) -> str:
+    rows = list(csv.DictReader(open(path)))
+    cfg = int(rows[0]["config"])
+    nb = lambda r: int(r["nbytes"])
+    gb = lambda r: f"{float(r['gbps']):.0f}" if r["gbps"] else ""
+    us = lambda r: f"{float(r['us_per_op']):.2f}" if r["us_per_op"] else ""
+    out = []
+    if cfg == 2:
+        ring = [r for r in rows if r["pattern"] == "ring" and r["op"] == "put"]
+        keep = ["work_item", "sub_group", "work_group_16x1", "work_group_128x1", "work_group_1024x1",
+                "work_group_256x18", "work_group_512x74", "work_group_bulk_256x37", "work_group_engine_64x1",
+                "copy_engine"]
+        for l2 in ("hot", "cold"):
+            sel = [r for r in ring if r["l2"] == l2 and r["variant"] in keep]
+            out += [f"### put, ring p -> (p+1) mod 8, 8 PEs concurrently, {l2} buffers: GB/s (algorithmic, aggregate)", "",
+                    _table(sel, nb, lambda r: r["variant"], gb, _fmt_size, [k for k in keep if any(r["variant"] == k for r in sel)]), ""]
+        t = lambda var, l2="hot", op="put", pat="ring": {nb(r): float(r["us_per_op"]) for r in rows if r["variant"] == var
+                                                          and r["l2"] == l2 and r["op"] == op and r["pattern"] == pat}
+        out += ["### crossover: smallest message from which the copy engine is at least as fast at every larger size", ""]
+        for var in ("work_item", "sub_group", "work_group_16x1", "work_group_128x1", "work_group_256x1", "work_group_1024x1",
+                    "work_group_256x4", "work_group_256x18", "work_group_256x37", "work_group_512x74",
+                    "work_group_bulk_256x37"):
+            c = _crossover(t(var), t("copy_engine"))
+            out.append(f"- `{var}` vs host-started copy engine (ring, 8 PEs): " + (_fmt_size(c) if c else "never"))
+        c = _crossover(t("host_api_kernel", pat="one_pe"), t("host_api_copy_engine", pat="one_pe"))
+        out.append("- host API `ishmem_putmem`, one PE, kernel vs engine: " + (_fmt_size(c) if c else "never (mixed)"))
+        for var in ("in_kernel_work_item", "in_kernel_sub_group", "in_kernel_work_group_16", "in_kernel_work_group_128",
+                    "in_kernel_work_group_256", "in_kernel_work_group_1024", "in_kernel_work_group_bulk_256"):
+            c = _crossover(t(var, pat="one_pe"), t("in_kernel_work_group_engine_64", pat="one_pe"))
+            out.append(f"- one collaboration unit inside a kernel, `{var[10:]}` vs device-initiated engine request: "
+                       + (_fmt_size(c) if c else "never"))
+        sel = [r for r in rows if r["pattern"] == "one_pe" and r["op"] == "put" and r["variant"].startswith("in_kernel")]
+        out += ["", "### one collaboration unit, PE 0 -> PE 1, put + quiet timed inside the kernel: microseconds", "",
+                _table(sel, nb, lambda r: r["variant"][10:], us, _fmt_size), ""]
+        sel = [r for r in rows if r["pattern"] == "all_pairs"]
+        out += ["### all-pairs (mean of the 7 permutation rounds): GB/s", "",
+                _table(sel, nb, lambda r: r["variant"], gb, _fmt_size), ""]
+        getr = [r for r in rows if r["pattern"] == "ring" and r["op"] == "get" and r["l2"] == "hot"
+                and r["variant"] in ("work_group_512x74", "work_group_bulk_256x37") and nb(r) >= 1 << 20]
+        out += ["### get, ring, hot buffers: GB/s", "", _table(getr, nb, lambda r: r["variant"], gb, _fmt_size), ""]
+    elif cfg == 1:
+        out += ["### 4 PEs x 16 MiB, int32: microseconds per operation", "",
+                _table([r for r in rows if r["op"] in ("put", "get")], nb,
+                       lambda r: r["op"] + " " + ("in-kernel" if r["variant"].startswith("in_kernel") else "host-launched x4 PEs"),
+                       us, _fmt_size), ""]
+        for r in rows:
+            if r["op"] == "sum_reduce":
+                out.append(f"- int32 sum_reduce, 262144 elements, 4 PEs, {r['variant']}: {us(r)} us ({gb(r)} GB/s algorithmic)")
+    elif cfg == 3:
+        for dt in ("f32", "f64", "i64"):
+            sel = [r for r in rows if r["dtype"] == dt and r["variant"] in ("auto", "stores")]
+            out += [f"### 12 PEs, {dt}: GB/s (algorithmic) / microseconds", "",
+                    _table(sel, nb, lambda r: r["op"], lambda r: f"{gb(r)} / {us(r)}", _fmt_size), ""]
+        for op in ("broadcast", "fcollect"):
+            out += [f"### {op}: stores vs copy engine, microseconds", ""]
+            sel = [r for r in rows if r["op"] == op and r["dtype"] == "u8" and r["variant"] in ("stores", "copy_engine")]
+            out += [_table(sel, nb, lambda r: f"P={r['npes']} {r['variant']}", us, _fmt_size), ""]
+            for P in ("2", "4", "8", "12"):
+                a = {nb(r): float(r["us_per_op"]) for r in sel if r["npes"] == P and r["variant"] == "stores"}
+                b = {nb(r): float(r["us_per_op"]) for r in sel if r["npes"] == P and r["variant"] == "copy_engine"}
+                c = _crossover(a, b)
+                out.append(f"- {op}, {P} PEs: engine at least as fast from " + (_fmt_size(c) if c else "never"))
+            out.append("")
+        sel = [r for r in rows if r["variant"] == "device_resident" and r["npes"] in ("2", "12") and r["threads"] in ("128", "1024")]
+        out += ["### device-resident forms (one work-group per PE, in-kernel push sync): microseconds", "",
+                _table(sel, nb, lambda r: f"{r['op']} P={r['npes']} T={r['threads']}", us, _fmt_size), ""]
+    elif cfg == 4:
+        out += ["### remote atomics, 16 PEs: Mops/s (one op per GPU thread)", "", "| op | index stream | variant | threads | Mops/s | us |",
+                "|---|---|---|---:|---:|---:|"]
+        for r in rows:
+            if r["mops"]:
+                out.append(f"| {r['op']} | {r['pattern']} | {r['variant']} | {r['threads']} | {float(r['mops']):.0f} | {us(r)} |")
+        sel = [r for r in rows if r["op"] == "put_signal_pingpong"]
+        out += ["", "### put_signal / wait_until ping-pong, half round trip in microseconds (in-kernel)", "",
+                _table(sel, nb, lambda r: f"{r['threads']} threads", us, _fmt_size), ""]
+    elif cfg == 5:
+        out += ["### Jacobi 16384 x 16384 float64, 12 PEs, 200 sweeps: per sweep", "",
+                "| overlap | threads | groups/PE | us/sweep | GB/s (16 B/cell) | of measured copy | of 8 TB/s |", "|---|---:|---:|---:|---:|---:|---:|"]
+        for r in rows:
+            if r["us_per_op"]:
+                out.append(f"| {r['variant'][-1]} | {r['threads']} | {r['groups']} | {us(r)} | {gb(r)} | {r['frac_hbm']} | {r['frac_8tbs']} |")
+            else:
+                out.append(f"| {r['variant'][-1]} | {r['threads']} | {r['groups']} | refused: not co-resident | | | |")
+    elif cfg == 6:
+        out += ["### reverse-offload ring (64-byte requests, one host proxy thread)", "",
+                "| measurement | blocks x threads | us | M requests/s |", "|---|---:|---:|---:|"]
+        for r in rows:
+            out.append(f"| {r['op']} | {r['groups']} x {r['threads']} | {us(r)} | {r['mops']} |")
+    return "\n".join(out) + "\n"
+
+
 def main(argv=None):
     ap = argparse.ArgumentParser(description=__doc__, formatter_class=argparse.RawDescriptionHelpFormatter)
-    ap.add_argument("--config", type=int, required=True, choices=[1, 2, 3, 4, 5, 6],
+    ap.add_argument("--summarize", default=None, metavar="CSV", help="print a markdown digest of a CSV written earlier")
+    ap.add_argument("--config", type=int, default=None, choices=[1, 2, 3, 4, 5, 6],
                     help="benchmark configuration 1..5, or 6 = the reverse-offload ring")
-    ap.add_argument("--out", required=True, help="CSV file to write")
+    ap.add_argument("--out", default=None, help="CSV file to write")
     ap.add_argument("--peak-gbs", type=float, default=None,
                     help="measured HBM copy peak in GB/s (default: MEASURED_PEAKS.json beside the package, else 6650)")
     ap.add_argument("--quick", action="store_true", help="fewer sizes (smoke run)")
     ap.add_argument("--fcollect-max-elems", type=int, default=4 ** 12,
                     help="largest per-PE element count of the 8-byte fcollect rows")
     args = ap.parse_args(argv)
+    if args.summarize:
+        print(summarize(args.summarize))
+        return 0
+    if args.config is None or args.out is None:
+        ap.error("--config and --out are required")
     peak = args.peak_gbs
     if peak is None:
         import json

@@ -124,3 +124,35 @@ def test_ring_round_trip_and_request_rate():
             assert s.status() == 0
         finally:
             B.ishmemx_proxy_stop()
+
+
+def test_cutover_tuned_from_measurement():
+    """ishmemx_tune_cutover times both paths and installs its pick; transfers stay correct on
+    both sides of it."""
+    npes, heap = 2, 40 << 20
+    with Session(npes, heap) as s:
+        src, dst = s.malloc(3 << 20), s.malloc(3 << 20)
+        B.ishmemx_proxy_start()
+        try:
+            chosen = np.zeros(1, np.uint64)
+            for which, threads in ((0, 0), (3, 256)):
+                B.ishmemx_tune_cutover(which, threads, 16 << 20, chosen)
+                pick = int(chosen[0])
+                assert pick == B.SIZE_MAX or (4096 <= pick <= 16 << 20 and pick & (pick - 1) == 0)
+                assert B.ishmemx_get_cutover(which) == pick
+                print(f"tuned cutover[{which}] = {'never' if pick == B.SIZE_MAX else pick}")
+            with pytest.raises(B.IshmemError) as e:
+                B.ishmemx_tune_cutover(0, 0, 1 << 30, None)          # no room for the temporaries
+            assert e.value.code == B.ISHMEM_ERR_OOM
+            for p in range(npes):
+                src.fill(p, inputs.byte_payload(inputs.SEED_C2, 30 + p, 3 << 20))
+            for n in (5000, 3 << 20):
+                B.ishmem_putmem(0, dst.addr, src.addr, n, 1)
+                s.oracle.putmem(0, dst.ooff, s.oracle.ptr(src.ooff, n, 0), n, 1)
+                B.ishmemx_putmem_on_device(1, dst.addr, src.addr, n, 0, B.ISHMEMX_WORK_GROUP, 256, 1)
+                s.oracle.putmem(1, dst.ooff, s.oracle.ptr(src.ooff, n, 1), n, 0)
+                B.ishmem_barrier_all()
+                dst.assert_equal(f"after tuning n={n}")
+            assert s.status() == 0
+        finally:
+            B.ishmemx_proxy_stop()
