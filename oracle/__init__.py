@@ -18,7 +18,8 @@ _SRC = _HERE / "ishmem_oracle.c"
 _LIB = _HERE / "libishmem_oracle.so"
 
 # element types / operators / comparisons: the oracle's own numbering
-T_INT32, T_INT64, T_FLOAT, T_DOUBLE, T_UINT32, T_UINT64 = range(6)
+(T_INT32, T_INT64, T_FLOAT, T_DOUBLE, T_UINT32, T_UINT64, T_INT8, T_UINT8, T_INT16,
+ T_UINT16) = range(10)
 R_SUM, R_MAX, R_MIN, R_PROD, R_AND, R_OR, R_XOR = range(7)
 (A_FETCH_ADD, A_ADD, A_FETCH_INC, A_INC, A_FETCH, A_SET, A_SWAP, A_COMPARE_SWAP,
  A_FETCH_AND, A_FETCH_OR, A_FETCH_XOR) = range(11)
@@ -28,7 +29,8 @@ C_EQ, C_NE, C_GT, C_GE, C_LT, C_LE = range(6)
 OK, ERR_INVALID_PE, ERR_NOT_SYMMETRIC, ERR_ALIGN, ERR_OOM, ERR_ARG = 0, -1, -2, -3, -4, -5
 
 NP_DTYPE = {T_INT32: np.int32, T_INT64: np.int64, T_FLOAT: np.float32, T_DOUBLE: np.float64,
-            T_UINT32: np.uint32, T_UINT64: np.uint64}
+            T_UINT32: np.uint32, T_UINT64: np.uint64, T_INT8: np.int8, T_UINT8: np.uint8,
+            T_INT16: np.int16, T_UINT16: np.uint16}
 
 
 def build(force: bool = False) -> Path:
@@ -61,6 +63,10 @@ def lib():
         L.oracle_reset_allocator.argtypes = [vp]
         L.oracle_putmem.argtypes = [vp, i, sz, vp, sz, i]
         L.oracle_getmem.argtypes = [vp, i, vp, sz, sz, i]
+        L.oracle_iput.argtypes = [vp, i, sz, vp, sz, sz, sz, sz, i]
+        L.oracle_iget.argtypes = [vp, i, vp, sz, sz, sz, sz, sz, i]
+        L.oracle_collectmem.argtypes = [vp, i, i, i, sz, sz, vp]
+        L.oracle_alltoallmem.argtypes = [vp, i, i, i, sz, sz, sz]
         L.oracle_p.argtypes = [vp, sz, vp, sz, i]
         L.oracle_g.argtypes = [vp, vp, sz, sz, i]
         L.oracle_putmem_signal.argtypes = [vp, i, sz, vp, sz, sz, u64, i, i]
@@ -155,6 +161,12 @@ class Oracle:
     def getmem(self, my_pe, dest, src_off, n, pe):
         _chk(self.L.oracle_getmem(self.h, my_pe, _addr(dest), src_off, n, pe))
 
+    def iput(self, my_pe, dest_off, src, dst, sst, nelems, esize, pe):
+        _chk(self.L.oracle_iput(self.h, my_pe, dest_off, _addr(src), dst, sst, nelems, esize, pe))
+
+    def iget(self, my_pe, dest, src_off, dst, sst, nelems, esize, pe):
+        _chk(self.L.oracle_iget(self.h, my_pe, _addr(dest), src_off, dst, sst, nelems, esize, pe))
+
     def p(self, dest_off, value: np.generic | np.ndarray, pe):
         v = np.ascontiguousarray(value).reshape(1)
         _chk(self.L.oracle_p(self.h, dest_off, v.ctypes.data, v.itemsize, pe))
@@ -203,6 +215,14 @@ class Oracle:
 
     def fcollectmem(self, team, dest_off, src_off, n):
         _chk(self.L.oracle_fcollectmem(self.h, *team, dest_off, src_off, n))
+
+    def collectmem(self, team, dest_off, src_off, nbytes):
+        sizes = np.ascontiguousarray(nbytes, dtype=np.uint64)
+        assert len(sizes) == team[2]
+        _chk(self.L.oracle_collectmem(self.h, *team, dest_off, src_off, sizes.ctypes.data))
+
+    def alltoallmem(self, team, dest_off, src_off, n):
+        _chk(self.L.oracle_alltoallmem(self.h, *team, dest_off, src_off, n))
 
     def reduce(self, team, dest_off, src_off, nreduce, op, dtype):
         _chk(self.L.oracle_reduce(self.h, *team, dest_off, src_off, nreduce, op, dtype))

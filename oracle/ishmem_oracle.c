@@ -18,7 +18,9 @@
  *
  * Parity pins (tests/test_oracle_*.py): put/get against Python's byte-at-a-time
  * model on tiny heaps, closed forms of PE-indexed patterns for reduce /
- * fcollect / broadcast, numpy wrap-around sums, conservation and chain checks
+ * fcollect / broadcast, numpy wrap-around sums (also for 8- and 16-bit elements), numpy strided
+ * slices for iput / iget, np.concatenate for collect, a block transpose for alltoall (with its
+ * involution property), conservation and chain checks
  * for atomics, Jacobi eigenmode decay and decomposition independence.
  * "parity unpinned": oracle_test (the comparison of wait_until) beyond its truth
  * table, and the root-writes-dest reading of broadcast (both readings offered).
@@ -38,7 +40,8 @@
 #define ORACLE_ERR_ARG (-5)
 
 /* element types of typed operations */
-enum { T_INT32 = 0, T_INT64 = 1, T_FLOAT = 2, T_DOUBLE = 3, T_UINT32 = 4, T_UINT64 = 5 };
+enum { T_INT32 = 0, T_INT64 = 1, T_FLOAT = 2, T_DOUBLE = 3, T_UINT32 = 4, T_UINT64 = 5,
+       T_INT8 = 6, T_UINT8 = 7, T_INT16 = 8, T_UINT16 = 9 };
 /* reduction operators (Section 3.7.2, "Reduction": min, max, sum, product, and/or/xor) */
 enum { R_SUM = 0, R_MAX = 1, R_MIN = 2, R_PROD = 3, R_AND = 4, R_OR = 5, R_XOR = 6 };
 /* atomic operations */
@@ -62,6 +65,8 @@ static size_t type_size(int t)
     switch (t) {
     case T_INT32: case T_FLOAT: case T_UINT32: return 4;
     case T_INT64: case T_DOUBLE: case T_UINT64: return 8;
+    case T_INT8: case T_UINT8: return 1;
+    case T_INT16: case T_UINT16: return 2;
     default: return 0;
     }
 }
@@ -155,6 +160,52 @@ int oracle_getmem(oracle_t *o, int my_pe, void *dest, size_t src_off, size_t n, 
     const unsigned char *s = o->heap[pe] + src_off;
     unsigned char *d = (unsigned char *)dest;
     for (size_t i = 0; i < n; ++i) d[i] = s[i];
+    return ORACLE_OK;
+}
+
+/* strided put (OpenSHMEM iput; "put ... that are blocked or strided", Section 3.7.1): element k
+ * of the source, taken every `sst` elements from `src`, becomes element k*dst of the symmetric
+ * object at `dest_off` on PE `pe`, k = 0..nelems-1.  Elements are `esize` bytes; strides are in
+ * elements and at least 1. */
+int oracle_iput(oracle_t *o, int my_pe, size_t dest_off, const void *src, size_t dst, size_t sst,
+                size_t nelems, size_t esize, int pe)
+{
+    int rc = check(o, 0, 0, my_pe);
+    if (rc) return rc;
+    if (dst < 1 || sst < 1 || esize < 1) return ORACLE_ERR_ARG;
+    if (nelems) {
+        if ((nelems - 1) > (o->heap_bytes / esize) / dst) return ORACLE_ERR_NOT_SYMMETRIC;
+        rc = check(o, dest_off, ((nelems - 1) * dst + 1) * esize, pe);
+        if (rc) return rc;
+    } else if ((rc = check(o, dest_off, 0, pe))) {
+        return rc;
+    }
+    const unsigned char *s = (const unsigned char *)src;
+    unsigned char *d = o->heap[pe] + dest_off;
+    for (size_t k = 0; k < nelems; ++k)
+        for (size_t b = 0; b < esize; ++b) d[k * dst * esize + b] = s[k * sst * esize + b];
+    return ORACLE_OK;
+}
+
+/* strided get (iget): element k*sst of the symmetric object at `src_off` on PE `pe` becomes
+ * element k*dst of the caller's `dest`. */
+int oracle_iget(oracle_t *o, int my_pe, void *dest, size_t src_off, size_t dst, size_t sst,
+                size_t nelems, size_t esize, int pe)
+{
+    int rc = check(o, 0, 0, my_pe);
+    if (rc) return rc;
+    if (dst < 1 || sst < 1 || esize < 1) return ORACLE_ERR_ARG;
+    if (nelems) {
+        if ((nelems - 1) > (o->heap_bytes / esize) / sst) return ORACLE_ERR_NOT_SYMMETRIC;
+        rc = check(o, src_off, ((nelems - 1) * sst + 1) * esize, pe);
+        if (rc) return rc;
+    } else if ((rc = check(o, src_off, 0, pe))) {
+        return rc;
+    }
+    const unsigned char *s = o->heap[pe] + src_off;
+    unsigned char *d = (unsigned char *)dest;
+    for (size_t k = 0; k < nelems; ++k)
+        for (size_t b = 0; b < esize; ++b) d[k * dst * esize + b] = s[k * sst * esize + b];
     return ORACLE_OK;
 }
 
@@ -345,6 +396,64 @@ int oracle_fcollectmem(oracle_t *o, int t_start, int t_stride, int t_size, size_
     return ORACLE_OK;
 }
 
+/* collect: like fcollect with contributions of different sizes ("collect (which is like MPI
+ * allgather)", Section 3.7.2) -- every member's dest is the concatenation, in team order, of
+ * the members' sources; member i contributes nbytes[i] bytes. */
+int oracle_collectmem(oracle_t *o, int t_start, int t_stride, int t_size, size_t dest_off,
+                      size_t src_off, const size_t *nbytes)
+{
+    int rc = team_check(o, t_start, t_stride, t_size);
+    if (rc) return rc;
+    size_t total = 0;
+    for (int i = 0; i < t_size; ++i) {
+        rc = check(o, src_off, nbytes[i], t_start + i * t_stride);
+        if (rc) return rc;
+        if (nbytes[i] > o->heap_bytes - total) return ORACLE_ERR_NOT_SYMMETRIC;
+        total += nbytes[i];
+    }
+    rc = check(o, dest_off, total, t_start);
+    if (rc) return rc;
+    unsigned char *snap = (unsigned char *)malloc(total + 1);
+    if (!snap) return ORACLE_ERR_OOM;
+    size_t at = 0;
+    for (int i = 0; i < t_size; ++i) {
+        memcpy(snap + at, o->heap[t_start + i * t_stride] + src_off, nbytes[i]);
+        at += nbytes[i];
+    }
+    for (int q = 0; q < t_size; ++q) {
+        unsigned char *d = o->heap[t_start + q * t_stride] + dest_off;
+        for (size_t k = 0; k < total; ++k) d[k] = snap[k];
+    }
+    free(snap);
+    return ORACLE_OK;
+}
+
+/* alltoall (OpenSHMEM 1.5 team collective): block i of member q's dest is block q of member
+ * i's source, blocks of n bytes: dest@q[i*n + k] = src@i[q*n + k]. */
+int oracle_alltoallmem(oracle_t *o, int t_start, int t_stride, int t_size, size_t dest_off,
+                       size_t src_off, size_t n)
+{
+    int rc = team_check(o, t_start, t_stride, t_size);
+    if (rc) return rc;
+    if (n && (size_t)t_size > o->heap_bytes / n) return ORACLE_ERR_NOT_SYMMETRIC;
+    const size_t all = n * (size_t)t_size;
+    rc = check(o, src_off, all, t_start);
+    if (rc) return rc;
+    rc = check(o, dest_off, all, t_start);
+    if (rc) return rc;
+    unsigned char *snap = (unsigned char *)malloc(all * (size_t)t_size + 1);
+    if (!snap) return ORACLE_ERR_OOM;
+    for (int i = 0; i < t_size; ++i)
+        memcpy(snap + (size_t)i * all, o->heap[t_start + i * t_stride] + src_off, all);
+    for (int q = 0; q < t_size; ++q) {
+        unsigned char *d = o->heap[t_start + q * t_stride] + dest_off;
+        for (int i = 0; i < t_size; ++i)
+            for (size_t k = 0; k < n; ++k) d[(size_t)i * n + k] = snap[(size_t)i * all + (size_t)q * n + k];
+    }
+    free(snap);
+    return ORACLE_OK;
+}
+
 /* One binary combine, `acc = acc op x`, in the element's own precision.
  * Integer sum and product wrap (computed unsigned); max/min keep the left
  * operand on ties: (x > acc) ? x : acc. */
@@ -365,6 +474,12 @@ COMBINE_INT(int32_t, uint32_t)
 COMBINE_INT(int64_t, uint64_t)
 COMBINE_INT(uint32_t, uint32_t)
 COMBINE_INT(uint64_t, uint64_t)
+/* 8- and 16-bit elements ("fixed-point datatypes from 8 to 64 bits"): the unsigned type of the
+ * same width keeps sum and product modulo 2^8 / 2^16 */
+COMBINE_INT(int8_t, uint8_t)
+COMBINE_INT(uint8_t, uint8_t)
+COMBINE_INT(int16_t, uint16_t)
+COMBINE_INT(uint16_t, uint16_t)
 
 #define COMBINE_FP(F)                                                   \
     static F combine_##F(int op, F acc, F x)                            \
@@ -413,6 +528,10 @@ int oracle_reduce(oracle_t *o, int t_start, int t_stride, int t_size, size_t des
         case T_UINT32: FOLD(uint32_t) break;
         case T_UINT64: FOLD(uint64_t) break;
         case T_FLOAT: FOLD(float) break;
+        case T_INT8: FOLD(int8_t) break;
+        case T_UINT8: FOLD(uint8_t) break;
+        case T_INT16: FOLD(int16_t) break;
+        case T_UINT16: FOLD(uint16_t) break;
         default: FOLD(double) break;
         }
 #undef FOLD
