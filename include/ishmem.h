@@ -97,6 +97,10 @@ typedef int ishmem_team_t;
 #define ISHMEM_T_DOUBLE 3
 #define ISHMEM_T_UINT32 4
 #define ISHMEM_T_UINT64 5
+#define ISHMEM_T_INT8 6
+#define ISHMEM_T_UINT8 7
+#define ISHMEM_T_INT16 8
+#define ISHMEM_T_UINT16 9
 
 /* reduce algorithms (Section 3.7.2, "Reduction") */
 #define ISHMEMX_REDUCE_AUTO 0
@@ -184,6 +188,31 @@ ISHMEM_DECL_RMA(uint32, uint32_t)
 ISHMEM_DECL_RMA(uint64, uint64_t)
 #undef ISHMEM_DECL_RMA
 
+/* Strided put / get (OpenSHMEM iput / iget; Section 3.7.1, "blocked or strided"): element k of
+ * the source, taken every `sst` elements, becomes element k*dst of the destination, k = 0 ..
+ * nelems-1.  Strides are in elements and at least 1; elem_size is 1, 2, 4, 8 or 16 bytes and both
+ * addresses must be aligned to it.  Symmetric side and ordering as for ishmem_putmem /
+ * ishmem_getmem; always a kernel of cooperating threads (no cutover). */
+int ishmemx_iputmem(int my_pe, void *dest, const void *src, size_t dst, size_t sst, size_t nelems,
+                    size_t elem_size, int pe);
+int ishmemx_igetmem(int my_pe, void *dest, const void *src, size_t dst, size_t sst, size_t nelems,
+                    size_t elem_size, int pe);
+#define ISHMEM_DECL_STRIDED(NAME, T)                                                          \
+    int ishmem_##NAME##_iput(int my_pe, T *dest, const T *src, size_t dst, size_t sst,        \
+                             size_t nelems, int pe);                                          \
+    int ishmem_##NAME##_iget(int my_pe, T *dest, const T *src, size_t dst, size_t sst,        \
+                             size_t nelems, int pe);
+ISHMEM_DECL_STRIDED(float, float)
+ISHMEM_DECL_STRIDED(double, double)
+ISHMEM_DECL_STRIDED(int, int)
+ISHMEM_DECL_STRIDED(long, long)
+ISHMEM_DECL_STRIDED(int32, int32_t)
+ISHMEM_DECL_STRIDED(int64, int64_t)
+ISHMEM_DECL_STRIDED(uint8, uint8_t)
+ISHMEM_DECL_STRIDED(uint32, uint32_t)
+ISHMEM_DECL_STRIDED(uint64, uint64_t)
+#undef ISHMEM_DECL_STRIDED
+
 /* Explicit thread-collaborative variants (Section 3.6; experiments of Section 4): a
  * kernel of `groups` blocks x `threads` threads is launched on my_pe's stream; the message
  * is cut into one contiguous slice per collaboration unit (thread / warp / block,
@@ -265,6 +294,20 @@ int ishmem_putmem_signal(int my_pe, void *dest, const void *src, size_t nbytes,
 /* Enqueues a bounded device-side wait on my_pe's stream until `*ivar`@my_pe cmp value.
  * On expiry the status word latches ISHMEM_ERR_TIMEOUT and the stream continues. */
 int ishmem_uint64_wait_until(int my_pe, uint64_t *ivar, int cmp, uint64_t value);
+/* One evaluation of the comparison on my_pe's copy of `ivar`, after everything already
+ * enqueued on my_pe's stream: HOST *result = 1 or 0.  Blocks the host. */
+int ishmem_uint64_test(int my_pe, uint64_t *ivar, int cmp, uint64_t value, int *result);
+/* Waits on `nelems` (at most 256) consecutive symmetric 64-bit words of my_pe (OpenSHMEM 1.5
+ * wait_until_all / _any / _some, without the optional status mask), bounded like
+ * ishmem_uint64_wait_until.  _all is stream-ordered.  _any writes the index of a satisfied word
+ * to HOST *index; _some waits for at least one and writes the ascending indices of all words
+ * satisfied at that moment to HOST indices[0..*count-1] (room for nelems).  _any and _some block
+ * the host and return ISHMEM_ERR_TIMEOUT when the wait gave up. */
+int ishmem_uint64_wait_until_all(int my_pe, uint64_t *ivars, size_t nelems, int cmp, uint64_t value);
+int ishmem_uint64_wait_until_any(int my_pe, uint64_t *ivars, size_t nelems, int cmp, uint64_t value,
+                                 size_t *index);
+int ishmem_uint64_wait_until_some(int my_pe, uint64_t *ivars, size_t nelems, size_t *indices, int cmp,
+                                  uint64_t value, size_t *count);
 /* fence: orders my_pe's earlier puts before its later ones per target (stream order
  * already gives this; kept for API parity).  quiet: completes all outstanding operations
  * of my_pe, including _nbi transfers on the copy engine, in stream order. */
@@ -329,6 +372,14 @@ int ishmemx_set_bcast_root_dest(int enable);
 /* fcollect: dest@q[i*nbytes:(i+1)*nbytes] = src@member_i for every member q (allgather
  * with equal contributions; push). */
 int ishmem_fcollectmem(ishmem_team_t team, void *dest, const void *src, size_t nbytes);
+/* collect: fcollect with contributions of different sizes ("collect (which is like MPI
+ * allgather)", Section 3.7.2): every member's dest becomes the concatenation, in team order, of
+ * the members' sources; member i contributes nbytes_per_member[i] bytes (HOST array of team-size
+ * entries -- all PEs live in this process, so the sizes need no exchange).  Push. */
+int ishmem_collectmem(ishmem_team_t team, void *dest, const void *src, const size_t *nbytes_per_member);
+/* alltoall (OpenSHMEM 1.5): dest@q[i*nbytes + k] = src@member_i[q*nbytes + k]: block q of member
+ * i's source lands in block i of member q's dest.  dest and src must not overlap.  Push. */
+int ishmem_alltoallmem(ishmem_team_t team, void *dest, const void *src, size_t nbytes);
 /* reduce: dest@q[j] = ((src@m0[j] op src@m1[j]) op ...) op src@m_{P-1}[j], folded in team
  * order (floating point bit-exact in that order), for every member q.  dest and src may
  * not overlap unless identical, which is handled with snapshot semantics only by the
@@ -352,6 +403,15 @@ ISHMEM_DECL_REDUCE_BITS(int32, int32_t)
 ISHMEM_DECL_REDUCE_BITS(int64, int64_t)
 ISHMEM_DECL_REDUCE_BITS(uint32, uint32_t)
 ISHMEM_DECL_REDUCE_BITS(uint64, uint64_t)
+/* "fixed-point datatypes from 8 to 64 bits" (Section 3.7.2): sum and product modulo 2^8 / 2^16 */
+ISHMEM_DECL_REDUCE_ARITH(int8, int8_t)
+ISHMEM_DECL_REDUCE_ARITH(uint8, uint8_t)
+ISHMEM_DECL_REDUCE_ARITH(int16, int16_t)
+ISHMEM_DECL_REDUCE_ARITH(uint16, uint16_t)
+ISHMEM_DECL_REDUCE_BITS(int8, int8_t)
+ISHMEM_DECL_REDUCE_BITS(uint8, uint8_t)
+ISHMEM_DECL_REDUCE_BITS(int16, int16_t)
+ISHMEM_DECL_REDUCE_BITS(uint16, uint16_t)
 #undef ISHMEM_DECL_REDUCE
 #undef ISHMEM_DECL_REDUCE_ARITH
 #undef ISHMEM_DECL_REDUCE_BITS
@@ -362,7 +422,7 @@ int ishmemx_set_collective_geometry(int groups_per_pe, int threads);
  * the device routine ishmemx_{broadcastmem,fcollectmem,reduce,sync_all}_work_group of
  * ishmem_device.cuh, with in-kernel push synchronisation (for tests and latency
  * measurements of the device API itself).  which: 0 broadcast, 1 fcollect, 2 reduce
- * (op/dtype as above), 3 sync_all repeated `repeat` times. */
+ * (op/dtype as above), 3 sync_all, 4 alltoall; the call is repeated `repeat` times. */
 int ishmemx_collective_on_device(int which, ishmem_team_t team, void *dest, const void *src,
                                  size_t n, int root, int op, int dtype, int threads, int repeat);
 

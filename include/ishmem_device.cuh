@@ -302,6 +302,35 @@ __device__ __forceinline__ void copy_bytes(char *d, const char *s, size_t n, uns
     for (size_t i = body + tid; i < n; i += nthr) stv<unsigned char>(d + i, ldv<unsigned char>(s + i));
 }
 
+/* Strided element copy (iput / iget, Section 3.7.1 "blocked or strided"): element k, taken every
+ * `sst` elements from s, goes to element k*dst of d, k = tid, tid+nthr, ...  ES = element size in
+ * bytes (1, 2, 4, 8 or 16); both addresses aligned to it. */
+template <int ES>
+__device__ __forceinline__ void strided_copy(char *d, const char *s, size_t dst, size_t sst, size_t nelems,
+                                             size_t tid, size_t nthr)
+{
+    for (size_t k = tid; k < nelems; k += nthr) {
+        char *pd = d + k * dst * ES;
+        const char *ps = s + k * sst * ES;
+        if (ES == 1) stv<unsigned char>(pd, ldv<unsigned char>(ps));
+        else if (ES == 2) stv<unsigned short>(pd, ldv<unsigned short>(ps));
+        else if (ES == 4) stv<unsigned>(pd, ldv<unsigned>(ps));
+        else if (ES == 8) stv<unsigned long long>(pd, ldv<unsigned long long>(ps));
+        else st16(pd, ld16(ps));
+    }
+}
+__device__ __forceinline__ void strided_copy_any(char *d, const char *s, size_t dst, size_t sst, size_t nelems,
+                                                 unsigned es, size_t tid, size_t nthr)
+{
+    switch (es) {
+    case 1: strided_copy<1>(d, s, dst, sst, nelems, tid, nthr); break;
+    case 2: strided_copy<2>(d, s, dst, sst, nelems, tid, nthr); break;
+    case 4: strided_copy<4>(d, s, dst, sst, nelems, tid, nthr); break;
+    case 8: strided_copy<8>(d, s, dst, sst, nelems, tid, nthr); break;
+    default: strided_copy<16>(d, s, dst, sst, nelems, tid, nthr); break;
+    }
+}
+
 /* ---- TMA bulk copy ring --------------------------------------------------------------- */
 
 __device__ __forceinline__ unsigned smem_u32(const void *p)
@@ -743,6 +772,46 @@ __device__ __forceinline__ void ishmemx_getmem_sub_group(const ishmem_ctx_t *ctx
     __syncwarp();
 }
 
+/* strided put / get (OpenSHMEM iput / iget): strides in elements, at least 1.  T of 1, 2, 4, 8
+ * or 16 bytes.  The plain forms are called by one thread, the _work_group forms by every thread
+ * of the block (they end with a block barrier). */
+template <typename T>
+__device__ __forceinline__ void ishmem_iput(const ishmem_ctx_t *ctx, T *dest, const T *src, size_t dst, size_t sst,
+                                            size_t nelems, int pe)
+{
+    char *r = ishmemi::translate(ctx, (char *)dest, pe);
+    if (r) ishmemi::strided_copy<sizeof(T)>(r, (const char *)src, dst, sst, nelems, 0, 1);
+}
+template <typename T>
+__device__ __forceinline__ void ishmem_iget(const ishmem_ctx_t *ctx, T *dest, const T *src, size_t dst, size_t sst,
+                                            size_t nelems, int pe)
+{
+    const char *r = ishmemi::translate(ctx, (const char *)src, pe);
+    if (r) ishmemi::strided_copy<sizeof(T)>((char *)dest, r, dst, sst, nelems, 0, 1);
+}
+template <typename T>
+__device__ __forceinline__ void ishmemx_iput_work_group(const ishmem_ctx_t *ctx, T *dest, const T *src, size_t dst,
+                                                        size_t sst, size_t nelems, int pe)
+{
+    char *r = ishmemi::translate(ctx, (char *)dest, pe);
+    if (r)
+        ishmemi::strided_copy<sizeof(T)>(r, (const char *)src, dst, sst, nelems,
+                                         threadIdx.x + blockDim.x * (threadIdx.y + blockDim.y * threadIdx.z),
+                                         blockDim.x * blockDim.y * blockDim.z);
+    __syncthreads();
+}
+template <typename T>
+__device__ __forceinline__ void ishmemx_iget_work_group(const ishmem_ctx_t *ctx, T *dest, const T *src, size_t dst,
+                                                        size_t sst, size_t nelems, int pe)
+{
+    const char *r = ishmemi::translate(ctx, (const char *)src, pe);
+    if (r)
+        ishmemi::strided_copy<sizeof(T)>((char *)dest, r, dst, sst, nelems,
+                                         threadIdx.x + blockDim.x * (threadIdx.y + blockDim.y * threadIdx.z),
+                                         blockDim.x * blockDim.y * blockDim.z);
+    __syncthreads();
+}
+
 /* work-group: every thread of the block takes part in a multi-threaded vectorised copy
  * (Sections 3.6, 3.7.1); with `staging` large aligned blocks are moved by TMA bulk copies
  * instead.  Returns 0 or ISHMEM_ERR_TIMEOUT (same value in every thread).  On return the
@@ -939,6 +1008,71 @@ __device__ __forceinline__ int ishmem_uint64_test(const ishmem_ctx_t *, const un
     return ishmemi::compare(ishmemi::ld_acquire(ivar), cmp, value) ? 1 : 0;
 }
 
+/* Waits on `nelems` consecutive 64-bit words of the calling PE (OpenSHMEM 1.5 wait_until_all /
+ * _any / _some; without the optional status mask).  One thread calls.  All three are bounded
+ * by ctx->wait_limit_ns and return 0 or ISHMEM_ERR_TIMEOUT (latched).
+ * _all: every word satisfies the comparison.
+ * _any: *index = some word that does (the lowest one found in a scan from 0).
+ * _some: waits until at least one does, then lists ALL that do at that moment in indices[]
+ *        (ascending, room for nelems entries) and their number in *count. */
+__device__ __forceinline__ int ishmem_uint64_wait_until_all(const ishmem_ctx_t *ctx, const unsigned long long *ivars,
+                                                            size_t nelems, int cmp, unsigned long long value)
+{
+    ishmemi::deadline dl(ctx->wait_limit_ns);
+    size_t k = 0;
+    while (k < nelems) {
+        if (ishmemi::compare(ishmemi::ld_acquire(ivars + k), cmp, value)) {
+            ++k;
+            continue;
+        }
+        if (dl.expired()) {
+            ishmemi::latch_error(ctx, ISHMEM_ERR_TIMEOUT);
+            return ISHMEM_ERR_TIMEOUT;
+        }
+        if (dl.polls > 64u) __nanosleep(32);
+    }
+    return 0;
+}
+__device__ __forceinline__ int ishmem_uint64_wait_until_any(const ishmem_ctx_t *ctx, const unsigned long long *ivars,
+                                                            size_t nelems, int cmp, unsigned long long value,
+                                                            size_t *index)
+{
+    ishmemi::deadline dl(ctx->wait_limit_ns);
+    if (nelems == 0) return 0;
+    for (;;) {
+        for (size_t k = 0; k < nelems; ++k)
+            if (ishmemi::compare(ishmemi::ld_acquire(ivars + k), cmp, value)) {
+                *index = k;
+                return 0;
+            }
+        if (dl.expired()) break;
+        if (dl.polls > 64u) __nanosleep(32);
+    }
+    ishmemi::latch_error(ctx, ISHMEM_ERR_TIMEOUT);
+    return ISHMEM_ERR_TIMEOUT;
+}
+__device__ __forceinline__ int ishmem_uint64_wait_until_some(const ishmem_ctx_t *ctx, const unsigned long long *ivars,
+                                                             size_t nelems, size_t *indices, int cmp,
+                                                             unsigned long long value, size_t *count)
+{
+    ishmemi::deadline dl(ctx->wait_limit_ns);
+    *count = 0;
+    if (nelems == 0) return 0;
+    for (;;) {
+        size_t n = 0;
+        for (size_t k = 0; k < nelems; ++k)
+            if (ishmemi::compare(ishmemi::ld_acquire(ivars + k), cmp, value)) indices[n++] = k;
+        if (n) {
+            *count = n;
+            return 0;
+        }
+        if (dl.expired()) break;
+        if (dl.polls > 64u) __nanosleep(32);
+    }
+    ishmemi::latch_error(ctx, ISHMEM_ERR_TIMEOUT);
+    return ISHMEM_ERR_TIMEOUT;
+}
+
 /* ---- remote atomics (scalar: no work-group forms, Section 3.6) --------------------------- */
 /* T in {int, unsigned, long long, unsigned long long, long, unsigned long, int32_t, ...}
  * of 4 or 8 bytes.  Relaxed at .gpu scope; ordering comes from fence / quiet. */
@@ -1103,6 +1237,32 @@ template <typename T, int OP>
 struct folder<T, OP, true> {
     static __device__ __forceinline__ T f(T a, T x) { return combine_bits<T, OP>(a, x); }
 };
+/* 8- and 16-bit integers are promoted to int by the arithmetic operators; sum and product are
+ * taken in unsigned int (no signed overflow) and cut back to the element's width */
+#define ISHMEMI_NARROW_FOLDER(T)                                                                   \
+    template <int OP>                                                                              \
+    struct folder<T, OP, false> {                                                                  \
+        static __device__ __forceinline__ T f(T a, T x)                                            \
+        {                                                                                          \
+            if (OP == ISHMEM_OP_SUM) return (T)((unsigned)a + (unsigned)x);                        \
+            if (OP == ISHMEM_OP_PROD) return (T)((unsigned)a * (unsigned)x);                       \
+            return combine<T, OP>(a, x);                                                           \
+        }                                                                                          \
+    };                                                                                             \
+    template <int OP>                                                                              \
+    struct folder<T, OP, true> {                                                                   \
+        static __device__ __forceinline__ T f(T a, T x)                                            \
+        {                                                                                          \
+            if (OP == ISHMEM_OP_AND) return (T)((unsigned)a & (unsigned)x);                        \
+            if (OP == ISHMEM_OP_OR) return (T)((unsigned)a | (unsigned)x);                         \
+            return (T)((unsigned)a ^ (unsigned)x);                                                 \
+        }                                                                                          \
+    };
+ISHMEMI_NARROW_FOLDER(signed char)
+ISHMEMI_NARROW_FOLDER(unsigned char)
+ISHMEMI_NARROW_FOLDER(short)
+ISHMEMI_NARROW_FOLDER(unsigned short)
+#undef ISHMEMI_NARROW_FOLDER
 /* signed integer sum/prod must wrap: do them unsigned */
 template <int OP>
 struct folder<int, OP, false> {
@@ -1431,6 +1591,23 @@ __device__ __forceinline__ int ishmemx_fcollectmem_work_group(const ishmem_ctx_t
     if (ok && me >= 0)
         ishmemi::push_bytes((char *)dest + (size_t)me * nbytes, delta, t.size, -1, (const char *)src,
                             nbytes, ishmemi::block_tid(), ishmemi::block_nthr());
+    int rc = ishmemx_team_sync_work_group(ctx, team);
+    return ok ? rc : ISHMEM_ERR_INVALID_PE;
+}
+
+/* alltoall: every member stores block q of its source into block `my index` of member q's dest
+ * (push, destinations in the inner loop like broadcast), then the team synchronises. */
+__device__ __forceinline__ int ishmemx_alltoallmem_work_group(const ishmem_ctx_t *ctx, ishmem_team_t team,
+                                                              void *dest, const void *src, size_t nbytes)
+{
+    __shared__ long long delta[ISHMEM_MAX_PES];
+    const ishmemi_team t = ctx->teams[team];
+    const int me = ishmemi::team_index(t, ctx->my_pe);
+    const bool ok = ishmemi::team_deltas(ctx, t, delta);
+    if (ok && me >= 0)
+        for (int q = 0; q < t.size; ++q)
+            ishmemi::copy_bytes((char *)dest + delta[q] + (size_t)me * nbytes, (const char *)src + (size_t)q * nbytes,
+                                nbytes, ishmemi::block_tid(), ishmemi::block_nthr());
     int rc = ishmemx_team_sync_work_group(ctx, team);
     return ok ? rc : ISHMEM_ERR_INVALID_PE;
 }

@@ -41,7 +41,7 @@ ISHMEM_CMP_EQ, ISHMEM_CMP_NE, ISHMEM_CMP_GT, ISHMEM_CMP_GE, ISHMEM_CMP_LT, ISHME
 (ISHMEM_OP_SUM, ISHMEM_OP_MAX, ISHMEM_OP_MIN, ISHMEM_OP_PROD, ISHMEM_OP_AND, ISHMEM_OP_OR,
  ISHMEM_OP_XOR) = range(7)
 (ISHMEM_T_INT32, ISHMEM_T_INT64, ISHMEM_T_FLOAT, ISHMEM_T_DOUBLE, ISHMEM_T_UINT32,
- ISHMEM_T_UINT64) = range(6)
+ ISHMEM_T_UINT64, ISHMEM_T_INT8, ISHMEM_T_UINT8, ISHMEM_T_INT16, ISHMEM_T_UINT16) = range(10)
 ISHMEMX_REDUCE_AUTO, ISHMEMX_REDUCE_DUPLICATED, ISHMEMX_REDUCE_SPLIT = range(3)
 SIZE_MAX = 2**64 - 1
 
@@ -82,8 +82,8 @@ _CT = {"i": C.c_int, "z": C.c_size_t, "p": _Ptr, "u64": C.c_uint64, "i64": C.c_i
 _RMA_TYPES = {"float": "f", "double": "d", "int": "i", "long": "l", "int32": "i32", "int64": "i64",
               "uint8": "u8", "uint32": "u32", "uint64": "u64"}
 _AMO_TYPES = {"int32": "i32", "int64": "i64", "uint32": "u32", "uint64": "u64"}
-_REDUCE_ARITH = ["int32", "int64", "uint32", "uint64", "float", "double"]
-_REDUCE_BITS = ["int32", "int64", "uint32", "uint64"]
+_REDUCE_ARITH = ["int32", "int64", "uint32", "uint64", "float", "double", "int8", "uint8", "int16", "uint16"]
+_REDUCE_BITS = ["int32", "int64", "uint32", "uint64", "int8", "uint8", "int16", "uint16"]
 
 
 def _signatures() -> dict[str, tuple[str, list[str]]]:
@@ -125,6 +125,14 @@ def _signatures() -> dict[str, tuple[str, list[str]]]:
         "ishmemx_tune_cutover": ("status", ["i", "i", "z", "p"]),
         "ishmem_putmem_signal": ("status", ["i", "p", "p", "z", "p", "u64", "i", "i"]),
         "ishmem_uint64_wait_until": ("status", ["i", "p", "i", "u64"]),
+        "ishmemx_iputmem": ("status", ["i", "p", "p", "z", "z", "z", "z", "i"]),
+        "ishmemx_igetmem": ("status", ["i", "p", "p", "z", "z", "z", "z", "i"]),
+        "ishmem_uint64_test": ("status", ["i", "p", "i", "u64", "p"]),
+        "ishmem_uint64_wait_until_all": ("status", ["i", "p", "z", "i", "u64"]),
+        "ishmem_uint64_wait_until_any": ("status", ["i", "p", "z", "i", "u64", "p"]),
+        "ishmem_uint64_wait_until_some": ("status", ["i", "p", "z", "p", "i", "u64", "p"]),
+        "ishmem_collectmem": ("status", ["i", "p", "p", "p"]),
+        "ishmem_alltoallmem": ("status", ["i", "p", "p", "z"]),
         "ishmem_fence": ("status", ["i"]),
         "ishmem_quiet": ("status", ["i"]),
         "ishmem_team_sync": ("status", ["i"]),
@@ -154,6 +162,8 @@ def _signatures() -> dict[str, tuple[str, list[str]]]:
     for name, t in _RMA_TYPES.items():
         for op in ("put", "get", "put_nbi", "get_nbi"):
             S[f"ishmem_{name}_{op}"] = ("status", ["i", "p", "p", "z", "i"])
+        S[f"ishmem_{name}_iput"] = ("status", ["i", "p", "p", "z", "z", "z", "i"])
+        S[f"ishmem_{name}_iget"] = ("status", ["i", "p", "p", "z", "z", "z", "i"])
         S[f"ishmem_{name}_p"] = ("status", ["i", "p", t, "i"])
         S[f"ishmem_{name}_g"] = ("status", ["i", "p", "p", "i"])
     for name, t in _AMO_TYPES.items():

@@ -62,6 +62,47 @@ __global__ void __launch_bounds__(1024) k_fcollect(const ishmem_ctx_t *ctxs, col
                      local_of(ctxs, ctx, a.src), a.n, st, g, (size_t)a.groups, a.push_tile);
 }
 
+/* ---- collect: fcollect with a size and an offset per member ------------------------------------ */
+struct collect_args {
+    ishmem_team_t team;
+    char *dest;
+    const char *src;
+    int groups;
+    unsigned tile;
+    unsigned long long nbytes[ISHMEM_MAX_PES], offset[ISHMEM_MAX_PES];
+};
+__global__ void __launch_bounds__(1024) k_collect(const ishmem_ctx_t *ctxs, collect_args a)
+{
+    __shared__ long long delta[ISHMEM_MAX_PES];
+    const ishmemi_team t = ctxs[0].teams[a.team];
+    const unsigned me = blockIdx.x % (unsigned)t.size, g = blockIdx.x / (unsigned)t.size;
+    const ishmem_ctx_t *ctx = ctxs + (t.start + (int)me * t.stride);
+    if (!ishmemi::team_deltas(ctx, t, delta)) return;
+    ishmemx_staging_t st = {nullptr, 0};
+    ishmemi::wg_push(ctx, local_of(ctxs, ctx, a.dest) + a.offset[me], delta, t.size, -1, local_of(ctxs, ctx, a.src),
+                     (size_t)a.nbytes[me], st, g, (size_t)a.groups, a.tile);
+}
+
+/* ---- alltoall: member i's blocks store block q of its source into block i of member q's dest ---- */
+__global__ void __launch_bounds__(1024) k_alltoall(const ishmem_ctx_t *ctxs, coll_args a)
+{
+    __shared__ long long delta[ISHMEM_MAX_PES];
+    const ishmemi_team t = ctxs[0].teams[a.team];
+    const unsigned me = blockIdx.x % (unsigned)t.size, g = blockIdx.x / (unsigned)t.size;
+    const ishmem_ctx_t *ctx = ctxs + (t.start + (int)me * t.stride);
+    if (!ishmemi::team_deltas(ctx, t, delta)) return;
+    const char *src = local_of(ctxs, ctx, a.src);
+    char *dest = local_of(ctxs, ctx, a.dest) + (size_t)me * a.n;
+    /* (destination, tile) pairs dealt round-robin, the destination running fastest so that
+     * consecutive tiles go to different PEs */
+    const size_t tile = a.push_tile, per = (a.n + tile - 1) / tile, total = per * (size_t)t.size;
+    for (size_t k = g; k < total; k += (size_t)a.groups) {
+        const size_t q = k % (size_t)t.size, o = (k / (size_t)t.size) * tile;
+        const size_t len = a.n - o < tile ? a.n - o : tile;
+        ishmemi::copy_bytes(dest + delta[q] + o, src + q * a.n + o, len, threadIdx.x, blockDim.x);
+    }
+}
+
 /* ---- reduce ------------------------------------------------------------------------------- */
 /* split: member q owns a contiguous address range, folds it from all sources in team order
  * and stores the result into every member's dest (traffic: each source and each dest once).
@@ -143,6 +184,10 @@ static reduce_kernel_t pick_reduce(int op, int dtype)
     case ISHMEM_T_UINT64: return pick_int<unsigned long long>(op);
     case ISHMEM_T_FLOAT: return pick_arith<float>(op);
     case ISHMEM_T_DOUBLE: return pick_arith<double>(op);
+    case ISHMEM_T_INT8: return pick_int<signed char>(op);
+    case ISHMEM_T_UINT8: return pick_int<unsigned char>(op);
+    case ISHMEM_T_INT16: return pick_int<short>(op);
+    case ISHMEM_T_UINT16: return pick_int<unsigned short>(op);
     default: return nullptr;
     }
 }
@@ -151,12 +196,14 @@ static size_t dtype_size(int dtype)
     switch (dtype) {
     case ISHMEM_T_INT32: case ISHMEM_T_UINT32: case ISHMEM_T_FLOAT: return 4;
     case ISHMEM_T_INT64: case ISHMEM_T_UINT64: case ISHMEM_T_DOUBLE: return 8;
+    case ISHMEM_T_INT8: case ISHMEM_T_UINT8: return 1;
+    case ISHMEM_T_INT16: case ISHMEM_T_UINT16: return 2;
     default: return 0;
     }
 }
 
 /* ---- device-resident forms: one work-group per member, in-kernel push sync ---------------- */
-/* WHICH: 0 broadcast, 1 fcollect, 2 reduce<T, OP>, 3 sync */
+/* WHICH: 0 broadcast, 1 fcollect, 2 reduce<T, OP>, 3 sync, 4 alltoall */
 template <int WHICH, typename T, int OP>
 __global__ void __launch_bounds__(1024) k_collective_on_device(const ishmem_ctx_t *ctxs, coll_args a)
 {
@@ -169,6 +216,7 @@ __global__ void __launch_bounds__(1024) k_collective_on_device(const ishmem_ctx_
         if (WHICH == 0) rc = ishmemx_broadcastmem_work_group(ctx, a.team, d, s, a.n, a.root);
         else if (WHICH == 1) rc = ishmemx_fcollectmem_work_group(ctx, a.team, d, s, a.n);
         else if (WHICH == 2) rc = ishmemx_reduce_work_group<T, OP>(ctx, a.team, (T *)d, (const T *)s, a.n);
+        else if (WHICH == 4) rc = ishmemx_alltoallmem_work_group(ctx, a.team, d, s, a.n);
         else rc = ishmemx_team_sync_work_group(ctx, a.team);
         if (rc) return; /* the error is latched; every member gives up the same way */
     }
@@ -200,6 +248,7 @@ static reduce_kernel_t pick_dev(int which, int op, int dtype)
     if (which == 0) return k_collective_on_device<0, int, 0>;
     if (which == 1) return k_collective_on_device<1, int, 0>;
     if (which == 3) return k_collective_on_device<3, int, 0>;
+    if (which == 4) return k_collective_on_device<4, int, 0>;
     switch (dtype) {
     case ISHMEM_T_INT32: return pick_dev_int<int>(op);
     case ISHMEM_T_INT64: return pick_dev_int<long long>(op);
@@ -207,6 +256,10 @@ static reduce_kernel_t pick_dev(int which, int op, int dtype)
     case ISHMEM_T_UINT64: return pick_dev_int<unsigned long long>(op);
     case ISHMEM_T_FLOAT: return pick_dev_arith<float>(op);
     case ISHMEM_T_DOUBLE: return pick_dev_arith<double>(op);
+    case ISHMEM_T_INT8: return pick_dev_int<signed char>(op);
+    case ISHMEM_T_UINT8: return pick_dev_int<unsigned char>(op);
+    case ISHMEM_T_INT16: return pick_dev_int<short>(op);
+    case ISHMEM_T_UINT16: return pick_dev_int<unsigned short>(op);
     default: return nullptr;
     }
 }
@@ -405,6 +458,87 @@ extern "C" int ishmem_fcollectmem(ishmem_team_t team, void *dest, const void *sr
     return rc;
 }
 
+extern "C" int ishmem_collectmem(ishmem_team_t team, void *dest, const void *src, const size_t *nbytes_per_member)
+{
+    auto &g = g_ishmem;
+    ISHMEMI_REQUIRE_INIT();
+    ishmemi_team t;
+    int rc = team_of(team, &t);
+    if (rc) return rc;
+    if (!nbytes_per_member) return ISHMEM_ERR_ARG;
+    collect_args a = {};
+    size_t total = 0, largest = 0;
+    for (int i = 0; i < t.size; ++i) {
+        const size_t n = nbytes_per_member[i];
+        if (n > g.heap_bytes || total > g.heap_bytes - n) return ISHMEM_ERR_NOT_SYMMETRIC;
+        a.nbytes[i] = n;
+        a.offset[i] = total;
+        total += n;
+        if (n > largest) largest = n;
+    }
+    if ((rc = check_sym2(dest, total, src, largest))) return rc;
+    const char *d = (const char *)dest, *sp = (const char *)src;
+    if (total && d < sp + largest && sp < d + total) return ISHMEM_ERR_ARG;
+    cudaStream_t s;
+    if ((rc = ishmemi_team_stream_begin(team, &s))) return rc;
+    if (total) {
+        a.team = team;
+        a.dest = (char *)dest;
+        a.src = sp;
+        const bool shaped = g.coll_groups > 0;
+        push_shape sh = push_geometry(largest < ((size_t)1 << 20) ? largest : ((size_t)1 << 20) - 1, t.size, t.size,
+                                      (const void *)k_collect); /* loads/stores only: sizes differ per member */
+        if (!shaped && largest >= ((size_t)1 << 20)) {
+            size_t cap = ((size_t)g.sm_count * 4 + t.size - 1) / t.size, want = (largest + 16383) / 16384;
+            sh.blocks_per_member = (int)(want < cap ? want : cap);
+            sh.tile = 16384;
+            sh.staging = 0;
+            sh.threads = g.coll_threads;
+        }
+        a.groups = sh.blocks_per_member;
+        a.tile = sh.tile;
+        k_collect<<<a.groups * t.size, sh.threads, 0, s>>>(g.d_ctx, a);
+        ishmemi_count_launch();
+        rc = ishmemi_check_launch("k_collect");
+    }
+    ishmemi_team_stream_end();
+    return rc;
+}
+
+extern "C" int ishmem_alltoallmem(ishmem_team_t team, void *dest, const void *src, size_t nbytes)
+{
+    auto &g = g_ishmem;
+    ISHMEMI_REQUIRE_INIT();
+    ishmemi_team t;
+    int rc = team_of(team, &t);
+    if (rc) return rc;
+    if (nbytes && (size_t)t.size > (size_t)-1 / nbytes) return ISHMEM_ERR_ARG;
+    const size_t all = nbytes * t.size;
+    if ((rc = check_sym2(dest, all, src, all))) return rc;
+    const char *d = (const char *)dest, *sp = (const char *)src;
+    if (all && d < sp + all && sp < d + all) return ISHMEM_ERR_ARG;
+    cudaStream_t s;
+    if ((rc = ishmemi_team_stream_begin(team, &s))) return rc;
+    if (nbytes) {
+        coll_args a = {};
+        a.team = team;
+        a.dest = (char *)dest;
+        a.src = sp;
+        a.n = nbytes;
+        size_t tile = 16384;
+        const size_t cap = ((size_t)g.sm_count * 4 + t.size - 1) / t.size;
+        while (tile > 2048 && (all + tile - 1) / tile < cap) tile >>= 1;
+        size_t want = ((nbytes + tile - 1) / tile) * t.size;
+        a.push_tile = (unsigned)tile;
+        a.groups = g.coll_groups > 0 ? g.coll_groups : (int)(want < cap ? (want < 1 ? 1 : want) : cap);
+        k_alltoall<<<a.groups * t.size, all <= 65536 ? 256 : g.coll_threads, 0, s>>>(g.d_ctx, a);
+        ishmemi_count_launch();
+        rc = ishmemi_check_launch("k_alltoall");
+    }
+    ishmemi_team_stream_end();
+    return rc;
+}
+
 extern "C" int ishmemx_reduce(ishmem_team_t team, void *dest, const void *src, size_t nreduce, int op, int dtype,
                               int algorithm)
 {
@@ -506,6 +640,14 @@ ISHMEMI_DEF_REDUCE_BITS(int32, int32_t, ISHMEM_T_INT32)
 ISHMEMI_DEF_REDUCE_BITS(int64, int64_t, ISHMEM_T_INT64)
 ISHMEMI_DEF_REDUCE_BITS(uint32, uint32_t, ISHMEM_T_UINT32)
 ISHMEMI_DEF_REDUCE_BITS(uint64, uint64_t, ISHMEM_T_UINT64)
+ISHMEMI_DEF_REDUCE_ARITH(int8, int8_t, ISHMEM_T_INT8)
+ISHMEMI_DEF_REDUCE_ARITH(uint8, uint8_t, ISHMEM_T_UINT8)
+ISHMEMI_DEF_REDUCE_ARITH(int16, int16_t, ISHMEM_T_INT16)
+ISHMEMI_DEF_REDUCE_ARITH(uint16, uint16_t, ISHMEM_T_UINT16)
+ISHMEMI_DEF_REDUCE_BITS(int8, int8_t, ISHMEM_T_INT8)
+ISHMEMI_DEF_REDUCE_BITS(uint8, uint8_t, ISHMEM_T_UINT8)
+ISHMEMI_DEF_REDUCE_BITS(int16, int16_t, ISHMEM_T_INT16)
+ISHMEMI_DEF_REDUCE_BITS(uint16, uint16_t, ISHMEM_T_UINT16)
 
 extern "C" int ishmemx_collective_on_device(int which, ishmem_team_t team, void *dest, const void *src, size_t n,
                                             int root, int op, int dtype, int threads, int repeat)
@@ -515,7 +657,7 @@ extern "C" int ishmemx_collective_on_device(int which, ishmem_team_t team, void 
     ishmemi_team t;
     int rc = team_of(team, &t);
     if (rc) return rc;
-    if (which < 0 || which > 3 || threads < 32 || threads > 1024 || repeat < 1) return ISHMEM_ERR_ARG;
+    if (which < 0 || which > 4 || threads < 32 || threads > 1024 || repeat < 1) return ISHMEM_ERR_ARG;
     if (which != 3) {
         size_t es = 1;
         if (which == 2) {
@@ -525,7 +667,7 @@ extern "C" int ishmemx_collective_on_device(int which, ishmem_team_t team, void 
         }
         if (which == 0 && (root < 0 || root >= t.size)) return ISHMEM_ERR_INVALID_PE;
         if (n > (size_t)-1 / (es * t.size)) return ISHMEM_ERR_ARG;
-        size_t sbytes = n * es, dbytes = which == 1 ? sbytes * t.size : sbytes;
+        size_t sbytes = (which == 4 ? n * t.size : n * es), dbytes = (which == 1 || which == 4) ? n * es * t.size : sbytes;
         if ((rc = check_sym2(dest, dbytes, src, sbytes))) return rc;
         const char *d = (const char *)dest, *sp = (const char *)src;
         if (d < sp + sbytes && sp < d + dbytes) return ISHMEM_ERR_ARG;

@@ -122,6 +122,46 @@ __global__ void k_wait_until(const ishmem_ctx_t *ctxs, int my_pe, const unsigned
     ishmem_uint64_wait_until(ctxs + my_pe, ivar, cmp, value);
 }
 
+/* strided put/get: the blocks of the launch share the elements, one element per thread and step */
+__global__ void __launch_bounds__(256) k_strided(const ishmem_ctx_t *ctxs, int my_pe, char *dest, const char *src,
+                                                 size_t dst, size_t sst, size_t nelems, unsigned es, int pe, int is_get)
+{
+    const ishmem_ctx_t *ctx = ctxs + my_pe;
+    char *d = dest;
+    const char *s = src;
+    if (is_get) s = ishmem_ptr(ctx, src, pe);
+    else d = ishmem_ptr(ctx, dest, pe);
+    if (!d || !s) return;
+    ishmemi::strided_copy_any(d, s, dst, sst, nelems, es, (size_t)blockIdx.x * blockDim.x + threadIdx.x,
+                              (size_t)gridDim.x * blockDim.x);
+}
+
+/* which: 0 all, 1 any, 2 some; results (index / count + indices) go to host-mapped memory */
+__global__ void k_wait_many(const ishmem_ctx_t *ctxs, int my_pe, const unsigned long long *ivars, size_t nelems,
+                            int cmp, unsigned long long value, int which, unsigned long long *out)
+{
+    const ishmem_ctx_t *ctx = ctxs + my_pe;
+    if (which == 0) {
+        ishmem_uint64_wait_until_all(ctx, ivars, nelems, cmp, value);
+    } else if (which == 1) {
+        size_t idx = 0;
+        int rc = ishmem_uint64_wait_until_any(ctx, ivars, nelems, cmp, value, &idx);
+        out[0] = (unsigned long long)(long long)rc;
+        out[1] = idx;
+    } else {
+        size_t cnt = 0;
+        int rc = ishmem_uint64_wait_until_some(ctx, ivars, nelems, (size_t *)(out + 2), cmp, value, &cnt);
+        out[0] = (unsigned long long)(long long)rc;
+        out[1] = cnt;
+    }
+}
+
+__global__ void k_test(const ishmem_ctx_t *ctxs, int my_pe, const unsigned long long *ivar, int cmp,
+                       unsigned long long value, int *out)
+{
+    *out = ishmem_uint64_test(ctxs + my_pe, ivar, cmp, value);
+}
+
 /* ---- launch helpers --------------------------------------------------------------------- */
 
 static unsigned g_bulk_smem = 0;
@@ -325,6 +365,60 @@ ISHMEMI_DEF_RMA(uint8, uint8_t)
 ISHMEMI_DEF_RMA(uint32, uint32_t)
 ISHMEMI_DEF_RMA(uint64, uint64_t)
 
+static int strided(int my_pe, void *dest, const void *src, size_t dst, size_t sst, size_t nelems, size_t es, int pe,
+                   bool is_get)
+{
+    ISHMEMI_REQUIRE_INIT();
+    if (ishmemi_check_pe(my_pe) || ishmemi_check_pe(pe)) return ISHMEM_ERR_INVALID_PE;
+    if (es != 1 && es != 2 && es != 4 && es != 8 && es != 16) return ISHMEM_ERR_ARG;
+    if (dst < 1 || sst < 1) return ISHMEM_ERR_ARG;
+    if (nelems == 0) return ISHMEM_OK;
+    if (!dest || !src) return ISHMEM_ERR_ARG;
+    if (((uintptr_t)dest | (uintptr_t)src) % es) return ISHMEM_ERR_ALIGN;
+    if ((nelems - 1) > ((size_t)-1 / es - 1) / (dst > sst ? dst : sst)) return ISHMEM_ERR_ARG;
+    const size_t dspan = ((nelems - 1) * dst + 1) * es, sspan = ((nelems - 1) * sst + 1) * es;
+    if (ishmemi_sym_offset(is_get ? src : (const void *)dest, is_get ? sspan : dspan) < 0)
+        return ISHMEM_ERR_NOT_SYMMETRIC;
+    char *dl = ishmemi_localise(dest, dspan, my_pe);
+    const char *sl = ishmemi_localise(src, sspan, my_pe);
+    size_t blocks = (nelems + 255) / 256, cap = (size_t)g_ishmem.sm_count * 8;
+    if (blocks > cap) blocks = cap;
+    k_strided<<<(unsigned)blocks, 256, 0, ishmemi_pe_stream_for_op(my_pe)>>>(g_ishmem.d_ctx, my_pe, dl, sl, dst, sst,
+                                                                             nelems, (unsigned)es, pe, is_get ? 1 : 0);
+    ishmemi_count_launch();
+    return ishmemi_check_launch("k_strided");
+}
+extern "C" int ishmemx_iputmem(int my_pe, void *dest, const void *src, size_t dst, size_t sst, size_t nelems,
+                               size_t elem_size, int pe)
+{
+    return strided(my_pe, dest, src, dst, sst, nelems, elem_size, pe, false);
+}
+extern "C" int ishmemx_igetmem(int my_pe, void *dest, const void *src, size_t dst, size_t sst, size_t nelems,
+                               size_t elem_size, int pe)
+{
+    return strided(my_pe, dest, src, dst, sst, nelems, elem_size, pe, true);
+}
+#define ISHMEMI_DEF_STRIDED(NAME, T)                                                                          \
+    extern "C" int ishmem_##NAME##_iput(int my_pe, T *dest, const T *src, size_t dst, size_t sst, size_t nelems, \
+                                        int pe)                                                               \
+    {                                                                                                         \
+        return strided(my_pe, dest, src, dst, sst, nelems, sizeof(T), pe, false);                             \
+    }                                                                                                         \
+    extern "C" int ishmem_##NAME##_iget(int my_pe, T *dest, const T *src, size_t dst, size_t sst, size_t nelems, \
+                                        int pe)                                                               \
+    {                                                                                                         \
+        return strided(my_pe, dest, src, dst, sst, nelems, sizeof(T), pe, true);                              \
+    }
+ISHMEMI_DEF_STRIDED(float, float)
+ISHMEMI_DEF_STRIDED(double, double)
+ISHMEMI_DEF_STRIDED(int, int)
+ISHMEMI_DEF_STRIDED(long, long)
+ISHMEMI_DEF_STRIDED(int32, int32_t)
+ISHMEMI_DEF_STRIDED(int64, int64_t)
+ISHMEMI_DEF_STRIDED(uint8, uint8_t)
+ISHMEMI_DEF_STRIDED(uint32, uint32_t)
+ISHMEMI_DEF_STRIDED(uint64, uint64_t)
+
 static int on_device(int my_pe, void *dest, const void *src, size_t n, int pe, int level, int threads,
                      int groups, bool is_get)
 {
@@ -466,6 +560,66 @@ extern "C" int ishmem_uint64_wait_until(int my_pe, uint64_t *ivar, int cmp, uint
     k_wait_until<<<1, 1, 0, ishmemi_pe_stream_for_op(my_pe)>>>(g_ishmem.d_ctx, my_pe, il, cmp, value);
     ishmemi_count_launch();
     return ishmemi_check_launch("k_wait_until");
+}
+
+extern "C" int ishmem_uint64_test(int my_pe, uint64_t *ivar, int cmp, uint64_t value, int *result)
+{
+    ISHMEMI_REQUIRE_INIT();
+    if (ishmemi_check_pe(my_pe)) return ISHMEM_ERR_INVALID_PE;
+    if ((uintptr_t)ivar % 8) return ISHMEM_ERR_ALIGN;
+    if (ishmemi_sym_offset(ivar, 8) < 0) return ISHMEM_ERR_NOT_SYMMETRIC;
+    if (cmp < ISHMEM_CMP_EQ || cmp > ISHMEM_CMP_LE || !result) return ISHMEM_ERR_ARG;
+    const unsigned long long *il = (const unsigned long long *)ishmemi_localise(ivar, 8, my_pe);
+    cudaStream_t s = ishmemi_pe_stream_for_op(my_pe);
+    k_test<<<1, 1, 0, s>>>(g_ishmem.d_ctx, my_pe, il, cmp, value, (int *)g_ishmem.h_pinned);
+    ishmemi_count_launch();
+    int rc = ishmemi_check_launch("k_test");
+    if (rc) return rc;
+    ISHMEMI_CUDA(cudaStreamSynchronize(s));
+    *result = *(int *)g_ishmem.h_pinned;
+    return ISHMEM_OK;
+}
+
+static int wait_many(int my_pe, uint64_t *ivars, size_t nelems, int cmp, uint64_t value, int which, size_t *index,
+                     size_t *indices, size_t *count)
+{
+    ISHMEMI_REQUIRE_INIT();
+    if (ishmemi_check_pe(my_pe)) return ISHMEM_ERR_INVALID_PE;
+    if ((uintptr_t)ivars % 8) return ISHMEM_ERR_ALIGN;
+    if (nelems > 256) return ISHMEM_ERR_ARG;
+    if (ishmemi_sym_offset(ivars, nelems * 8) < 0) return ISHMEM_ERR_NOT_SYMMETRIC;
+    if (cmp < ISHMEM_CMP_EQ || cmp > ISHMEM_CMP_LE) return ISHMEM_ERR_ARG;
+    if ((which == 1 && !index) || (which == 2 && (!indices || !count))) return ISHMEM_ERR_ARG;
+    const unsigned long long *il = (const unsigned long long *)ishmemi_localise(ivars, nelems * 8, my_pe);
+    cudaStream_t s = ishmemi_pe_stream_for_op(my_pe);
+    unsigned long long *out = (unsigned long long *)g_ishmem.h_pinned; /* 4096 B: 2 + 256 words */
+    k_wait_many<<<1, 1, 0, s>>>(g_ishmem.d_ctx, my_pe, il, nelems, cmp, value, which, out);
+    ishmemi_count_launch();
+    int rc = ishmemi_check_launch("k_wait_many");
+    if (rc || which == 0) return rc;
+    ISHMEMI_CUDA(cudaStreamSynchronize(s));
+    if ((long long)out[0]) return (int)(long long)out[0];
+    if (which == 1) {
+        *index = (size_t)out[1];
+    } else {
+        *count = (size_t)out[1];
+        for (size_t k = 0; k < *count; ++k) indices[k] = (size_t)out[2 + k];
+    }
+    return ISHMEM_OK;
+}
+extern "C" int ishmem_uint64_wait_until_all(int my_pe, uint64_t *ivars, size_t nelems, int cmp, uint64_t value)
+{
+    return wait_many(my_pe, ivars, nelems, cmp, value, 0, nullptr, nullptr, nullptr);
+}
+extern "C" int ishmem_uint64_wait_until_any(int my_pe, uint64_t *ivars, size_t nelems, int cmp, uint64_t value,
+                                            size_t *index)
+{
+    return wait_many(my_pe, ivars, nelems, cmp, value, 1, index, nullptr, nullptr);
+}
+extern "C" int ishmem_uint64_wait_until_some(int my_pe, uint64_t *ivars, size_t nelems, size_t *indices, int cmp,
+                                             uint64_t value, size_t *count)
+{
+    return wait_many(my_pe, ivars, nelems, cmp, value, 2, nullptr, indices, count);
 }
 
 extern "C" int ishmem_fence(int my_pe)
