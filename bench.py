@@ -200,7 +200,7 @@ def run_ours(args) -> dict:
         B.ishmem_uint64_p(0, ppsig, 0, 0)
         B.ishmem_uint64_p(1, ppsig, 0, 1)
         B.ishmemx_pingpong(0, 1, ppdata, ppsig, S["pp_bytes"], S["pp_rounds"], 256, rtt, bad)
-        B.ishmemx_int64_atomic_fetch_add_batch(table, word, inc, fetched, NOPS_FADD, 256, 1)
+        B.ishmemx_int64_atomic_fetch_add_batch(table, word, inc, fetched, NOPS_FADD, 1024, 2)
         B.ishmemx_int64_atomic_compare_swap_batch(table, cword, ccond, cval, fetched, NOPS_CAS, 256)
         B.ishmem_broadcastmem(B.ISHMEM_TEAM_WORLD, dst, src, S["bcast"], 0)
         B.ishmem_fcollectmem(B.ISHMEM_TEAM_WORLD, dst, src, S["fcollect"])
@@ -307,7 +307,9 @@ def breakdown(B, torch, team_stream, env) -> dict:
         "broadcast": lambda: B.ishmem_broadcastmem(W, dst, src, S["bcast"], 0),
         "fcollect": lambda: B.ishmem_fcollectmem(W, dst, src, S["fcollect"]),
         "reduce_f32": lambda: B.ishmem_float_sum_reduce(W, dst, src, S["reduce_f32"]),
-        "fetch_add": lambda: B.ishmemx_int64_atomic_fetch_add_batch(table, word, inc, fetched, NOPS_FADD, 256, 1),
+        "fetch_add": lambda: B.ishmemx_int64_atomic_fetch_add_batch(table, word, inc, fetched, NOPS_FADD, 1024, 2),
+        "fetch_add_warp_aggregation": lambda: B.ishmemx_int64_atomic_fetch_add_batch(table, word, inc, fetched,
+                                                                                       NOPS_FADD, 256, 1),
         "fetch_add_no_aggregation": lambda: B.ishmemx_int64_atomic_fetch_add_batch(table, word, inc, fetched,
                                                                                      NOPS_FADD, 256, 0),
         "compare_swap": lambda: B.ishmemx_int64_atomic_compare_swap_batch(table, cword, ccond, cval, fetched,
@@ -316,7 +318,8 @@ def breakdown(B, torch, team_stream, env) -> dict:
     res = {}
     for name, fn in ops.items():
         ms = timed(fn)
-        key = {"copy_engine_put": "put", "fetch_add_no_aggregation": "fetch_add"}.get(name, name)
+        key = {"copy_engine_put": "put", "fetch_add_no_aggregation": "fetch_add",
+               "fetch_add_warp_aggregation": "fetch_add"}.get(name, name)
         entry = {"ms": round(ms, 4), "GB/s": round(nbytes[key] / (ms * 1e-3) / 1e9, 1)}
         if "fetch_add" in name:
             entry["Mops/s"] = round(NOPS_FADD / (ms * 1e-3) / 1e6, 1)

@@ -352,9 +352,13 @@ ISHMEM_DECL_AMO(uint64, uint64_t)
 /* Device-initiated batches (one op per GPU thread, "issued from all threads"): op i is
  * issued by PE (i mod npes); word w of the table lives on PE (w mod npes) at
  * table + 8*(w div npes).  word_idx/inc/cond/value/fetched are device arrays of `nops`
- * entries (fetched may be NULL).  aggregate != 0 lets the lanes of a warp that hit the same
- * word combine into one atomic and rebuild their fetched values (still one valid
- * serialisation).  One launch on the team stream. */
+ * entries (fetched may be NULL).  aggregate = 0: one atomic per op.  aggregate = 1: the lanes
+ * of a warp that hit the same word combine into one atomic.  aggregate = 2: the ops of a whole
+ * block (8 per thread) that hit the same word combine in shared-memory accumulators (2048
+ * direct-mapped slots; ops whose slot is taken by another word go to the table directly) and
+ * one atomic per used slot reaches the table.  In every mode each op's fetched value is the one
+ * it would have seen in one valid serialisation, and the final table is the same.  One launch
+ * on the team stream. */
 int ishmemx_int64_atomic_fetch_add_batch(int64_t *table, const int32_t *word_idx,
                                          const int64_t *inc, int64_t *fetched, size_t nops,
                                          int threads, int aggregate);

@@ -101,28 +101,130 @@ ISHMEMI_DEF_AMO(uint32, uint32_t, unsigned)
 ISHMEMI_DEF_AMO(uint64, uint64_t, unsigned long long)
 
 /* ---- device-initiated batches ---------------------------------------------------------- */
-/* Block b belongs to PE (b mod npes); its threads issue that PE's ops i = k*npes + pe in
- * order, one per thread.  Word w lives on PE (w mod npes), slot (w div npes). */
+/* Op i is issued by PE (i mod npes): the thread that handles it uses that PE's context for the
+ * address translation.  Consecutive threads take consecutive ops (coalesced reads of the op
+ * stream).  Word w lives on PE (w mod npes), slot (w div npes). */
 
-template <bool AGGREGATE>
+#define AMO_BLOCK_SLOTS 2048 /* shared-memory accumulators of the block-level aggregation */
+#define AMO_BLOCK_OPT 8      /* ops per thread in that mode */
+
+__device__ __forceinline__ long long *table_of(const ishmem_ctx_t *ctxs, const ishmem_ctx_t *ctx, long long *table0)
+{
+    return (long long *)((char *)table0 + (ctx->heap_base - ctxs[0].heap_base));
+}
+
+/* Lanes of the warp (those in `act`) that hit the same word w combine: on return `total` is the
+ * sum of the group's increments, `before` the sum over the group's lower lanes (what this lane
+ * would find added already if the group's ops ran back to back in lane order), and the result
+ * is the group's lowest lane, which issues the one atomic.  Called by every lane in `act`. */
+__device__ __forceinline__ unsigned warp_combine(unsigned act, int w, long long v, long long *total, long long *before)
+{
+    const unsigned lane = threadIdx.x & 31u;
+    const unsigned peers = __match_any_sync(act, w);
+    long long bef = 0, tot = 0;
+    unsigned rest = peers;
+    /* round r: every lane reads the increment of its r-th peer; the number of rounds is the
+     * largest group in the warp, so the shuffles stay converged */
+    const unsigned rounds = __reduce_max_sync(act, (unsigned)__popc(peers));
+#pragma unroll 1
+    for (unsigned r = 0; r < rounds; ++r) {
+        const unsigned src = rest ? (unsigned)(__ffs(rest) - 1) : lane;
+        const long long x = __shfl_sync(act, v, src);
+        if (rest) {
+            tot += x;
+            if (src < lane) bef += x;
+            rest &= rest - 1;
+        }
+    }
+    *total = tot;
+    *before = bef;
+    return (unsigned)__ffs(peers) - 1;
+}
+
+/* MODE 0: one atomic per op.  MODE 1: lanes of a warp that hit the same word combine into one
+ * atomic.  MODE 2: the ops of a block (AMO_BLOCK_OPT per thread) that hit the same word combine,
+ * first within each warp, then in a direct-mapped table of shared-memory accumulators; one
+ * global atomic per used slot.
+ * In every mode each op gets the value it would have fetched in ONE valid serialisation. */
+template <int MODE>
 __global__ void __launch_bounds__(1024) k_fetch_add_batch(const ishmem_ctx_t *ctxs, long long *table0,
                                                           const int *word_idx, const long long *inc,
                                                           long long *fetched, size_t nops)
 {
     const int npes = ctxs[0].npes;
-    const int my = (int)(blockIdx.x % (unsigned)npes);
-    const ishmem_ctx_t *ctx = ctxs + my;
-    const size_t k = (size_t)(blockIdx.x / (unsigned)npes) * blockDim.x + threadIdx.x;
-    const size_t i = k * (size_t)npes + (size_t)my;
+    if (MODE == 2) {
+        __shared__ int tag[AMO_BLOCK_SLOTS];
+        __shared__ unsigned long long acc[AMO_BLOCK_SLOTS];
+        for (unsigned k = threadIdx.x; k < AMO_BLOCK_SLOTS; k += blockDim.x) {
+            tag[k] = -1;
+            acc[k] = 0ull;
+        }
+        __syncthreads();
+        const size_t base = (size_t)blockIdx.x * blockDim.x * AMO_BLOCK_OPT;
+        long long mine[AMO_BLOCK_OPT]; /* value fetched from shared memory, or from the table if direct */
+        int slot[AMO_BLOCK_OPT];       /* slot used, -1: went straight to the table, -2: no op */
+#pragma unroll
+        for (int j = 0; j < AMO_BLOCK_OPT; ++j) {
+            const size_t i = base + (size_t)j * blockDim.x + threadIdx.x;
+            const bool active = i < nops;
+            const unsigned act = __ballot_sync(0xffffffffu, active);
+            slot[j] = -2;
+            mine[j] = 0;
+            if (active) {
+                const int w = word_idx[i];
+                const long long v = inc[i];
+                long long total, before;
+                const unsigned leader = warp_combine(act, w, v, &total, &before);
+                long long got = 0;
+                int sl = -1;
+                if ((threadIdx.x & 31u) == leader) {
+                    sl = w & (AMO_BLOCK_SLOTS - 1);
+                    const int seen = atomicCAS(&tag[sl], -1, w);
+                    if (seen == -1 || seen == w) {
+                        got = (long long)atomicAdd(&acc[sl], (unsigned long long)total);
+                    } else { /* slot taken by another word: the group goes to the table itself */
+                        const ishmem_ctx_t *ctx = ctxs + (int)(i % (size_t)npes);
+                        got = ishmem_atomic_fetch_add<long long>(ctx, table_of(ctxs, ctx, table0) + w / npes, total,
+                                                                 w % npes);
+                        sl = -1;
+                    }
+                }
+                mine[j] = __shfl_sync(act, got, leader) + before;
+                slot[j] = __shfl_sync(act, sl, leader);
+            }
+        }
+        __syncthreads();
+        /* one atomic per used slot carries the block's total; the slot then holds the value the
+         * table had before it */
+        const ishmem_ctx_t *bctx = ctxs + (int)(blockIdx.x % (unsigned)npes);
+        for (unsigned k = threadIdx.x; k < AMO_BLOCK_SLOTS; k += blockDim.x) {
+            const int w = tag[k];
+            if (w >= 0)
+                acc[k] = (unsigned long long)ishmem_atomic_fetch_add<long long>(
+                    bctx, table_of(ctxs, bctx, table0) + w / npes, (long long)acc[k], w % npes);
+        }
+        __syncthreads();
+        if (fetched) {
+#pragma unroll
+            for (int j = 0; j < AMO_BLOCK_OPT; ++j) {
+                const size_t i = base + (size_t)j * blockDim.x + threadIdx.x;
+                if (slot[j] >= 0) fetched[i] = (long long)acc[slot[j]] + mine[j];
+                else if (slot[j] == -1) fetched[i] = mine[j];
+            }
+        }
+        return;
+    }
+    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     const bool active = i < nops;
-    long long *table = (long long *)((char *)table0 + (ctx->heap_base - ctxs[0].heap_base));
+    const ishmem_ctx_t *ctx = ctxs + (int)(i % (size_t)npes);
+    long long *table = table_of(ctxs, ctx, table0);
     int w = 0;
     long long v = 0;
     if (active) {
         w = word_idx[i];
         v = inc[i];
     }
-    if (!AGGREGATE) {
+    if (MODE == 0) {
         if (active) {
             long long old = ishmem_atomic_fetch_add<long long>(ctx, table + w / npes, v, w % npes);
             if (fetched) fetched[i] = old;
@@ -135,23 +237,8 @@ __global__ void __launch_bounds__(1024) k_fetch_add_batch(const ishmem_ctx_t *ct
     const unsigned lane = threadIdx.x & 31u;
     const unsigned act = __ballot_sync(0xffffffffu, active);
     if (!active) return;
-    const unsigned peers = __match_any_sync(act, w);
-    const unsigned leader = __ffs(peers) - 1;
-    long long before = 0, total = 0; /* sum over peers in lower lanes; sum over all peers */
-    unsigned rest = peers;
-    /* round r: every lane reads the increment of its r-th peer; the number of rounds is the
-     * largest group in the warp, so the shuffles stay converged */
-    const unsigned rounds = __reduce_max_sync(act, (unsigned)__popc(peers));
-#pragma unroll 1
-    for (unsigned r = 0; r < rounds; ++r) {
-        const unsigned src = rest ? (unsigned)(__ffs(rest) - 1) : lane;
-        const long long x = __shfl_sync(act, v, src);
-        if (rest) {
-            total += x;
-            if (src < lane) before += x;
-            rest &= rest - 1;
-        }
-    }
+    long long before = 0, total = 0;
+    const unsigned leader = warp_combine(act, w, v, &total, &before);
     long long base = 0;
     if (lane == leader) base = ishmem_atomic_fetch_add<long long>(ctx, table + w / npes, total, w % npes);
     base = __shfl_sync(act, base, leader);
@@ -164,26 +251,23 @@ __global__ void __launch_bounds__(1024) k_compare_swap_batch(const ishmem_ctx_t 
                                                              size_t nops)
 {
     const int npes = ctxs[0].npes;
-    const int my = (int)(blockIdx.x % (unsigned)npes);
-    const ishmem_ctx_t *ctx = ctxs + my;
-    const size_t k = (size_t)(blockIdx.x / (unsigned)npes) * blockDim.x + threadIdx.x;
-    const size_t i = k * (size_t)npes + (size_t)my;
+    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= nops) return;
-    long long *table = (long long *)((char *)table0 + (ctx->heap_base - ctxs[0].heap_base));
+    const ishmem_ctx_t *ctx = ctxs + (int)(i % (size_t)npes);
+    long long *table = table_of(ctxs, ctx, table0);
     const int w = word_idx[i];
     long long old = ishmem_atomic_compare_swap<long long>(ctx, table + w / npes, cond[i], value[i], w % npes);
     if (fetched) fetched[i] = old;
 }
 
-static int batch_geometry(size_t nops, int threads, unsigned *blocks)
+static int batch_geometry(size_t nops, int threads, int ops_per_thread, unsigned *blocks)
 {
-    auto &g = g_ishmem;
     if (threads < 32 || threads > 1024 || threads % 32) return ISHMEM_ERR_ARG;
-    size_t per_pe = (nops + g.npes - 1) / g.npes;
-    size_t bpp = (per_pe + threads - 1) / threads;
-    if (bpp == 0) bpp = 1;
-    if (bpp * g.npes > 0x7fffffffull) return ISHMEM_ERR_ARG;
-    *blocks = (unsigned)(bpp * g.npes);
+    const size_t per_block = (size_t)threads * ops_per_thread;
+    size_t b = (nops + per_block - 1) / per_block;
+    if (b == 0) b = 1;
+    if (b > 0x7fffffffull) return ISHMEM_ERR_ARG;
+    *blocks = (unsigned)b;
     return ISHMEM_OK;
 }
 
@@ -195,18 +279,22 @@ extern "C" int ishmemx_int64_atomic_fetch_add_batch(int64_t *table, const int32_
     if (!word_idx || !inc) return ISHMEM_ERR_ARG;
     if ((uintptr_t)table % 8) return ISHMEM_ERR_ALIGN;
     if (ishmemi_sym_offset(table, 8) < 0) return ISHMEM_ERR_NOT_SYMMETRIC;
+    if (aggregate < 0 || aggregate > 2) return ISHMEM_ERR_ARG;
     unsigned blocks;
-    int rc = batch_geometry(nops, threads, &blocks);
+    int rc = batch_geometry(nops, threads, aggregate == 2 ? AMO_BLOCK_OPT : 1, &blocks);
     if (rc) return rc;
     cudaStream_t s;
     if ((rc = ishmemi_team_stream_begin(ISHMEM_TEAM_WORLD, &s))) return rc;
     if (nops) {
-        if (aggregate)
-            k_fetch_add_batch<true><<<blocks, threads, 0, s>>>(g.d_ctx, (long long *)table, word_idx,
-                                                               (const long long *)inc, (long long *)fetched, nops);
+        if (aggregate == 2)
+            k_fetch_add_batch<2><<<blocks, threads, 0, s>>>(g.d_ctx, (long long *)table, word_idx,
+                                                            (const long long *)inc, (long long *)fetched, nops);
+        else if (aggregate == 1)
+            k_fetch_add_batch<1><<<blocks, threads, 0, s>>>(g.d_ctx, (long long *)table, word_idx,
+                                                            (const long long *)inc, (long long *)fetched, nops);
         else
-            k_fetch_add_batch<false><<<blocks, threads, 0, s>>>(g.d_ctx, (long long *)table, word_idx,
-                                                                (const long long *)inc, (long long *)fetched, nops);
+            k_fetch_add_batch<0><<<blocks, threads, 0, s>>>(g.d_ctx, (long long *)table, word_idx,
+                                                            (const long long *)inc, (long long *)fetched, nops);
         ishmemi_count_launch();
         rc = ishmemi_check_launch("k_fetch_add_batch");
     }
@@ -224,7 +312,7 @@ extern "C" int ishmemx_int64_atomic_compare_swap_batch(int64_t *table, const int
     if ((uintptr_t)table % 8) return ISHMEM_ERR_ALIGN;
     if (ishmemi_sym_offset(table, 8) < 0) return ISHMEM_ERR_NOT_SYMMETRIC;
     unsigned blocks;
-    int rc = batch_geometry(nops, threads, &blocks);
+    int rc = batch_geometry(nops, threads, 1, &blocks);
     if (rc) return rc;
     cudaStream_t s;
     if ((rc = ishmemi_team_stream_begin(ISHMEM_TEAM_WORLD, &s))) return rc;

@@ -402,11 +402,11 @@ def sweep_c4(args, out):
                "one_word": np.zeros(nops, dtype=np.int32)}
     for sname, idx in streams.items():
         word = torch.from_numpy(idx).cuda()
-        for agg in (1, 0):
+        for agg in (2, 1, 0):
             for fet, fname in ((fetched, "fetch_add"), (None, "add")):
                 for threads in (256, 1024):
                     us, it = T(lambda i: B.ishmemx_int64_atomic_fetch_add_batch(table, word, inc, fet, nops, threads, agg))
-                    out.add(config=4, op=fname, pattern=sname, variant="aggregate" if agg else "plain",
+                    out.add(config=4, op=fname, pattern=sname, variant=("plain", "aggregate_warp", "aggregate_block")[agg],
                             threads=threads, npes=npes, dtype="i64", nbytes=8, l2="hot", iters=it, us_per_op=us,
                             mops=round(nops / us, 1), note=f"{nops} ops on {nwords} words")
     nops_c, nwords_c = 1 << 20, 1024

@@ -58,7 +58,7 @@ def test_host_initiated_atomics_all_ops():
         assert e.value.code == B.ISHMEM_ERR_ALIGN
 
 
-@pytest.mark.parametrize("aggregate", [0, 1])
+@pytest.mark.parametrize("aggregate", [0, 1, 2])
 @pytest.mark.parametrize("nops,nwords", [(100_003, 257), (1 << 22, 4096)])
 def test_config4_fetch_add_batch(nops, nwords, aggregate):
     """Config 4: 16 PEs, Zipf(1.1) targets spread round-robin over PEs, increments in
