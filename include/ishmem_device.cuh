@@ -66,6 +66,7 @@ struct ishmemi_proxy_t {
     unsigned long long *nbi_seen;          /* device [npes]: last value of nbi_done[pe] any thread has seen */
     const unsigned long long *nbi_done;    /* host [npes]: non-blocking requests of each PE completed */
     unsigned long long wg_cutover;         /* work-group put/get of at least this size use the engine */
+    unsigned long long hybrid_head;        /* bytes the work-group copies itself while the engine starts on the rest */
 };
 
 /* Per-PE context, resident in device memory (Section 3.7.1: a separate GPU-side copy of
@@ -262,6 +263,29 @@ __device__ __forceinline__ void copy_vec16(char *d, const char *s, size_t nvec, 
     for (; i < nvec; i += nthr) st16(d + i * 16, ld16(s + i * 16));
 }
 
+/* Fewer than 16 bytes at the edge of a vector copy: d and s are congruent mod 16, so the widest
+ * power-of-two word that d is aligned to and that still fits is valid for both; at most
+ * 1 + 2 + 4 + 8 bytes going up to a boundary or 8 + 4 + 2 + 1 coming down from one.  One thread. */
+__device__ __forceinline__ void copy_edge(char *d, const char *s, size_t n)
+{
+    while (n) {
+        const unsigned a = (unsigned)(uintptr_t)d;
+        if (n >= 8 && (a & 7u) == 0) {
+            stv<unsigned long long>(d, ldv<unsigned long long>(s));
+            d += 8, s += 8, n -= 8;
+        } else if (n >= 4 && (a & 3u) == 0) {
+            stv<unsigned>(d, ldv<unsigned>(s));
+            d += 4, s += 4, n -= 4;
+        } else if (n >= 2 && (a & 1u) == 0) {
+            stv<unsigned short>(d, ldv<unsigned short>(s));
+            d += 2, s += 2, n -= 2;
+        } else {
+            stv<unsigned char>(d, ldv<unsigned char>(s));
+            d += 1, s += 1, n -= 1;
+        }
+    }
+}
+
 /* General copy by `nthr` cooperating threads (nthr = 1: a single work-item).  Picks the
  * widest access both addresses allow: when dest and src are congruent mod 16 the head is
  * peeled to a 16-byte boundary and the body moves 16-byte vectors; otherwise the widest
@@ -275,15 +299,11 @@ __device__ __forceinline__ void copy_bytes(char *d, const char *s, size_t n, uns
     if (rel == 0) {
         size_t head = (size_t)((16u - ((unsigned)(uintptr_t)d & 15u)) & 15u);
         if (head > n) head = n;
-        for (size_t i = tid; i < head; i += nthr) stv<unsigned char>(d + i, ldv<unsigned char>(s + i));
-        d += head;
-        s += head;
-        n -= head;
-        const size_t nvec = n >> 4;
-        copy_vec16<UNROLL>(d, s, nvec, tid, nthr);
-        const size_t done = nvec << 4;
-        for (size_t i = done + tid; i < n; i += nthr)
-            stv<unsigned char>(d + i, ldv<unsigned char>(s + i));
+        const size_t nvec = (n - head) >> 4, tail = n - head - (nvec << 4);
+        /* the two ragged edges go to the first and the last thread, in the widest words */
+        if (tid == 0) copy_edge(d, s, head);
+        if (tid == nthr - 1) copy_edge(d + head + (nvec << 4), s + head + (nvec << 4), tail);
+        copy_vec16<UNROLL>(d + head, s + head, nvec, tid, nthr);
         return;
     }
     /* W = widest power of two (< 16) dividing the distance between the two addresses */
@@ -627,8 +647,24 @@ __device__ __forceinline__ int wg_copy(const ishmem_ctx_t *ctx, char *d, const c
         /* cutover (Sections 3.2 and 3.7.1): above the tuned size the group leader asks the host
          * to start the copy engine, after a group barrier that makes the source valid */
         __shared__ int rc_engine;
+        __shared__ unsigned long long ticket;
+        /* hybrid form (a refinement the paper sketches): the engine gets the tail of the message
+         * and, while it starts up, the group moves the head by loads and stores */
+        size_t head = ctx->proxy->hybrid_head < n ? (size_t)ctx->proxy->hybrid_head & ~(size_t)255 : 0;
+        if (!complete) head = 0; /* the non-blocking form returns at once */
         __syncthreads();
-        if (tid == 0) rc_engine = proxy_copy(ctx, d, s, n, complete);
+        if (tid == 0) {
+            if (head) {
+                ticket = atomicAdd(ctx->proxy->comp_alloc, 1ull);
+                rc_engine = proxy_post(ctx, ISHMEMI_REQ_COPY, d + head, s + head, n - head, nullptr, 0, ticket + 1);
+            } else {
+                rc_engine = proxy_copy(ctx, d, s, n, complete);
+            }
+        }
+        if (head) {
+            copy_bytes(d, s, head, tid, nthr);
+            if (tid == 0 && rc_engine == 0) rc_engine = proxy_wait(ctx, ticket);
+        }
         __syncthreads();
         return rc_engine;
     }
@@ -963,10 +999,9 @@ __device__ __forceinline__ int ishmemx_putmem_signal_work_group(
     int rc = ISHMEM_ERR_INVALID_PE;
     if (r && rs) rc = ishmemi::wg_copy(ctx, r, (const char *)src, nbytes, staging, true);
     __syncthreads();
-    if (r && rs && ishmemi::block_tid() == 0) {
-        ishmemi::fence_acq_rel_gpu();
-        ishmemi::signal_update(rs, signal, sig_op);
-    }
+    /* the release below is cumulative: it also covers the other threads' stores, which the
+     * block barrier has ordered before it */
+    if (r && rs && ishmemi::block_tid() == 0) ishmemi::signal_update(rs, signal, sig_op);
     return rc;
 }
 __device__ __forceinline__ unsigned long long ishmem_signal_fetch(const ishmem_ctx_t *,

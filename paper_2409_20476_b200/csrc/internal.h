@@ -49,6 +49,7 @@ struct ishmemi_state {
     ishmemi_team teams[ISHMEM_MAX_TEAMS] = {};
     size_t cutover[3] = {0, 0, 0};
     size_t wg_cutover = (size_t)-1; /* device-initiated work-group put/get: bytes from which the engine is used */
+    size_t hybrid_head = 0;         /* ... and bytes of the head the group copies itself meanwhile */
     int coll_groups = 0, coll_threads = 512;
     int bcast_root_dest = 1;
     unsigned long long wait_limit_ns = 2000000000ull;
@@ -88,6 +89,6 @@ int ishmemi_check_launch(const char *what);      /* cudaGetLastError -> status *
 int ishmemi_engine_copy(int my_pe, void *dst, const void *src, size_t n, bool blocking);
 /* reverse-offload proxy (proxy.cu) */
 void ishmemi_proxy_finalize();
-void ishmemi_proxy_set_cutover(size_t nbytes);
+void ishmemi_proxy_set_cutover(size_t nbytes, size_t hybrid_head);
 
 #endif

@@ -45,11 +45,12 @@ __global__ void __launch_bounds__(1024) k_pingpong(const ishmem_ctx_t *ctxs, int
             if (ishmemx_uint64_wait_until_work_group(ctx, sig, ISHMEM_CMP_GE, (unsigned long long)r)) break;
         } else {
             if (ishmemx_uint64_wait_until_work_group(ctx, sig, ISHMEM_CMP_GE, (unsigned long long)r)) break;
+            /* the leader checks the stamps while the others already start on the reply (both only
+             * read this buffer; the leader signals last, after the barrier inside the put) */
             if (threadIdx.x == 0) {
                 if (w0 && *w0 != (unsigned long long)r) ++bad;
                 if (w1 && *w1 != (unsigned long long)r) ++bad;
             }
-            __syncthreads();
             ishmemx_putmem_signal_work_group(ctx, data, data, nbytes, sig, (unsigned long long)r,
                                              ISHMEM_SIGNAL_SET, other);
         }

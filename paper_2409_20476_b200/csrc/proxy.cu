@@ -176,6 +176,7 @@ extern "C" int ishmemx_proxy_start(void)
     h.comp = g_px.comp;
     h.nbi_done = g_px.nbi_done;
     h.wg_cutover = g.wg_cutover;
+    h.hybrid_head = g.hybrid_head;
     rc = ishmemi_cuda(cudaMemcpy(g_px.d_proxy, &h, sizeof(h), cudaMemcpyHostToDevice), "cudaMemcpy(proxy)");
     if (rc) {
         proxy_release();
@@ -213,11 +214,12 @@ void ishmemi_proxy_finalize()
     if (g_px.running) ishmemx_proxy_stop();
 }
 
-void ishmemi_proxy_set_cutover(size_t nbytes)
+void ishmemi_proxy_set_cutover(size_t nbytes, size_t hybrid_head)
 {
     if (!g_px.running) return;
     cudaDeviceSynchronize();
     g_px.h_proxy.wg_cutover = nbytes;
+    g_px.h_proxy.hybrid_head = hybrid_head;
     cudaMemcpy(g_px.d_proxy, &g_px.h_proxy, sizeof(g_px.h_proxy), cudaMemcpyHostToDevice);
 }
 

@@ -96,10 +96,7 @@ __global__ void __launch_bounds__(1024) k_rma(const ishmem_ctx_t *ctxs, rma_args
         __syncthreads();
         if (threadIdx.x == 0) {
             unsigned long long *rs = ishmem_ptr(ctx, a.sig, target);
-            if (rs) {
-                ishmemi::fence_acq_rel_gpu();
-                ishmemi::signal_update(rs, a.sig_value, a.sig_op);
-            }
+            if (rs) ishmemi::signal_update(rs, a.sig_value, a.sig_op); /* release: cumulative over the block */
         }
     }
 }

@@ -202,6 +202,7 @@ static int init_common(int npes, size_t heap_bytes, void *external)
     g.cutover[1] = (env = getenv("ISHMEM_CUTOVER_BCAST")) ? strtoull(env, nullptr, 0) : (size_t)-1;
     g.cutover[2] = (env = getenv("ISHMEM_CUTOVER_FCOLLECT")) ? strtoull(env, nullptr, 0) : (size_t)-1;
     g.wg_cutover = (env = getenv("ISHMEM_CUTOVER_WORK_GROUP")) ? strtoull(env, nullptr, 0) : (size_t)-1;
+    g.hybrid_head = 0;
     if ((env = getenv("ISHMEM_WAIT_TIMEOUT_NS"))) g.wait_limit_ns = strtoull(env, nullptr, 0);
     g.launches = 0;
     g.initialised = true;
@@ -483,10 +484,11 @@ extern "C" int ishmem_team_n_pes(ishmem_team_t team)
 extern "C" int ishmemx_set_cutover(int which, size_t nbytes)
 {
     ISHMEMI_REQUIRE_INIT();
-    if (which < 0 || which > 3) return ISHMEM_ERR_ARG;
-    if (which == 3) {
-        g_ishmem.wg_cutover = nbytes;
-        ishmemi_proxy_set_cutover(nbytes);
+    if (which < 0 || which > 4) return ISHMEM_ERR_ARG;
+    if (which >= 3) {
+        if (which == 3) g_ishmem.wg_cutover = nbytes;
+        else g_ishmem.hybrid_head = nbytes;
+        ishmemi_proxy_set_cutover(g_ishmem.wg_cutover, g_ishmem.hybrid_head);
         return ISHMEM_OK;
     }
     g_ishmem.cutover[which] = nbytes;
@@ -495,6 +497,7 @@ extern "C" int ishmemx_set_cutover(int which, size_t nbytes)
 extern "C" size_t ishmemx_get_cutover(int which)
 {
     if (which == 3) return g_ishmem.wg_cutover;
+    if (which == 4) return g_ishmem.hybrid_head;
     return (which < 0 || which > 2) ? 0 : g_ishmem.cutover[which];
 }
 extern "C" int ishmemx_set_bcast_root_dest(int enable)

@@ -213,6 +213,21 @@ def sweep_c2(args, out):
                 out.add(config=2, op=op, pattern="one_pe", variant="in_kernel_" + name, level=level, threads=threads,
                         groups=1, npes=1, dtype="u8", nbytes=n, l2="hot", iters=iters, us_per_op=float(ns[0]) / 1e3,
                         alg_bytes=2 * n, note="device global timer, op + quiet")
+    # hybrid put: above the cutover the engine takes the tail while the group copies the head
+    B.ishmemx_set_cutover(3, 256 << 10)
+    for head in (512 << 10, 1 * MiB, 2 * MiB):
+        B.ishmemx_set_cutover(4, head)
+        for n in sizes:
+            if n < MiB or n > 64 * MiB:
+                continue
+            iters = int(max(4, min(200, (64 * MiB) // n)))
+            B.ishmemx_rma_latency(0, dst, src, n, 1, 0, WG, 1024, iters, ns)
+            B.ishmemx_rma_latency(0, dst, src, n, 1, 0, WG, 1024, iters, ns)
+            out.add(config=2, op="put", pattern="one_pe", variant=f"in_kernel_hybrid_1024_head_{head >> 10}K", level=WG,
+                    threads=1024, groups=1, npes=1, dtype="u8", nbytes=n, l2="hot", iters=iters,
+                    us_per_op=float(ns[0]) / 1e3, alg_bytes=2 * n, note="device global timer, op + quiet")
+    B.ishmemx_set_cutover(4, 0)
+    B.ishmemx_set_cutover(3, B.SIZE_MAX)
     assert B.ishmemx_status(1) == 0
     B.ishmemx_proxy_stop()
     B.ishmem_finalize()

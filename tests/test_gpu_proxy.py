@@ -91,6 +91,19 @@ def test_cutover_inside_the_work_group_calls():
                 B.ishmem_barrier_all()
                 heaps_equal(s, f"cutover put n={n}")
                 assert stats()[1] - before == engine_copies
+            # hybrid: the group copies the first 20000 bytes (rounded down to 19968) itself
+            B.ishmemx_set_cutover(4, 20_000)
+            assert B.ishmemx_get_cutover(4) == 20_000
+            for n in (299_999, 40_000, 19_000):
+                before = stats()[1]
+                B.ishmemx_putmem_on_device(1, dst.addr + 7, src.addr + 7, n, 0, B.ISHMEMX_WORK_GROUP, 128, 1)
+                s.oracle.putmem(1, dst.ooff + 7, s.oracle.ptr(src.ooff + 7, n, 1), n, 0)
+                B.ishmemx_getmem_on_device(2, src.addr + 9, dst.addr + 9, n, 0, B.ISHMEMX_WORK_GROUP, 128, 1)
+                s.oracle.getmem(2, s.oracle.ptr(src.ooff + 9, n, 2), dst.ooff + 9, n, 0)
+                B.ishmem_barrier_all()
+                heaps_equal(s, f"hybrid put/get n={n}")
+                assert stats()[1] - before == (2 if n >= 32 << 10 else 0)
+            B.ishmemx_set_cutover(4, 0)
             # in-kernel ping-pong with every put_signal going through the engine
             B.ishmemx_set_cutover(3, 0)
             rtt, bad = np.zeros(1), np.zeros(1, dtype=np.uint64)
