@@ -241,7 +241,9 @@ int ishmemx_putmem_spmd_copy_engine(void *dest, const void *src, size_t nbytes, 
 /* Cutover sizes in bytes (Section 4: tuned from measurement; for the collaborative calls
  * it depends on the number of threads).  which: 0 = host-initiated put/get, 1 = broadcast,
  * 2 = fcollect, 3 = device-initiated work-group put/get (takes effect while the host proxy of
- * ishmemx_proxy_start runs).  SIZE_MAX = never use the copy engine (the default), 0 = always.
+ * ishmemx_proxy_start runs).  SIZE_MAX = never use the copy engine, 0 = always.  Defaults, from
+ * the size sweep on B200: 4 MiB for which = 0, SIZE_MAX for the others (environment overrides:
+ * ISHMEM_CUTOVER_PUT, _BCAST, _FCOLLECT, _WORK_GROUP).
  * which = 4 is not a threshold but the hybrid head: a blocking work-group put/get above cutover 3
  * gives the engine everything past the first `nbytes` bytes (rounded down to 256) and copies
  * that head itself meanwhile, hiding the engine's start-up; 0 (the default) = engine only. */

@@ -196,9 +196,12 @@ static int init_common(int npes, size_t heap_bytes, void *external)
     g.free_blocks.clear();
     g.used_blocks.clear();
     g.free_blocks[0] = heap_bytes;
-    /* default cutovers: see ishmemx_set_cutover; tuned from the committed size sweep */
+    /* default cutovers, from the committed size sweep on B200 (ishmemx_tune_cutover re-measures):
+     * a host-initiated put/get of one PE is at least as fast on the copy engine from 4 MiB on
+     * (5.8 against 6.1 us there, 6.3 against 5.6 TB/s at 256 MiB); the push collectives and
+     * the device-initiated work-group calls never are, so they stay on loads and stores */
     const char *env;
-    g.cutover[0] = (env = getenv("ISHMEM_CUTOVER_PUT")) ? strtoull(env, nullptr, 0) : (size_t)-1;
+    g.cutover[0] = (env = getenv("ISHMEM_CUTOVER_PUT")) ? strtoull(env, nullptr, 0) : ((size_t)4 << 20);
     g.cutover[1] = (env = getenv("ISHMEM_CUTOVER_BCAST")) ? strtoull(env, nullptr, 0) : (size_t)-1;
     g.cutover[2] = (env = getenv("ISHMEM_CUTOVER_FCOLLECT")) ? strtoull(env, nullptr, 0) : (size_t)-1;
     g.wg_cutover = (env = getenv("ISHMEM_CUTOVER_WORK_GROUP")) ? strtoull(env, nullptr, 0) : (size_t)-1;

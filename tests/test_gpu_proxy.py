@@ -169,3 +169,26 @@ def test_cutover_tuned_from_measurement():
             assert s.status() == 0
         finally:
             B.ishmemx_proxy_stop()
+
+
+def test_many_work_groups_post_at_once():
+    """296 work-groups (37 per PE) each post one slice of an 8 MiB message at the same time and
+    quiet on their PE's completion counter; ring pattern, whole output checked on the device,
+    twice in a row (the second launch is queued behind the first)."""
+    npes, n = 8, 8 << 20
+    with Session(npes, 2 * n + (1 << 20), with_oracle=False) as s:
+        src, dst = s.malloc(n), s.malloc(n)
+        for p in range(npes):
+            src.gpu(p).copy_(torch.from_numpy(inputs.block_values("u8", inputs.SEED_C2, p, 0, n)))
+        s.sync()
+        B.ishmemx_proxy_start()
+        try:
+            for shift in (1, 3):
+                B.ishmemx_putmem_spmd(dst.addr, src.addr, n, shift, B.ISHMEMX_WORK_GROUP_ENGINE, 64, 37)
+            s.sync()
+            for p in range(npes):
+                assert torch.equal(dst.gpu((p + 3) % npes), src.gpu(p)), p
+            assert stats()[1] == 2 * 37 * npes
+            assert s.status() == 0
+        finally:
+            B.ishmemx_proxy_stop()
