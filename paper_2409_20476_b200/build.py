@@ -63,6 +63,23 @@ def build(force: bool = False, verbose: bool = False, ptxas_info: bool = False) 
     return LIB
 
 
+def build_user_kernel_example(force: bool = False) -> Path:
+    """Compiles tests/csrc/user_kernel.cu -- a kernel of a library USER, built only against the
+    public headers -- into tests/libuser_kernel.so (used by the GPU tests)."""
+    src = ROOT / "tests" / "csrc" / "user_kernel.cu"
+    out = ROOT / "tests" / "libuser_kernel.so"
+    newest = max(src.stat().st_mtime, max(f.stat().st_mtime for f in (ROOT / "include").glob("*")))
+    if not force and out.exists() and out.stat().st_mtime >= newest:
+        return out
+    tmp = out.with_suffix(f".so.{os.getpid()}")
+    subprocess.run([nvcc(), "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "-shared",
+                    "-Xcompiler", "-fPIC", "-I", str(ROOT / "include"), str(src), "-o", str(tmp), "-lcudart_static",
+                    "-ldl", "-lpthread", "-lrt"], check=True)
+    os.replace(tmp, out)
+    return out
+
+
 if __name__ == "__main__":
     build(force="--force" in sys.argv, verbose=True, ptxas_info="--ptxas" in sys.argv)
+    build_user_kernel_example(force="--force" in sys.argv)
     print(LIB)
