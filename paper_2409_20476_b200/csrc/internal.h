@@ -41,6 +41,7 @@ struct ishmemi_state {
     bool pe_dirty[ISHMEM_MAX_PES] = {};
     bool nbi_pending[ISHMEM_MAX_PES] = {};
     unsigned long long team_seq = 0;
+    unsigned long long team_event_seq = 0; /* team_seq value ev_team was last recorded for */
     unsigned long long pe_seen_team[ISHMEM_MAX_PES] = {};
 
     /* symmetric allocator: offset -> size of free and of used blocks */

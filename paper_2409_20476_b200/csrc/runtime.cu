@@ -59,6 +59,13 @@ cudaStream_t ishmemi_pe_stream_for_op(int pe)
 {
     auto &g = g_ishmem;
     if (g.pe_seen_team[pe] != g.team_seq) {
+        /* the event is recorded only now, when somebody needs it: it then covers everything the
+         * team stream holds (at least the launch this PE has not seen), and back-to-back team
+         * launches pay for no event at all */
+        if (g.team_event_seq != g.team_seq) {
+            cudaEventRecord(g.ev_team, g.team_stream);
+            g.team_event_seq = g.team_seq;
+        }
         cudaStreamWaitEvent(g.pe_stream[pe], g.ev_team, 0);
         g.pe_seen_team[pe] = g.team_seq;
     }
@@ -97,9 +104,7 @@ int ishmemi_team_stream_begin(ishmem_team_t team, cudaStream_t *out)
 
 void ishmemi_team_stream_end()
 {
-    auto &g = g_ishmem;
-    cudaEventRecord(g.ev_team, g.team_stream);
-    ++g.team_seq;
+    ++g_ishmem.team_seq; /* PE streams order themselves after it lazily (ishmemi_pe_stream_for_op) */
 }
 
 int ishmemi_engine_copy(int my_pe, void *dst, const void *src, size_t n, bool blocking)
@@ -193,6 +198,7 @@ static int init_common(int npes, size_t heap_bytes, void *external)
     g.owns_team_stream = true;
     ISHMEMI_CUDA(cudaEventCreateWithFlags(&g.ev_team, cudaEventDisableTiming));
     g.team_seq = 0;
+    g.team_event_seq = 0;
     g.free_blocks.clear();
     g.used_blocks.clear();
     g.free_blocks[0] = heap_bytes;
