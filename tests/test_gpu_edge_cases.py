@@ -1,0 +1,124 @@
+"""Degenerate and extreme shapes against the oracle: one PE, the maximum number of PEs,
+zero-length operations, strided teams, sizes around the kernels' internal thresholds."""
+import numpy as np
+import pytest
+import torch
+
+import oracle as orc
+from paper_2409_20476_b200 import binding as B
+from paper_2409_20476_b200 import inputs
+from tests.gpu_util import Session, heaps_equal
+
+pytestmark = pytest.mark.gpu
+W = B.ISHMEM_TEAM_WORLD
+
+
+def run_everything(s, npes, n, team=None, oteam=None):
+    """one pass of every collective and a put/get ring of n bytes on both sides"""
+    o = s.oracle
+    team = W if team is None else team
+    oteam = o.world if oteam is None else oteam
+    P = oteam[2]
+    src, dst = s.malloc(max(n * P, 64)), s.malloc(max(n * P * P, 64))
+    for p in range(npes):
+        src.fill(p, inputs.byte_payload(inputs.SEED_C2, 200 + p, max(n * P, 64)))
+    for p in range(npes):
+        t = (p + 1) % npes
+        B.ishmem_putmem(p, dst.addr, src.addr, n, t)
+        o.putmem(p, dst.ooff, o.ptr(src.ooff, n, p), n, t)
+    B.ishmem_barrier_all()
+    for p in range(npes):
+        t = (p + npes - 1) % npes
+        B.ishmem_getmem(p, dst.addr + n, src.addr, n, t)
+        o.getmem(p, o.ptr(dst.ooff + n, n, p), src.ooff, n, t)
+    B.ishmem_barrier_all()
+    heaps_equal(s, f"put/get ring npes={npes} n={n}")
+    B.ishmem_broadcastmem(team, dst.addr, src.addr, n, P - 1)
+    o.broadcastmem(oteam, dst.ooff, src.ooff, n, P - 1)
+    heaps_equal(s, "broadcast")
+    B.ishmem_fcollectmem(team, dst.addr, src.addr, n)
+    o.fcollectmem(oteam, dst.ooff, src.ooff, n)
+    heaps_equal(s, "fcollect")
+    B.ishmem_alltoallmem(team, dst.addr, src.addr, n)
+    o.alltoallmem(oteam, dst.ooff, src.ooff, n)
+    heaps_equal(s, "alltoall")
+    sizes = [(n * (i % 3)) // 2 for i in range(P)]
+    B.ishmem_collectmem(team, dst.addr, src.addr, np.array(sizes, dtype=np.uint64))
+    o.collectmem(oteam, dst.ooff, src.ooff, sizes)
+    heaps_equal(s, "collect")
+    for alg in (B.ISHMEMX_REDUCE_SPLIT, B.ISHMEMX_REDUCE_DUPLICATED):
+        B.ishmemx_reduce(team, dst.addr, src.addr, n // 8, B.ISHMEM_OP_XOR, B.ISHMEM_T_UINT64, alg)
+        o.reduce(oteam, dst.ooff, src.ooff, n // 8, orc.R_XOR, orc.T_UINT64)
+        # (the payload is random bytes: as floats they would contain NaNs, whose payloads are outside
+        # the bit-exact contract, so the arithmetic fold here is the wrapping int32 sum)
+        B.ishmemx_reduce(team, dst.addr + 8 * (n // 8 + 1), src.addr, n // 4, B.ISHMEM_OP_SUM, B.ISHMEM_T_INT32, alg)
+        o.reduce(oteam, dst.ooff + 8 * (n // 8 + 1), src.ooff, n // 4, orc.R_SUM, orc.T_INT32)
+        heaps_equal(s, f"reduce alg={alg}")
+    B.ishmem_team_sync(team)
+    assert s.status() == 0
+
+
+@pytest.mark.parametrize("n", [0, 8, 4104])
+def test_a_single_pe_is_a_valid_job(n):
+    """P = 1: every collective degenerates to a local copy (reduce of one source = that source)."""
+    with Session(1, 1 << 18) as s:
+        run_everything(s, 1, n)
+
+
+@pytest.mark.parametrize("n", [0, 16, 1032])
+def test_the_maximum_number_of_pes(n):
+    """64 PEs (ISHMEM_MAX_PES): translation tables, push sync and the collectives at full width."""
+    npes = B.ISHMEM_MAX_PES
+    with Session(npes, (1 << 16) + n * npes * npes * 2) as s:
+        run_everything(s, npes, n)
+        with pytest.raises(B.IshmemError) as e:
+            B.ishmem_putmem(0, s.malloc(64).addr, s.malloc(64).addr, 8, npes)
+        assert e.value.code == B.ISHMEM_ERR_INVALID_PE
+
+
+def test_more_pes_than_the_library_supports_is_refused():
+    heap = torch.zeros(65 * 4096, dtype=torch.uint8, device="cuda")
+    with pytest.raises(B.IshmemError) as e:
+        B.ishmemx_init_external(B.ISHMEM_MAX_PES + 1, 4096, heap.data_ptr())
+    assert e.value.code == B.ISHMEM_ERR_ARG
+
+
+def test_strided_teams_only_touch_their_members():
+    npes = 12
+    with Session(npes, 1 << 20) as s:
+        team = B.ishmem_team_split_strided(W, 2, 4, 3)                 # PEs 2, 6, 10
+        assert B.ishmem_team_n_pes(team) == 3
+        run_everything(s, npes, 2056, team, (2, 4, 3))
+        sub = B.ishmem_team_split_strided(team, 1, 1, 2)                # PEs 6, 10 of the parent
+        src, dst = s.malloc(4096), s.malloc(8192)
+        for p in range(npes):
+            src.fill(p, inputs.byte_payload(inputs.SEED_C3, 300 + p, 4096))
+        B.ishmem_fcollectmem(sub, dst.addr, src.addr, 3000)
+        s.oracle.fcollectmem((6, 4, 2), dst.ooff, src.ooff, 3000)
+        heaps_equal(s, "team of a team")
+        B.ishmem_team_destroy(sub)
+        B.ishmem_team_destroy(team)
+        assert B.ishmem_team_split_strided(W, 0, 5, 4) == B.ISHMEM_TEAM_INVALID     # 0, 5, 10, 15: outside
+        assert s.status() == 0
+
+
+@pytest.mark.parametrize("n", [16383, 16384, 16385, (1 << 20) - 1, (1 << 20) + 16, (4 << 20) + 1])
+def test_sizes_around_the_internal_thresholds(n):
+    """bulk-ring minimum (16 KiB), the 1 MiB push threshold, the 4 MiB host cutover"""
+    npes = 4
+    with Session(npes, 3 * n + (1 << 20)) as s:
+        src, dst = s.malloc(n + 32), s.malloc(2 * n + 64)
+        for p in range(npes):
+            src.fill(p, inputs.byte_payload(inputs.SEED_C2, 400 + p, n + 32))
+        for p in range(npes):
+            B.ishmem_putmem(p, dst.addr + 1, src.addr + 1, n, (p + 1) % npes)               # default cutover
+            s.oracle.putmem(p, dst.ooff + 1, s.oracle.ptr(src.ooff + 1, n, p), n, (p + 1) % npes)
+        B.ishmemx_putmem_spmd(dst.addr + n + 16, src.addr + 16, n, 2, B.ISHMEMX_WORK_GROUP_BULK, 256, 2)
+        for p in range(npes):
+            s.oracle.putmem(p, dst.ooff + n + 16, s.oracle.ptr(src.ooff + 16, n, p), n, (p + 2) % npes)
+        B.ishmem_barrier_all()
+        heaps_equal(s, f"puts n={n}")
+        B.ishmem_broadcastmem(W, dst.addr, src.addr, n, 1)
+        s.oracle.broadcastmem(s.oracle.world, dst.ooff, src.ooff, n, 1)
+        heaps_equal(s, f"broadcast n={n}")
+        assert s.status() == 0
