@@ -114,7 +114,10 @@ typedef int ishmem_team_t;
  * ishmem_init allocates the heap with cudaMalloc; ishmemx_init_external uses
  * npes*heap_bytes bytes at `base` (device memory, 256-byte aligned, owned by the caller,
  * e.g. a torch tensor; cf. the external-heap registration of Section 3.5) and does
- * not clear it.  ISHMEM_ERR_ARG if already initialised. */
+ * not clear it.  ISHMEM_ERR_ARG if already initialised.  ishmem_init(npes, 0) takes the heap
+ * size per PE from the environment variable ISHMEM_SYMMETRIC_SIZE (bytes).  Other variables read
+ * at initialisation: ISHMEM_CUTOVER_{PUT,BCAST,FCOLLECT,WORK_GROUP} (bytes, "never" or "always";
+ * see ishmemx_set_cutover) and ISHMEM_WAIT_TIMEOUT_NS (see ishmemx_set_wait_limit_ns). */
 int ishmem_init(int npes, size_t heap_bytes);
 int ishmemx_init_external(int npes, size_t heap_bytes, void *base);
 /* Waits for all streams, frees everything the library allocated. */

@@ -126,11 +126,24 @@ int ishmemi_engine_copy(int my_pe, void *dst, const void *src, size_t n, bool bl
 
 /* ---- lifecycle -------------------------------------------------------------------------- */
 
+/* a size from the environment: a number of bytes (0x.. accepted), or "never" / "always" */
+static bool env_size(const char *name, size_t *out)
+{
+    const char *v = getenv(name);
+    if (!v || !*v) return false;
+    if (!strcmp(v, "never")) *out = (size_t)-1;
+    else if (!strcmp(v, "always")) *out = 0;
+    else *out = (size_t)strtoull(v, nullptr, 0);
+    return true;
+}
+
 static int init_common(int npes, size_t heap_bytes, void *external)
 {
     auto &g = g_ishmem;
     if (g.initialised) return ISHMEM_ERR_ARG;
-    if (npes < 1 || npes > ISHMEM_MAX_PES || heap_bytes == 0) return ISHMEM_ERR_ARG;
+    /* ishmem_init(npes, 0): the heap size comes from ISHMEM_SYMMETRIC_SIZE (bytes per PE) */
+    if (heap_bytes == 0 && !external) env_size("ISHMEM_SYMMETRIC_SIZE", &heap_bytes);
+    if (npes < 1 || npes > ISHMEM_MAX_PES || heap_bytes == 0 || heap_bytes == (size_t)-1) return ISHMEM_ERR_ARG;
     int ndev = 0;
     if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev == 0) {
         g.last_cuda_error = "no CUDA device: this library has no CPU path";
@@ -206,13 +219,17 @@ static int init_common(int npes, size_t heap_bytes, void *external)
      * a host-initiated put/get of one PE is at least as fast on the copy engine from 4 MiB on
      * (5.8 against 6.1 us there, 6.3 against 5.6 TB/s at 256 MiB); the push collectives and
      * the device-initiated work-group calls never are, so they stay on loads and stores */
-    const char *env;
-    g.cutover[0] = (env = getenv("ISHMEM_CUTOVER_PUT")) ? strtoull(env, nullptr, 0) : ((size_t)4 << 20);
-    g.cutover[1] = (env = getenv("ISHMEM_CUTOVER_BCAST")) ? strtoull(env, nullptr, 0) : (size_t)-1;
-    g.cutover[2] = (env = getenv("ISHMEM_CUTOVER_FCOLLECT")) ? strtoull(env, nullptr, 0) : (size_t)-1;
-    g.wg_cutover = (env = getenv("ISHMEM_CUTOVER_WORK_GROUP")) ? strtoull(env, nullptr, 0) : (size_t)-1;
+    g.cutover[0] = (size_t)4 << 20;
+    g.cutover[1] = g.cutover[2] = g.wg_cutover = (size_t)-1;
+    env_size("ISHMEM_CUTOVER_PUT", &g.cutover[0]);
+    env_size("ISHMEM_CUTOVER_BCAST", &g.cutover[1]);
+    env_size("ISHMEM_CUTOVER_FCOLLECT", &g.cutover[2]);
+    env_size("ISHMEM_CUTOVER_WORK_GROUP", &g.wg_cutover);
+    {
+        size_t ns = 0;
+        if (env_size("ISHMEM_WAIT_TIMEOUT_NS", &ns) && ns && ns != (size_t)-1) g.wait_limit_ns = ns;
+    }
     g.hybrid_head = 0;
-    if ((env = getenv("ISHMEM_WAIT_TIMEOUT_NS"))) g.wait_limit_ns = strtoull(env, nullptr, 0);
     g.launches = 0;
     g.initialised = true;
     ishmemi_push_ctx();

@@ -154,3 +154,19 @@ def test_config4_pingpong(threads):
         assert s.status() == 0
         with pytest.raises(B.IshmemError):
             B.ishmemx_pingpong(2, 2, data.addr, sig.addr, 8, 1, 32, None, None)
+
+
+def test_pingpong_100k_rounds_no_signal_overtakes_its_payload():
+    """Memory-model soak: 10^5 round trips at every payload size 8 B..64 KiB; each round stamps
+    its number into the first and last word of the payload, and the receiver counts stamps that
+    do not match the signalled round."""
+    with Session(2, 1 << 18, with_oracle=False) as s:
+        data, sig = s.malloc(1 << 16), s.malloc(64)
+        rtt, bad = np.zeros(1), np.zeros(1, dtype=np.uint64)
+        for n in inputs.message_sizes(3, 16):
+            B.ishmem_uint64_p(0, sig.addr, 0, 0)
+            B.ishmem_uint64_p(1, sig.addr, 0, 1)
+            B.ishmemx_pingpong(0, 1, data.addr, sig.addr, n, 100_000, 256, rtt, bad)
+            assert bad[0] == 0, (n, int(bad[0]))
+            assert sig.read(0, np.uint64)[0] == 100_000 and sig.read(1, np.uint64)[0] == 100_000
+        assert s.status() == 0

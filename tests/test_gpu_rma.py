@@ -288,3 +288,26 @@ def test_device_timed_latency_program_moves_the_data(level):
             B.ishmemx_rma_latency(1, dst.addr, src.addr, 8, 7, 0, LEVELS[level], 64, 1, ns)
         assert e.value.code == B.ISHMEM_ERR_INVALID_PE
         assert s.status() == 0
+
+
+def test_environment_variables_at_initialisation(monkeypatch):
+    monkeypatch.setenv("ISHMEM_SYMMETRIC_SIZE", str(3 << 20))
+    monkeypatch.setenv("ISHMEM_CUTOVER_PUT", "never")
+    monkeypatch.setenv("ISHMEM_CUTOVER_BCAST", "always")
+    monkeypatch.setenv("ISHMEM_CUTOVER_FCOLLECT", "0x10000")
+    B.ishmem_init(2, 0)
+    try:
+        assert B.ishmemx_heap_bytes() == 3 << 20 and B.ishmem_n_pes() == 2
+        assert B.ishmemx_get_cutover(0) == B.SIZE_MAX and B.ishmemx_get_cutover(1) == 0
+        assert B.ishmemx_get_cutover(2) == 0x10000 and B.ishmemx_get_cutover(3) == B.SIZE_MAX
+        a = B.ishmem_calloc(16, 8)
+        B.ishmem_int64_p(0, a + 8, -5, 1)
+        out = np.zeros(1, np.int64)
+        B.ishmem_int64_g(0, out, a + 8, 1)
+        assert out[0] == -5
+    finally:
+        B.ishmem_finalize()
+    monkeypatch.delenv("ISHMEM_SYMMETRIC_SIZE")
+    with pytest.raises(B.IshmemError) as e:
+        B.ishmem_init(2, 0)
+    assert e.value.code == B.ISHMEM_ERR_ARG
