@@ -631,10 +631,6 @@ static int jacobi_launch(double *buf0, double *buf1, uint64_t *sig, size_t ny, s
          * and a deeper window; everything else the 1024-thread instance */
         const bool wide = threads <= 512 && nblocks <= (size_t)g.sm_count;
         void *kernel = wide ? (void *)k_jacobi<512, 8> : (void *)k_jacobi<1024, 4>;
-        static const char *env_depth = getenv("ISHMEM_JACOBI_DEPTH");
-        if (wide && env_depth && atoi(env_depth) == 12) kernel = (void *)k_jacobi<512, 12>;
-        if (wide && env_depth && atoi(env_depth) == 16) kernel = (void *)k_jacobi<512, 16>;
-        if (wide && env_depth && atoi(env_depth) == 4) kernel = (void *)k_jacobi<512, 4>;
         rc = ishmemi_cuda(cudaLaunchCooperativeKernel(kernel, dim3((unsigned)nblocks), dim3(threads), params, 0, s),
                           "cudaLaunchCooperativeKernel(jacobi)");
     }
