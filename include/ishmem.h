@@ -332,6 +332,19 @@ int ishmem_barrier_all(void);
 ishmem_team_t ishmem_team_split_strided(ishmem_team_t parent, int start, int stride, int size);
 int ishmem_team_destroy(ishmem_team_t team);
 int ishmem_team_n_pes(ishmem_team_t team);
+/* Index of world PE `pe` inside `team`, or -1 when it is not a member (OpenSHMEM's team_my_pe, with
+ * the PE explicit because all PEs live in this process). */
+int ishmem_team_my_pe(ishmem_team_t team, int pe);
+/* The PE with index `src_pe` in src_team, expressed as an index in dest_team; -1 when it is not
+ * a member of dest_team or an argument is invalid. */
+int ishmem_team_translate_pe(ishmem_team_t src_team, int src_pe, ishmem_team_t dest_team);
+/* Library identification (OpenSHMEM info routines): the OpenSHMEM level the API follows, and a
+ * name of at most ISHMEM_MAX_NAME_LEN - 1 characters copied to HOST `name`. */
+#define ISHMEM_MAJOR_VERSION 1
+#define ISHMEM_MINOR_VERSION 5
+#define ISHMEM_MAX_NAME_LEN 64
+void ishmem_info_get_version(int *major, int *minor);
+void ishmem_info_get_name(char *name);
 
 /* --------------------------------------------------------------- remote atomics --- */
 

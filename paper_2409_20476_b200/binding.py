@@ -141,6 +141,10 @@ def _signatures() -> dict[str, tuple[str, list[str]]]:
         "ishmem_team_split_strided": ("int", ["i", "i", "i", "i"]),
         "ishmem_team_destroy": ("status", ["i"]),
         "ishmem_team_n_pes": ("int", ["i"]),
+        "ishmem_team_my_pe": ("int", ["i", "i"]),
+        "ishmem_team_translate_pe": ("int", ["i", "i", "i"]),
+        "ishmem_info_get_version": ("void", ["p", "p"]),
+        "ishmem_info_get_name": ("void", ["p"]),
         "ishmemx_int64_atomic_fetch_add_batch": ("status", ["p", "p", "p", "p", "z", "i", "i"]),
         "ishmemx_int64_atomic_compare_swap_batch": ("status", ["p", "p", "p", "p", "p", "z", "i"]),
         "ishmem_broadcastmem": ("status", ["i", "p", "p", "z", "i"]),
@@ -211,6 +215,8 @@ def lib() -> C.CDLL:
             if ret == "status":
                 f.restype = C.c_int
                 f.errcheck = _status_check(name)
+            elif ret == "void":
+                f.restype = None
             elif ret == "int":
                 f.restype = C.c_int
             elif ret == "ptr":

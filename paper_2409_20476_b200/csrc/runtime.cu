@@ -507,6 +507,37 @@ extern "C" int ishmem_team_n_pes(ishmem_team_t team)
     return g.teams[team].size;
 }
 
+static int index_in(const ishmemi_team &t, int pe)
+{
+    const int d = pe - t.start;
+    if (d < 0 || d % t.stride) return -1;
+    return d / t.stride < t.size ? d / t.stride : -1;
+}
+extern "C" int ishmem_team_my_pe(ishmem_team_t team, int pe)
+{
+    auto &g = g_ishmem;
+    if (!g.initialised || team < 0 || team >= ISHMEM_MAX_TEAMS || !g.teams[team].valid || ishmemi_check_pe(pe)) return -1;
+    return index_in(g.teams[team], pe);
+}
+extern "C" int ishmem_team_translate_pe(ishmem_team_t src_team, int src_pe, ishmem_team_t dest_team)
+{
+    auto &g = g_ishmem;
+    if (!g.initialised || src_team < 0 || src_team >= ISHMEM_MAX_TEAMS || !g.teams[src_team].valid) return -1;
+    if (dest_team < 0 || dest_team >= ISHMEM_MAX_TEAMS || !g.teams[dest_team].valid) return -1;
+    const ishmemi_team &s = g.teams[src_team];
+    if (src_pe < 0 || src_pe >= s.size) return -1;
+    return index_in(g.teams[dest_team], s.start + src_pe * s.stride);
+}
+extern "C" void ishmem_info_get_version(int *major, int *minor)
+{
+    if (major) *major = ISHMEM_MAJOR_VERSION;
+    if (minor) *minor = ISHMEM_MINOR_VERSION;
+}
+extern "C" void ishmem_info_get_name(char *name)
+{
+    if (name) strncpy(name, "ishmem for B200 (sm_100a), after Intel SHMEM", ISHMEM_MAX_NAME_LEN - 1), name[ISHMEM_MAX_NAME_LEN - 1] = 0;
+}
+
 extern "C" int ishmemx_set_cutover(int which, size_t nbytes)
 {
     ISHMEMI_REQUIRE_INIT();

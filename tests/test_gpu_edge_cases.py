@@ -96,6 +96,14 @@ def test_strided_teams_only_touch_their_members():
         B.ishmem_fcollectmem(sub, dst.addr, src.addr, 3000)
         s.oracle.fcollectmem((6, 4, 2), dst.ooff, src.ooff, 3000)
         heaps_equal(s, "team of a team")
+        assert [B.ishmem_team_my_pe(team, p) for p in (2, 6, 10, 3, 11)] == [0, 1, 2, -1, -1]
+        assert [B.ishmem_team_my_pe(sub, p) for p in (2, 6, 10)] == [-1, 0, 1]
+        assert B.ishmem_team_translate_pe(sub, 1, team) == 2 and B.ishmem_team_translate_pe(team, 0, sub) == -1
+        assert B.ishmem_team_translate_pe(team, 2, W) == 10 and B.ishmem_team_translate_pe(W, 7, team) == -1
+        major, minor, name = np.zeros(1, np.int32), np.zeros(1, np.int32), np.zeros(64, np.uint8)
+        B.ishmem_info_get_version(major, minor)
+        B.ishmem_info_get_name(name)
+        assert (major[0], minor[0]) == (1, 5) and bytes(name).split(b"\0")[0].startswith(b"ishmem")
         B.ishmem_team_destroy(sub)
         B.ishmem_team_destroy(team)
         assert B.ishmem_team_split_strided(W, 0, 5, 4) == B.ISHMEM_TEAM_INVALID     # 0, 5, 10, 15: outside
