@@ -506,10 +506,12 @@ int ishmemx_jacobi(double *buf0, double *buf1, uint64_t *sig, size_t ny, size_t 
 int ishmemx_jacobi_noalloc(double *buf0, double *buf1, uint64_t *sig, size_t ny, size_t nx, int iters,
                            int overlap, int groups_per_pe, int threads, double *residual_sq_host);
 
-/* Host-buffer convenience for end-to-end measurements: copy `nbytes` from HOST `src_host`
- * into src@p for every PE p (per-PE stride `nbytes` in the host buffer), run
- * ishmemx_putmem_spmd(dest, src, nbytes, shift, level, threads, groups), and copy every
- * dest@p back to HOST `dest_host`.  Blocks the host. */
+/* Host-buffer convenience for end-to-end measurements: for every PE p, copy `nbytes` from HOST
+ * `src_host` (per-PE stride `nbytes`) into src@p, let PE p put it to dest@((p + shift) mod npes)
+ * (device call of the given level with `groups` work-groups of `threads` threads), and copy that
+ * destination back to HOST `dest_host` (same layout).  Each PE's three steps run on its own
+ * stream, so transfers in the two directions overlap between PEs; with pinned host memory the
+ * copies are asynchronous.  Blocks the host until everything has arrived. */
 int ishmemx_host_put_ring(void *dest_host, const void *src_host, void *dest, void *src,
                           size_t nbytes, int shift, int level, int threads, int groups);
 

@@ -647,12 +647,36 @@ extern "C" int ishmemx_host_put_ring(void *dest_host, const void *src_host, void
     ISHMEMI_REQUIRE_INIT();
     auto &g = g_ishmem;
     if (!dest_host || !src_host) return ISHMEM_ERR_ARG;
-    int rc;
-    for (int p = 0; p < g.npes; ++p)
-        if ((rc = ishmemx_heap_write(p, src, (const char *)src_host + (size_t)p * nbytes, nbytes))) return rc;
-    if ((rc = ishmemx_putmem_spmd(dest, src, nbytes, shift, level, threads, groups))) return rc;
-    for (int p = 0; p < g.npes; ++p)
-        if ((rc = ishmemx_heap_read(p, (char *)dest_host + (size_t)p * nbytes, dest, nbytes))) return rc;
-    for (int p = 0; p < g.npes; ++p) ISHMEMI_CUDA(cudaStreamSynchronize(g.pe_stream[p]));
-    return ISHMEM_OK;
+    if (groups < 1 || shift < 0) return ISHMEM_ERR_ARG;
+    long long doff = ishmemi_sym_offset(dest, nbytes), soff = ishmemi_sym_offset(src, nbytes);
+    if (doff < 0 || soff < 0) return ISHMEM_ERR_NOT_SYMMETRIC;
+    /* One pipeline per PE on that PE's stream: payload in, the PE's put, and the copy back of the
+     * destination that put has just filled.  The pipelines of different PEs overlap, so the bus
+     * carries host-to-device and device-to-host traffic at the same time. */
+    int rc = ISHMEM_OK;
+    for (int p = 0; p < g.npes && !rc; ++p) {
+        const int t = (p + shift) % g.npes;
+        cudaStream_t s = ishmemi_pe_stream_for_op(p);
+        rc = ishmemi_cuda(cudaMemcpyAsync(g.base + (size_t)p * g.heap_bytes + (size_t)soff,
+                                          (const char *)src_host + (size_t)p * nbytes, nbytes, cudaMemcpyHostToDevice, s),
+                          "cudaMemcpyAsync(H2D)");
+        if (rc) break;
+        rma_args a = {};
+        a.dest = g.base + (size_t)p * g.heap_bytes + (size_t)doff; /* my_pe's copy: translated to t in the kernel */
+        a.src = g.base + (size_t)p * g.heap_bytes + (size_t)soff;
+        a.nbytes = nbytes;
+        a.my_pe = p;
+        a.pe = t;
+        a.groups = groups;
+        if (nbytes) rc = launch_rma(s, a, level, threads, (unsigned)groups);
+        if (rc) break;
+        rc = ishmemi_cuda(cudaMemcpyAsync((char *)dest_host + (size_t)t * nbytes,
+                                          g.base + (size_t)t * g.heap_bytes + (size_t)doff, nbytes, cudaMemcpyDeviceToHost, s),
+                          "cudaMemcpyAsync(D2H)");
+    }
+    for (int p = 0; p < g.npes; ++p) {
+        int rc2 = ishmemi_cuda(cudaStreamSynchronize(g.pe_stream[p]), "cudaStreamSynchronize");
+        if (!rc) rc = rc2;
+    }
+    return rc;
 }

@@ -311,3 +311,26 @@ def test_environment_variables_at_initialisation(monkeypatch):
     with pytest.raises(B.IshmemError) as e:
         B.ishmem_init(2, 0)
     assert e.value.code == B.ISHMEM_ERR_ARG
+
+
+@pytest.mark.parametrize("pinned", [True, False])
+def test_host_put_ring_with_host_buffers(pinned):
+    """The end-to-end entry point: host payloads in, ring put on the device, destinations back
+    on the host -- against the oracle's puts, with pinned and with pageable host memory."""
+    npes, n = 5, 70_001
+    with Session(npes, 1 << 19) as s:
+        src, dst = s.malloc(n), s.malloc(n)
+        hsrc = torch.from_numpy(np.concatenate([inputs.byte_payload(inputs.SEED_C2, 500 + p, n) for p in range(npes)]))
+        hdst = torch.zeros(npes * n, dtype=torch.uint8)
+        if pinned:
+            hsrc, hdst = hsrc.pin_memory(), hdst.pin_memory()
+        for level, shift in (("work_group", 1), ("work_group_bulk", 3)):
+            B.ishmemx_host_put_ring(hdst.data_ptr(), hsrc.data_ptr(), dst.addr, src.addr, n, shift, LEVELS[level], 256, 2)
+            for p in range(npes):
+                s.oracle.view(src.ooff, n, p)[:] = hsrc[p * n:(p + 1) * n].numpy()
+                s.oracle.putmem(p, dst.ooff, s.oracle.ptr(src.ooff, n, p), n, (p + shift) % npes)
+            heaps_equal(s, f"host_put_ring {level}")
+            for p in range(npes):
+                t = (p + shift) % npes
+                assert torch.equal(hdst[t * n:(t + 1) * n], hsrc[p * n:(p + 1) * n]), (level, p)
+        assert s.status() == 0
