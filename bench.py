@@ -201,7 +201,7 @@ def run_ours(args) -> dict:
         B.ishmem_uint64_p(1, ppsig, 0, 1)
         B.ishmemx_pingpong(0, 1, ppdata, ppsig, S["pp_bytes"], S["pp_rounds"], 256, rtt, bad)
         B.ishmemx_int64_atomic_fetch_add_batch(table, word, inc, fetched, NOPS_FADD, 1024, 2)
-        B.ishmemx_int64_atomic_compare_swap_batch(table, cword, ccond, cval, fetched, NOPS_CAS, 256)
+        B.ishmemx_int64_atomic_compare_swap_batch(table, cword, ccond, cval, fetched, NOPS_CAS, 256, 1)
         B.ishmem_broadcastmem(B.ISHMEM_TEAM_WORLD, dst, src, S["bcast"], 0)
         B.ishmem_fcollectmem(B.ISHMEM_TEAM_WORLD, dst, src, S["fcollect"])
         B.ishmem_float_sum_reduce(B.ISHMEM_TEAM_WORLD, dst, src, S["reduce_f32"])
@@ -313,17 +313,19 @@ def breakdown(B, torch, team_stream, env) -> dict:
         "fetch_add_no_aggregation": lambda: B.ishmemx_int64_atomic_fetch_add_batch(table, word, inc, fetched,
                                                                                      NOPS_FADD, 256, 0),
         "compare_swap": lambda: B.ishmemx_int64_atomic_compare_swap_batch(table, cword, ccond, cval, fetched,
-                                                                          NOPS_CAS, 256),
+                                                                          NOPS_CAS, 256, 1),
+        "compare_swap_no_aggregation": lambda: B.ishmemx_int64_atomic_compare_swap_batch(table, cword, ccond, cval,
+                                                                                         fetched, NOPS_CAS, 256, 0),
     }
     res = {}
     for name, fn in ops.items():
         ms = timed(fn)
         key = {"copy_engine_put": "put", "fetch_add_no_aggregation": "fetch_add",
-               "fetch_add_warp_aggregation": "fetch_add"}.get(name, name)
+               "fetch_add_warp_aggregation": "fetch_add", "compare_swap_no_aggregation": "compare_swap"}.get(name, name)
         entry = {"ms": round(ms, 4), "GB/s": round(nbytes[key] / (ms * 1e-3) / 1e9, 1)}
         if "fetch_add" in name:
             entry["Mops/s"] = round(NOPS_FADD / (ms * 1e-3) / 1e6, 1)
-        if name == "compare_swap":
+        if name.startswith("compare_swap"):
             entry["Mops/s"] = round(NOPS_CAS / (ms * 1e-3) / 1e6, 1)
         res[name] = entry
     return res

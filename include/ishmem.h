@@ -383,9 +383,12 @@ ISHMEM_DECL_AMO(uint64, uint64_t)
 int ishmemx_int64_atomic_fetch_add_batch(int64_t *table, const int32_t *word_idx,
                                          const int64_t *inc, int64_t *fetched, size_t nops,
                                          int threads, int aggregate);
+/* compare_swap: aggregate = 1 lets the lanes of a warp that hit the same word act as one group
+ * whose operations are applied back to back in lane order by a single compare-and-swap of the
+ * word (a read alone when the group changes nothing); aggregate = 0: one atomic per op. */
 int ishmemx_int64_atomic_compare_swap_batch(int64_t *table, const int32_t *word_idx,
                                             const int64_t *cond, const int64_t *value,
-                                            int64_t *fetched, size_t nops, int threads);
+                                            int64_t *fetched, size_t nops, int threads, int aggregate);
 
 /* ------------------------------------------------- collectives (Section 3.7.2) --- */
 

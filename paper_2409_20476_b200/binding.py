@@ -146,7 +146,7 @@ def _signatures() -> dict[str, tuple[str, list[str]]]:
         "ishmem_info_get_version": ("void", ["p", "p"]),
         "ishmem_info_get_name": ("void", ["p"]),
         "ishmemx_int64_atomic_fetch_add_batch": ("status", ["p", "p", "p", "p", "z", "i", "i"]),
-        "ishmemx_int64_atomic_compare_swap_batch": ("status", ["p", "p", "p", "p", "p", "z", "i"]),
+        "ishmemx_int64_atomic_compare_swap_batch": ("status", ["p", "p", "p", "p", "p", "z", "i", "i"]),
         "ishmem_broadcastmem": ("status", ["i", "p", "p", "z", "i"]),
         "ishmemx_set_bcast_root_dest": ("status", ["i"]),
         "ishmem_fcollectmem": ("status", ["i", "p", "p", "z"]),

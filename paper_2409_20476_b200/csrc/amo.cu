@@ -245,6 +245,13 @@ __global__ void __launch_bounds__(1024) k_fetch_add_batch(const ishmem_ctx_t *ct
     if (fetched) fetched[i] = base + before;
 }
 
+/* AGGREGATE: the lanes of a warp that hit the same word act as one group whose compare-and-swaps
+ * are applied back to back in lane order: the group's lowest lane reads the word, runs the chain
+ * on that value (each op sees the state its predecessors left and swaps if it equals its
+ * condition) and installs the end state with ONE compare-and-swap against the value it read,
+ * retrying when somebody else got in between.  The successful swap (or, when the chain changes
+ * nothing, the read) is the point at which the whole group takes effect. */
+template <bool AGGREGATE>
 __global__ void __launch_bounds__(1024) k_compare_swap_batch(const ishmem_ctx_t *ctxs, long long *table0,
                                                              const int *word_idx, const long long *cond,
                                                              const long long *value, long long *fetched,
@@ -252,12 +259,53 @@ __global__ void __launch_bounds__(1024) k_compare_swap_batch(const ishmem_ctx_t 
 {
     const int npes = ctxs[0].npes;
     const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= nops) return;
+    const bool active = i < nops;
     const ishmem_ctx_t *ctx = ctxs + (int)(i % (size_t)npes);
     long long *table = table_of(ctxs, ctx, table0);
+    if (!AGGREGATE) {
+        if (!active) return;
+        const int w = word_idx[i];
+        long long old = ishmem_atomic_compare_swap<long long>(ctx, table + w / npes, cond[i], value[i], w % npes);
+        if (fetched) fetched[i] = old;
+        return;
+    }
+    __shared__ long long sh_cond[1024], sh_val[1024], sh_old[1024];
+    const unsigned lane = threadIdx.x & 31u, wbase = threadIdx.x & ~31u;
+    const unsigned act = __ballot_sync(0xffffffffu, active);
+    if (!active) return;
     const int w = word_idx[i];
-    long long old = ishmem_atomic_compare_swap<long long>(ctx, table + w / npes, cond[i], value[i], w % npes);
-    if (fetched) fetched[i] = old;
+    sh_cond[threadIdx.x] = cond[i];
+    sh_val[threadIdx.x] = value[i];
+    const unsigned peers = __match_any_sync(act, w);
+    __syncwarp(act);
+    if (lane == (unsigned)__ffs(peers) - 1) {
+        long long *target = ishmem_ptr(ctx, table + w / npes, w % npes);
+        if (target) {
+            for (int tries = 0;; ++tries) {
+                const long long cur = ishmem_atomic_fetch<long long>(ctx, table + w / npes, w % npes);
+                long long state = cur;
+                for (unsigned rest = peers; rest; rest &= rest - 1) {
+                    const unsigned k = wbase + (unsigned)__ffs(rest) - 1;
+                    sh_old[k] = state;
+                    if (state == sh_cond[k]) state = sh_val[k];
+                }
+                if (state == cur) break; /* the chain leaves the word as it is */
+                if ((long long)atomicCAS((unsigned long long *)target, (unsigned long long)cur,
+                                         (unsigned long long)state) == cur)
+                    break;
+                if (tries == 4096) { /* give way: apply the ops one by one */
+                    for (unsigned rest = peers; rest; rest &= rest - 1) {
+                        const unsigned k = wbase + (unsigned)__ffs(rest) - 1;
+                        sh_old[k] = (long long)atomicCAS((unsigned long long *)target, (unsigned long long)sh_cond[k],
+                                                         (unsigned long long)sh_val[k]);
+                    }
+                    break;
+                }
+            }
+        }
+    }
+    __syncwarp(act);
+    if (fetched) fetched[i] = sh_old[threadIdx.x];
 }
 
 static int batch_geometry(size_t nops, int threads, int ops_per_thread, unsigned *blocks)
@@ -304,11 +352,11 @@ extern "C" int ishmemx_int64_atomic_fetch_add_batch(int64_t *table, const int32_
 
 extern "C" int ishmemx_int64_atomic_compare_swap_batch(int64_t *table, const int32_t *word_idx,
                                                        const int64_t *cond, const int64_t *value,
-                                                       int64_t *fetched, size_t nops, int threads)
+                                                       int64_t *fetched, size_t nops, int threads, int aggregate)
 {
     ISHMEMI_REQUIRE_INIT();
     auto &g = g_ishmem;
-    if (!word_idx || !cond || !value) return ISHMEM_ERR_ARG;
+    if (!word_idx || !cond || !value || aggregate < 0 || aggregate > 1) return ISHMEM_ERR_ARG;
     if ((uintptr_t)table % 8) return ISHMEM_ERR_ALIGN;
     if (ishmemi_sym_offset(table, 8) < 0) return ISHMEM_ERR_NOT_SYMMETRIC;
     unsigned blocks;
@@ -317,9 +365,14 @@ extern "C" int ishmemx_int64_atomic_compare_swap_batch(int64_t *table, const int
     cudaStream_t s;
     if ((rc = ishmemi_team_stream_begin(ISHMEM_TEAM_WORLD, &s))) return rc;
     if (nops) {
-        k_compare_swap_batch<<<blocks, threads, 0, s>>>(g.d_ctx, (long long *)table, word_idx,
-                                                        (const long long *)cond, (const long long *)value,
-                                                        (long long *)fetched, nops);
+        if (aggregate)
+            k_compare_swap_batch<true><<<blocks, threads, 0, s>>>(g.d_ctx, (long long *)table, word_idx,
+                                                                  (const long long *)cond, (const long long *)value,
+                                                                  (long long *)fetched, nops);
+        else
+            k_compare_swap_batch<false><<<blocks, threads, 0, s>>>(g.d_ctx, (long long *)table, word_idx,
+                                                                   (const long long *)cond, (const long long *)value,
+                                                                   (long long *)fetched, nops);
         ishmemi_count_launch();
         rc = ishmemi_check_launch("k_compare_swap_batch");
     }

@@ -429,10 +429,12 @@ def sweep_c4(args, out):
     cval = torch.arange(1, nops_c + 1, dtype=torch.int64, device="cuda")
     for cname, ccond in (("claim_cond_0", torch.zeros(nops_c, dtype=torch.int64, device="cuda")),
                          ("never_matches", torch.full((nops_c,), -7, dtype=torch.int64, device="cuda"))):
-        us, it = T(lambda i: B.ishmemx_int64_atomic_compare_swap_batch(table, cword, ccond, cval, fetched, nops_c, 256))
-        out.add(config=4, op="compare_swap", pattern="zipf1.1", variant=cname, threads=256, npes=npes, dtype="i64",
-                nbytes=8, l2="hot", iters=it, us_per_op=us, mops=round(nops_c / us, 1),
-                note=f"{nops_c} ops on {nwords_c} words")
+        for agg in (1, 0):
+            us, it = T(lambda i: B.ishmemx_int64_atomic_compare_swap_batch(table, cword, ccond, cval, fetched, nops_c,
+                                                                           256, agg))
+            out.add(config=4, op="compare_swap", pattern="zipf1.1", variant=cname + ("_aggregate_warp" if agg else "_plain"),
+                    threads=256, npes=npes, dtype="i64", nbytes=8, l2="hot", iters=it, us_per_op=us,
+                    mops=round(nops_c / us, 1), note=f"{nops_c} ops on {nwords_c} words")
     rtt, bad = np.zeros(1), np.zeros(1, dtype=np.uint64)
     rounds = 1000
     for threads in (32, 256, 1024):

@@ -81,7 +81,8 @@ def test_config4_fetch_add_batch(nops, nwords, aggregate):
         assert s.status() == 0
 
 
-def test_config4_compare_swap_batch():
+@pytest.mark.parametrize("aggregate", [0, 1])
+def test_config4_compare_swap_batch(aggregate):
     """2^20 compare_swap ops on 1024 words.  (i) claim: every op tries 0 -> id+1; exactly one
     op per touched word wins and everybody else sees the winner.  (ii) a CAS that cannot
     succeed leaves the table alone (bit-exact against the oracle)."""
@@ -93,7 +94,7 @@ def test_config4_compare_swap_batch():
         value = np.arange(1, nops + 1, dtype=np.int64)
         d = [torch.from_numpy(a).cuda() for a in (word, cond, value)]
         d_fetched = torch.full((nops,), -1, dtype=torch.int64, device="cuda")
-        B.ishmemx_int64_atomic_compare_swap_batch(table.addr, d[0], d[1], d[2], d_fetched, nops, 256)
+        B.ishmemx_int64_atomic_compare_swap_batch(table.addr, d[0], d[1], d[2], d_fetched, nops, 256, aggregate)
         s.sync()
         fetched = d_fetched.cpu().numpy()
         final = np.zeros(nwords, dtype=np.int64)
@@ -114,7 +115,7 @@ def test_config4_compare_swap_batch():
             table.fill(p, final[p::npes].copy())
         cond2 = np.full(nops, -1, dtype=np.int64)
         d_cond2 = torch.from_numpy(cond2).cuda()
-        B.ishmemx_int64_atomic_compare_swap_batch(table.addr, d[0], d_cond2, d[2], d_fetched, nops, 512)
+        B.ishmemx_int64_atomic_compare_swap_batch(table.addr, d[0], d_cond2, d[2], d_fetched, nops, 512, aggregate)
         exp_fetched = s.oracle.compare_swap_batch(table.ooff, word, cond2, value)
         heaps_equal(s, "cas no-op")
         assert np.array_equal(d_fetched.cpu().numpy(), exp_fetched)
@@ -169,4 +170,37 @@ def test_pingpong_100k_rounds_no_signal_overtakes_its_payload():
             B.ishmemx_pingpong(0, 1, data.addr, sig.addr, n, 100_000, 256, rtt, bad)
             assert bad[0] == 0, (n, int(bad[0]))
             assert sig.read(0, np.uint64)[0] == 100_000 and sig.read(1, np.uint64)[0] == 100_000
+        assert s.status() == 0
+
+
+@pytest.mark.parametrize("aggregate", [0, 1])
+def test_compare_swap_token_passing_is_linearisable(aggregate):
+    """Op k tries CAS(word, k, k+1) on its word, for k = 0..K-1 in a shuffled order, several
+    words at once.  Whatever the interleaving, an op can only succeed when the word holds exactly
+    k, so the successful ops of a word must be 0..m-1 (m = final value), each of them must have
+    fetched its own k, and every failed op must have fetched something else."""
+    npes, nwords, K = 16, 48, 4096
+    rng = inputs.rng_for(inputs.SEED_C4, 77)
+    word = np.repeat(np.arange(nwords, dtype=np.int32), K)
+    k = np.tile(np.arange(K, dtype=np.int64), nwords)
+    perm = rng.permutation(word.size)
+    word, k = word[perm].copy(), k[perm].copy()
+    with Session(npes, 1 << 16, with_oracle=False) as s:
+        table = s.malloc(8 * nwords // npes)
+        d = [torch.from_numpy(a).cuda() for a in (word, k, k + 1)]
+        fetched = torch.full((word.size,), -1, dtype=torch.int64, device="cuda")
+        for _ in range(3):                                  # later passes continue where the word stands
+            B.ishmemx_int64_atomic_compare_swap_batch(table.addr, d[0], d[1], d[2], fetched, word.size, 1024, aggregate)
+            s.sync()
+            f = fetched.cpu().numpy()
+            final = np.zeros(nwords, dtype=np.int64)
+            for p in range(npes):
+                final[p::npes] = table.read(p, np.int64)
+            ok = f == k
+            for w in range(nwords):
+                sel = word == w
+                won = np.sort(k[sel][ok[sel]])
+                assert won.size == 0 or won[-1] == final[w] - 1, (w, final[w])
+                assert np.array_equal(won, np.arange(final[w] - won.size, final[w])), w
+            assert (final > 0).all()
         assert s.status() == 0
