@@ -306,16 +306,18 @@ int ishmem_uint64_wait_until(int my_pe, uint64_t *ivar, int cmp, uint64_t value)
  * enqueued on my_pe's stream: HOST *result = 1 or 0.  Blocks the host. */
 int ishmem_uint64_test(int my_pe, uint64_t *ivar, int cmp, uint64_t value, int *result);
 /* Waits on `nelems` (at most 256) consecutive symmetric 64-bit words of my_pe (OpenSHMEM 1.5
- * wait_until_all / _any / _some, without the optional status mask), bounded like
- * ishmem_uint64_wait_until.  _all is stream-ordered.  _any writes the index of a satisfied word
- * to HOST *index; _some waits for at least one and writes the ascending indices of all words
- * satisfied at that moment to HOST indices[0..*count-1] (room for nelems).  _any and _some block
- * the host and return ISHMEM_ERR_TIMEOUT when the wait gave up. */
-int ishmem_uint64_wait_until_all(int my_pe, uint64_t *ivars, size_t nelems, int cmp, uint64_t value);
-int ishmem_uint64_wait_until_any(int my_pe, uint64_t *ivars, size_t nelems, int cmp, uint64_t value,
-                                 size_t *index);
-int ishmem_uint64_wait_until_some(int my_pe, uint64_t *ivars, size_t nelems, size_t *indices, int cmp,
-                                  uint64_t value, size_t *count);
+ * wait_until_all / _any / _some), bounded like ishmem_uint64_wait_until.  `status` is the
+ * standard's mask: a DEVICE array of nelems ints (or NULL) -- words whose entry is non-zero are
+ * left out.  _all is stream-ordered.  _any writes the index of a satisfied word to HOST *index;
+ * _some waits for at least one and writes the ascending indices of all words satisfied at that
+ * moment to HOST indices[0..*count-1] (room for nelems).  _any and _some block the host and
+ * return ISHMEM_ERR_TIMEOUT when the wait gave up. */
+int ishmem_uint64_wait_until_all(int my_pe, uint64_t *ivars, size_t nelems, const int *status, int cmp,
+                                 uint64_t value);
+int ishmem_uint64_wait_until_any(int my_pe, uint64_t *ivars, size_t nelems, const int *status, int cmp,
+                                 uint64_t value, size_t *index);
+int ishmem_uint64_wait_until_some(int my_pe, uint64_t *ivars, size_t nelems, size_t *indices, const int *status,
+                                  int cmp, uint64_t value, size_t *count);
 /* fence: orders my_pe's earlier puts before its later ones per target (stream order
  * already gives this; kept for API parity).  quiet: completes all outstanding operations
  * of my_pe, including _nbi transfers on the copy engine, in stream order. */
@@ -408,6 +410,23 @@ int ishmem_collectmem(ishmem_team_t team, void *dest, const void *src, const siz
 /* alltoall (OpenSHMEM 1.5): dest@q[i*nbytes + k] = src@member_i[q*nbytes + k]: block q of member
  * i's source lands in block i of member q's dest.  dest and src must not overlap.  Push. */
 int ishmem_alltoallmem(ishmem_team_t team, void *dest, const void *src, size_t nbytes);
+/* Typed names of the four data-movement collectives (counts in elements; addresses aligned to
+ * the element). */
+#define ISHMEM_DECL_COLL(NAME, T)                                                                          \
+    int ishmem_##NAME##_broadcast(ishmem_team_t team, T *dest, const T *src, size_t nelems, int root);      \
+    int ishmem_##NAME##_fcollect(ishmem_team_t team, T *dest, const T *src, size_t nelems);                 \
+    int ishmem_##NAME##_collect(ishmem_team_t team, T *dest, const T *src, const size_t *nelems_per_member); \
+    int ishmem_##NAME##_alltoall(ishmem_team_t team, T *dest, const T *src, size_t nelems);
+ISHMEM_DECL_COLL(float, float)
+ISHMEM_DECL_COLL(double, double)
+ISHMEM_DECL_COLL(int, int)
+ISHMEM_DECL_COLL(long, long)
+ISHMEM_DECL_COLL(int32, int32_t)
+ISHMEM_DECL_COLL(int64, int64_t)
+ISHMEM_DECL_COLL(uint8, uint8_t)
+ISHMEM_DECL_COLL(uint32, uint32_t)
+ISHMEM_DECL_COLL(uint64, uint64_t)
+#undef ISHMEM_DECL_COLL
 /* reduce: dest@q[j] = ((src@m0[j] op src@m1[j]) op ...) op src@m_{P-1}[j], folded in team
  * order (floating point bit-exact in that order), for every member q.  dest and src may
  * not overlap unless identical, which is handled with snapshot semantics only by the

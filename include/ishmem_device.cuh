@@ -1044,19 +1044,21 @@ __device__ __forceinline__ int ishmem_uint64_test(const ishmem_ctx_t *, const un
 }
 
 /* Waits on `nelems` consecutive 64-bit words of the calling PE (OpenSHMEM 1.5 wait_until_all /
- * _any / _some; without the optional status mask).  One thread calls.  All three are bounded
+ * _any / _some).  `status` (may be nullptr) is OpenSHMEM's mask: words whose status entry is
+ * non-zero are left out of the wait.  One thread calls.  All three are bounded
  * by ctx->wait_limit_ns and return 0 or ISHMEM_ERR_TIMEOUT (latched).
  * _all: every word satisfies the comparison.
  * _any: *index = some word that does (the lowest one found in a scan from 0).
  * _some: waits until at least one does, then lists ALL that do at that moment in indices[]
  *        (ascending, room for nelems entries) and their number in *count. */
 __device__ __forceinline__ int ishmem_uint64_wait_until_all(const ishmem_ctx_t *ctx, const unsigned long long *ivars,
-                                                            size_t nelems, int cmp, unsigned long long value)
+                                                            size_t nelems, int cmp, unsigned long long value,
+                                                            const int *status = nullptr)
 {
     ishmemi::deadline dl(ctx->wait_limit_ns);
     size_t k = 0;
     while (k < nelems) {
-        if (ishmemi::compare(ishmemi::ld_acquire(ivars + k), cmp, value)) {
+        if ((status && status[k]) || ishmemi::compare(ishmemi::ld_acquire(ivars + k), cmp, value)) {
             ++k;
             continue;
         }
@@ -1070,13 +1072,13 @@ __device__ __forceinline__ int ishmem_uint64_wait_until_all(const ishmem_ctx_t *
 }
 __device__ __forceinline__ int ishmem_uint64_wait_until_any(const ishmem_ctx_t *ctx, const unsigned long long *ivars,
                                                             size_t nelems, int cmp, unsigned long long value,
-                                                            size_t *index)
+                                                            size_t *index, const int *status = nullptr)
 {
     ishmemi::deadline dl(ctx->wait_limit_ns);
     if (nelems == 0) return 0;
     for (;;) {
         for (size_t k = 0; k < nelems; ++k)
-            if (ishmemi::compare(ishmemi::ld_acquire(ivars + k), cmp, value)) {
+            if (!(status && status[k]) && ishmemi::compare(ishmemi::ld_acquire(ivars + k), cmp, value)) {
                 *index = k;
                 return 0;
             }
@@ -1088,7 +1090,8 @@ __device__ __forceinline__ int ishmem_uint64_wait_until_any(const ishmem_ctx_t *
 }
 __device__ __forceinline__ int ishmem_uint64_wait_until_some(const ishmem_ctx_t *ctx, const unsigned long long *ivars,
                                                              size_t nelems, size_t *indices, int cmp,
-                                                             unsigned long long value, size_t *count)
+                                                             unsigned long long value, size_t *count,
+                                                             const int *status = nullptr)
 {
     ishmemi::deadline dl(ctx->wait_limit_ns);
     *count = 0;
@@ -1096,7 +1099,8 @@ __device__ __forceinline__ int ishmem_uint64_wait_until_some(const ishmem_ctx_t 
     for (;;) {
         size_t n = 0;
         for (size_t k = 0; k < nelems; ++k)
-            if (ishmemi::compare(ishmemi::ld_acquire(ivars + k), cmp, value)) indices[n++] = k;
+            if (!(status && status[k]) && ishmemi::compare(ishmemi::ld_acquire(ivars + k), cmp, value))
+                indices[n++] = k;
         if (n) {
             *count = n;
             return 0;

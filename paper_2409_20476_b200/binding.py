@@ -128,9 +128,9 @@ def _signatures() -> dict[str, tuple[str, list[str]]]:
         "ishmemx_iputmem": ("status", ["i", "p", "p", "z", "z", "z", "z", "i"]),
         "ishmemx_igetmem": ("status", ["i", "p", "p", "z", "z", "z", "z", "i"]),
         "ishmem_uint64_test": ("status", ["i", "p", "i", "u64", "p"]),
-        "ishmem_uint64_wait_until_all": ("status", ["i", "p", "z", "i", "u64"]),
-        "ishmem_uint64_wait_until_any": ("status", ["i", "p", "z", "i", "u64", "p"]),
-        "ishmem_uint64_wait_until_some": ("status", ["i", "p", "z", "p", "i", "u64", "p"]),
+        "ishmem_uint64_wait_until_all": ("status", ["i", "p", "z", "p", "i", "u64"]),
+        "ishmem_uint64_wait_until_any": ("status", ["i", "p", "z", "p", "i", "u64", "p"]),
+        "ishmem_uint64_wait_until_some": ("status", ["i", "p", "z", "p", "p", "i", "u64", "p"]),
         "ishmem_collectmem": ("status", ["i", "p", "p", "p"]),
         "ishmem_alltoallmem": ("status", ["i", "p", "p", "z"]),
         "ishmem_fence": ("status", ["i"]),
@@ -166,6 +166,10 @@ def _signatures() -> dict[str, tuple[str, list[str]]]:
     for name, t in _RMA_TYPES.items():
         for op in ("put", "get", "put_nbi", "get_nbi"):
             S[f"ishmem_{name}_{op}"] = ("status", ["i", "p", "p", "z", "i"])
+        S[f"ishmem_{name}_broadcast"] = ("status", ["i", "p", "p", "z", "i"])
+        S[f"ishmem_{name}_fcollect"] = ("status", ["i", "p", "p", "z"])
+        S[f"ishmem_{name}_collect"] = ("status", ["i", "p", "p", "p"])
+        S[f"ishmem_{name}_alltoall"] = ("status", ["i", "p", "p", "z"])
         S[f"ishmem_{name}_iput"] = ("status", ["i", "p", "p", "z", "z", "z", "i"])
         S[f"ishmem_{name}_iget"] = ("status", ["i", "p", "p", "z", "z", "z", "i"])
         S[f"ishmem_{name}_p"] = ("status", ["i", "p", t, "i"])

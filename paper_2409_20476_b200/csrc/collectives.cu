@@ -539,6 +539,55 @@ extern "C" int ishmem_alltoallmem(ishmem_team_t team, void *dest, const void *sr
     return rc;
 }
 
+template <typename T>
+static int typed_collect(ishmem_team_t team, T *dest, const T *src, const size_t *nelems)
+{
+    ISHMEMI_REQUIRE_INIT();
+    ishmemi_team t;
+    int rc = team_of(team, &t);
+    if (rc) return rc;
+    if (!nelems) return ISHMEM_ERR_ARG;
+    if (((uintptr_t)dest | (uintptr_t)src) % sizeof(T)) return ISHMEM_ERR_ALIGN;
+    size_t bytes[ISHMEM_MAX_PES];
+    for (int i = 0; i < t.size; ++i) {
+        if (nelems[i] > (size_t)-1 / sizeof(T)) return ISHMEM_ERR_ARG;
+        bytes[i] = nelems[i] * sizeof(T);
+    }
+    return ishmem_collectmem(team, dest, src, bytes);
+}
+#define ISHMEMI_DEF_COLL(NAME, T)                                                                                   \
+    extern "C" int ishmem_##NAME##_broadcast(ishmem_team_t team, T *dest, const T *src, size_t nelems, int root)     \
+    {                                                                                                                \
+        if (((uintptr_t)dest | (uintptr_t)src) % sizeof(T)) return ISHMEM_ERR_ALIGN;                                 \
+        if (nelems > (size_t)-1 / sizeof(T)) return ISHMEM_ERR_ARG;                                                  \
+        return ishmem_broadcastmem(team, dest, src, nelems * sizeof(T), root);                                       \
+    }                                                                                                                \
+    extern "C" int ishmem_##NAME##_fcollect(ishmem_team_t team, T *dest, const T *src, size_t nelems)                \
+    {                                                                                                                \
+        if (((uintptr_t)dest | (uintptr_t)src) % sizeof(T)) return ISHMEM_ERR_ALIGN;                                 \
+        if (nelems > (size_t)-1 / sizeof(T)) return ISHMEM_ERR_ARG;                                                  \
+        return ishmem_fcollectmem(team, dest, src, nelems * sizeof(T));                                              \
+    }                                                                                                                \
+    extern "C" int ishmem_##NAME##_collect(ishmem_team_t team, T *dest, const T *src, const size_t *nelems)          \
+    {                                                                                                                \
+        return typed_collect<T>(team, dest, src, nelems);                                                            \
+    }                                                                                                                \
+    extern "C" int ishmem_##NAME##_alltoall(ishmem_team_t team, T *dest, const T *src, size_t nelems)                \
+    {                                                                                                                \
+        if (((uintptr_t)dest | (uintptr_t)src) % sizeof(T)) return ISHMEM_ERR_ALIGN;                                 \
+        if (nelems > (size_t)-1 / sizeof(T)) return ISHMEM_ERR_ARG;                                                  \
+        return ishmem_alltoallmem(team, dest, src, nelems * sizeof(T));                                              \
+    }
+ISHMEMI_DEF_COLL(float, float)
+ISHMEMI_DEF_COLL(double, double)
+ISHMEMI_DEF_COLL(int, int)
+ISHMEMI_DEF_COLL(long, long)
+ISHMEMI_DEF_COLL(int32, int32_t)
+ISHMEMI_DEF_COLL(int64, int64_t)
+ISHMEMI_DEF_COLL(uint8, uint8_t)
+ISHMEMI_DEF_COLL(uint32, uint32_t)
+ISHMEMI_DEF_COLL(uint64, uint64_t)
+
 extern "C" int ishmemx_reduce(ishmem_team_t team, void *dest, const void *src, size_t nreduce, int op, int dtype,
                               int algorithm)
 {

@@ -135,19 +135,19 @@ __global__ void __launch_bounds__(256) k_strided(const ishmem_ctx_t *ctxs, int m
 
 /* which: 0 all, 1 any, 2 some; results (index / count + indices) go to host-mapped memory */
 __global__ void k_wait_many(const ishmem_ctx_t *ctxs, int my_pe, const unsigned long long *ivars, size_t nelems,
-                            int cmp, unsigned long long value, int which, unsigned long long *out)
+                            int cmp, unsigned long long value, int which, unsigned long long *out, const int *status)
 {
     const ishmem_ctx_t *ctx = ctxs + my_pe;
     if (which == 0) {
-        ishmem_uint64_wait_until_all(ctx, ivars, nelems, cmp, value);
+        ishmem_uint64_wait_until_all(ctx, ivars, nelems, cmp, value, status);
     } else if (which == 1) {
         size_t idx = 0;
-        int rc = ishmem_uint64_wait_until_any(ctx, ivars, nelems, cmp, value, &idx);
+        int rc = ishmem_uint64_wait_until_any(ctx, ivars, nelems, cmp, value, &idx, status);
         out[0] = (unsigned long long)(long long)rc;
         out[1] = idx;
     } else {
         size_t cnt = 0;
-        int rc = ishmem_uint64_wait_until_some(ctx, ivars, nelems, (size_t *)(out + 2), cmp, value, &cnt);
+        int rc = ishmem_uint64_wait_until_some(ctx, ivars, nelems, (size_t *)(out + 2), cmp, value, &cnt, status);
         out[0] = (unsigned long long)(long long)rc;
         out[1] = cnt;
     }
@@ -577,8 +577,8 @@ extern "C" int ishmem_uint64_test(int my_pe, uint64_t *ivar, int cmp, uint64_t v
     return ISHMEM_OK;
 }
 
-static int wait_many(int my_pe, uint64_t *ivars, size_t nelems, int cmp, uint64_t value, int which, size_t *index,
-                     size_t *indices, size_t *count)
+static int wait_many(int my_pe, uint64_t *ivars, size_t nelems, const int *status, int cmp, uint64_t value, int which,
+                     size_t *index, size_t *indices, size_t *count)
 {
     ISHMEMI_REQUIRE_INIT();
     if (ishmemi_check_pe(my_pe)) return ISHMEM_ERR_INVALID_PE;
@@ -590,7 +590,7 @@ static int wait_many(int my_pe, uint64_t *ivars, size_t nelems, int cmp, uint64_
     const unsigned long long *il = (const unsigned long long *)ishmemi_localise(ivars, nelems * 8, my_pe);
     cudaStream_t s = ishmemi_pe_stream_for_op(my_pe);
     unsigned long long *out = (unsigned long long *)g_ishmem.h_pinned; /* 4096 B: 2 + 256 words */
-    k_wait_many<<<1, 1, 0, s>>>(g_ishmem.d_ctx, my_pe, il, nelems, cmp, value, which, out);
+    k_wait_many<<<1, 1, 0, s>>>(g_ishmem.d_ctx, my_pe, il, nelems, cmp, value, which, out, status);
     ishmemi_count_launch();
     int rc = ishmemi_check_launch("k_wait_many");
     if (rc || which == 0) return rc;
@@ -604,19 +604,20 @@ static int wait_many(int my_pe, uint64_t *ivars, size_t nelems, int cmp, uint64_
     }
     return ISHMEM_OK;
 }
-extern "C" int ishmem_uint64_wait_until_all(int my_pe, uint64_t *ivars, size_t nelems, int cmp, uint64_t value)
+extern "C" int ishmem_uint64_wait_until_all(int my_pe, uint64_t *ivars, size_t nelems, const int *status, int cmp,
+                                            uint64_t value)
 {
-    return wait_many(my_pe, ivars, nelems, cmp, value, 0, nullptr, nullptr, nullptr);
+    return wait_many(my_pe, ivars, nelems, status, cmp, value, 0, nullptr, nullptr, nullptr);
 }
-extern "C" int ishmem_uint64_wait_until_any(int my_pe, uint64_t *ivars, size_t nelems, int cmp, uint64_t value,
-                                            size_t *index)
+extern "C" int ishmem_uint64_wait_until_any(int my_pe, uint64_t *ivars, size_t nelems, const int *status, int cmp,
+                                            uint64_t value, size_t *index)
 {
-    return wait_many(my_pe, ivars, nelems, cmp, value, 1, index, nullptr, nullptr);
+    return wait_many(my_pe, ivars, nelems, status, cmp, value, 1, index, nullptr, nullptr);
 }
-extern "C" int ishmem_uint64_wait_until_some(int my_pe, uint64_t *ivars, size_t nelems, size_t *indices, int cmp,
-                                             uint64_t value, size_t *count)
+extern "C" int ishmem_uint64_wait_until_some(int my_pe, uint64_t *ivars, size_t nelems, size_t *indices,
+                                             const int *status, int cmp, uint64_t value, size_t *count)
 {
-    return wait_many(my_pe, ivars, nelems, cmp, value, 2, nullptr, indices, count);
+    return wait_many(my_pe, ivars, nelems, status, cmp, value, 2, nullptr, indices, count);
 }
 
 extern "C" int ishmem_fence(int my_pe)

@@ -84,6 +84,19 @@ def test_collect_and_alltoall_12_pes():
         heaps_equal(s, "alltoall_work_group")
         with pytest.raises(B.IshmemError):
             B.ishmem_alltoallmem(B.ISHMEM_TEAM_WORLD, src.addr + 8, src.addr, 64)   # overlap
+        # typed names (counts in elements)
+        B.ishmem_double_broadcast(B.ISHMEM_TEAM_WORLD, dst.addr, src.addr, 1000, 3)
+        s.oracle.broadcastmem(s.oracle.world, dst.ooff, src.ooff, 8000, 3)
+        B.ishmem_int32_fcollect(team, dst.addr, src.addr, 777)
+        s.oracle.fcollectmem((1, 3, 4), dst.ooff, src.ooff, 4 * 777)
+        B.ishmem_uint64_alltoall(team, dst.addr + 64, src.addr, 99)
+        s.oracle.alltoallmem((1, 3, 4), dst.ooff + 64, src.ooff, 8 * 99)
+        B.ishmem_float_collect(team, dst.addr + 8, src.addr + 4, np.array([3, 0, 1000, 17], dtype=np.uint64))
+        s.oracle.collectmem((1, 3, 4), dst.ooff + 8, src.ooff + 4, [12, 0, 4000, 68])
+        heaps_equal(s, "typed collectives")
+        with pytest.raises(B.IshmemError) as e:
+            B.ishmem_double_fcollect(team, dst.addr + 4, src.addr, 8)
+        assert e.value.code == B.ISHMEM_ERR_ALIGN
         B.ishmem_team_destroy(team)
         assert s.status() == 0
 
@@ -136,20 +149,32 @@ def test_test_and_multi_word_waits():
                     B.ishmem_uint64_test(0, iv.addr + 8 * word, cmp_l, v, res)
                     assert bool(res[0]) == s.oracle.test(0, iv.ooff + 8 * word, cmp_o, v), (cmp_l, word, v)
         idx, cnt, found = np.zeros(1, np.uint64), np.zeros(1, np.uint64), np.zeros(8, np.uint64)
-        B.ishmem_uint64_wait_until_any(0, iv.addr, 8, B.ISHMEM_CMP_GE, 7, idx)
+        B.ishmem_uint64_wait_until_any(0, iv.addr, 8, None, B.ISHMEM_CMP_GE, 7, idx)
         assert idx[0] == 2
-        B.ishmem_uint64_wait_until_any(0, iv.addr, 8, B.ISHMEM_CMP_GT, 7, idx)
+        B.ishmem_uint64_wait_until_any(0, iv.addr, 8, None, B.ISHMEM_CMP_GT, 7, idx)
         assert idx[0] == 5
-        B.ishmem_uint64_wait_until_some(0, iv.addr, 8, found, B.ISHMEM_CMP_NE, 0, cnt)
+        B.ishmem_uint64_wait_until_some(0, iv.addr, 8, found, None, B.ISHMEM_CMP_NE, 0, cnt)
         assert cnt[0] == 2 and list(found[:2]) == [2, 5]
-        B.ishmem_uint64_wait_until_all(0, iv.addr, 8, B.ISHMEM_CMP_LE, 9)
+        # the status mask takes words out of the wait: word 2 masked -> only word 5 qualifies
+        mask = torch.zeros(8, dtype=torch.int32, device="cuda")
+        mask[2] = 1
+        torch.cuda.synchronize()
+        B.ishmem_uint64_wait_until_any(0, iv.addr, 8, mask, B.ISHMEM_CMP_NE, 0, idx)
+        assert idx[0] == 5
+        B.ishmem_uint64_wait_until_some(0, iv.addr, 8, found, mask, B.ISHMEM_CMP_NE, 0, cnt)
+        assert cnt[0] == 1 and found[0] == 5
+        allbut = torch.ones(8, dtype=torch.int32, device="cuda")
+        allbut[2] = allbut[5] = 0
+        torch.cuda.synchronize()
+        B.ishmem_uint64_wait_until_all(0, iv.addr, 8, allbut, B.ISHMEM_CMP_GE, 7)     # only words 2 and 5 count
+        B.ishmem_uint64_wait_until_all(0, iv.addr, 8, None, B.ISHMEM_CMP_LE, 9)
         assert s.status() == 0
         # nothing on PE 1 satisfies these: bounded waits give up and say so
         with pytest.raises(B.IshmemError) as e:
-            B.ishmem_uint64_wait_until_any(1, iv.addr, 8, B.ISHMEM_CMP_NE, 0, idx)
+            B.ishmem_uint64_wait_until_any(1, iv.addr, 8, None, B.ISHMEM_CMP_NE, 0, idx)
         assert e.value.code == B.ISHMEM_ERR_TIMEOUT
         assert s.status() == B.ISHMEM_ERR_TIMEOUT
-        B.ishmem_uint64_wait_until_all(0, iv.addr, 8, B.ISHMEM_CMP_NE, 0)
+        B.ishmem_uint64_wait_until_all(0, iv.addr, 8, None, B.ISHMEM_CMP_NE, 0)
         assert s.status() == B.ISHMEM_ERR_TIMEOUT
         with pytest.raises(B.IshmemError):
-            B.ishmem_uint64_wait_until_all(0, iv.addr, 257, B.ISHMEM_CMP_NE, 0)
+            B.ishmem_uint64_wait_until_all(0, iv.addr, 257, None, B.ISHMEM_CMP_NE, 0)
