@@ -214,3 +214,46 @@ def test_config5_jacobi_16384_200_iterations_sampled_cells():
             r = ci - firsts[p] + 1
             got = fin.gpu(p)[(r * n + cj) * 8:(r * n + cj + 1) * 8].cpu().numpy().view(np.float64)[0]
             assert np.float64(got).tobytes() == np.float64(exp).tobytes(), (ci, cj, got, exp)
+
+
+def test_large_alltoall_collect_and_narrow_reduce():
+    """Sizes that take the large-message launch shapes: alltoall of 8 MiB blocks and collect of
+    up to 24 MiB per member on 8 PEs (whole output checked on the device), uint8 sum / xor of
+    64 Mi elements through the TMA fold ring (all PEs identical + oracle windows)."""
+    npes, nblk = 8, 8 * MiB
+    rng = np.random.default_rng(11)
+    with Session(npes, 2 * npes * nblk + 4 * MiB, with_oracle=False) as s:
+        src, dst = s.malloc(npes * nblk), s.malloc(npes * nblk)
+        fill_full(src, "u8", inputs.SEED_C3, npes * nblk, npes)
+        B.ishmem_alltoallmem(B.ISHMEM_TEAM_WORLD, dst.addr, src.addr, nblk)
+        s.sync()
+        for q in range(npes):
+            for i in range(npes):
+                assert torch.equal(dst.gpu(q)[i * nblk:(i + 1) * nblk], src.gpu(i)[q * nblk:(q + 1) * nblk]), (q, i)
+        sizes = [(3 * MiB * (i % 4)) + 4096 * i + (i % 3) for i in range(npes)]          # 0 .. ~9 MiB, ragged
+        sizes[5] = 24 * MiB + 5
+        assert sum(sizes) <= npes * nblk
+        B.ishmem_collectmem(B.ISHMEM_TEAM_WORLD, dst.addr, src.addr, np.array(sizes, dtype=np.uint64))
+        s.sync()
+        at = 0
+        for i in range(npes):
+            for q in (0, 3, 7):
+                assert torch.equal(dst.gpu(q)[at:at + sizes[i]], src.gpu(i)[:sizes[i]]), (q, i)
+            at += sizes[i]
+        # narrow-type reduce at a size that uses the shared-memory fold ring
+        n = 64 * MiB
+        o = orc.Oracle(npes, 1 << 14)
+        try:
+            for lop, oop in ((B.ISHMEM_OP_SUM, orc.R_SUM), (B.ISHMEM_OP_XOR, orc.R_XOR), (B.ISHMEM_OP_MAX, orc.R_MAX)):
+                B.ishmemx_reduce(B.ISHMEM_TEAM_WORLD, dst.addr, src.addr, n, lop, B.ISHMEM_T_UINT8, B.ISHMEMX_REDUCE_AUTO)
+                s.sync()
+                for q in range(1, npes):
+                    assert torch.equal(dst.gpu(q)[:n], dst.gpu(0)[:n]), (lop, q)
+                for off in windows(n, 4096, rng, extra=[n // 2, n // 8 * 3]):
+                    for p in range(npes):
+                        o.view(0, 4096, p)[:] = inputs.block_values("u8", inputs.SEED_C3, p, off, 4096)
+                    o.reduce(o.world, 8192, 0, 4096, oop, orc.T_UINT8)
+                    assert np.array_equal(dst.gpu(5)[off:off + 4096].cpu().numpy(), o.view(8192, 4096, 5)), (lop, off)
+        finally:
+            o.close()
+        assert s.status() == 0
