@@ -86,6 +86,7 @@ __global__ void __launch_bounds__(1024) k_collect(const ishmem_ctx_t *ctxs, coll
 /* ---- alltoall: member i's blocks store block q of its source into block i of member q's dest ---- */
 __global__ void __launch_bounds__(1024) k_alltoall(const ishmem_ctx_t *ctxs, coll_args a)
 {
+    extern __shared__ __align__(128) unsigned char dyn_smem[];
     __shared__ long long delta[ISHMEM_MAX_PES];
     const ishmemi_team t = ctxs[0].teams[a.team];
     const unsigned me = blockIdx.x % (unsigned)t.size, g = blockIdx.x / (unsigned)t.size;
@@ -99,7 +100,14 @@ __global__ void __launch_bounds__(1024) k_alltoall(const ishmem_ctx_t *ctxs, col
     for (size_t k = g; k < total; k += (size_t)a.groups) {
         const size_t q = k % (size_t)t.size, o = (k / (size_t)t.size) * tile;
         const size_t len = a.n - o < tile ? a.n - o : tile;
-        ishmemi::copy_bytes(dest + delta[q] + o, src + q * a.n + o, len, threadIdx.x, blockDim.x);
+        if (a.staging_bytes) {
+            /* large blocks: every tile streams through the TMA ring of this block */
+            ishmemx_staging_t st = {dyn_smem, a.staging_bytes};
+            if (ishmemi::wg_copy(ctx, dest + delta[q] + o, src + q * a.n + o, len, st, true)) return;
+            __syncthreads(); /* the ring's shared memory is reused by the next tile */
+        } else {
+            ishmemi::copy_bytes(dest + delta[q] + o, src + q * a.n + o, len, threadIdx.x, blockDim.x);
+        }
     }
 }
 
@@ -531,7 +539,24 @@ extern "C" int ishmem_alltoallmem(ishmem_team_t team, void *dest, const void *sr
         size_t want = ((nbytes + tile - 1) / tile) * t.size;
         a.push_tile = (unsigned)tile;
         a.groups = g.coll_groups > 0 ? g.coll_groups : (int)(want < cap ? (want < 1 ? 1 : want) : cap);
-        k_alltoall<<<a.groups * t.size, all <= 65536 ? 256 : g.coll_threads, 0, s>>>(g.d_ctx, a);
+        int threads = all <= 65536 ? 256 : g.coll_threads;
+        /* from 1 MiB of loads plus stores per SM on: one block per SM, 512 KiB tiles through the
+         * TMA ring (the same copy routine as the work-group put) */
+        static unsigned smem = 0;
+        if (g.coll_groups == 0 && 2 * all * (size_t)t.size >= ((size_t)g.sm_count << 20)) {
+            unsigned want_smem = 192 * 1024 + 128;
+            if (want_smem > g.max_dyn_smem) want_smem = (unsigned)g.max_dyn_smem;
+            if (smem == want_smem ||
+                cudaFuncSetAttribute(k_alltoall, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)want_smem) == cudaSuccess) {
+                smem = want_smem;
+                a.staging_bytes = want_smem;
+                a.push_tile = 512u << 10;
+                size_t per_sm = (size_t)g.sm_count / t.size;
+                a.groups = (int)(per_sm < 1 ? 1 : per_sm);
+                threads = 128;
+            }
+        }
+        k_alltoall<<<a.groups * t.size, threads, a.staging_bytes, s>>>(g.d_ctx, a);
         ishmemi_count_launch();
         rc = ishmemi_check_launch("k_alltoall");
     }

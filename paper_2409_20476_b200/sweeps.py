@@ -372,6 +372,10 @@ def sweep_c3(args, out):
                             l2="hot", iters=it, us_per_op=us, alg_bytes=nb)
         B.ishmemx_set_cutover(1, B.SIZE_MAX)
         B.ishmemx_set_cutover(2, B.SIZE_MAX)
+        for n in [4 ** k for k in range(1, 13) if 4 ** k * P <= 8 * max_el]:
+            us, it = T(lambda i: B.ishmem_alltoallmem(team, dst, src, n))
+            out.add(config=3, op="alltoall", pattern="team", variant="stores", npes=P, dtype="u8", nbytes=n, l2="hot",
+                    iters=it, us_per_op=us, alg_bytes=2 * P * P * n, note="nbytes = one block; P*P blocks move")
         # device-resident forms: one work-group per PE, push sync inside the kernel, `rep` calls per launch
         rep = 50
         for threads in (128, 256, 1024):
@@ -601,6 +605,10 @@ def summarize(path) -> str:
                 c = _crossover(a, b)
                 out.append(f"- {op}, {P} PEs: engine at least as fast from " + (_fmt_size(c) if c else "never"))
             out.append("")
+        sel = [r for r in rows if r["op"] == "alltoall"]
+        if sel:
+            out += ["### alltoall (block size per pair; P x P blocks move): GB/s (algorithmic 2 P^2 n) / microseconds", "",
+                    _table(sel, nb, lambda r: f"P={r['npes']}", lambda r: f"{gb(r)} / {us(r)}", _fmt_size), ""]
         sel = [r for r in rows if r["variant"] == "device_resident" and r["npes"] in ("2", "12") and r["threads"] in ("128", "1024")]
         out += ["### device-resident forms (one work-group per PE, in-kernel push sync): microseconds", "",
                 _table(sel, nb, lambda r: f"{r['op']} P={r['npes']} T={r['threads']}", us, _fmt_size), ""]
