@@ -332,6 +332,13 @@ int ishmem_sync_all(void);
 int ishmem_barrier_all(void);
 /* Strided sub-team of a parent team; returns the new team or ISHMEM_TEAM_INVALID. */
 ishmem_team_t ishmem_team_split_strided(ishmem_team_t parent, int start, int stride, int size);
+/* 2-D split (OpenSHMEM 1.5 team_split_2d): the parent's members are laid out row-major with
+ * `xrange` columns; *xaxis_team receives the team of parent member `parent_index`'s row (stride 1)
+ * and *yaxis_team that of its column (stride xrange).  Each call creates two new teams (destroy
+ * them with ishmem_team_destroy).  ISHMEM_ERR_ARG when an argument is invalid or the team table
+ * is full (in which case nothing is created). */
+int ishmem_team_split_2d(ishmem_team_t parent, int xrange, int parent_index, ishmem_team_t *xaxis_team,
+                         ishmem_team_t *yaxis_team);
 int ishmem_team_destroy(ishmem_team_t team);
 int ishmem_team_n_pes(ishmem_team_t team);
 /* Index of world PE `pe` inside `team`, or -1 when it is not a member (OpenSHMEM's team_my_pe, with
@@ -469,7 +476,9 @@ int ishmemx_set_collective_geometry(int groups_per_pe, int threads);
  * the device routine ishmemx_{broadcastmem,fcollectmem,reduce,sync_all}_work_group of
  * ishmem_device.cuh, with in-kernel push synchronisation (for tests and latency
  * measurements of the device API itself).  which: 0 broadcast, 1 fcollect, 2 reduce
- * (op/dtype as above), 3 sync_all, 4 alltoall; the call is repeated `repeat` times. */
+ * (op/dtype as above), 3 sync_all, 4 alltoall, 5 collect with the sizes exchanged inside the
+ * kernel (member i contributes n * ((i mod 3) + 1) / 3 bytes); the call is repeated `repeat`
+ * times. */
 int ishmemx_collective_on_device(int which, ishmem_team_t team, void *dest, const void *src,
                                  size_t n, int root, int op, int dtype, int threads, int repeat);
 

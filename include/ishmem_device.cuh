@@ -84,6 +84,7 @@ struct ishmem_ctx_t {
      * the other members, sync_epoch[team] counts the syncs this PE has begun */
     unsigned long long *sync_arrive;
     unsigned long long *sync_epoch;
+    unsigned long long *collect_sizes; /* [ISHMEM_MAX_PES]: contributions announced by the members of a collect */
     long long internal_stride; /* bytes between consecutive PEs' internal regions */
     ishmemi_team teams[ISHMEM_MAX_TEAMS];
     int *status;                       /* one word shared by all PEs; first error wins */
@@ -1632,6 +1633,47 @@ __device__ __forceinline__ int ishmemx_fcollectmem_work_group(const ishmem_ctx_t
                             nbytes, ishmemi::block_tid(), ishmemi::block_nthr());
     int rc = ishmemx_team_sync_work_group(ctx, team);
     return ok ? rc : ISHMEM_ERR_INVALID_PE;
+}
+
+/* collect: every member contributes `my_nbytes` bytes (they may differ); every member's dest ends
+ * up with the concatenation in team order.  The sizes are exchanged first -- each member stores
+ * its size into a slot of every member's internal region and the team synchronises -- then every
+ * member pushes its source to its offset in every dest, and a second synchronisation completes
+ * the call.  *total (may be nullptr) receives the gathered size. */
+__device__ __forceinline__ int ishmemx_collectmem_work_group(const ishmem_ctx_t *ctx, ishmem_team_t team, void *dest,
+                                                             const void *src, size_t my_nbytes, size_t *total = nullptr)
+{
+    __shared__ long long delta[ISHMEM_MAX_PES];
+    __shared__ unsigned long long my_offset, all_bytes;
+    const ishmemi_team t = ctx->teams[team];
+    const int me = ishmemi::team_index(t, ctx->my_pe);
+    const bool ok = ishmemi::team_deltas(ctx, t, delta) && me >= 0;
+    const unsigned tid = ishmemi::block_tid(), nthr = ishmemi::block_nthr();
+    if (ok)
+        for (unsigned i = tid; i < (unsigned)t.size; i += nthr) {
+            const int pe = t.start + (int)i * t.stride;
+            unsigned long long *slot = (unsigned long long *)((char *)(ctx->collect_sizes + me) +
+                                                              (long long)(pe - ctx->my_pe) * ctx->internal_stride);
+            ishmemi::st_relaxed(slot, (unsigned long long)my_nbytes);
+        }
+    int rc = ishmemx_team_sync_work_group(ctx, team); /* release/acquire: all sizes have arrived */
+    if (ok && rc == 0) {
+        if (tid == 0) {
+            unsigned long long off = 0, sum = 0;
+            for (int i = 0; i < t.size; ++i) {
+                const unsigned long long n = ishmemi::ld_relaxed(ctx->collect_sizes + i);
+                if (i < me) off += n;
+                sum += n;
+            }
+            my_offset = off;
+            all_bytes = sum;
+        }
+        __syncthreads();
+        ishmemi::push_bytes((char *)dest + my_offset, delta, t.size, -1, (const char *)src, my_nbytes, tid, nthr);
+        if (total) *total = (size_t)all_bytes;
+    }
+    int rc2 = ishmemx_team_sync_work_group(ctx, team);
+    return !ok ? ISHMEM_ERR_INVALID_PE : (rc ? rc : rc2);
 }
 
 /* alltoall: every member stores block q of its source into block `my index` of member q's dest

@@ -139,6 +139,7 @@ def _signatures() -> dict[str, tuple[str, list[str]]]:
         "ishmem_sync_all": ("status", []),
         "ishmem_barrier_all": ("status", []),
         "ishmem_team_split_strided": ("int", ["i", "i", "i", "i"]),
+        "ishmem_team_split_2d": ("status", ["i", "i", "i", "p", "p"]),
         "ishmem_team_destroy": ("status", ["i"]),
         "ishmem_team_n_pes": ("int", ["i"]),
         "ishmem_team_my_pe": ("int", ["i", "i"]),

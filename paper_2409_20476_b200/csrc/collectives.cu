@@ -211,7 +211,8 @@ static size_t dtype_size(int dtype)
 }
 
 /* ---- device-resident forms: one work-group per member, in-kernel push sync ---------------- */
-/* WHICH: 0 broadcast, 1 fcollect, 2 reduce<T, OP>, 3 sync, 4 alltoall */
+/* WHICH: 0 broadcast, 1 fcollect, 2 reduce<T, OP>, 3 sync, 4 alltoall, 5 collect (member i of the
+ * team contributes n * ((i mod 3) + 1) / 3 bytes: a fixed ragged pattern for tests) */
 template <int WHICH, typename T, int OP>
 __global__ void __launch_bounds__(1024) k_collective_on_device(const ishmem_ctx_t *ctxs, coll_args a)
 {
@@ -225,6 +226,7 @@ __global__ void __launch_bounds__(1024) k_collective_on_device(const ishmem_ctx_
         else if (WHICH == 1) rc = ishmemx_fcollectmem_work_group(ctx, a.team, d, s, a.n);
         else if (WHICH == 2) rc = ishmemx_reduce_work_group<T, OP>(ctx, a.team, (T *)d, (const T *)s, a.n);
         else if (WHICH == 4) rc = ishmemx_alltoallmem_work_group(ctx, a.team, d, s, a.n);
+        else if (WHICH == 5) rc = ishmemx_collectmem_work_group(ctx, a.team, d, s, a.n * (size_t)(blockIdx.x % 3 + 1) / 3);
         else rc = ishmemx_team_sync_work_group(ctx, a.team);
         if (rc) return; /* the error is latched; every member gives up the same way */
     }
@@ -257,6 +259,7 @@ static reduce_kernel_t pick_dev(int which, int op, int dtype)
     if (which == 1) return k_collective_on_device<1, int, 0>;
     if (which == 3) return k_collective_on_device<3, int, 0>;
     if (which == 4) return k_collective_on_device<4, int, 0>;
+    if (which == 5) return k_collective_on_device<5, int, 0>;
     switch (dtype) {
     case ISHMEM_T_INT32: return pick_dev_int<int>(op);
     case ISHMEM_T_INT64: return pick_dev_int<long long>(op);
@@ -732,7 +735,7 @@ extern "C" int ishmemx_collective_on_device(int which, ishmem_team_t team, void 
     ishmemi_team t;
     int rc = team_of(team, &t);
     if (rc) return rc;
-    if (which < 0 || which > 4 || threads < 32 || threads > 1024 || repeat < 1) return ISHMEM_ERR_ARG;
+    if (which < 0 || which > 5 || threads < 32 || threads > 1024 || repeat < 1) return ISHMEM_ERR_ARG;
     if (which != 3) {
         size_t es = 1;
         if (which == 2) {
@@ -742,7 +745,7 @@ extern "C" int ishmemx_collective_on_device(int which, ishmem_team_t team, void 
         }
         if (which == 0 && (root < 0 || root >= t.size)) return ISHMEM_ERR_INVALID_PE;
         if (n > (size_t)-1 / (es * t.size)) return ISHMEM_ERR_ARG;
-        size_t sbytes = (which == 4 ? n * t.size : n * es), dbytes = (which == 1 || which == 4) ? n * es * t.size : sbytes;
+        size_t sbytes = (which == 4 ? n * t.size : n * es), dbytes = (which == 1 || which == 4 || which == 5) ? n * es * t.size : sbytes;
         if ((rc = check_sym2(dest, dbytes, src, sbytes))) return rc;
         const char *d = (const char *)dest, *sp = (const char *)src;
         if (d < sp + sbytes && sp < d + dbytes) return ISHMEM_ERR_ARG;

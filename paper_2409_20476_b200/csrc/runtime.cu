@@ -194,6 +194,7 @@ static int init_common(int npes, size_t heap_bytes, void *external)
         char *mine = g.d_internal + (size_t)p * ISHMEMI_INTERNAL_BYTES;
         c.sync_arrive = (unsigned long long *)mine;
         c.sync_epoch = (unsigned long long *)(mine + 8 * ISHMEM_MAX_TEAMS);
+        c.collect_sizes = (unsigned long long *)(mine + 16 * ISHMEM_MAX_TEAMS);
         c.internal_stride = ISHMEMI_INTERNAL_BYTES;
         c.status = g.d_status;
     }
@@ -487,6 +488,31 @@ extern "C" ishmem_team_t ishmem_team_split_strided(ishmem_team_t parent, int sta
             return t;
         }
     return ISHMEM_TEAM_INVALID;
+}
+
+extern "C" int ishmem_team_split_2d(ishmem_team_t parent, int xrange, int parent_index, ishmem_team_t *xaxis_team,
+                                    ishmem_team_t *yaxis_team)
+{
+    auto &g = g_ishmem;
+    ISHMEMI_REQUIRE_INIT();
+    if (parent < 0 || parent >= ISHMEM_MAX_TEAMS || !g.teams[parent].valid || !xaxis_team || !yaxis_team)
+        return ISHMEM_ERR_ARG;
+    const int size = g.teams[parent].size;
+    if (xrange < 1 || parent_index < 0 || parent_index >= size) return ISHMEM_ERR_ARG;
+    if (xrange > size) xrange = size;
+    const int x = parent_index % xrange, y = parent_index / xrange;
+    const int row_size = (size - y * xrange) < xrange ? size - y * xrange : xrange;
+    const int col_size = (size - x + xrange - 1) / xrange;
+    ishmem_team_t tx = ishmem_team_split_strided(parent, y * xrange, 1, row_size);
+    if (tx == ISHMEM_TEAM_INVALID) return ISHMEM_ERR_ARG;
+    ishmem_team_t ty = ishmem_team_split_strided(parent, x, xrange, col_size);
+    if (ty == ISHMEM_TEAM_INVALID) {
+        ishmem_team_destroy(tx);
+        return ISHMEM_ERR_ARG;
+    }
+    *xaxis_team = tx;
+    *yaxis_team = ty;
+    return ISHMEM_OK;
 }
 
 extern "C" int ishmem_team_destroy(ishmem_team_t team)

@@ -82,6 +82,11 @@ def test_collect_and_alltoall_12_pes():
         B.ishmemx_collective_on_device(4, B.ISHMEM_TEAM_WORLD, dst.addr, src.addr, 3001, 0, 0, 0, 256, 1)
         s.oracle.alltoallmem(s.oracle.world, dst.ooff, src.ooff, 3001)
         heaps_equal(s, "alltoall_work_group")
+        # collect with the sizes exchanged inside the kernel (member i gives n * ((i mod 3) + 1) / 3 bytes), twice
+        for n in (3000, 10):
+            B.ishmemx_collective_on_device(5, B.ISHMEM_TEAM_WORLD, dst.addr, src.addr, n, 0, 0, 0, 128, 2)
+            s.oracle.collectmem(s.oracle.world, dst.ooff, src.ooff, [n * (i % 3 + 1) // 3 for i in range(npes)])
+            heaps_equal(s, f"collect_work_group n={n}")
         with pytest.raises(B.IshmemError):
             B.ishmem_alltoallmem(B.ISHMEM_TEAM_WORLD, src.addr + 8, src.addr, 64)   # overlap
         # typed names (counts in elements)

@@ -130,3 +130,29 @@ def test_sizes_around_the_internal_thresholds(n):
         s.oracle.broadcastmem(s.oracle.world, dst.ooff, src.ooff, n, 1)
         heaps_equal(s, f"broadcast n={n}")
         assert s.status() == 0
+
+
+def test_two_dimensional_team_split():
+    """12 PEs as a 3 x 4 grid (xrange 4), and a ragged 5-column split of the same 12."""
+    npes = 12
+    with Session(npes, 1 << 18) as s:
+        src, dst = s.malloc(4096), s.malloc(16384)
+        for p in range(npes):
+            src.fill(p, inputs.byte_payload(inputs.SEED_C3, 600 + p, 4096))
+        tx, ty = np.zeros(1, np.int32), np.zeros(1, np.int32)
+        B.ishmem_team_split_2d(W, 4, 6, tx, ty)                 # PE 6 = (x 2, y 1)
+        assert [B.ishmem_team_my_pe(int(tx[0]), p) for p in range(npes)] == [-1] * 4 + [0, 1, 2, 3] + [-1] * 4
+        assert [B.ishmem_team_my_pe(int(ty[0]), p) for p in range(npes)] == [-1, -1, 0, -1, -1, -1, 1, -1, -1, -1, 2, -1]
+        B.ishmem_fcollectmem(int(tx[0]), dst.addr, src.addr, 1000)
+        s.oracle.fcollectmem((4, 1, 4), dst.ooff, src.ooff, 1000)
+        B.ishmemx_reduce(int(ty[0]), dst.addr + 8192, src.addr, 500, B.ISHMEM_OP_XOR, B.ISHMEM_T_UINT64, B.ISHMEMX_REDUCE_AUTO)
+        s.oracle.reduce((2, 4, 3), dst.ooff + 8192, src.ooff, 500, orc.R_XOR, orc.T_UINT64)
+        heaps_equal(s, "2-D teams")
+        B.ishmem_team_destroy(int(tx[0]))
+        B.ishmem_team_destroy(int(ty[0]))
+        B.ishmem_team_split_2d(W, 5, 11, tx, ty)                # ragged: rows 0-4, 5-9, 10-11; PE 11 = (x 1, y 2)
+        assert B.ishmem_team_n_pes(int(tx[0])) == 2 and B.ishmem_team_n_pes(int(ty[0])) == 3
+        assert B.ishmem_team_my_pe(int(tx[0]), 10) == 0 and B.ishmem_team_my_pe(int(ty[0]), 6) == 1
+        with pytest.raises(B.IshmemError):
+            B.ishmem_team_split_2d(W, 0, 0, tx, ty)
+        assert s.status() == 0
