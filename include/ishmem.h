@@ -233,7 +233,10 @@ int ishmemx_putmem_copy_engine(int my_pe, void *dest, const void *src, size_t nb
 int ishmemx_getmem_copy_engine(int my_pe, void *dest, const void *src, size_t nbytes, int pe);
 /* SPMD form: ONE launch on the team stream in which every PE p runs the same device call
  * with target (p + shift) mod npes -- shift 1 is the ring pattern, shifts 1..npes-1 in turn
- * the all-pairs pattern.  `groups` blocks per PE.  dest and src are symmetric. */
+ * the all-pairs pattern.  `groups` blocks per PE; groups == 0 lets the library size the grid so
+ * that every block gets one tile of threads x 128 bytes (blocks start in index order and sweep one
+ * short window of memory together: the fastest shape for large messages on B200, and what
+ * ishmem_putmem chooses by itself).  dest and src are symmetric. */
 int ishmemx_putmem_spmd(void *dest, const void *src, size_t nbytes, int shift, int level,
                         int threads, int groups);
 int ishmemx_getmem_spmd(void *dest, const void *src, size_t nbytes, int shift, int level,
@@ -539,7 +542,8 @@ int ishmemx_jacobi_noalloc(double *buf0, double *buf1, uint64_t *sig, size_t ny,
 
 /* Host-buffer convenience for end-to-end measurements: for every PE p, copy `nbytes` from HOST
  * `src_host` (per-PE stride `nbytes`) into src@p, let PE p put it to dest@((p + shift) mod npes)
- * (device call of the given level with `groups` work-groups of `threads` threads), and copy that
+ * (device call of the given level with `groups` work-groups of `threads` threads; groups == 0: one
+ * tile of threads x 128 bytes per work-group), and copy that
  * destination back to HOST `dest_host` (same layout).  Each PE's three steps run on its own
  * stream, so transfers in the two directions overlap between PEs; with pinned host memory the
  * copies are asynchronous.  Blocks the host until everything has arrived. */

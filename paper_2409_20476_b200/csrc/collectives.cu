@@ -286,47 +286,34 @@ static int team_of(ishmem_team_t team, ishmemi_team *out)
 }
 
 /* Launch shape of a push collective (broadcast: 1 pushing member; fcollect: `members`), each
- * pushing `bytes` to `ndst` destinations.
- *  - loads/stores (small and medium messages): tiles dealt round-robin to the blocks; the tile
- *    shrinks from 16 KiB down to 2 KiB so that a medium message still reaches every SM;
- *  - TMA push ring (one elected thread per block moves the data): only when every block of a
- *    full grid (one per SM) gets at least 1 MiB of loads plus stores. */
+ * pushing `bytes` to `ndst` destinations by loads and stores: one tile per block.  Blocks start in
+ * index order, so at any moment the running blocks cover one short contiguous window of the source
+ * and of every destination; on this GPU that order moves more bytes per second than a resident
+ * grid whose blocks each stream a long range of their own, by loads and stores or by the TMA ring
+ * (broadcast of 256 MiB to 12 PEs: 6.5 against 5.6 TB/s).  The tile is 8 KiB -- one 16-byte vector
+ * per thread of a 512-thread block, stored to every destination -- and shrinks down to 2 KiB so
+ * that a medium message still reaches every SM twice. */
 struct push_shape {
     int blocks_per_member, threads;
     unsigned staging, tile;
 };
-static push_shape push_geometry(size_t bytes, int members, int ndst, const void *kernel)
+static push_shape push_geometry(size_t bytes, int members, int ndst)
 {
     auto &g = g_ishmem;
     push_shape sh = {1, g.coll_threads, 0, 16384};
-    static unsigned smem = 0;
-    if (!smem) {
-        unsigned want = 192 * 1024 + 128;
-        if (want > g.max_dyn_smem) want = (unsigned)g.max_dyn_smem;
-        smem = want;
-    }
     if (g.coll_groups > 0) { /* caller-shaped */
         sh.blocks_per_member = g.coll_groups;
         return sh;
     }
-    const size_t work = bytes * (size_t)(1 + ndst) * (size_t)members;
-    size_t cap = (size_t)g.sm_count / members;
-    if (cap < 1) cap = 1;
-    if (work >= (size_t)g.sm_count << 20 &&
-        cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) == cudaSuccess) {
-        sh.staging = smem;
-        sh.threads = 128;
-        sh.blocks_per_member = (int)cap;
-        return sh;
-    }
-    /* loads/stores: aim at two blocks per SM, at least one tile each */
-    cap = ((size_t)g.sm_count * 2 + members - 1) / members;
-    size_t tile = (bytes / cap + 2047) & ~(size_t)2047;
+    const size_t aim = ((size_t)g.sm_count * 2 + members - 1) / members;
+    size_t tile = (bytes / aim + 2047) & ~(size_t)2047;
     if (tile < 2048) tile = 2048;
-    if (tile > 16384) tile = 16384;
+    if (tile > 8192) tile = 8192;
+    if (sh.threads > 512) sh.threads = 512;
     size_t want = (bytes + tile - 1) / tile;
+    const size_t most = (size_t)0x7fffffff / (size_t)members; /* grid limit */
     sh.tile = (unsigned)tile;
-    sh.blocks_per_member = (int)(want < 1 ? 1 : (want < cap * 2 ? want : cap * 2));
+    sh.blocks_per_member = (int)(want < 1 ? 1 : (want < most ? want : most));
     if (bytes <= 4096 * (size_t)ndst && sh.threads > 256) sh.threads = 256;
     return sh;
 }
@@ -415,7 +402,7 @@ extern "C" int ishmem_broadcastmem(ishmem_team_t team, void *dest, const void *s
         a.src = (const char *)src;
         a.n = nbytes;
         a.root = root;
-        const push_shape sh = push_geometry(nbytes, 1, t.size, (const void *)k_broadcast);
+        const push_shape sh = push_geometry(nbytes, 1, t.size);
         a.staging_bytes = sh.staging;
         a.push_tile = sh.tile;
         k_broadcast<<<sh.blocks_per_member, sh.threads, sh.staging, s>>>(g.d_ctx, a);
@@ -457,7 +444,7 @@ extern "C" int ishmem_fcollectmem(ishmem_team_t team, void *dest, const void *sr
         a.dest = (char *)dest;
         a.src = (const char *)src;
         a.n = nbytes;
-        const push_shape sh = push_geometry(nbytes, t.size, t.size, (const void *)k_fcollect);
+        const push_shape sh = push_geometry(nbytes, t.size, t.size);
         a.groups = sh.blocks_per_member;
         a.staging_bytes = sh.staging;
         a.push_tile = sh.tile;
@@ -496,16 +483,7 @@ extern "C" int ishmem_collectmem(ishmem_team_t team, void *dest, const void *src
         a.team = team;
         a.dest = (char *)dest;
         a.src = sp;
-        const bool shaped = g.coll_groups > 0;
-        push_shape sh = push_geometry(largest < ((size_t)1 << 20) ? largest : ((size_t)1 << 20) - 1, t.size, t.size,
-                                      (const void *)k_collect); /* loads/stores only: sizes differ per member */
-        if (!shaped && largest >= ((size_t)1 << 20)) {
-            size_t cap = ((size_t)g.sm_count * 4 + t.size - 1) / t.size, want = (largest + 16383) / 16384;
-            sh.blocks_per_member = (int)(want < cap ? want : cap);
-            sh.tile = 16384;
-            sh.staging = 0;
-            sh.threads = g.coll_threads;
-        }
+        const push_shape sh = push_geometry(largest, t.size, t.size); /* sized for the largest contribution */
         a.groups = sh.blocks_per_member;
         a.tile = sh.tile;
         k_collect<<<a.groups * t.size, sh.threads, 0, s>>>(g.d_ctx, a);
@@ -536,29 +514,16 @@ extern "C" int ishmem_alltoallmem(ishmem_team_t team, void *dest, const void *sr
         a.dest = (char *)dest;
         a.src = sp;
         a.n = nbytes;
-        size_t tile = 16384;
-        const size_t cap = ((size_t)g.sm_count * 4 + t.size - 1) / t.size;
-        while (tile > 2048 && (all + tile - 1) / tile < cap) tile >>= 1;
+        /* one (destination, tile) pair per block, the tile shrinking from 32 to 2 KiB while the
+         * grid would not fill every SM four times */
+        size_t tile = 32768;
+        const size_t aim = ((size_t)g.sm_count * 4 + t.size - 1) / t.size;
+        while (tile > 2048 && (all + tile - 1) / tile < aim) tile >>= 1;
         size_t want = ((nbytes + tile - 1) / tile) * t.size;
+        const size_t most = (size_t)0x7fffffff / (size_t)t.size;
         a.push_tile = (unsigned)tile;
-        a.groups = g.coll_groups > 0 ? g.coll_groups : (int)(want < cap ? (want < 1 ? 1 : want) : cap);
-        int threads = all <= 65536 ? 256 : g.coll_threads;
-        /* from 1 MiB of loads plus stores per SM on: one block per SM, 512 KiB tiles through the
-         * TMA ring (the same copy routine as the work-group put) */
-        static unsigned smem = 0;
-        if (g.coll_groups == 0 && 2 * all * (size_t)t.size >= ((size_t)g.sm_count << 20)) {
-            unsigned want_smem = 192 * 1024 + 128;
-            if (want_smem > g.max_dyn_smem) want_smem = (unsigned)g.max_dyn_smem;
-            if (smem == want_smem ||
-                cudaFuncSetAttribute(k_alltoall, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)want_smem) == cudaSuccess) {
-                smem = want_smem;
-                a.staging_bytes = want_smem;
-                a.push_tile = 512u << 10;
-                size_t per_sm = (size_t)g.sm_count / t.size;
-                a.groups = (int)(per_sm < 1 ? 1 : per_sm);
-                threads = 128;
-            }
-        }
+        a.groups = g.coll_groups > 0 ? g.coll_groups : (int)(want < 1 ? 1 : (want < most ? want : most));
+        const int threads = (all <= 65536 || g.coll_groups == 0) ? 256 : g.coll_threads;
         k_alltoall<<<a.groups * t.size, threads, a.staging_bytes, s>>>(g.d_ctx, a);
         ishmemi_count_launch();
         rc = ishmemi_check_launch("k_alltoall");
@@ -648,36 +613,31 @@ extern "C" int ishmemx_reduce(ishmem_team_t team, void *dest, const void *src, s
         a.n = nreduce;
         a.duplicated = (algorithm == ISHMEMX_REDUCE_DUPLICATED);
         const size_t per_member = a.duplicated ? bytes : bytes / t.size + 1;
-        /* loads/stores: tiles of threads x tile_vpt vectors dealt round-robin over all blocks.
-         * Small inputs take one vector per thread in 256-thread blocks, so that a few hundred
-         * KiB already occupy every SM; large ones 512 threads x 2 vectors, 4 blocks per SM. */
+        /* loads/stores, one tile of threads x tile_vpt vectors per block (blocks start in index
+         * order, so the running blocks sweep one contiguous window of every source and
+         * destination).  Small inputs take one vector per thread, so that a few hundred KiB
+         * already occupy every SM; large ones two. */
         int threads = g.coll_threads > 512 ? 512 : g.coll_threads;
         a.tile_vpt = 2;
         const size_t nvec = (bytes + 15) / 16;
         if (g.coll_groups > 0) {
             a.groups = g.coll_groups;
         } else {
-            size_t blocks;
-            if (nvec <= (size_t)g.sm_count * 2 * 256 * (a.duplicated ? t.size : 1)) {
-                threads = threads > 256 ? 256 : threads;
-                a.tile_vpt = 1;
-                blocks = (nvec + threads - 1) / threads;
-            } else {
-                blocks = (nvec + (size_t)threads * 2 - 1) / ((size_t)threads * 2);
-                if (blocks > (size_t)g.sm_count * 6) blocks = (size_t)g.sm_count * 6; /* measured: 6 > 4 by 5 % */
-            }
+            threads = threads > 128 ? 128 : threads;
+            if (nvec <= (size_t)g.sm_count * 4 * 128 * (a.duplicated ? t.size : 1)) a.tile_vpt = 1;
+            size_t blocks = (nvec + (size_t)threads * a.tile_vpt - 1) / ((size_t)threads * a.tile_vpt);
             /* the grid is groups x members blocks (in the duplicated form each member's `groups`
              * blocks sweep all tiles, so the tiles per block come out the same) */
             blocks = (blocks + t.size - 1) / t.size;
-            a.groups = (int)(blocks < 1 ? 1 : blocks);
+            const size_t most = (size_t)0x7fffffff / (size_t)t.size;
+            a.groups = (int)(blocks < 1 ? 1 : (blocks < most ? blocks : most));
         }
-        /* Loads/stores over round-robin tiles are the default; from 48 MiB per source on the TMA
-         * fold ring (one block per SM) is faster (12 PEs: 6.2 against 6.0 TB/s at 64 MiB per
-         * source, but 3.6 against 5.7 at 16 MiB).  ISHMEM_REDUCE_BULK=0/1 forces. */
+        /* ISHMEM_REDUCE_BULK=1 selects the TMA fold ring instead (one resident block per SM, three
+         * stages of P tiles in shared memory): 6.2 TB/s at 12 PEs x 256 MiB where the tiles above
+         * reach 6.5. */
         static const char *env_bulk = getenv("ISHMEM_REDUCE_BULK");
-        const bool use_bulk = env_bulk ? atoi(env_bulk) != 0 : (!a.duplicated && bytes >= ((size_t)48 << 20));
+        const bool use_bulk = env_bulk && atoi(env_bulk) != 0 && !a.duplicated;
         if (use_bulk && g.coll_groups == 0 && per_member >= (1u << 20) && t.size <= 48) {
-            /* large: TMA ring, one block per SM */
             unsigned want = 192 * 1024 + 128;
             if (want > g.max_dyn_smem) want = (unsigned)g.max_dyn_smem;
             if (cudaFuncSetAttribute((const void *)k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)want) ==
