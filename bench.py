@@ -207,10 +207,10 @@ def run_ours(args) -> dict:
         B.ishmem_float_sum_reduce(B.ISHMEM_TEAM_WORLD, dst, src, S["reduce_f32"])
         B.ishmem_int32_sum_reduce(B.ISHMEM_TEAM_WORLD, dst, src, S["reduce_i32"])
         for p in range(NPES):
-            B.ishmem_uint64_p(p, jsig, 0, p)
-            B.ishmem_uint64_p(p, jsig + 8, 0, p)
+            for w in range(4):
+                B.ishmem_uint64_p(p, jsig + 8 * w, 0, p)
         B.ishmemx_jacobi(jb0, jb1, jsig, S["jacobi_n"], S["jacobi_n"], S["jacobi_sweeps"], 1,
-                         args.jacobi_groups, 512, res)
+                         args.jacobi_groups, 0, res)
         B.ishmem_barrier_all()
 
     for _ in range(max(args.warmup, 3)):
@@ -516,7 +516,7 @@ def run_profile_jacobi(args) -> dict:
     heap_bytes = 2 * nbytes + MiB
     heap = torch.zeros(NPES * heap_bytes, dtype=torch.uint8, device="cuda")
     B.ishmemx_init_external(NPES, heap_bytes, heap.data_ptr())
-    b0, b1, sig = B.ishmem_malloc(nbytes), B.ishmem_malloc(nbytes), B.ishmem_calloc(2, 8)
+    b0, b1, sig = B.ishmem_malloc(nbytes), B.ishmem_malloc(nbytes), B.ishmem_calloc(4, 8)
     grid = inputs.jacobi_grid(inputs.SEED_C5, n, n)
     for p in range(NPES):
         o = p * heap_bytes + (b0 - heap.data_ptr()) + n * 8
@@ -532,7 +532,7 @@ def run_profile_jacobi(args) -> dict:
         torch.cuda.synchronize()
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         a.record(ts)
-        B.ishmemx_jacobi(b0, b1, sig, n, n, sweeps, 1, args.jacobi_groups, 512, res)
+        B.ishmemx_jacobi(b0, b1, sig, n, n, sweeps, 1, args.jacobi_groups, 0, res)
         b.record(ts)
         torch.cuda.synchronize()
         times.append(a.elapsed_time(b))

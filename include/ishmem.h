@@ -510,14 +510,21 @@ int ishmemx_rma_latency(int my_pe, void *dest, const void *src, size_t nbytes, i
 
 /* Overlap workload: `iters` sweeps of the 5-point Jacobi update on an ny x nx float64
  * grid cut into npes row strips (the first ny mod npes strips have one more row), in one
- * persistent co-resident launch: each sweep every PE sends its first and last rows to the
- * neighbours' halo rows with in-kernel work-group put_signal, updates its interior rows
- * meanwhile, waits for its own halos, then updates its edge rows.  buf0/buf1: symmetric,
- * (ceil(ny/npes)+2)*nx doubles each, strip row r at local row r+1 of buf0 on entry (buf1
- * is overwritten); sig: symmetric, 2 words, zero on entry.  overlap = 0 disables the
- * interior-first ordering (exchange, wait, then compute).  The final strips are in buf0
- * if iters is even, else buf1.  residual_sq_host (HOST, may be NULL) receives
- * ||u_iters - u_(iters-1)||_2^2 over the interior.  Blocks the host. */
+ * persistent co-resident launch of npes x groups_per_pe blocks: each sweep every PE sends its
+ * first and last rows to the neighbours' halo rows with in-kernel work-group put_signal, updates
+ * its interior rows meanwhile, waits for its own halos, then updates its edge rows.  buf0/buf1:
+ * symmetric, (ceil(ny/npes)+2)*nx doubles each, strip row r at local row r+1 of buf0 on entry
+ * (buf1 is overwritten); sig: symmetric, 4 words, zero on entry.  overlap = 0 disables the
+ * interior-first ordering (exchange, wait, then compute).
+ * threads: threads per block (a multiple of 32 up to 1024) -- the blocks of a PE then take
+ * bands of rows, and one of them sends each halo row -- or 0: the library shapes the blocks; they
+ * then take ranges of 60-column tiles, one warp per tile, every block sends its columns of the
+ * halo rows, and the warps of a PE move down the strip together (a few per cent faster).
+ * groups_per_pe is clamped to the rows (tiles) of the shortest strip.  The environment variable
+ * ISHMEM_JACOBI_SPLIT=rows|columns forces one of the two forms.
+ * The final strips are in buf0 if iters is even, else buf1.  residual_sq_host (HOST, may be
+ * NULL) receives ||u_iters - u_(iters-1)||_2^2 over the interior.  Blocks the host.
+ * ISHMEM_ERR_NOT_CORESIDENT when the blocks cannot all be resident at once. */
 int ishmemx_jacobi(double *buf0, double *buf1, uint64_t *sig, size_t ny, size_t nx, int iters,
                    int overlap, int groups_per_pe, int threads, double *residual_sq_host);
 

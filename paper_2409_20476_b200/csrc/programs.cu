@@ -271,6 +271,7 @@ struct jacobi_args {
     unsigned long long *done;     /* scratch [npes*groups]: sweeps completed by each block */
     double *partial;              /* scratch [npes*groups]: residual partial sums */
     int sliding;                  /* even nx: interior rows by the register sliding window */
+    int colsplit;                 /* the blocks of a PE split the strip by columns (else by rows) */
 };
 
 __device__ __forceinline__ void strip_of(size_t ny, int npes, int pe, size_t *first, size_t *rows)
@@ -283,15 +284,17 @@ __device__ __forceinline__ void strip_of(size_t ny, int npes, int pe, size_t *fi
 /* One local row r of the strip: nxt[r] = sweep(cur[r-1..r+1]); boundary cells are copied.
  * Adds the squared update to *acc when want_res. */
 __device__ __forceinline__ void jacobi_row(const double *cur, double *nxt, size_t r, size_t nx, bool fixed_row,
-                                           unsigned tid, unsigned nthr, bool want_res, double *acc)
+                                           unsigned tid, unsigned nthr, bool want_res, double *acc, size_t c_lo = 0,
+                                           size_t c_hi = ~(size_t)0)
 {
     const double *up = cur + (r - 1) * nx, *mid = cur + r * nx, *dn = cur + (r + 1) * nx;
     double *out = nxt + r * nx;
+    if (c_hi > nx) c_hi = nx;
     if (fixed_row) {
-        for (size_t j = tid; j < nx; j += nthr) out[j] = mid[j];
+        for (size_t j = c_lo + tid; j < c_hi; j += nthr) out[j] = mid[j];
         return;
     }
-    if ((nx & 1) == 0) {
+    if ((nx & 1) == 0 && c_lo == 0 && c_hi == nx) {
         const size_t half = nx >> 1;
         for (size_t c = tid; c < half; c += nthr) {
             const size_t j = c << 1;
@@ -312,7 +315,7 @@ __device__ __forceinline__ void jacobi_row(const double *cur, double *nxt, size_
         }
         return;
     }
-    for (size_t j = tid; j < nx; j += nthr) {
+    for (size_t j = c_lo + tid; j < c_hi; j += nthr) {
         double v = mid[j];
         if (j > 0 && j + 1 < nx) v = 0.25 * ((up[j] + dn[j]) + (mid[j - 1] + mid[j + 1]));
         out[j] = v;
@@ -337,16 +340,16 @@ __device__ __forceinline__ void jacobi_row(const double *cur, double *nxt, size_
  * grid's first and last row (kept as they are), or ~0u when they lie outside this strip.
  * Returns this thread's share of the squared update when want_res. */
 template <int DEPTH>
-static __device__ __noinline__ double jacobi_march(const double *cur, double *nxt, unsigned ra, unsigned rb,
-                                                   unsigned fixed0, unsigned fixed1, unsigned nx, bool want_res)
+__device__ __forceinline__ double jacobi_march_tiles(const double *cur, double *nxt, unsigned ra, unsigned rb,
+                                                     unsigned fixed0, unsigned fixed1, unsigned nx, bool want_res,
+                                                     unsigned t_lo, unsigned t_hi)
 {
     double acc = 0.0;
     if (rb <= ra) return acc;
     const unsigned lane = threadIdx.x & 31u, nwarps = blockDim.x >> 5;
-    const unsigned ntiles = (nx + 59u) / 60u;
     const unsigned full = 0xffffffffu;
     const double2 zero = make_double2(0.0, 0.0);
-    for (unsigned t = threadIdx.x >> 5; t < ntiles; t += nwarps) {
+    for (unsigned t = t_lo + (threadIdx.x >> 5); t < t_hi; t += nwarps) {
         const int jl = (int)(t * 60u) - 2 + 2 * (int)lane; /* first column of this lane's pair */
         const bool ld_ok = jl >= 0 && jl < (int)nx;
         const bool st_ok = ld_ok && lane >= 1 && lane <= 30;
@@ -402,21 +405,37 @@ static __device__ __noinline__ double jacobi_march(const double *cur, double *nx
     return acc;
 }
 
+/* out of line, so that the window gets a register allocation of its own: all tiles of the rows
+ * (two values fewer to carry), or the tiles [t_lo, t_hi) */
+template <int DEPTH>
+static __device__ __noinline__ double jacobi_march(const double *cur, double *nxt, unsigned ra, unsigned rb,
+                                                   unsigned fixed0, unsigned fixed1, unsigned nx, bool want_res)
+{
+    return jacobi_march_tiles<DEPTH>(cur, nxt, ra, rb, fixed0, fixed1, nx, want_res, 0u, (nx + 59u) / 60u);
+}
+template <int DEPTH>
+static __device__ __noinline__ double jacobi_march_range(const double *cur, double *nxt, unsigned ra, unsigned rb,
+                                                         unsigned fixed0, unsigned fixed1, unsigned nx, bool want_res,
+                                                         unsigned t_lo, unsigned t_hi)
+{
+    return jacobi_march_tiles<DEPTH>(cur, nxt, ra, rb, fixed0, fixed1, nx, want_res, t_lo, t_hi);
+}
+
 /* The first and the last row of a block's range (local rows rA and rB; rB == ~0u: only rA), which
  * are computed after the neighbours' rows have arrived.  Same 60-column tiles and shuffles as
  * jacobi_march; the loads of U tiles x 2 rows x 3 source rows are all issued before the first
  * use, since there is nothing to slide along. */
 template <int U>
 __device__ __forceinline__ double jacobi_edge_rows(const double *cur, double *nxt, unsigned rA, unsigned rB,
-                                                   unsigned fixed0, unsigned fixed1, unsigned nx, bool want_res)
+                                                   unsigned fixed0, unsigned fixed1, unsigned nx, bool want_res,
+                                                   unsigned t_lo, unsigned ntiles)
 {
     double acc = 0.0;
     const unsigned lane = threadIdx.x & 31u, nwarps = blockDim.x >> 5;
-    const unsigned ntiles = (nx + 59u) / 60u;
     const unsigned full = 0xffffffffu;
     const double2 zero = make_double2(0.0, 0.0);
     const unsigned rows[2] = {rA, rB};
-    for (unsigned t0 = (threadIdx.x >> 5) * U; t0 < ntiles; t0 += nwarps * U) {
+    for (unsigned t0 = t_lo + (threadIdx.x >> 5) * U; t0 < ntiles; t0 += nwarps * U) {
         double2 up[U][2], mid[U][2], dn[U][2];
 #pragma unroll
         for (int k = 0; k < U; ++k) {
@@ -460,7 +479,18 @@ __device__ __forceinline__ double jacobi_edge_rows(const double *cur, double *nx
 }
 
 /* MAXT: largest block the instance may be launched with (it fixes the registers per thread);
- * DEPTH: rows in flight per lane in the sliding window */
+ * DEPTH: rows in flight per lane in the sliding window.
+ *
+ * The G blocks of a PE share its strip in one of two ways.
+ *  - by rows (colsplit = 0): block g takes a band of rows and walks every column tile of it;
+ *    it sends the strip's first / last row when it owns them, and before its band's two edge
+ *    rows it waits for the blocks above and below (or the neighbour PE's halo).
+ *  - by columns (colsplit = 1): block g takes a range of 60-column tiles and walks them down the
+ *    whole strip, one warp per tile when the block is large enough, so that the warps of a PE
+ *    advance together through one band of rows (a short contiguous window of memory, which this
+ *    GPU serves faster than many scattered streams).  Every block sends its columns of the first
+ *    and last row (the signal counts the pieces), and at the start of a sweep waits for the
+ *    blocks left and right of it, whose columns its outermost tiles overlap by two. */
 template <int MAXT, int DEPTH>
 __global__ void __launch_bounds__(MAXT) k_jacobi(const ishmem_ctx_t *ctxs, jacobi_args a)
 {
@@ -474,8 +504,14 @@ __global__ void __launch_bounds__(MAXT) k_jacobi(const ishmem_ctx_t *ctxs, jacob
     double *b[2] = {(double *)local_of(ctxs, ctx, a.buf0), (double *)local_of(ctxs, ctx, a.buf1)};
     unsigned long long *sig = (unsigned long long *)local_of(ctxs, ctx, a.sig);
     const size_t nx = a.nx;
-    /* this block's local rows [r0, r1) out of 1..rows */
-    const size_t r0 = 1 + rows * (size_t)g / (size_t)G, r1 = 1 + rows * (size_t)(g + 1) / (size_t)G;
+    const bool cols = a.colsplit != 0;
+    /* this block's local rows [r0, r1) out of 1..rows, and its tiles [t_lo, t_hi) of 60 columns */
+    const size_t r0 = cols ? 1 : 1 + rows * (size_t)g / (size_t)G;
+    const size_t r1 = cols ? rows + 1 : 1 + rows * (size_t)(g + 1) / (size_t)G;
+    const unsigned ntiles = (unsigned)((nx + 59) / 60);
+    const unsigned t_lo = cols ? (unsigned)((size_t)ntiles * (size_t)g / (size_t)G) : 0u;
+    const unsigned t_hi = cols ? (unsigned)((size_t)ntiles * (size_t)(g + 1) / (size_t)G) : ntiles;
+    const size_t c_lo = (size_t)t_lo * 60, c_hi = ((size_t)t_hi * 60 < nx) ? (size_t)t_hi * 60 : nx;
     unsigned long long *done = a.done + (size_t)p * G;
     double acc = 0.0;
     __shared__ int give_up;
@@ -484,53 +520,100 @@ __global__ void __launch_bounds__(MAXT) k_jacobi(const ishmem_ctx_t *ctxs, jacob
     /* local numbers of the grid's first and last row when they belong to this strip */
     const unsigned fixed0 = (first == 0) ? 1u : ~0u;
     const unsigned fixed1 = (first + rows == a.ny) ? (unsigned)rows : ~0u;
+    /* Halo signals.  By rows one block sends the whole row and SETs the word to the sweep number.
+     * By columns every block sends its piece and ADDs 1, and the words alternate with the parity
+     * of the sweep (sig[2], sig[3] for even sweeps): a PE can receive pieces of the next sweep
+     * while it still waits for one of this sweep -- never of the sweep after that, which needs
+     * this PE's own next halo -- so a word only ever counts sweeps up to the one waited for. */
     if (tid == 0) give_up = 0;
     __syncthreads();
+
+    /* rows [ra, rb) of this block's columns */
+    auto sweep_rows = [&](const double *cur, double *nxt, size_t ra, size_t rb, bool want_res) {
+        if (rb <= ra) return;
+        if (slide) {
+            acc += cols ? jacobi_march_range<DEPTH>(cur, nxt, (unsigned)ra, (unsigned)rb, fixed0, fixed1, (unsigned)nx,
+                                                    want_res, t_lo, t_hi)
+                        : jacobi_march<DEPTH>(cur, nxt, (unsigned)ra, (unsigned)rb, fixed0, fixed1, (unsigned)nx,
+                                              want_res);
+        } else {
+            for (size_t r = ra; r < rb; ++r) {
+                const size_t gi = first + r - 1;
+                jacobi_row(cur, nxt, r, nx, gi == 0 || gi == a.ny - 1, tid, nthr, want_res, &acc, c_lo, c_hi);
+            }
+        }
+    };
+    /* the two rows rA and rB (rB == ~0: only rA) of this block's columns */
+    auto two_rows = [&](const double *cur, double *nxt, size_t rA, size_t rB, bool want_res) {
+        if (slide) {
+            acc += jacobi_edge_rows<(MAXT <= 512) ? 2 : 1>(cur, nxt, (unsigned)rA, rB == ~(size_t)0 ? ~0u : (unsigned)rB,
+                                                           fixed0, fixed1, (unsigned)nx, want_res, t_lo, t_hi);
+        } else {
+            sweep_rows(cur, nxt, rA, rA + 1, want_res);
+            if (rB != ~(size_t)0) sweep_rows(cur, nxt, rB, rB + 1, want_res);
+        }
+    };
+    /* block `other` of this PE has finished sweep it - 1 */
+    auto wait_block = [&](int other, int it, ishmemi::deadline &dl) -> int {
+        while (ishmemi::ld_acquire(done + other) < (unsigned long long)it)
+            if (dl.expired()) return ISHMEM_ERR_TIMEOUT;
+        return 0;
+    };
 
     for (int it = 0; it < a.iters; ++it) {
         const double *cur = b[it & 1];
         double *nxt = b[(it + 1) & 1];
         const unsigned long long round = (unsigned long long)it + 1;
         const bool want_res = (it == a.iters - 1);
-        /* (a) halo rows of the current sweep go out first: my first row to the bottom halo of
-         * the PE above, my last row to the top halo of the PE below */
-        if (g == 0 && p > 0)
-            ishmemx_putmem_signal_work_group(ctx, (void *)(cur + (rows_above + 1) * nx), cur + nx, nx * 8,
-                                             sig + 1, round, ISHMEM_SIGNAL_SET, p - 1);
-        if (g == G - 1 && p + 1 < P)
-            ishmemx_putmem_signal_work_group(ctx, (void *)cur, cur + rows * nx, nx * 8, sig + 0, round,
-                                             ISHMEM_SIGNAL_SET, p + 1);
-        /* (b) rows that need nobody else's data of this sweep */
-        if (a.overlap) {
-            if (slide) {
-                if (r1 > r0 + 2)
-                    acc += jacobi_march<DEPTH>(cur, nxt, (unsigned)r0 + 1, (unsigned)r1 - 1, fixed0, fixed1, (unsigned)nx,
-                                           want_res);
-            } else {
-                for (size_t r = r0 + 1; r + 1 < r1; ++r) {
-                    const size_t gi = first + r - 1;
-                    jacobi_row(cur, nxt, r, nx, gi == 0 || gi == a.ny - 1, tid, nthr, want_res, &acc);
+        if (cols && G > 1) {
+            /* the blocks left and right have finished the previous sweep: their columns next to
+             * mine are current, and they no longer read the columns I am about to overwrite */
+            if (tid == 0) {
+                ishmemi::deadline dl(ctx->wait_limit_ns);
+                int rc = (g > 0) ? wait_block(g - 1, it, dl) : 0;
+                if (!rc && g < G - 1) rc = wait_block(g + 1, it, dl);
+                if (rc) {
+                    ishmemi::latch_error(ctx, rc);
+                    give_up = 1;
                 }
             }
+            __syncthreads();
+            if (give_up) break;
         }
+        /* (a) halo rows of the current sweep go out first: my first row to the bottom halo of
+         * the PE above, my last row to the top halo of the PE below */
+        unsigned long long *sig_top = sig + 0, *sig_bottom = sig + 1; /* halo from above / below arrived */
+        unsigned long long expect = round;
+        if (cols) {
+            sig_top += 2 * (it & 1);
+            sig_bottom += 2 * (it & 1);
+            expect = (unsigned long long)G * (unsigned long long)(it / 2 + 1);
+            if (p > 0)
+                ishmemx_putmem_signal_work_group(ctx, (void *)(cur + (rows_above + 1) * nx + c_lo), cur + nx + c_lo,
+                                                 (c_hi - c_lo) * 8, sig_bottom, 1, ISHMEM_SIGNAL_ADD, p - 1);
+            if (p + 1 < P)
+                ishmemx_putmem_signal_work_group(ctx, (void *)(cur + c_lo), cur + rows * nx + c_lo, (c_hi - c_lo) * 8,
+                                                 sig_top, 1, ISHMEM_SIGNAL_ADD, p + 1);
+        } else {
+            if (g == 0 && p > 0)
+                ishmemx_putmem_signal_work_group(ctx, (void *)(cur + (rows_above + 1) * nx), cur + nx, nx * 8, sig + 1,
+                                                 round, ISHMEM_SIGNAL_SET, p - 1);
+            if (g == G - 1 && p + 1 < P)
+                ishmemx_putmem_signal_work_group(ctx, (void *)cur, cur + rows * nx, nx * 8, sig + 0, round,
+                                                 ISHMEM_SIGNAL_SET, p + 1);
+        }
+        /* (b) rows that need nobody else's data of this sweep */
+        if (a.overlap && r1 > r0 + 2) sweep_rows(cur, nxt, r0 + 1, r1 - 1, want_res);
         /* (c) wait for the rows above and below this block's range: neighbouring blocks of
          * the same PE publish a sweep counter, neighbouring PEs signal their halo */
         if (tid == 0) {
             int rc = 0;
             ishmemi::deadline dl(ctx->wait_limit_ns);
-            if (g > 0) {
-                while (ishmemi::ld_acquire(done + g - 1) < (unsigned long long)it)
-                    if (dl.expired()) { rc = ISHMEM_ERR_TIMEOUT; break; }
-            } else if (p > 0) {
-                rc = ishmem_uint64_wait_until(ctx, sig + 0, ISHMEM_CMP_GE, round);
-            }
+            if (!cols && g > 0) rc = wait_block(g - 1, it, dl);
+            else if (p > 0) rc = ishmem_uint64_wait_until(ctx, sig_top, ISHMEM_CMP_GE, expect);
             if (!rc) {
-                if (g < G - 1) {
-                    while (ishmemi::ld_acquire(done + g + 1) < (unsigned long long)it)
-                        if (dl.expired()) { rc = ISHMEM_ERR_TIMEOUT; break; }
-                } else if (p + 1 < P) {
-                    rc = ishmem_uint64_wait_until(ctx, sig + 1, ISHMEM_CMP_GE, round);
-                }
+                if (!cols && g < G - 1) rc = wait_block(g + 1, it, dl);
+                else if (p + 1 < P) rc = ishmem_uint64_wait_until(ctx, sig_bottom, ISHMEM_CMP_GE, expect);
             }
             if (rc) {
                 ishmemi::latch_error(ctx, rc);
@@ -540,28 +623,8 @@ __global__ void __launch_bounds__(MAXT) k_jacobi(const ishmem_ctx_t *ctxs, jacob
         __syncthreads();
         if (give_up) break;
         /* (d) the remaining rows */
-        if (slide && !a.overlap) {
-            acc += jacobi_march<DEPTH>(cur, nxt, (unsigned)r0, (unsigned)r1, fixed0, fixed1, (unsigned)nx, want_res);
-        } else if (slide) {
-            if (r1 > r0)
-                acc += jacobi_edge_rows<(MAXT <= 512) ? 2 : 1>(cur, nxt, (unsigned)r0,
-                                                               (r1 - 1 > r0) ? (unsigned)r1 - 1 : ~0u, fixed0, fixed1,
-                                                               (unsigned)nx, want_res);
-        } else if (a.overlap) {
-            if (r1 > r0) {
-                size_t gi = first + r0 - 1;
-                jacobi_row(cur, nxt, r0, nx, gi == 0 || gi == a.ny - 1, tid, nthr, want_res, &acc);
-                if (r1 - 1 > r0) {
-                    gi = first + (r1 - 1) - 1;
-                    jacobi_row(cur, nxt, r1 - 1, nx, gi == 0 || gi == a.ny - 1, tid, nthr, want_res, &acc);
-                }
-            }
-        } else {
-            for (size_t r = r0; r < r1; ++r) {
-                const size_t gi = first + r - 1;
-                jacobi_row(cur, nxt, r, nx, gi == 0 || gi == a.ny - 1, tid, nthr, want_res, &acc);
-            }
-        }
+        if (!a.overlap) sweep_rows(cur, nxt, r0, r1, want_res);
+        else if (r1 > r0) two_rows(cur, nxt, r0, (r1 - 1 > r0) ? r1 - 1 : ~(size_t)0, want_res);
         /* (e) publish this sweep */
         __syncthreads();
         if (tid == 0) {
@@ -581,20 +644,33 @@ __global__ void __launch_bounds__(MAXT) k_jacobi(const ishmem_ctx_t *ctxs, jacob
     }
 }
 
+/* How the blocks of a PE share its strip: by columns when the library shapes the blocks itself
+ * (threads == 0: one warp per column tile), by rows when the caller gives the block size (any
+ * size then keeps all its warps busy).  ISHMEM_JACOBI_SPLIT=rows / columns overrides; read at
+ * every call. */
+static bool jacobi_by_columns(int threads)
+{
+    const char *env = getenv("ISHMEM_JACOBI_SPLIT");
+    if (env && !strcmp(env, "rows")) return false;
+    if (env && !strcmp(env, "columns")) return true;
+    return threads == 0;
+}
+
 /* argument checks shared by the two entry points; *groups_per_pe is clamped to the shortest strip */
 static int jacobi_check(double *buf0, double *buf1, uint64_t *sig, size_t ny, size_t nx, int iters,
                         int *groups_per_pe, int threads)
 {
     auto &g = g_ishmem;
     const int P = g.npes;
-    if (ny < 3 || nx < 3 || iters < 0 || (size_t)P > ny) return ISHMEM_ERR_ARG;
-    if (threads < 32 || threads > 1024 || threads % 32 || *groups_per_pe < 1) return ISHMEM_ERR_ARG;
+    if (ny < 3 || nx < 3 || nx > 0x7fffff00u || ny > 0x7fffff00u || iters < 0 || (size_t)P > ny) return ISHMEM_ERR_ARG;
+    if (threads < 0 || threads > 1024 || threads % 32 || *groups_per_pe < 1) return ISHMEM_ERR_ARG;
     const size_t rows_min = ny / P, rows_max = (ny + P - 1) / P;
-    if ((size_t)*groups_per_pe > rows_min) *groups_per_pe = (int)rows_min;
+    const size_t most = jacobi_by_columns(threads) ? (nx + 59) / 60 : rows_min; /* a tile or a row per block at least */
+    if ((size_t)*groups_per_pe > most) *groups_per_pe = (int)most;
     const size_t bytes = (rows_max + 2) * nx * 8;
     if ((uintptr_t)buf0 % 16 || (uintptr_t)buf1 % 16 || (uintptr_t)sig % 8) return ISHMEM_ERR_ALIGN;
     if (ishmemi_sym_offset(buf0, bytes) < 0 || ishmemi_sym_offset(buf1, bytes) < 0 ||
-        ishmemi_sym_offset(sig, 16) < 0)
+        ishmemi_sym_offset(sig, 32) < 0)
         return ISHMEM_ERR_NOT_SYMMETRIC;
     return ISHMEM_OK;
 }
@@ -622,15 +698,28 @@ static int jacobi_launch(double *buf0, double *buf1, uint64_t *sig, size_t ny, s
     a.groups = groups_per_pe;
     a.done = (unsigned long long *)scratch;
     a.partial = (double *)((char *)scratch + nblocks * 8);
-    a.sliding = (nx % 2 == 0 && nx < 0x7fffffffu && ny < 0x7fffffffu);
+    a.sliding = (nx % 2 == 0);
+    a.colsplit = jacobi_by_columns(threads);
+    if (threads == 0) {
+        /* by columns: one warp per tile when that fits a block, else the fewest equal rounds;
+         * by rows: 512 */
+        threads = 512;
+        if (a.colsplit) {
+            const size_t tiles = ((nx + 59) / 60 + groups_per_pe - 1) / groups_per_pe;
+            const size_t cap = nblocks <= (size_t)g.sm_count ? 23 : 16, rounds = (tiles + cap - 1) / cap;
+            threads = 32 * (int)((tiles + rounds - 1) / rounds);
+        }
+    }
     const ishmem_ctx_t *ctxs = g.d_ctx;
     void *params[] = {(void *)&ctxs, (void *)&a};
     if (!rc)
     {
         /* blocks of at most 512 threads that have an SM to themselves get 128 registers per thread
          * and a deeper window; everything else the 1024-thread instance */
-        const bool wide = threads <= 512 && nblocks <= (size_t)g.sm_count;
-        void *kernel = wide ? (void *)k_jacobi<512, 8> : (void *)k_jacobi<1024, 4>;
+        const bool alone = nblocks <= (size_t)g.sm_count;
+        void *kernel = (alone && threads <= 512) ? (void *)k_jacobi<512, 7>
+                       : (alone && threads <= 736) ? (void *)k_jacobi<736, 5>
+                                                   : (void *)k_jacobi<1024, 4>;
         rc = ishmemi_cuda(cudaLaunchCooperativeKernel(kernel, dim3((unsigned)nblocks), dim3(threads), params, 0, s),
                           "cudaLaunchCooperativeKernel(jacobi)");
     }

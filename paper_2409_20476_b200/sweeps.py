@@ -126,6 +126,8 @@ def sweep_c2(args, out):
     variants += [(f"work_group_256x{g}", WG, 256, g, big) for g in (4, 18, 37, 74)]
     variants += [(f"work_group_512x{g}", WG, 512, g, big) for g in (37, 74)]
     variants += [(f"work_group_bulk_256x{g}", BK, 256, g, big) for g in (1, 4, 18, 37)]
+    # groups = 0: the library sizes the grid, one tile of threads x 128 bytes per block
+    variants += [("work_group_tiled_256", WG, 256, 0, big)]
     # device-initiated copy engine: each work-group's leader posts its slice to the host proxy
     B.ishmemx_proxy_start()
     B.ishmemx_set_wait_limit_ns(200_000_000)      # a lost reply costs 0.2 s, not 2 s, and shows in the status
@@ -149,7 +151,7 @@ def sweep_c2(args, out):
                 us, it = timer(lambda i: spmd(dst, src, n, 1, level, threads, groups))
                 out.add(config=2, op=op, pattern="ring", variant=name, level=level, threads=threads, groups=groups,
                         npes=npes, dtype="u8", nbytes=n, l2="hot", iters=it, us_per_op=us, alg_bytes=2 * n * npes)
-                if groups >= 18 and n < big:
+                if (groups >= 18 or groups == 0) and n < big:
                     nsl, stride = slots(n)
                     us, it = T(lambda i: spmd(dst + (i % nsl) * stride, src + (i % nsl) * stride, n, 1, level,
                                               threads, groups))
@@ -168,8 +170,8 @@ def sweep_c2(args, out):
             out.add(config=2, op="put", pattern="ring", variant="copy_engine", npes=npes, dtype="u8", nbytes=n,
                     l2="cold", iters=it, us_per_op=us, alg_bytes=2 * n * npes)
     # all-pairs: 7 permutation rounds p -> (p+r) mod 8 per operation
-    for name, level, threads, groups in (("work_group_bulk_256x37", BK, 256, 37), ("work_group_512x74", WG, 512, 74),
-                                          ("copy_engine", None, 0, 0)):
+    for name, level, threads, groups in (("work_group_tiled_256", WG, 256, 0), ("work_group_bulk_256x37", BK, 256, 37),
+                                          ("work_group_512x74", WG, 512, 74), ("copy_engine", None, 0, 0)):
         for n in sizes:
             def rounds(i, n=n):
                 for r in range(1, npes):
@@ -468,7 +470,7 @@ def sweep_c5(args, out):
     nbytes = (rows_max + 2) * n * 8
     heap_bytes = 2 * nbytes + MiB
     heap, stream = _session(torch, B, npes, heap_bytes)
-    b0, b1, sig = B.ishmem_malloc(nbytes), B.ishmem_malloc(nbytes), B.ishmem_calloc(2, 8)
+    b0, b1, sig = B.ishmem_malloc(nbytes), B.ishmem_malloc(nbytes), B.ishmem_calloc(4, 8)
     base, extra = divmod(n, npes)
     res = np.zeros(1)
 
@@ -485,12 +487,12 @@ def sweep_c5(args, out):
     load()
     for overlap in (1, 0):
         for groups in (6, 12, 24):
-            for threads in (256, 512, 1024):
+            for threads in (0, 256, 512, 1024):       # 0: blocks shaped by the library, strip split by columns
                 if npes * groups * threads > 148 * 2048:
                     continue
                 for p in range(npes):
-                    B.ishmem_uint64_p(p, sig, 0, p)
-                    B.ishmem_uint64_p(p, sig + 8, 0, p)
+                    for w in range(4):
+                        B.ishmem_uint64_p(p, sig + 8 * w, 0, p)
                 a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                 torch.cuda.synchronize()
                 a.record(stream)
@@ -552,8 +554,8 @@ def summarize(path) -> str:
     if cfg == 2:
         ring = [r for r in rows if r["pattern"] == "ring" and r["op"] == "put"]
         keep = ["work_item", "sub_group", "work_group_16x1", "work_group_128x1", "work_group_1024x1",
-                "work_group_256x18", "work_group_512x74", "work_group_bulk_256x37", "work_group_engine_64x1",
-                "copy_engine"]
+                "work_group_256x18", "work_group_512x74", "work_group_bulk_256x37", "work_group_tiled_256",
+                "work_group_engine_64x1", "copy_engine"]
         for l2 in ("hot", "cold"):
             sel = [r for r in ring if r["l2"] == l2 and r["variant"] in keep]
             out += [f"### put, ring p -> (p+1) mod 8, 8 PEs concurrently, {l2} buffers: GB/s (algorithmic, aggregate)", "",
@@ -563,7 +565,7 @@ def summarize(path) -> str:
         out += ["### crossover: smallest message from which the copy engine is at least as fast at every larger size", ""]
         for var in ("work_item", "sub_group", "work_group_16x1", "work_group_128x1", "work_group_256x1", "work_group_1024x1",
                     "work_group_256x4", "work_group_256x18", "work_group_256x37", "work_group_512x74",
-                    "work_group_bulk_256x37"):
+                    "work_group_bulk_256x37", "work_group_tiled_256"):
             c = _crossover(t(var), t("copy_engine"))
             out.append(f"- `{var}` vs host-started copy engine (ring, 8 PEs): " + (_fmt_size(c) if c else "never"))
         c = _crossover(t("host_api_kernel", pat="one_pe"), t("host_api_copy_engine", pat="one_pe"))
@@ -580,7 +582,8 @@ def summarize(path) -> str:
         out += ["### all-pairs (mean of the 7 permutation rounds): GB/s", "",
                 _table(sel, nb, lambda r: r["variant"], gb, _fmt_size), ""]
         getr = [r for r in rows if r["pattern"] == "ring" and r["op"] == "get" and r["l2"] == "hot"
-                and r["variant"] in ("work_group_512x74", "work_group_bulk_256x37") and nb(r) >= 1 << 20]
+                and r["variant"] in ("work_group_512x74", "work_group_bulk_256x37", "work_group_tiled_256")
+                and nb(r) >= 1 << 20]
         out += ["### get, ring, hot buffers: GB/s", "", _table(getr, nb, lambda r: r["variant"], gb, _fmt_size), ""]
     elif cfg == 1:
         out += ["### 4 PEs x 16 MiB, int32: microseconds per operation", "",

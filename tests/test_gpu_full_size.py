@@ -198,7 +198,10 @@ def test_config5_jacobi_16384_200_iterations_sampled_cells():
             rows = firsts[p + 1] - firsts[p]
             b0.gpu(p)[n * 8:(rows + 1) * n * 8].copy_(torch.from_numpy(grid[firsts[p]:firsts[p + 1]].view(np.uint8).ravel()))
         s.sync()
-        B.ishmemx_jacobi(b0.addr, b1.addr, sig.addr, n, n, iters, 1, 12, 512, None)
+        for p in range(npes):
+            sig.fill(p, np.zeros(64, np.uint8))
+        s.sync()
+        B.ishmemx_jacobi(b0.addr, b1.addr, sig.addr, n, n, iters, 1, 12, 0, None)
         assert s.status() == 0
         rng = np.random.default_rng(10)
         cells = [(1, 1), (n - 2, n - 2), (1, n // 2), (n // 2, 1), (0, 5), (7, n - 1)]

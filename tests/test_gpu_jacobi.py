@@ -25,6 +25,7 @@ def run_gpu(grid, npes, iters, overlap, groups, threads):
             strip = np.zeros((rows_max + 2, nx))
             strip[1:rows + 1] = grid[first:first + rows]
             b0.fill(p, strip)
+            sig.fill(p, np.zeros(64, np.uint8))
             first += rows
         res = np.zeros(1)
         B.ishmemx_jacobi(b0.addr, b1.addr, sig.addr, ny, nx, iters, overlap, groups, threads, res)
@@ -39,18 +40,32 @@ def run_gpu(grid, npes, iters, overlap, groups, threads):
         return out, res[0]
 
 
+@pytest.mark.parametrize("split", ["columns", "rows"])
 @pytest.mark.parametrize("overlap", [1, 0])
 @pytest.mark.parametrize("ny,nx,npes,groups,threads", [
-    (64, 48, 12, 1, 128), (200, 130, 12, 3, 128), (257, 33, 5, 4, 128),       # odd nx: row-by-row path
+    (64, 48, 12, 1, 128), (200, 131, 12, 3, 128), (257, 33, 5, 4, 128),       # odd nx: row-by-row path
     (40, 40, 1, 2, 128), (1000, 512, 12, 8, 128), (301, 1234, 7, 3, 256),      # sliding window, 128 registers
-    (600, 256, 12, 13, 128), (300, 4096, 4, 2, 1024), (97, 62, 3, 5, 1024)])   # sliding window, 64 registers
-def test_jacobi_matches_oracle(ny, nx, npes, groups, threads, overlap):
+    (600, 256, 12, 13, 128), (300, 4096, 4, 2, 1024), (97, 62, 3, 5, 1024),    # sliding window, 64 registers
+    (120, 2880, 6, 6, 0), (90, 1442, 3, 2, 0), (60, 5000, 2, 4, 640),          # threads chosen by the library; 80 registers
+    (36, 600, 12, 12, 32), (50, 121, 4, 3, 64)])                               # one tile per block; odd nx by columns
+def test_jacobi_matches_oracle(ny, nx, npes, groups, threads, overlap, split, monkeypatch):
+    monkeypatch.setenv("ISHMEM_JACOBI_SPLIT", split)
     grid = inputs.jacobi_grid(inputs.SEED_C5, ny, nx)
     iters = 21
     exp, exp_res = orc.jacobi(grid, iters)
     got, res = run_gpu(grid, npes, iters, overlap, groups, threads)
     assert got.tobytes() == exp.tobytes()
     assert abs(res - exp_res) <= 1e-6 * exp_res
+
+
+def test_jacobi_default_split_and_repeated_calls():
+    """Without ISHMEM_JACOBI_SPLIT the library splits by columns when it shapes the blocks (threads = 0)
+    and by rows otherwise; both give the oracle's grid, call after call on the same heap."""
+    grid = inputs.jacobi_grid(inputs.SEED_C5, 150, 1860)
+    exp, _ = orc.jacobi(grid, 9)
+    for groups, threads in ((5, 0), (5, 96), (40, 0), (2, 0)):
+        got, _ = run_gpu(grid, 6, 9, 1, groups, threads)
+        assert got.tobytes() == exp.tobytes(), (groups, threads)
 
 
 def test_jacobi_even_iterations_and_zero():
@@ -64,7 +79,7 @@ def test_jacobi_even_iterations_and_zero():
 def test_refused_coresident_launch_leaves_the_library_usable():
     """A persistent launch that cannot be co-resident is refused with NOT_CORESIDENT; the
     refusal must not leak into the next call."""
-    npes, ny, nx = 12, 4800, 16
+    npes, ny, nx = 12, 4800, 60 * 400        # 400 rows and 400 column tiles per strip: no clamping of the groups
     nbytes = (ny // npes + 2) * nx * 8
     with Session(npes, 2 * nbytes + (1 << 16), with_oracle=False) as s:
         b0, b1, sig = s.malloc(nbytes), s.malloc(nbytes), s.malloc(64)

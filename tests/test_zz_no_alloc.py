@@ -66,7 +66,7 @@ def test_noalloc_matches_regular_entry_point_twice():
 
 
 def test_noalloc_rejects_launches_beyond_its_fixed_scratch():
-    npes, ny, nx = 12, 12 * 200, 64
+    npes, ny, nx = 12, 12 * 200, 60 * 171    # enough rows and column tiles that 171 groups are not clamped
     rows_max = ny // npes
     nbytes = (rows_max + 2) * nx * 8
     with Session(npes, 2 * nbytes + (1 << 16), with_oracle=False) as s:
