@@ -148,6 +148,7 @@ def run_ours(args) -> dict:
         view = heap[p * HEAP:(p + 1) * HEAP]
         view[:MSG].view(-1, 16 * MiB)[:] = blk
         view[MSG:] = 0
+        view[MSG - 256:MSG] = 0          # a zero source for resetting signal words (end of src)
     # the Jacobi strips live at the start of src: a proper float64 grid (config 5 recipe)
     jn = sizes()["jacobi_n"]
     grid = inputs.jacobi_grid(inputs.SEED_C5, jn, jn)
@@ -167,6 +168,7 @@ def run_ours(args) -> dict:
     rows_max = -(-S["jacobi_n"] // NPES)
     jac_bytes = (rows_max + 2) * S["jacobi_n"] * 8
     jb0, jb1, jsig = src, dst + MiB, dst + 512 * 1024
+    zeros = src + MSG - 256
     rtt, bad, res = np.zeros(1), np.zeros(1, dtype=np.uint64), np.zeros(1)
     ev = lambda: torch.cuda.Event(enable_timing=True)  # noqa: E731
     put_ev, get_ev = [], []
@@ -206,9 +208,8 @@ def run_ours(args) -> dict:
         B.ishmem_fcollectmem(B.ISHMEM_TEAM_WORLD, dst, src, S["fcollect"])
         B.ishmem_float_sum_reduce(B.ISHMEM_TEAM_WORLD, dst, src, S["reduce_f32"])
         B.ishmem_int32_sum_reduce(B.ISHMEM_TEAM_WORLD, dst, src, S["reduce_i32"])
-        for p in range(NPES):
-            for w in range(4):
-                B.ishmem_uint64_p(p, jsig + 8 * w, 0, p)
+        # the four halo signal words of every PE back to zero: one put-to-self from the zeroed end of src
+        B.ishmemx_putmem_spmd(jsig, zeros, 32, 0, B.ISHMEMX_WORK_GROUP, 32, 1)
         B.ishmemx_jacobi(jb0, jb1, jsig, S["jacobi_n"], S["jacobi_n"], S["jacobi_sweeps"], 1,
                          args.jacobi_groups, 0, res)
         B.ishmem_barrier_all()
@@ -277,7 +278,7 @@ def run_ours(args) -> dict:
 
 # DRAM bytes per launch of the put kernel: ncu capture of the 8 x 32 MiB case (reads scale with the
 # bytes copied; writes are the algorithmic bytes minus the ~52 MB tail that stays in L2)
-TRAFFIC_PER_LAUNCH = {"tiled": None, "bulk": 4.24e9, "ldst": None}
+TRAFFIC_PER_LAUNCH = {"tiled": 4.24e9, "bulk": 4.24e9, "ldst": None}
 KERNEL_FORM = {"tiled": "loads/stores, one 32 KiB tile per block", "bulk": "TMA ring, resident blocks",
                "ldst": "loads/stores, resident blocks"}
 
@@ -504,41 +505,42 @@ def run_profile_case(args) -> dict:
 
 
 def run_profile_jacobi(args) -> dict:
-    """Small Jacobi case for profiler captures: 8 PEs, 4096 x 4096 float64 (two buffers of
-    128 MiB: larger than L2), `--steps` launches of 4 sweeps each in the benchmark's shape."""
+    """Small Jacobi case for profiler captures: 8 PEs, 2048 x 16384 float64 (full-width rows as in config 5,
+    two buffers of 256 MiB: larger than L2), `--steps` launches of 4 sweeps each; with --jacobi-groups 17 or
+    fewer the library splits the strips by columns, as it does at full size."""
     import torch
     from paper_2409_20476_b200 import binding as B
     from paper_2409_20476_b200 import inputs
 
-    n, sweeps = 4096, 4
-    rows = n // NPES
-    nbytes = (rows + 2) * n * 8
+    ny, nx, sweeps = 2048, 16384, 4
+    rows = ny // NPES
+    nbytes = (rows + 2) * nx * 8
     heap_bytes = 2 * nbytes + MiB
     heap = torch.zeros(NPES * heap_bytes, dtype=torch.uint8, device="cuda")
     B.ishmemx_init_external(NPES, heap_bytes, heap.data_ptr())
     b0, b1, sig = B.ishmem_malloc(nbytes), B.ishmem_malloc(nbytes), B.ishmem_calloc(4, 8)
-    grid = inputs.jacobi_grid(inputs.SEED_C5, n, n)
+    grid = inputs.jacobi_grid(inputs.SEED_C5, ny, nx)
     for p in range(NPES):
-        o = p * heap_bytes + (b0 - heap.data_ptr()) + n * 8
-        heap[o:o + rows * n * 8].copy_(torch.from_numpy(grid[p * rows:(p + 1) * rows].view(np.uint8).ravel()))
+        o = p * heap_bytes + (b0 - heap.data_ptr()) + nx * 8
+        heap[o:o + rows * nx * 8].copy_(torch.from_numpy(grid[p * rows:(p + 1) * rows].view(np.uint8).ravel()))
     torch.cuda.synchronize()
     ts = torch.cuda.Stream()
     B.ishmemx_set_stream(-1, ts.cuda_stream)
     res, times = np.zeros(1), []
     for _ in range(2 + args.steps):
         for p in range(NPES):
-            B.ishmem_uint64_p(p, sig, 0, p)
-            B.ishmem_uint64_p(p, sig + 8, 0, p)
+            for w in range(4):
+                B.ishmem_uint64_p(p, sig + 8 * w, 0, p)
         torch.cuda.synchronize()
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         a.record(ts)
-        B.ishmemx_jacobi(b0, b1, sig, n, n, sweeps, 1, args.jacobi_groups, 0, res)
+        B.ishmemx_jacobi(b0, b1, sig, ny, nx, sweeps, 1, args.jacobi_groups, 0, res)
         b.record(ts)
         torch.cuda.synchronize()
         times.append(a.elapsed_time(b))
     status = B.ishmemx_status(1)
     B.ishmem_finalize()
-    return {"profile_case": "jacobi", "n": n, "sweeps_per_launch": sweeps, "status": status,
+    return {"profile_case": "jacobi", "ny": ny, "nx": nx, "sweeps_per_launch": sweeps, "status": status,
             "ms": [round(t, 4) for t in times[2:]]}
 
 

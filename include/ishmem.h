@@ -517,9 +517,10 @@ int ishmemx_rma_latency(int my_pe, void *dest, const void *src, size_t nbytes, i
  * (buf1 is overwritten); sig: symmetric, 4 words, zero on entry.  overlap = 0 disables the
  * interior-first ordering (exchange, wait, then compute).
  * threads: threads per block (a multiple of 32 up to 1024) -- the blocks of a PE then take
- * bands of rows, and one of them sends each halo row -- or 0: the library shapes the blocks; they
- * then take ranges of 60-column tiles, one warp per tile, every block sends its columns of the
- * halo rows, and the warps of a PE move down the strip together (a few per cent faster).
+ * bands of rows, and one of them sends each halo row -- or 0: the library shapes the blocks; when
+ * the grid is wide enough for 16 tiles of 60 columns per block they then take ranges of tiles, one
+ * warp per tile, every block sends its columns of the halo rows, and the warps of a PE move down
+ * the strip together (a few per cent faster); narrower grids get 512 threads and bands of rows.
  * groups_per_pe is clamped to the rows (tiles) of the shortest strip.  The environment variable
  * ISHMEM_JACOBI_SPLIT=rows|columns forces one of the two forms.
  * The final strips are in buf0 if iters is even, else buf1.  residual_sq_host (HOST, may be

@@ -645,27 +645,29 @@ __global__ void __launch_bounds__(MAXT) k_jacobi(const ishmem_ctx_t *ctxs, jacob
 }
 
 /* How the blocks of a PE share its strip: by columns when the library shapes the blocks itself
- * (threads == 0: one warp per column tile), by rows when the caller gives the block size (any
- * size then keeps all its warps busy).  ISHMEM_JACOBI_SPLIT=rows / columns overrides; read at
- * every call. */
-static bool jacobi_by_columns(int threads)
+ * (threads == 0) and every block gets at least 16 column tiles, one warp each; by rows when the
+ * caller gives the block size, or when the grid is too narrow to fill the blocks with tiles (a
+ * block then walks all tiles of its band, and any block size keeps its warps busy).
+ * ISHMEM_JACOBI_SPLIT=rows / columns overrides; read at every call. */
+static bool jacobi_by_columns(int threads, size_t nx, int groups_per_pe)
 {
     const char *env = getenv("ISHMEM_JACOBI_SPLIT");
     if (env && !strcmp(env, "rows")) return false;
     if (env && !strcmp(env, "columns")) return true;
-    return threads == 0;
+    return threads == 0 && (nx + 59) / 60 >= (size_t)groups_per_pe * 16;
 }
 
 /* argument checks shared by the two entry points; *groups_per_pe is clamped to the shortest strip */
 static int jacobi_check(double *buf0, double *buf1, uint64_t *sig, size_t ny, size_t nx, int iters,
-                        int *groups_per_pe, int threads)
+                        int *groups_per_pe, int threads, bool *by_columns)
 {
     auto &g = g_ishmem;
     const int P = g.npes;
     if (ny < 3 || nx < 3 || nx > 0x7fffff00u || ny > 0x7fffff00u || iters < 0 || (size_t)P > ny) return ISHMEM_ERR_ARG;
     if (threads < 0 || threads > 1024 || threads % 32 || *groups_per_pe < 1) return ISHMEM_ERR_ARG;
     const size_t rows_min = ny / P, rows_max = (ny + P - 1) / P;
-    const size_t most = jacobi_by_columns(threads) ? (nx + 59) / 60 : rows_min; /* a tile or a row per block at least */
+    *by_columns = jacobi_by_columns(threads, nx, *groups_per_pe);
+    const size_t most = *by_columns ? (nx + 59) / 60 : rows_min; /* a tile or a row per block at least */
     if ((size_t)*groups_per_pe > most) *groups_per_pe = (int)most;
     const size_t bytes = (rows_max + 2) * nx * 8;
     if ((uintptr_t)buf0 % 16 || (uintptr_t)buf1 % 16 || (uintptr_t)sig % 8) return ISHMEM_ERR_ALIGN;
@@ -678,7 +680,7 @@ static int jacobi_check(double *buf0, double *buf1, uint64_t *sig, size_t ny, si
 /* clears the scratch, launches the persistent kernel on the team stream and waits for it;
  * `scratch` holds nblocks sweep counters followed by nblocks residual partials */
 static int jacobi_launch(double *buf0, double *buf1, uint64_t *sig, size_t ny, size_t nx, int iters, int overlap,
-                         int groups_per_pe, int threads, void *scratch, jacobi_args *out_args)
+                         int groups_per_pe, int threads, bool by_columns, void *scratch, jacobi_args *out_args)
 {
     auto &g = g_ishmem;
     const size_t nblocks = (size_t)g.npes * groups_per_pe;
@@ -699,7 +701,7 @@ static int jacobi_launch(double *buf0, double *buf1, uint64_t *sig, size_t ny, s
     a.done = (unsigned long long *)scratch;
     a.partial = (double *)((char *)scratch + nblocks * 8);
     a.sliding = (nx % 2 == 0);
-    a.colsplit = jacobi_by_columns(threads);
+    a.colsplit = by_columns;
     if (threads == 0) {
         /* by columns: one warp per tile when that fits a block, else the fewest equal rounds;
          * by rows: 512 */
@@ -735,14 +737,15 @@ extern "C" int ishmemx_jacobi(double *buf0, double *buf1, uint64_t *sig, size_t 
 {
     ISHMEMI_REQUIRE_INIT();
     auto &g = g_ishmem;
-    int rc = jacobi_check(buf0, buf1, sig, ny, nx, iters, &groups_per_pe, threads);
+    bool by_columns = false;
+    int rc = jacobi_check(buf0, buf1, sig, ny, nx, iters, &groups_per_pe, threads, &by_columns);
     if (rc) return rc;
     const size_t nblocks = (size_t)g.npes * groups_per_pe;
     /* scratch: per-block sweep counters and residual partials */
     char *scratch = nullptr;
     ISHMEMI_CUDA(cudaMalloc((void **)&scratch, nblocks * 16));
     jacobi_args a;
-    rc = jacobi_launch(buf0, buf1, sig, ny, nx, iters, overlap, groups_per_pe, threads, scratch, &a);
+    rc = jacobi_launch(buf0, buf1, sig, ny, nx, iters, overlap, groups_per_pe, threads, by_columns, scratch, &a);
     if (!rc && residual_sq_host) {
         std::vector<double> part(nblocks);
         rc = ishmemi_cuda(cudaMemcpy(part.data(), a.partial, nblocks * 8, cudaMemcpyDeviceToHost), "cudaMemcpy");
@@ -787,7 +790,8 @@ extern "C" int ishmemx_jacobi_noalloc(double *buf0, double *buf1, uint64_t *sig,
 {
     ISHMEMI_REQUIRE_INIT();
     auto &g = g_ishmem;
-    int rc = jacobi_check(buf0, buf1, sig, ny, nx, iters, &groups_per_pe, threads);
+    bool by_columns = false;
+    int rc = jacobi_check(buf0, buf1, sig, ny, nx, iters, &groups_per_pe, threads, &by_columns);
     if (rc == ISHMEM_ERR_ARG) return rc;
     const size_t nblocks = (size_t)g.npes * groups_per_pe;
     if (nblocks > ISHMEMX_JACOBI_NOALLOC_MAX_BLOCKS) {
@@ -799,7 +803,7 @@ extern "C" int ishmemx_jacobi_noalloc(double *buf0, double *buf1, uint64_t *sig,
     if ((rc = jacobi_scratch_for_current_device(&scratch))) return rc;
     /* the array keeps the previous call's counters; jacobi_launch clears the part this call uses */
     jacobi_args a;
-    rc = jacobi_launch(buf0, buf1, sig, ny, nx, iters, overlap, groups_per_pe, threads, scratch, &a);
+    rc = jacobi_launch(buf0, buf1, sig, ny, nx, iters, overlap, groups_per_pe, threads, by_columns, scratch, &a);
     if (!rc && residual_sq_host) {
         double part[ISHMEMX_JACOBI_NOALLOC_MAX_BLOCKS];
         rc = ishmemi_cuda(cudaMemcpy(part, a.partial, nblocks * 8, cudaMemcpyDeviceToHost), "cudaMemcpy");

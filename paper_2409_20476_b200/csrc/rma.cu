@@ -228,12 +228,16 @@ static void auto_geometry(size_t n, int *threads, unsigned *blocks, int *level)
         *blocks = (unsigned)((n + 16383) / 16384);
         *level = ISHMEMX_WORK_GROUP;
     } else {
-        /* one 32 KiB tile per block.  Blocks start in index order, so the running blocks sweep one
+        /* one tile (32 KiB for large messages) per block.  Blocks start in index order, so the running blocks sweep one
          * short window of the source and of the destination; measured on B200 that moves more
          * bytes per second (6.8 TB/s at 256 MiB per PE) than a resident grid streaming long slices,
          * by loads and stores or through the TMA ring (6.4) */
         *threads = 256;
-        size_t b = (n + 32767) / 32768;
+        /* 128 bytes per thread when that still gives every SM four blocks, down to 16 for messages
+         * of a few MiB, which need the parallelism more than the long bursts */
+        size_t per_thread = 128;
+        while (per_thread > 16 && n / (256 * per_thread) < (size_t)g_ishmem.sm_count * 4) per_thread >>= 1;
+        const size_t tile = 256 * per_thread, b = (n + tile - 1) / tile;
         *blocks = (unsigned)(b < 0x7fffffffu ? b : 0x7fffffffu);
         *level = ISHMEMX_WORK_GROUP;
     }

@@ -59,11 +59,11 @@ def test_jacobi_matches_oracle(ny, nx, npes, groups, threads, overlap, split, mo
 
 
 def test_jacobi_default_split_and_repeated_calls():
-    """Without ISHMEM_JACOBI_SPLIT the library splits by columns when it shapes the blocks (threads = 0)
-    and by rows otherwise; both give the oracle's grid, call after call on the same heap."""
-    grid = inputs.jacobi_grid(inputs.SEED_C5, 150, 1860)
+    """Without ISHMEM_JACOBI_SPLIT the library splits by columns when it shapes the blocks (threads = 0) and
+    each gets 16 tiles or more, by rows otherwise; both give the oracle's grid."""
+    grid = inputs.jacobi_grid(inputs.SEED_C5, 150, 2400)         # 40 column tiles
     exp, _ = orc.jacobi(grid, 9)
-    for groups, threads in ((5, 0), (5, 96), (40, 0), (2, 0)):
+    for groups, threads in ((2, 0), (5, 0), (5, 96), (40, 0)):    # by columns (20 tiles per block), then by rows
         got, _ = run_gpu(grid, 6, 9, 1, groups, threads)
         assert got.tobytes() == exp.tobytes(), (groups, threads)
 
