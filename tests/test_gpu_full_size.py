@@ -50,19 +50,21 @@ def windows(n, width, rng, extra=()):
     return sorted(pts)
 
 
-@pytest.mark.parametrize("level,threads,groups", [("bulk", 256, 37), ("ldst", 512, 74)])
+@pytest.mark.parametrize("level,threads,groups", [("tiled", 256, 0), ("bulk", 256, 37), ("ldst", 512, 74)])
 def test_config2_put_get_256mib_ring_and_all_pairs(level, threads, groups):
     """Config 2 at its largest size: 8 PEs x 512 MiB heap, 256 MiB uint8 messages, ring and the
-    7 all-pairs rounds, in the geometry the benchmark launches (and the ldst alternative)."""
+    7 all-pairs rounds, in the geometry the benchmark launches (groups = 0: one tile of threads x 128
+    bytes per block) and in the two resident-grid alternatives."""
     npes, heap, n = 8, 512 * MiB, 256 * MiB
-    lv = {"bulk": B.ISHMEMX_WORK_GROUP_BULK, "ldst": B.ISHMEMX_WORK_GROUP}[level]
+    lv = {"tiled": B.ISHMEMX_WORK_GROUP, "bulk": B.ISHMEMX_WORK_GROUP_BULK, "ldst": B.ISHMEMX_WORK_GROUP}[level]
     rng = np.random.default_rng(7)
     with Session(npes, heap, with_oracle=False) as s:
         src, dst = s.malloc(n), s.malloc(n)
         fill_full(src, "u8", inputs.SEED_C2, n, npes)
-        per = -(-n // groups)
+        nslices = groups if groups else n // (threads * 128)
+        per = -(-n // nslices)
         per = (per + 127) // 128 * 128
-        offs = windows(n, 4096, rng, extra=[per * g for g in (1, 2, groups // 2, groups - 1)])
+        offs = windows(n, 4096, rng, extra=[per * g for g in (1, 2, nslices // 2, nslices - 1)])
         for shift in range(1, npes):
             B.ishmemx_putmem_spmd(dst.addr, src.addr, n, shift, lv, threads, groups)
             s.sync()

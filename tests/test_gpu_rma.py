@@ -128,6 +128,36 @@ def test_spmd_ring_and_all_pairs(level):
         assert s.status() == 0
 
 
+@pytest.mark.parametrize("threads", [32, 256, 1024])
+def test_spmd_grid_sized_by_the_library(threads):
+    """groups = 0: one tile of threads x 128 bytes per block.  Ragged sizes around the tile size and
+    misaligned, non-congruent addresses against the oracle; the heaps are compared whole."""
+    npes, heap = 5, 4 << 20
+    tile = threads * 128
+    with Session(npes, heap) as s:
+        src, dst = s.malloc(1 << 20), s.malloc(1 << 20)
+        for p in range(npes):
+            src.fill(p, inputs.byte_payload(inputs.SEED_C2, p, 1 << 20))
+        cases = [(0, 0, 1), (0, 0, tile - 1), (0, 0, tile), (3, 3, tile + 1), (16, 5, 3 * tile + 77),
+                 (1, 2, 7 * tile - 13), (0, 8, 500_000), (0, 0, 0)]
+        for k, (doff, soff, n) in enumerate(cases):
+            shift = 1 + k % (npes - 1)
+            B.ishmemx_putmem_spmd(dst.addr + doff, src.addr + soff, n, shift, B.ISHMEMX_WORK_GROUP, threads, 0)
+            for p in range(npes):
+                s.oracle.putmem(p, dst.ooff + doff, s.oracle.ptr(src.ooff + soff, n, p), n, (p + shift) % npes)
+            dst.assert_equal(f"put case {k}")
+        B.ishmemx_getmem_spmd(src.addr + 32, dst.addr + 1, 2 * tile + 5, 2, B.ISHMEMX_WORK_GROUP, threads, 0)
+        for p in range(npes):
+            s.oracle.getmem(p, s.oracle.ptr(src.ooff + 32, 2 * tile + 5, p), dst.ooff + 1, 2 * tile + 5, (p + 2) % npes)
+        heaps_equal(s, f"threads {threads}")
+        # the host API picks the same shape by itself above 256 KiB
+        B.ishmem_putmem(0, dst.addr + 7, src.addr + 7, 900_001, 3)
+        s.oracle.putmem(0, dst.ooff + 7, s.oracle.ptr(src.ooff + 7, 900_001, 0), 900_001, 3)
+        B.ishmem_barrier_all()
+        heaps_equal(s, "host api")
+        assert s.status() == 0
+
+
 @pytest.mark.parametrize("level", ["work_item", "sub_group", "work_group", "work_group_bulk"])
 def test_misaligned_brute_force(level):
     """Every source/destination alignment mod 16 with ragged lengths, private and symmetric
