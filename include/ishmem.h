@@ -509,23 +509,29 @@ int ishmemx_rma_latency(int my_pe, void *dest, const void *src, size_t nbytes, i
                         int level, int threads, int iters, double *ns_per_op);
 
 /* Overlap workload: `iters` sweeps of the 5-point Jacobi update on an ny x nx float64
- * grid cut into npes row strips (the first ny mod npes strips have one more row), in one
- * persistent co-resident launch of npes x groups_per_pe blocks: each sweep every PE sends its
- * first and last rows to the neighbours' halo rows with in-kernel work-group put_signal, updates
- * its interior rows meanwhile, waits for its own halos, then updates its edge rows.  buf0/buf1:
+ * grid cut into npes row strips (the first ny mod npes strips have one more row): each sweep
+ * every PE sends its first and last rows to the neighbours' halo rows with in-kernel work-group
+ * put_signal, updates its interior rows meanwhile, and updates its edge rows once its own halos
+ * have arrived.  buf0/buf1:
  * symmetric, (ceil(ny/npes)+2)*nx doubles each, strip row r at local row r+1 of buf0 on entry
  * (buf1 is overwritten); sig: symmetric, 4 words, zero on entry.  overlap = 0 disables the
  * interior-first ordering (exchange, wait, then compute).
- * threads: threads per block (a multiple of 32 up to 1024) -- the blocks of a PE then take
- * bands of rows, and one of them sends each halo row -- or 0: the library shapes the blocks; when
- * the grid is wide enough for 16 tiles of 60 columns per block they then take ranges of tiles, one
- * warp per tile, every block sends its columns of the halo rows, and the warps of a PE move down
- * the strip together (a few per cent faster); narrower grids get 512 threads and bands of rows.
- * groups_per_pe is clamped to the rows (tiles) of the shortest strip.  The environment variable
- * ISHMEM_JACOBI_SPLIT=rows|columns forces one of the two forms.
+ * threads = 0 (and an even nx): the library shapes the launches itself -- ONE LAUNCH PER SWEEP, whose
+ * first blocks send the halo rows (in-kernel work-group put_signal) and whose other blocks each
+ * take 16 rows of 8 neighbouring 60-column tiles, numbered so that the blocks sweep the grid in
+ * launch order; only the first and the last band of a strip wait for a halo, the interior never
+ * does.  This is the fastest form (6.6 TB/s at 16384^2); groups_per_pe is not used by it and
+ * nothing needs to be co-resident.
+ * threads > 0 (a multiple of 32 up to 1024): one persistent co-resident launch of
+ * npes x groups_per_pe blocks of that size for all sweeps; the blocks of a PE take bands of rows,
+ * one of them sends each halo row, and neighbouring blocks hand over through flags.
+ * ISHMEM_ERR_NOT_CORESIDENT when the blocks cannot all be resident at once.  The environment
+ * variable ISHMEM_JACOBI_SPLIT=rows|columns selects the persistent kernel also for threads = 0,
+ * with the strips cut by rows, or by ranges of column tiles (one warp per tile; every block then
+ * sends its columns of the halo rows); groups_per_pe is clamped to the rows (tiles) of the
+ * shortest strip.
  * The final strips are in buf0 if iters is even, else buf1.  residual_sq_host (HOST, may be
- * NULL) receives ||u_iters - u_(iters-1)||_2^2 over the interior.  Blocks the host.
- * ISHMEM_ERR_NOT_CORESIDENT when the blocks cannot all be resident at once. */
+ * NULL) receives ||u_iters - u_(iters-1)||_2^2 over the interior.  Blocks the host. */
 int ishmemx_jacobi(double *buf0, double *buf1, uint64_t *sig, size_t ny, size_t nx, int iters,
                    int overlap, int groups_per_pe, int threads, double *residual_sq_host);
 
@@ -544,6 +550,9 @@ int ishmemx_jacobi(double *buf0, double *buf1, uint64_t *sig, size_t ny, size_t 
  *   - All calls share the one array.  It still holds the previous call's contents, so each
  *     call clears the part it uses first; two calls whose kernels overlap on the GPU (from
  *     two host threads, say) would race on it -- serialise them.
+ *   - It always runs the persistent kernel (threads = 0: strips cut by column tiles when the grid
+ *     is wide enough, else by rows with 512 threads); the one-launch-per-sweep form keeps one
+ *     residual term per tile block and does not fit the fixed array.
  * Arguments, results and error codes are otherwise those of ishmemx_jacobi. */
 int ishmemx_jacobi_noalloc(double *buf0, double *buf1, uint64_t *sig, size_t ny, size_t nx, int iters,
                            int overlap, int groups_per_pe, int threads, double *residual_sq_host);

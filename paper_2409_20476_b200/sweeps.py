@@ -485,29 +485,39 @@ def sweep_c5(args, out):
             first += rows
 
     load()
+    import os
+    # (variant, ISHMEM_JACOBI_SPLIT, threads, groups): the library's own choice (one launch per sweep), the
+    # persistent kernel with strips cut by column tiles, and the persistent kernel with caller-shaped blocks
+    variants = [("per_sweep_tiles", None, 0, 1)]
+    variants += [("persistent_columns", "columns", 0, g) for g in (6, 12)]
+    variants += [("persistent_rows", "rows", t, g) for g in (6, 12, 24) for t in (256, 512, 1024)]
     for overlap in (1, 0):
-        for groups in (6, 12, 24):
-            for threads in (0, 256, 512, 1024):       # 0: blocks shaped by the library, strip split by columns
-                if npes * groups * threads > 148 * 2048:
-                    continue
-                for p in range(npes):
-                    for w in range(4):
-                        B.ishmem_uint64_p(p, sig + 8 * w, 0, p)
-                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                torch.cuda.synchronize()
-                a.record(stream)
-                try:
-                    B.ishmemx_jacobi(b0, b1, sig, n, n, iters, overlap, groups, threads, res)
-                except B.IshmemError as e:
-                    out.add(config=5, op="jacobi", variant=f"overlap={overlap}", threads=threads, groups=groups,
-                            npes=npes, dtype="f64", nbytes=n * n * 8, note=str(e))
-                    continue
-                b.record(stream)
-                torch.cuda.synchronize()
-                us = a.elapsed_time(b) * 1e3 / iters
-                out.add(config=5, op="jacobi", pattern=f"{n}x{n}", variant=f"overlap={overlap}", threads=threads,
-                        groups=groups, npes=npes, dtype="f64", nbytes=n * n * 8, l2="cold", iters=iters, us_per_op=us,
-                        alg_bytes=16 * n * n, note=f"per sweep; residual_sq {res[0]:.6e} (grid keeps evolving)")
+        for variant, split, threads, groups in variants:
+            if npes * groups * threads > 148 * 2048:
+                continue
+            if split is None:
+                os.environ.pop("ISHMEM_JACOBI_SPLIT", None)
+            else:
+                os.environ["ISHMEM_JACOBI_SPLIT"] = split
+            for p in range(npes):
+                for w in range(4):
+                    B.ishmem_uint64_p(p, sig + 8 * w, 0, p)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            a.record(stream)
+            try:
+                B.ishmemx_jacobi(b0, b1, sig, n, n, iters, overlap, groups, threads, res)
+            except B.IshmemError as e:
+                out.add(config=5, op="jacobi", variant=f"{variant} overlap={overlap}", threads=threads, groups=groups,
+                        npes=npes, dtype="f64", nbytes=n * n * 8, note=str(e))
+                continue
+            b.record(stream)
+            torch.cuda.synchronize()
+            us = a.elapsed_time(b) * 1e3 / iters
+            out.add(config=5, op="jacobi", pattern=f"{n}x{n}", variant=f"{variant} overlap={overlap}", threads=threads,
+                    groups=groups, npes=npes, dtype="f64", nbytes=n * n * 8, l2="cold", iters=iters, us_per_op=us,
+                    alg_bytes=16 * n * n, note=f"per sweep; residual_sq {res[0]:.6e} (grid keeps evolving)")
+    os.environ.pop("ISHMEM_JACOBI_SPLIT", None)
     assert B.ishmemx_status(1) == 0
     B.ishmem_finalize()
 
@@ -626,12 +636,15 @@ def summarize(path) -> str:
                 _table(sel, nb, lambda r: f"{r['threads']} threads", us, _fmt_size), ""]
     elif cfg == 5:
         out += ["### Jacobi 16384 x 16384 float64, 12 PEs, 200 sweeps: per sweep", "",
-                "| overlap | threads | groups/PE | us/sweep | GB/s (16 B/cell) | of measured copy | of 8 TB/s |", "|---|---:|---:|---:|---:|---:|---:|"]
+                "| form | overlap | threads | groups/PE | us/sweep | GB/s (16 B/cell) | of measured copy | of 8 TB/s |",
+                "|---|---|---:|---:|---:|---:|---:|---:|"]
         for r in rows:
+            form, ov = r["variant"].rsplit(" overlap=", 1) if " overlap=" in r["variant"] else ("", r["variant"][-1])
+            shape = f"| {form} | {ov} | {r['threads'] if r['threads'] != '0' else 'library'} | {r['groups'] if form != 'per_sweep_tiles' else '-'} |"
             if r["us_per_op"]:
-                out.append(f"| {r['variant'][-1]} | {r['threads']} | {r['groups']} | {us(r)} | {gb(r)} | {r['frac_hbm']} | {r['frac_8tbs']} |")
+                out.append(f"{shape} {us(r)} | {gb(r)} | {r['frac_hbm']} | {r['frac_8tbs']} |")
             else:
-                out.append(f"| {r['variant'][-1]} | {r['threads']} | {r['groups']} | refused: not co-resident | | | |")
+                out.append(f"{shape} refused: not co-resident | | | |")
     elif cfg == 6:
         out += ["### reverse-offload ring (64-byte requests, one host proxy thread)", "",
                 "| measurement | blocks x threads | us | M requests/s |", "|---|---:|---:|---:|"]

@@ -40,7 +40,7 @@ def run_gpu(grid, npes, iters, overlap, groups, threads):
         return out, res[0]
 
 
-@pytest.mark.parametrize("split", ["columns", "rows"])
+@pytest.mark.parametrize("split", ["sweeps", "columns", "rows"])
 @pytest.mark.parametrize("overlap", [1, 0])
 @pytest.mark.parametrize("ny,nx,npes,groups,threads", [
     (64, 48, 12, 1, 128), (200, 131, 12, 3, 128), (257, 33, 5, 4, 128),       # odd nx: row-by-row path
@@ -49,7 +49,13 @@ def run_gpu(grid, npes, iters, overlap, groups, threads):
     (120, 2880, 6, 6, 0), (90, 1442, 3, 2, 0), (60, 5000, 2, 4, 640),          # threads chosen by the library; 80 registers
     (36, 600, 12, 12, 32), (50, 121, 4, 3, 64)])                               # one tile per block; odd nx by columns
 def test_jacobi_matches_oracle(ny, nx, npes, groups, threads, overlap, split, monkeypatch):
-    monkeypatch.setenv("ISHMEM_JACOBI_SPLIT", split)
+    """split: the persistent kernel with the strips cut by columns or by rows, or `sweeps`: the form the
+    library picks by itself for threads = 0 and even nx (one launch per sweep, one tile per warp)."""
+    if split == "sweeps":
+        monkeypatch.delenv("ISHMEM_JACOBI_SPLIT", raising=False)
+        threads = 0
+    else:
+        monkeypatch.setenv("ISHMEM_JACOBI_SPLIT", split)
     grid = inputs.jacobi_grid(inputs.SEED_C5, ny, nx)
     iters = 21
     exp, exp_res = orc.jacobi(grid, iters)
@@ -59,13 +65,24 @@ def test_jacobi_matches_oracle(ny, nx, npes, groups, threads, overlap, split, mo
 
 
 def test_jacobi_default_split_and_repeated_calls():
-    """Without ISHMEM_JACOBI_SPLIT the library splits by columns when it shapes the blocks (threads = 0) and
-    each gets 16 tiles or more, by rows otherwise; both give the oracle's grid."""
+    """Without ISHMEM_JACOBI_SPLIT: threads = 0 launches once per sweep, a given block size runs the persistent
+    kernel with the strips cut by rows; both give the oracle's grid."""
     grid = inputs.jacobi_grid(inputs.SEED_C5, 150, 2400)         # 40 column tiles
     exp, _ = orc.jacobi(grid, 9)
-    for groups, threads in ((2, 0), (5, 0), (5, 96), (40, 0)):    # by columns (20 tiles per block), then by rows
+    for groups, threads in ((2, 0), (5, 0), (5, 96), (40, 0)):    # one launch per sweep; (5, 96): persistent, by rows
         got, _ = run_gpu(grid, 6, 9, 1, groups, threads)
         assert got.tobytes() == exp.tobytes(), (groups, threads)
+
+
+def test_jacobi_per_sweep_many_bands_and_residual():
+    """The per-sweep form on strips of several 32-row bands and tile groups, with strips of unequal length,
+    odd and even iteration counts; final grid bit-exact, residual within 1e-6 relative."""
+    grid = inputs.jacobi_grid(inputs.SEED_C5, 1000, 1100)
+    for npes, iters in ((7, 5), (3, 12), (1, 3)):
+        exp, exp_res = orc.jacobi(grid, iters)
+        got, res = run_gpu(grid, npes, iters, 1, 1, 0)
+        assert got.tobytes() == exp.tobytes(), (npes, iters)
+        assert abs(res - exp_res) <= 1e-6 * exp_res
 
 
 def test_jacobi_even_iterations_and_zero():
