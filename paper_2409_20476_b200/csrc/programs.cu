@@ -659,7 +659,9 @@ __global__ void __launch_bounds__(MAXT) k_jacobi(const ishmem_ctx_t *ctxs, jacob
  * needs the halo from above and only the last one the halo from below: their blocks wait (bounded)
  * for the signal first, which the senders -- started long before them -- have raised by then, while
  * the interior bands never wait: the exchange overlaps the interior update.  The launch boundary
- * orders one sweep after the other; nothing needs to be co-resident. */
+ * orders one sweep after the other; nothing needs to be co-resident.  The senders have the lowest
+ * block numbers and wait for nothing, so a block that waits for them can only hold an SM after all of
+ * them have started; and every wait gives up after the context's time limit in any case. */
 #define JACOBI_PIECES 8u
 /* sender block b of a sweep: piece (b mod JACOBI_PIECES) of a PE's first or last row.  Out of line,
  * like the full-featured window below, so that the common path of k_jacobi_sweep keeps its
@@ -671,7 +673,7 @@ static __device__ __noinline__ void jacobi_send_piece(const ishmem_ctx_t *ctxs, 
      * a reference to the kernel's argument block would put it on every thread's stack) */
     const int P = ctxs[0].npes;
     {
-        /* sender: piece `piece` of PE p's first row (up == 0) or last row (up == 1) */
+        /* piece `piece` of PE p's first row (down == 0) or last row (down == 1) */
         const int p = (int)(b / (2u * JACOBI_PIECES)), down = (int)((b / JACOBI_PIECES) & 1u);
         const unsigned piece = b % JACOBI_PIECES;
         const ishmem_ctx_t *ctx = ctxs + p;
