@@ -666,31 +666,37 @@ __global__ void __launch_bounds__(MAXT) k_jacobi(const ishmem_ctx_t *ctxs, jacob
 /* sender block b of a sweep: piece (b mod JACOBI_PIECES) of a PE's first or last row.  Out of line,
  * like the full-featured window below, so that the common path of k_jacobi_sweep keeps its
  * registers to itself. */
-static __device__ __noinline__ void jacobi_send_piece(const ishmem_ctx_t *ctxs, const double *cur0, unsigned long long *sig0,
-                                                      size_t ny, size_t nx, unsigned b)
+static __device__ __noinline__ void jacobi_send_piece(const ishmem_ctx_t *ctxs, const double *cur0, double *nxt0,
+                                                      unsigned long long *sig0, size_t ny, size_t nx, unsigned b)
 {
-    /* cur0, sig0: PE 0's copies of the sweep's source buffer and of the signal words (by value:
-     * a reference to the kernel's argument block would put it on every thread's stack) */
+    /* cur0, nxt0, sig0: PE 0's copies of the source buffer, of the other buffer (two-sweep passes
+     * only, else null) and of the signal words.  By value: a reference to the kernel's argument
+     * block would put it on every thread's stack.
+     * One sweep per launch: 2 x JACOBI_PIECES blocks per PE send its first row up and its last row
+     * down, into the halo rows of the neighbours' source buffers.  Two sweeps per launch: twice as
+     * many; the second set sends the second and the second-to-last row into the halo rows of the
+     * neighbours' OTHER buffer, which nothing else uses during the pass. */
     const int P = ctxs[0].npes;
-    {
-        /* piece `piece` of PE p's first row (down == 0) or last row (down == 1) */
-        const int p = (int)(b / (2u * JACOBI_PIECES)), down = (int)((b / JACOBI_PIECES) & 1u);
-        const unsigned piece = b % JACOBI_PIECES;
-        const ishmem_ctx_t *ctx = ctxs + p;
-        size_t first, rows, rows_above = 0, f2;
-        strip_of(ny, P, p, &first, &rows);
-        if (p > 0) strip_of(ny, P, p - 1, &f2, &rows_above);
-        const double *cur = (const double *)local_of(ctxs, ctx, cur0);
-        unsigned long long *sig = (unsigned long long *)local_of(ctxs, ctx, sig0);
-        const size_t per = ((nx + JACOBI_PIECES - 1) / JACOBI_PIECES + 1) & ~(size_t)1; /* even: 16-byte pieces */
-        const size_t c_lo = per * piece < nx ? per * piece : nx, c_hi = c_lo + per < nx ? c_lo + per : nx;
-        if (!down && p > 0) /* my first row -> bottom halo of the PE above */
-            ishmemx_putmem_signal_work_group(ctx, (void *)(cur + (rows_above + 1) * nx + c_lo), cur + nx + c_lo,
-                                             (c_hi - c_lo) * 8, sig + 1, 1, ISHMEM_SIGNAL_ADD, p - 1);
-        if (down && p + 1 < P) /* my last row -> top halo of the PE below */
-            ishmemx_putmem_signal_work_group(ctx, (void *)(cur + c_lo), cur + rows * nx + c_lo, (c_hi - c_lo) * 8,
-                                             sig + 0, 1, ISHMEM_SIGNAL_ADD, p + 1);
-    }
+    const unsigned per_pe = (nxt0 ? 4u : 2u) * JACOBI_PIECES;
+    const int p = (int)(b / per_pe), down = (int)((b / JACOBI_PIECES) & 1u), second = (int)((b % per_pe) / (2u * JACOBI_PIECES));
+    const unsigned piece = b % JACOBI_PIECES;
+    const ishmem_ctx_t *ctx = ctxs + p;
+    size_t first, rows, rows_above = 0, f2;
+    strip_of(ny, P, p, &first, &rows);
+    if (p > 0) strip_of(ny, P, p - 1, &f2, &rows_above);
+    const double *cur = (const double *)local_of(ctxs, ctx, cur0);
+    /* the destination is named by the calling PE's copy of the buffer that receives it */
+    double *into = second ? (double *)local_of(ctxs, ctx, nxt0) : (double *)cur;
+    unsigned long long *sig = (unsigned long long *)local_of(ctxs, ctx, sig0);
+    const size_t per = ((nx + JACOBI_PIECES - 1) / JACOBI_PIECES + 1) & ~(size_t)1; /* even: 16-byte pieces */
+    const size_t c_lo = per * piece < nx ? per * piece : nx, c_hi = c_lo + per < nx ? c_lo + per : nx;
+    if (!down && p > 0) /* my first (second) row -> bottom halo of the PE above */
+        ishmemx_putmem_signal_work_group(ctx, (void *)(into + (rows_above + 1) * nx + c_lo),
+                                         cur + (size_t)(second ? 2 : 1) * nx + c_lo, (c_hi - c_lo) * 8, sig + 1, 1,
+                                         ISHMEM_SIGNAL_ADD, p - 1);
+    if (down && p + 1 < P) /* my last (second-to-last) row -> top halo of the PE below */
+        ishmemx_putmem_signal_work_group(ctx, (void *)(into + c_lo), cur + (rows - (second ? 1 : 0)) * nx + c_lo,
+                                         (c_hi - c_lo) * 8, sig + 0, 1, ISHMEM_SIGNAL_ADD, p + 1);
 }
 static __device__ __noinline__ double jacobi_march_one(const double *cur, double *nxt, unsigned ra, unsigned rb,
                                                        unsigned fixed0, unsigned fixed1, unsigned nx, bool want_res,
@@ -699,18 +705,20 @@ static __device__ __noinline__ double jacobi_march_one(const double *cur, double
     return jacobi_march_tiles<4>(cur, nxt, ra, rb, fixed0, fixed1, nx, want_res, t_lo, t_hi);
 }
 
-__global__ void __launch_bounds__(256, 4) k_jacobi_sweep(const ishmem_ctx_t *ctxs, jacobi_args a, int it, unsigned band_rows,
+__global__ void __launch_bounds__(256, 4) k_jacobi_sweep(const ishmem_ctx_t *ctxs, jacobi_args a, int flip,
+                                                          unsigned long long arrived, int last, unsigned band_rows,
                                                           unsigned bands, unsigned tile_groups, int P, size_t heap_stride)
 {
+    /* flip: the sweep reads buf1 and writes buf0 (else buf0 -> buf1); arrived: what the halo words
+     * count once this sweep's pieces are in; last: the residual is wanted. */
     /* P and the distance between two PEs' heaps come as arguments: a tile block lives for a few
      * microseconds, too short to start with a chain of look-ups in the context */
     const unsigned tid = threadIdx.x;
     const size_t nx = a.nx;
     const unsigned nsend = (unsigned)P * 2u * JACOBI_PIECES;
-    const unsigned long long arrived = (unsigned long long)JACOBI_PIECES * ((unsigned long long)it + 1);
     unsigned b = blockIdx.x;
     if (b < nsend) {
-        jacobi_send_piece(ctxs, (it & 1) ? a.buf1 : a.buf0, a.sig, a.ny, nx, b);
+        jacobi_send_piece(ctxs, flip ? a.buf1 : a.buf0, nullptr, a.sig, a.ny, nx, b);
         return;
     }
     b -= nsend;
@@ -738,21 +746,165 @@ __global__ void __launch_bounds__(256, 4) k_jacobi_sweep(const ishmem_ctx_t *ctx
             __syncthreads();
             if (give_up) return;
         }
-        const double *cur = (const double *)((const char *)((it & 1) ? a.buf1 : a.buf0) + (size_t)p * heap_stride);
-        double *nxt = (double *)((char *)((it & 1) ? a.buf0 : a.buf1) + (size_t)p * heap_stride);
+        const double *cur = (const double *)((const char *)(flip ? a.buf1 : a.buf0) + (size_t)p * heap_stride);
+        double *nxt = (double *)((char *)(flip ? a.buf0 : a.buf1) + (size_t)p * heap_stride);
         const unsigned fixed0 = (first == 0) ? 1u : ~0u;
         const unsigned fixed1 = (first + rows == (unsigned)a.ny) ? rows : ~0u;
         /* this block's tiles: warp w takes tile t_lo + w */
         const unsigned ntiles = (unsigned)((nx + 59) / 60), t_lo = tg * (blockDim.x >> 5);
         const unsigned t_hi = t_lo + (blockDim.x >> 5) < ntiles ? t_lo + (blockDim.x >> 5) : ntiles;
         const bool has_fixed = (fixed0 >= ra && fixed0 < rb) || (fixed1 >= ra && fixed1 < rb);
-        if (it == a.iters - 1 || has_fixed) /* the last sweep, and the two bands with a boundary row */
-            acc = jacobi_march_one(cur, nxt, ra, rb, fixed0, fixed1, (unsigned)nx, it == a.iters - 1, t_lo, t_hi);
+        if (last || has_fixed) /* the last sweep, and the two bands with a boundary row */
+            acc = jacobi_march_one(cur, nxt, ra, rb, fixed0, fixed1, (unsigned)nx, last != 0, t_lo, t_hi);
         else
             jacobi_march_tiles<4, false, false>(cur, nxt, ra, rb, ~0u, ~0u, (unsigned)nx, false, t_lo, t_hi);
     }
-    if (it == a.iters - 1) {
+    if (last) {
         /* residual partial of this block, summed in a fixed order */
+        __shared__ double red[8];
+        for (int o = 16; o > 0; o >>= 1) acc += __shfl_down_sync(0xffffffffu, acc, o);
+        if ((tid & 31u) == 0) red[tid >> 5] = acc;
+        __syncthreads();
+        if (tid == 0) {
+            double sum = 0.0;
+            for (unsigned w = 0; w < (blockDim.x >> 5); ++w) sum += red[w];
+            a.partial[b] = sum;
+        }
+    }
+}
+
+/* ---- two sweeps per launch -------------------------------------------------------------------
+ * Every element of the source is read once and the result of the SECOND sweep written once: half
+ * the memory traffic per sweep.  A warp's window now carries two time levels.  It loads 64 columns
+ * of rows ra-2 .. rb+1 of u(t); from each new row it forms the row above it of u(t+1) (valid in
+ * lanes 1..30), keeps two rows of that level in registers as well, and from each new u(t+1) row
+ * forms the row above of u(t+2) (valid in lanes 2..29: 56 output columns per tile), which is
+ * stored.  The same expression, in the same order, gives every value, so the result is
+ * bit-identical to two single sweeps; values in the shrinking border of a tile are recomputed by
+ * the neighbouring tile.  Rows -1 and rows+2 (the second halo) are read from the halo rows of the
+ * destination buffer, where this pass's senders put them. */
+template <int DEPTH>
+__device__ __forceinline__ double jacobi_march2(const double *cur, double *nxt, unsigned ra, unsigned rb, unsigned rows,
+                                                unsigned fixed0, unsigned fixed1, unsigned nx, bool want_res,
+                                                unsigned t_lo, unsigned t_hi)
+{
+    double acc = 0.0;
+    if (rb <= ra) return acc;
+    const unsigned lane = threadIdx.x & 31u;
+    const unsigned full = 0xffffffffu;
+    const double2 zero = make_double2(0.0, 0.0);
+    const unsigned t = t_lo + (threadIdx.x >> 5);
+    if (t >= t_hi) return acc;
+    const int jl = (int)(t * 56u) - 4 + 2 * (int)lane; /* first column of this lane's pair */
+    const bool ld_ok = jl >= 0 && jl < (int)nx;
+    const bool st_ok = ld_ok && lane >= 2 && lane <= 29;
+    const unsigned j = ld_ok ? (unsigned)jl : 0u;
+    /* row r of u(t), r = -1 .. rows+2 (local numbering): the strip and its first halo rows in cur,
+     * the second halo rows in the halo rows of nxt */
+    int r_in = (int)ra - 2;
+    auto fetch = [&]() -> double2 {
+        const double *row = (r_in < 0)                 ? nxt
+                            : (r_in > (int)rows + 1)   ? nxt + (size_t)(rows + 1) * nx
+                                                       : cur + (size_t)r_in * nx;
+        ++r_in;
+        return ld_ok ? *(const double2 *)(row + j) : zero;
+    };
+    double2 a0 = fetch(), b0 = fetch(); /* u(t) rows ra-2, ra-1 */
+    double2 f[DEPTH];
+#pragma unroll
+    for (int s = 0; s < DEPTH; ++s) f[s] = (r_in <= (int)rb + 1) ? fetch() : zero;
+    double ml0 = __shfl_up_sync(full, b0.y, 1), mr0 = __shfl_down_sync(full, b0.x, 1);
+    double2 a1 = zero, b1 = zero; /* u(t+1) rows r-2, r-1 */
+    double ml1 = 0.0, mr1 = 0.0;
+    double *po = nxt + (size_t)ra * nx + j;
+    for (unsigned r = ra - 1; r <= rb; r += DEPTH) { /* r: the u(t+1) row formed in this step */
+#pragma unroll
+        for (int s = 0; s < DEPTH; ++s) {
+            const unsigned rr = r + s;
+            if (rr <= rb) { /* uniform over the warp */
+                const double2 c0 = f[s]; /* u(t) row rr + 1 */
+                if (r_in <= (int)rb + 1) f[s] = fetch();
+                double2 n1 = b0;
+                if (rr != fixed0 && rr != fixed1) {
+                    if (j != 0) n1.x = 0.25 * ((a0.x + c0.x) + (ml0 + b0.y));
+                    if (j + 2 != nx) n1.y = 0.25 * ((a0.y + c0.y) + (b0.x + mr0));
+                }
+                const double nl = __shfl_up_sync(full, n1.y, 1), nr = __shfl_down_sync(full, n1.x, 1);
+                if (rr >= ra + 1) { /* u(t+2) row rr - 1 from u(t+1) rows rr-2, rr-1, rr */
+                    double2 o = b1;
+                    if (rr - 1 != fixed0 && rr - 1 != fixed1) {
+                        if (j != 0) o.x = 0.25 * ((a1.x + n1.x) + (ml1 + b1.y));
+                        if (j + 2 != nx) o.y = 0.25 * ((a1.y + n1.y) + (b1.x + mr1));
+                        if (want_res && st_ok) {
+                            const double dx = o.x - b1.x, dy = o.y - b1.y;
+                            acc += dx * dx;
+                            acc += dy * dy;
+                        }
+                    }
+                    if (st_ok) *(double2 *)po = o;
+                    po += nx;
+                }
+                a1 = b1;
+                b1 = n1;
+                ml1 = nl;
+                mr1 = nr;
+                a0 = b0;
+                b0 = c0;
+                ml0 = __shfl_up_sync(full, c0.y, 1);
+                mr0 = __shfl_down_sync(full, c0.x, 1);
+            }
+        }
+    }
+    return acc;
+}
+
+/* one launch = two sweeps: sender blocks (two rows each way per PE), then one block per band of
+ * `band_rows` rows x 8 tiles of 56 columns, in launch order as in k_jacobi_sweep */
+__global__ void __launch_bounds__(256, 3) k_jacobi_pass2(const ishmem_ctx_t *ctxs, jacobi_args a, int flip,
+                                                          unsigned long long arrived, int last, unsigned band_rows,
+                                                          unsigned bands, unsigned tile_groups, int P, size_t heap_stride)
+{
+    const unsigned tid = threadIdx.x;
+    const size_t nx = a.nx;
+    const unsigned nsend = (unsigned)P * 4u * JACOBI_PIECES;
+    unsigned b = blockIdx.x;
+    if (b < nsend) {
+        jacobi_send_piece(ctxs, flip ? a.buf1 : a.buf0, flip ? a.buf0 : a.buf1, a.sig, a.ny, nx, b);
+        return;
+    }
+    b -= nsend;
+    const int p = (int)(b / (bands * tile_groups));
+    const unsigned band = (b / tile_groups) % bands, tg = b % tile_groups;
+    const ishmem_ctx_t *ctx = ctxs + p;
+    const unsigned base_rows = (unsigned)a.ny / (unsigned)P, extra = (unsigned)a.ny % (unsigned)P;
+    const unsigned rows = base_rows + ((unsigned)p < extra ? 1u : 0u);
+    const unsigned first = (unsigned)p * base_rows + ((unsigned)p < extra ? (unsigned)p : extra);
+    const unsigned ra = 1u + band * band_rows;
+    const unsigned rb = (ra + band_rows < rows + 1u) ? ra + band_rows : rows + 1u;
+    double acc = 0.0;
+    __shared__ int give_up;
+    if (ra < rb) {
+        /* the first band of a strip reads the two halo rows above it, the last one the two below */
+        const bool top = (band == 0 || !a.overlap) && p > 0, bottom = (rb == rows + 1u || !a.overlap) && p + 1 < P;
+        if (top || bottom) {
+            if (tid == 0) {
+                const unsigned long long *sig = (const unsigned long long *)local_of(ctxs, ctx, a.sig);
+                int rc = top ? ishmem_uint64_wait_until(ctx, sig + 0, ISHMEM_CMP_GE, arrived) : 0;
+                if (!rc && bottom) rc = ishmem_uint64_wait_until(ctx, sig + 1, ISHMEM_CMP_GE, arrived);
+                give_up = rc; /* the error is latched by the wait */
+            }
+            __syncthreads();
+            if (give_up) return;
+        }
+        const double *cur = (const double *)((const char *)(flip ? a.buf1 : a.buf0) + (size_t)p * heap_stride);
+        double *nxt = (double *)((char *)(flip ? a.buf0 : a.buf1) + (size_t)p * heap_stride);
+        const unsigned fixed0 = (first == 0) ? 1u : ~0u;
+        const unsigned fixed1 = (first + rows == (unsigned)a.ny) ? rows : ~0u;
+        const unsigned ntiles = (unsigned)((nx + 55) / 56), t_lo = tg * (blockDim.x >> 5);
+        const unsigned t_hi = t_lo + (blockDim.x >> 5) < ntiles ? t_lo + (blockDim.x >> 5) : ntiles;
+        acc = jacobi_march2<3>(cur, nxt, ra, rb, rows, fixed0, fixed1, (unsigned)nx, last != 0, t_lo, t_hi);
+    }
+    if (last) {
         __shared__ double red[8];
         for (int o = 16; o > 0; o >>= 1) acc += __shfl_down_sync(0xffffffffu, acc, o);
         if ((tid & 31u) == 0) red[tid >> 5] = acc;
@@ -855,22 +1007,43 @@ static int jacobi_launch(double *buf0, double *buf1, uint64_t *sig, size_t ny, s
 
 /* one launch per sweep (k_jacobi_sweep); `partial` receives one residual term per tile block */
 #define JACOBI_BAND_ROWS 16u /* measured at 16384^2: 8 rows 687 us, 12: 663, 16: 652, 20: 652, 24: 659, 32: 666, 64: 680 */
-static size_t jacobi_sweep_blocks(size_t ny, size_t nx, unsigned *bands, unsigned *tile_groups)
+/* two sweeps per launch: a band pays four extra rows instead of two, and the pass is bound by
+ * instructions rather than memory, so taller bands win (16384^2, per sweep: 16 rows 501 us, 32: 481,
+ * 64: 469, 128: 461) */
+#define JACOBI_BAND_ROWS2 64u
+static size_t jacobi_sweep_blocks(size_t ny, size_t nx, unsigned *bands, unsigned *tile_groups, unsigned tile_cols = 60)
 {
     auto &g = g_ishmem;
     const size_t rows_max = (ny + g.npes - 1) / g.npes;
-    *bands = (unsigned)((rows_max + JACOBI_BAND_ROWS - 1) / JACOBI_BAND_ROWS);
-    *tile_groups = (unsigned)(((nx + 59) / 60 + 7) / 8);
+    const unsigned band_rows = tile_cols == 60 ? JACOBI_BAND_ROWS : JACOBI_BAND_ROWS2;
+    *bands = (unsigned)((rows_max + band_rows - 1) / band_rows);
+    *tile_groups = (unsigned)(((nx + tile_cols - 1) / tile_cols + 7) / 8);
     return (size_t)g.npes * *bands * *tile_groups;
 }
+/* ISHMEM_JACOBI_FUSE=0 keeps one sweep per launch */
+static bool jacobi_fuse(size_t ny)
+{
+    const char *env = getenv("ISHMEM_JACOBI_FUSE");
+    if (env && atoi(env) == 0) return false;
+    return ny / (size_t)g_ishmem.npes >= 2; /* the second halo row must be a row of the neighbour's strip */
+}
+/* partial: room for jacobi_partial_slots() residual terms; *nterms: how many the last launch wrote */
+static size_t jacobi_partial_slots(size_t ny, size_t nx)
+{
+    unsigned b, t;
+    const size_t one = jacobi_sweep_blocks(ny, nx, &b, &t), two = jacobi_sweep_blocks(ny, nx, &b, &t, 56);
+    return one > two ? one : two;
+}
 static int jacobi_launch_sweeps(double *buf0, double *buf1, uint64_t *sig, size_t ny, size_t nx, int iters, int overlap,
-                                double *partial)
+                                double *partial, size_t *nterms)
 {
     auto &g = g_ishmem;
-    unsigned bands, tile_groups;
+    unsigned bands, tile_groups, bands2, tile_groups2;
     const size_t tile_blocks = jacobi_sweep_blocks(ny, nx, &bands, &tile_groups);
+    const size_t tile_blocks2 = jacobi_sweep_blocks(ny, nx, &bands2, &tile_groups2, 56);
     const size_t nblocks = (size_t)g.npes * 2 * JACOBI_PIECES + tile_blocks;
-    if (nblocks > 0x7fffffffu) return ISHMEM_ERR_ARG;
+    const size_t nblocks2 = (size_t)g.npes * 4 * JACOBI_PIECES + tile_blocks2;
+    if (nblocks > 0x7fffffffu || nblocks2 > 0x7fffffffu) return ISHMEM_ERR_ARG;
     cudaStream_t s;
     int rc = ishmemi_team_stream_begin(ISHMEM_TEAM_WORLD, &s);
     if (rc) return rc;
@@ -884,9 +1057,29 @@ static int jacobi_launch_sweeps(double *buf0, double *buf1, uint64_t *sig, size_
     a.overlap = overlap;
     a.partial = partial;
     a.sliding = 1;
-    for (int it = 0; it < iters && !rc; ++it) {
-        k_jacobi_sweep<<<(unsigned)nblocks, 256, 0, s>>>(g.d_ctx, a, it, JACOBI_BAND_ROWS, bands, tile_groups, g.npes,
-                                                         g.heap_bytes);
+    /* Every launch moves the grid from one buffer to the other, and the result has to end up where
+     * `iters` single sweeps would leave it (buf0 for an even count): an even number of two-sweep
+     * passes, then one to three single sweeps. */
+    int fused = jacobi_fuse(ny) ? iters / 2 : 0;
+    if (fused & 1) --fused;
+    int flip = 0, done = 0;
+    unsigned long long arrived = 0;
+    *nterms = 0;
+    while (done < iters && !rc) {
+        *nterms = fused > 0 ? tile_blocks2 : tile_blocks;
+        if (fused > 0) {
+            arrived += 2 * JACOBI_PIECES;
+            k_jacobi_pass2<<<(unsigned)nblocks2, 256, 0, s>>>(g.d_ctx, a, flip, arrived, done + 2 == iters, JACOBI_BAND_ROWS2,
+                                                              bands2, tile_groups2, g.npes, g.heap_bytes);
+            --fused;
+            done += 2;
+        } else {
+            arrived += JACOBI_PIECES;
+            k_jacobi_sweep<<<(unsigned)nblocks, 256, 0, s>>>(g.d_ctx, a, flip, arrived, done + 1 == iters, JACOBI_BAND_ROWS,
+                                                             bands, tile_groups, g.npes, g.heap_bytes);
+            done += 1;
+        }
+        flip ^= 1;
         ishmemi_count_launch();
         rc = ishmemi_check_launch("k_jacobi_sweep");
     }
@@ -911,17 +1104,16 @@ extern "C" int ishmemx_jacobi(double *buf0, double *buf1, uint64_t *sig, size_t 
     int rc = jacobi_check(buf0, buf1, sig, ny, nx, iters, &groups_per_pe, threads, &by_columns);
     if (rc) return rc;
     if (jacobi_per_sweep(threads, nx)) {
-        unsigned bands, tile_groups;
-        const size_t tile_blocks = jacobi_sweep_blocks(ny, nx, &bands, &tile_groups);
         double *partial = nullptr;
-        ISHMEMI_CUDA(cudaMalloc((void **)&partial, tile_blocks * 8));
-        rc = jacobi_launch_sweeps(buf0, buf1, sig, ny, nx, iters, overlap, partial);
+        size_t nterms = 0;
+        ISHMEMI_CUDA(cudaMalloc((void **)&partial, jacobi_partial_slots(ny, nx) * 8));
+        rc = jacobi_launch_sweeps(buf0, buf1, sig, ny, nx, iters, overlap, partial, &nterms);
         if (!rc && residual_sq_host) {
             double sum = 0.0;
-            if (iters > 0) {
-                std::vector<double> part(tile_blocks);
-                rc = ishmemi_cuda(cudaMemcpy(part.data(), partial, tile_blocks * 8, cudaMemcpyDeviceToHost), "cudaMemcpy");
-                for (size_t i = 0; i < tile_blocks; ++i) sum += part[i];
+            if (nterms) {
+                std::vector<double> part(nterms);
+                rc = ishmemi_cuda(cudaMemcpy(part.data(), partial, nterms * 8, cudaMemcpyDeviceToHost), "cudaMemcpy");
+                for (size_t i = 0; i < nterms; ++i) sum += part[i];
             }
             *residual_sq_host = sum;
         }

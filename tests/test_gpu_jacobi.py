@@ -40,7 +40,7 @@ def run_gpu(grid, npes, iters, overlap, groups, threads):
         return out, res[0]
 
 
-@pytest.mark.parametrize("split", ["sweeps", "columns", "rows"])
+@pytest.mark.parametrize("split", ["sweeps", "single_sweeps", "columns", "rows"])
 @pytest.mark.parametrize("overlap", [1, 0])
 @pytest.mark.parametrize("ny,nx,npes,groups,threads", [
     (64, 48, 12, 1, 128), (200, 131, 12, 3, 128), (257, 33, 5, 4, 128),       # odd nx: row-by-row path
@@ -50,9 +50,11 @@ def run_gpu(grid, npes, iters, overlap, groups, threads):
     (36, 600, 12, 12, 32), (50, 121, 4, 3, 64)])                               # one tile per block; odd nx by columns
 def test_jacobi_matches_oracle(ny, nx, npes, groups, threads, overlap, split, monkeypatch):
     """split: the persistent kernel with the strips cut by columns or by rows, or `sweeps`: the form the
-    library picks by itself for threads = 0 and even nx (one launch per sweep, one tile per warp)."""
-    if split == "sweeps":
+    library picks by itself for threads = 0 and even nx (one tile per warp, two sweeps per launch where the
+    count allows), or the same with one sweep per launch."""
+    if split in ("sweeps", "single_sweeps"):
         monkeypatch.delenv("ISHMEM_JACOBI_SPLIT", raising=False)
+        monkeypatch.setenv("ISHMEM_JACOBI_FUSE", "1" if split == "sweeps" else "0")
         threads = 0
     else:
         monkeypatch.setenv("ISHMEM_JACOBI_SPLIT", split)
@@ -75,10 +77,11 @@ def test_jacobi_default_split_and_repeated_calls():
 
 
 def test_jacobi_per_sweep_many_bands_and_residual():
-    """The per-sweep form on strips of several 32-row bands and tile groups, with strips of unequal length,
-    odd and even iteration counts; final grid bit-exact, residual within 1e-6 relative."""
+    """The launch-per-sweep form on strips of several bands and tile groups, with strips of unequal length and
+    iteration counts that end in a two-sweep pass or in one to three single sweeps; final grid bit-exact,
+    residual within 1e-6 relative."""
     grid = inputs.jacobi_grid(inputs.SEED_C5, 1000, 1100)
-    for npes, iters in ((7, 5), (3, 12), (1, 3)):
+    for npes, iters in ((7, 5), (3, 12), (1, 3), (5, 8), (12, 4), (2, 10)):     # 2, 6, 0, 4, 2, 4 two-sweep passes
         exp, exp_res = orc.jacobi(grid, iters)
         got, res = run_gpu(grid, npes, iters, 1, 1, 0)
         assert got.tobytes() == exp.tobytes(), (npes, iters)
