@@ -222,7 +222,9 @@ ISHMEM_DECL_STRIDED(uint64, uint64_t)
  * `level` = ISHMEMX_WORK_ITEM..ISHMEMX_WORK_GROUP_ENGINE) and every unit calls the device
  * routine ishmem_putmem / ishmemx_putmem_sub_group / ishmemx_putmem_work_group /
  * ishmemx_putmem_engine_work_group once on its slice.  threads in 1..1024, groups >= 1.
- * ISHMEMX_WORK_GROUP_ENGINE needs a running proxy (ISHMEM_ERR_ARG otherwise). */
+ * ISHMEMX_WORK_GROUP_ENGINE needs a running proxy (ISHMEM_ERR_ARG otherwise) and blocks the host
+ * until the kernel has finished: nothing may be queued behind a kernel that waits for the proxy
+ * (see ishmemx_proxy_start). */
 int ishmemx_putmem_on_device(int my_pe, void *dest, const void *src, size_t nbytes, int pe,
                              int level, int threads, int groups);
 int ishmemx_getmem_on_device(int my_pe, void *dest, const void *src, size_t nbytes, int pe,
@@ -516,12 +518,16 @@ int ishmemx_rma_latency(int my_pe, void *dest, const void *src, size_t nbytes, i
  * symmetric, (ceil(ny/npes)+2)*nx doubles each, strip row r at local row r+1 of buf0 on entry
  * (buf1 is overwritten); sig: symmetric, 4 words, zero on entry.  overlap = 0 disables the
  * interior-first ordering (exchange, wait, then compute).
- * threads = 0 (and an even nx): the library shapes the launches itself -- ONE LAUNCH PER SWEEP, whose
+ * threads = 0 (and an even nx): the library shapes the launches itself -- many short launches whose
  * first blocks send the halo rows (in-kernel work-group put_signal) and whose other blocks each
- * take 16 rows of 8 neighbouring 60-column tiles, numbered so that the blocks sweep the grid in
- * launch order; only the first and the last band of a strip wait for a halo, the interior never
- * does.  This is the fastest form (6.6 TB/s at 16384^2); groups_per_pe is not used by it and
- * nothing needs to be co-resident.
+ * take a band of rows of 8 neighbouring column tiles, one warp per tile, numbered so that the
+ * blocks sweep the grid in launch order; only the first and the last band of a strip wait for a
+ * halo, the interior never does.  Where the count allows, a launch does TWO sweeps (every element
+ * read once, the second result written once; two halo rows each way, the second one parked in the
+ * halo row of the buffer being written) -- an even number of such passes, then one to three
+ * single-sweep launches, so that the result ends in the buffer named below; 455 us per sweep at
+ * 16384^2 (single sweeps only, ISHMEM_JACOBI_FUSE=0: 652 us = the copy rate).  groups_per_pe is
+ * not used by this form and nothing needs to be co-resident.
  * threads > 0 (a multiple of 32 up to 1024): one persistent co-resident launch of
  * npes x groups_per_pe blocks of that size for all sweeps; the blocks of a PE take bands of rows,
  * one of them sends each halo row, and neighbouring blocks hand over through flags.

@@ -194,11 +194,26 @@ static int launch_rma(cudaStream_t s, rma_args a, int level, int threads, unsign
     case ISHMEMX_WORK_GROUP_ENGINE:
         if (g_ishmem.h_ctx[0].proxy == nullptr) return ISHMEM_ERR_ARG; /* no host proxy running */
         k_rma<ISHMEMX_WORK_GROUP_ENGINE><<<blocks, threads, 0, s>>>(ctxs, a);
-        break;
+        /* This kernel waits for the host proxy, and the proxy's copy needs a free hardware queue:
+         * work enqueued behind the kernel can end up in front of that copy (streams share the
+         * queues), which would stall both until the wait gives up.  So the call returns only when
+         * the kernel has finished -- nothing can be queued behind it. */
+        ishmemi_count_launch();
+        {
+            int rc = ishmemi_check_launch("k_rma");
+            if (rc) return rc;
+        }
+        return ishmemi_cuda(cudaStreamSynchronize(s), "cudaStreamSynchronize(engine level)");
     default: return ISHMEM_ERR_ARG;
     }
     ishmemi_count_launch();
-    return ishmemi_check_launch("k_rma");
+    int rc = ishmemi_check_launch("k_rma");
+    /* a work-group slice at or above the device-side cutover goes to the proxy as well: same rule */
+    const bool may_wait_for_proxy = (level == ISHMEMX_WORK_GROUP || level == ISHMEMX_WORK_GROUP_BULK) &&
+                                    g_ishmem.h_ctx[0].proxy != nullptr && g_ishmem.wg_cutover != (size_t)-1 &&
+                                    a.nbytes >= g_ishmem.wg_cutover;
+    if (!rc && may_wait_for_proxy) rc = ishmemi_cuda(cudaStreamSynchronize(s), "cudaStreamSynchronize(cutover)");
+    return rc;
 }
 
 /* Validates one RMA request and resolves addresses: the symmetric side must lie in the heap;

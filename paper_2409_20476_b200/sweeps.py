@@ -488,16 +488,18 @@ def sweep_c5(args, out):
     import os
     # (variant, ISHMEM_JACOBI_SPLIT, threads, groups): the library's own choice (one launch per sweep), the
     # persistent kernel with strips cut by column tiles, and the persistent kernel with caller-shaped blocks
-    variants = [("per_sweep_tiles", None, 0, 1)]
+    variants = [("launch_per_two_sweeps", None, 0, 1), ("launch_per_sweep", "single", 0, 1)]
     variants += [("persistent_columns", "columns", 0, g) for g in (6, 12)]
     variants += [("persistent_rows", "rows", t, g) for g in (6, 12, 24) for t in (256, 512, 1024)]
     for overlap in (1, 0):
         for variant, split, threads, groups in variants:
             if npes * groups * threads > 148 * 2048:
                 continue
-            if split is None:
-                os.environ.pop("ISHMEM_JACOBI_SPLIT", None)
-            else:
+            os.environ.pop("ISHMEM_JACOBI_SPLIT", None)
+            os.environ.pop("ISHMEM_JACOBI_FUSE", None)
+            if split == "single":
+                os.environ["ISHMEM_JACOBI_FUSE"] = "0"
+            elif split is not None:
                 os.environ["ISHMEM_JACOBI_SPLIT"] = split
             for p in range(npes):
                 for w in range(4):
@@ -518,6 +520,7 @@ def sweep_c5(args, out):
                     groups=groups, npes=npes, dtype="f64", nbytes=n * n * 8, l2="cold", iters=iters, us_per_op=us,
                     alg_bytes=16 * n * n, note=f"per sweep; residual_sq {res[0]:.6e} (grid keeps evolving)")
     os.environ.pop("ISHMEM_JACOBI_SPLIT", None)
+    os.environ.pop("ISHMEM_JACOBI_FUSE", None)
     assert B.ishmemx_status(1) == 0
     B.ishmem_finalize()
 
@@ -640,7 +643,7 @@ def summarize(path) -> str:
                 "|---|---|---:|---:|---:|---:|---:|---:|"]
         for r in rows:
             form, ov = r["variant"].rsplit(" overlap=", 1) if " overlap=" in r["variant"] else ("", r["variant"][-1])
-            shape = f"| {form} | {ov} | {r['threads'] if r['threads'] != '0' else 'library'} | {r['groups'] if form != 'per_sweep_tiles' else '-'} |"
+            shape = f"| {form} | {ov} | {r['threads'] if r['threads'] != '0' else 'library'} | {r['groups'] if not form.startswith('launch_per') else '-'} |"
             if r["us_per_op"]:
                 out.append(f"{shape} {us(r)} | {gb(r)} | {r['frac_hbm']} | {r['frac_8tbs']} |")
             else:

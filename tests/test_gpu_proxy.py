@@ -174,7 +174,7 @@ def test_cutover_tuned_from_measurement():
 def test_many_work_groups_post_at_once():
     """296 work-groups (37 per PE) each post one slice of an 8 MiB message at the same time and
     quiet on their PE's completion counter; ring pattern, whole output checked on the device,
-    twice in a row (the second launch is queued behind the first)."""
+    twice in a row."""
     npes, n = 8, 8 << 20
     with Session(npes, 2 * n + (1 << 20), with_oracle=False) as s:
         src, dst = s.malloc(n), s.malloc(n)
