@@ -501,9 +501,17 @@ def sweep_c5(args, out):
                 os.environ["ISHMEM_JACOBI_FUSE"] = "0"
             elif split is not None:
                 os.environ["ISHMEM_JACOBI_SPLIT"] = split
-            for p in range(npes):
-                for w in range(4):
-                    B.ishmem_uint64_p(p, sig + 8 * w, 0, p)
+            def reset_signals():
+                for p in range(npes):
+                    for w in range(4):
+                        B.ishmem_uint64_p(p, sig + 8 * w, 0, p)
+            try:
+                # a short untimed call first: the first launch of a kernel in a process loads its code
+                reset_signals()
+                B.ishmemx_jacobi(b0, b1, sig, n, n, 6, overlap, groups, threads, res)
+            except B.IshmemError:
+                pass
+            reset_signals()
             a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             torch.cuda.synchronize()
             a.record(stream)
