@@ -320,6 +320,9 @@ def breakdown(B, torch, team_stream, env) -> dict:
                                                                           NOPS_CAS, 256, 1),
         "compare_swap_no_aggregation": lambda: B.ishmemx_int64_atomic_compare_swap_batch(table, cword, ccond, cval,
                                                                                          fetched, NOPS_CAS, 256, 0),
+        "jacobi": lambda: (B.ishmemx_putmem_spmd(env["jsig"], env["zeros"], 32, 0, B.ISHMEMX_WORK_GROUP, 32, 1),
+                           B.ishmemx_jacobi(env["jb0"], env["jb1"], env["jsig"], S["jacobi_n"], S["jacobi_n"],
+                                            S["jacobi_sweeps"], 1, args.jacobi_groups, 0, None)),
     }
     res = {}
     for name, fn in ops.items():
