@@ -88,6 +88,18 @@ def test_jacobi_per_sweep_many_bands_and_residual():
         assert abs(res - exp_res) <= 1e-6 * exp_res
 
 
+def test_jacobi_two_sweep_passes_on_the_shortest_strips():
+    """Strips of two and three rows: the second halo row of a neighbour is its first or last row but one, and a
+    strip's single band is both its first and its last; 4 and 8 sweeps are all two-sweep passes."""
+    for ny, nx, npes in ((24, 120, 12), (31, 232, 10), (8, 64, 4)):
+        grid = inputs.jacobi_grid(inputs.SEED_C5, ny, nx)
+        for iters in (4, 8, 9):
+            exp, exp_res = orc.jacobi(grid, iters)
+            got, res = run_gpu(grid, npes, iters, 1, 1, 0)
+            assert got.tobytes() == exp.tobytes(), (ny, nx, npes, iters)
+            assert abs(res - exp_res) <= 1e-6 * exp_res
+
+
 def test_jacobi_even_iterations_and_zero():
     grid = inputs.jacobi_grid(inputs.SEED_C5, 96, 64)
     for iters in (0, 1, 2, 10):
