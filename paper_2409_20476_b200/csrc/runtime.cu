@@ -217,9 +217,10 @@ static int init_common(int npes, size_t heap_bytes, void *external)
     g.used_blocks.clear();
     g.free_blocks[0] = heap_bytes;
     /* default cutovers, from the committed size sweep on B200 (ishmemx_tune_cutover re-measures):
-     * a host-initiated put/get of one PE is at least as fast on the copy engine from 4 MiB on
-     * (5.8 against 6.1 us there, 6.3 against 5.6 TB/s at 256 MiB); the push collectives and
-     * the device-initiated work-group calls never are, so they stay on loads and stores */
+     * a host-initiated put/get of one PE is faster on the copy engine from 4 to 32 MiB (5.9 against
+     * 6.2 us at 4 MiB, 9.3 against 12.3 us at 32 MiB, back-to-back calls) and within a few per cent
+     * of the tiled kernel above that, while leaving the SMs free; the push collectives and the
+     * device-initiated work-group calls never gain, so they stay on loads and stores */
     g.cutover[0] = (size_t)4 << 20;
     g.cutover[1] = g.cutover[2] = g.wg_cutover = (size_t)-1;
     env_size("ISHMEM_CUTOVER_PUT", &g.cutover[0]);
