@@ -858,9 +858,103 @@ __device__ __forceinline__ double jacobi_march2(const double *cur, double *nxt, 
     return acc;
 }
 
+/* The two-level window with FOUR columns per lane (two pairs, A and B): a tile is 128 loaded and 120
+ * stored columns, the neighbours inside a lane cost nothing, and only the lane's outer neighbours
+ * travel by shuffle -- half the shuffles per cell of jacobi_march2, and 6 % instead of 12 % of the
+ * columns computed twice. */
+template <int DEPTH>
+__device__ __forceinline__ double jacobi_march2w(const double *cur, double *nxt, unsigned ra, unsigned rb, unsigned rows,
+                                                 unsigned fixed0, unsigned fixed1, unsigned nx, bool want_res,
+                                                 unsigned t_lo, unsigned t_hi)
+{
+    double acc = 0.0;
+    if (rb <= ra) return acc;
+    const unsigned lane = threadIdx.x & 31u;
+    const unsigned full = 0xffffffffu;
+    const double2 zero = make_double2(0.0, 0.0);
+    const unsigned t = t_lo + (threadIdx.x >> 5);
+    if (t >= t_hi) return acc;
+    const int jA = (int)(t * 120u) - 4 + 4 * (int)lane, jB = jA + 2; /* first columns of this lane's two pairs */
+    const bool okA = jA >= 0 && jA < (int)nx, okB = jB >= 0 && jB < (int)nx;
+    const bool stA = okA && lane >= 1 && lane <= 30, stB = okB && lane >= 1 && lane <= 30;
+    int r_in = (int)ra - 2;
+    auto fetch = [&](double2 &A, double2 &B) {
+        const double *row = (r_in < 0)               ? nxt
+                            : (r_in > (int)rows + 1) ? nxt + (size_t)(rows + 1) * nx
+                                                     : cur + (size_t)r_in * nx;
+        ++r_in;
+        A = okA ? *(const double2 *)(row + jA) : zero;
+        B = okB ? *(const double2 *)(row + jB) : zero;
+    };
+    double2 a0A, a0B, b0A, b0B;
+    fetch(a0A, a0B);
+    fetch(b0A, b0B);
+    double2 fA[DEPTH], fB[DEPTH];
+#pragma unroll
+    for (int s = 0; s < DEPTH; ++s) {
+        fA[s] = fB[s] = zero;
+        if (r_in <= (int)rb + 1) fetch(fA[s], fB[s]);
+    }
+    double ml0 = __shfl_up_sync(full, b0B.y, 1), mr0 = __shfl_down_sync(full, b0A.x, 1);
+    double2 a1A = zero, a1B = zero, b1A = zero, b1B = zero;
+    double ml1 = 0.0, mr1 = 0.0;
+    double *po = nxt + (size_t)ra * nx + (okA ? jA : 0);
+    for (unsigned r = ra - 1; r <= rb; r += DEPTH) {
+#pragma unroll
+        for (int s = 0; s < DEPTH; ++s) {
+            const unsigned rr = r + s;
+            if (rr <= rb) {
+                const double2 c0A = fA[s], c0B = fB[s];
+                if (r_in <= (int)rb + 1) fetch(fA[s], fB[s]);
+                double2 n1A = b0A, n1B = b0B;
+                if (rr != fixed0 && rr != fixed1) {
+                    if (jA != 0) n1A.x = 0.25 * ((a0A.x + c0A.x) + (ml0 + b0A.y));
+                    if (jA + 2 != (int)nx) n1A.y = 0.25 * ((a0A.y + c0A.y) + (b0A.x + b0B.x));
+                    n1B.x = 0.25 * ((a0B.x + c0B.x) + (b0A.y + b0B.y));
+                    if (jB + 2 != (int)nx) n1B.y = 0.25 * ((a0B.y + c0B.y) + (b0B.x + mr0));
+                }
+                const double nl = __shfl_up_sync(full, n1B.y, 1), nr = __shfl_down_sync(full, n1A.x, 1);
+                if (rr >= ra + 1) {
+                    double2 oA = b1A, oB = b1B;
+                    if (rr - 1 != fixed0 && rr - 1 != fixed1) {
+                        if (jA != 0) oA.x = 0.25 * ((a1A.x + n1A.x) + (ml1 + b1A.y));
+                        if (jA + 2 != (int)nx) oA.y = 0.25 * ((a1A.y + n1A.y) + (b1A.x + b1B.x));
+                        oB.x = 0.25 * ((a1B.x + n1B.x) + (b1A.y + b1B.y));
+                        if (jB + 2 != (int)nx) oB.y = 0.25 * ((a1B.y + n1B.y) + (b1B.x + mr1));
+                        if (want_res) {
+                            if (stA) {
+                                const double dx = oA.x - b1A.x, dy = oA.y - b1A.y;
+                                acc += dx * dx;
+                                acc += dy * dy;
+                            }
+                            if (stB) {
+                                const double dx = oB.x - b1B.x, dy = oB.y - b1B.y;
+                                acc += dx * dx;
+                                acc += dy * dy;
+                            }
+                        }
+                    }
+                    if (stA) *(double2 *)po = oA;
+                    if (stB) *(double2 *)(po + 2) = oB;
+                    po += nx;
+                }
+                a1A = b1A, a1B = b1B;
+                b1A = n1A, b1B = n1B;
+                ml1 = nl, mr1 = nr;
+                a0A = b0A, a0B = b0B;
+                b0A = c0A, b0B = c0B;
+                ml0 = __shfl_up_sync(full, c0B.y, 1);
+                mr0 = __shfl_down_sync(full, c0A.x, 1);
+            }
+        }
+    }
+    return acc;
+}
+
 /* one launch = two sweeps: sender blocks (two rows each way per PE), then one block per band of
  * `band_rows` rows x 8 tiles of 56 columns, in launch order as in k_jacobi_sweep */
-__global__ void __launch_bounds__(256, 3) k_jacobi_pass2(const ishmem_ctx_t *ctxs, jacobi_args a, int flip,
+template <bool WIDE>
+__global__ void __launch_bounds__(256, WIDE ? 2 : 3) k_jacobi_pass2(const ishmem_ctx_t *ctxs, jacobi_args a, int flip,
                                                           unsigned long long arrived, int last, unsigned band_rows,
                                                           unsigned bands, unsigned tile_groups, int P, size_t heap_stride)
 {
@@ -900,9 +994,10 @@ __global__ void __launch_bounds__(256, 3) k_jacobi_pass2(const ishmem_ctx_t *ctx
         double *nxt = (double *)((char *)(flip ? a.buf0 : a.buf1) + (size_t)p * heap_stride);
         const unsigned fixed0 = (first == 0) ? 1u : ~0u;
         const unsigned fixed1 = (first + rows == (unsigned)a.ny) ? rows : ~0u;
-        const unsigned ntiles = (unsigned)((nx + 55) / 56), t_lo = tg * (blockDim.x >> 5);
+        const unsigned ntiles = (unsigned)((nx + (WIDE ? 119 : 55)) / (WIDE ? 120 : 56)), t_lo = tg * (blockDim.x >> 5);
         const unsigned t_hi = t_lo + (blockDim.x >> 5) < ntiles ? t_lo + (blockDim.x >> 5) : ntiles;
-        acc = jacobi_march2<3>(cur, nxt, ra, rb, rows, fixed0, fixed1, (unsigned)nx, last != 0, t_lo, t_hi);
+        acc = WIDE ? jacobi_march2w<2>(cur, nxt, ra, rb, rows, fixed0, fixed1, (unsigned)nx, last != 0, t_lo, t_hi)
+                   : jacobi_march2<3>(cur, nxt, ra, rb, rows, fixed0, fixed1, (unsigned)nx, last != 0, t_lo, t_hi);
     }
     if (last) {
         __shared__ double red[8];
@@ -1040,7 +1135,15 @@ static int jacobi_launch_sweeps(double *buf0, double *buf1, uint64_t *sig, size_
     auto &g = g_ishmem;
     unsigned bands, tile_groups, bands2, tile_groups2;
     const size_t tile_blocks = jacobi_sweep_blocks(ny, nx, &bands, &tile_groups);
-    const size_t tile_blocks2 = jacobi_sweep_blocks(ny, nx, &bands2, &tile_groups2, 56);
+    /* four columns per lane (120-column tiles, 118 registers, two blocks per SM): 428 against 454 us per
+     * 16384^2 sweep for two columns per lane (56-column tiles), which ISHMEM_JACOBI_WIDE=0 selects */
+    bool wide = !(getenv("ISHMEM_JACOBI_WIDE") && atoi(getenv("ISHMEM_JACOBI_WIDE")) == 0);
+    /* ... unless the grid is too small to give every SM a few of the larger blocks (the variable
+     * set to 1 keeps the wide form regardless) */
+    if (wide && !getenv("ISHMEM_JACOBI_WIDE") &&
+        jacobi_sweep_blocks(ny, nx, &bands2, &tile_groups2, 120) < (size_t)g.sm_count * 4)
+        wide = false;
+    const size_t tile_blocks2 = jacobi_sweep_blocks(ny, nx, &bands2, &tile_groups2, wide ? 120 : 56);
     const size_t nblocks = (size_t)g.npes * 2 * JACOBI_PIECES + tile_blocks;
     const size_t nblocks2 = (size_t)g.npes * 4 * JACOBI_PIECES + tile_blocks2;
     if (nblocks > 0x7fffffffu || nblocks2 > 0x7fffffffu) return ISHMEM_ERR_ARG;
@@ -1069,8 +1172,14 @@ static int jacobi_launch_sweeps(double *buf0, double *buf1, uint64_t *sig, size_
         *nterms = fused > 0 ? tile_blocks2 : tile_blocks;
         if (fused > 0) {
             arrived += 2 * JACOBI_PIECES;
-            k_jacobi_pass2<<<(unsigned)nblocks2, 256, 0, s>>>(g.d_ctx, a, flip, arrived, done + 2 == iters, JACOBI_BAND_ROWS2,
-                                                              bands2, tile_groups2, g.npes, g.heap_bytes);
+            if (wide)
+                k_jacobi_pass2<true><<<(unsigned)nblocks2, 256, 0, s>>>(g.d_ctx, a, flip, arrived, done + 2 == iters,
+                                                                        JACOBI_BAND_ROWS2, bands2, tile_groups2, g.npes,
+                                                                        g.heap_bytes);
+            else
+                k_jacobi_pass2<false><<<(unsigned)nblocks2, 256, 0, s>>>(g.d_ctx, a, flip, arrived, done + 2 == iters,
+                                                                         JACOBI_BAND_ROWS2, bands2, tile_groups2, g.npes,
+                                                                         g.heap_bytes);
             --fused;
             done += 2;
         } else {

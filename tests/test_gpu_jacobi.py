@@ -40,7 +40,7 @@ def run_gpu(grid, npes, iters, overlap, groups, threads):
         return out, res[0]
 
 
-@pytest.mark.parametrize("split", ["sweeps", "single_sweeps", "columns", "rows"])
+@pytest.mark.parametrize("split", ["sweeps", "sweeps_two_columns_per_lane", "single_sweeps", "columns", "rows"])
 @pytest.mark.parametrize("overlap", [1, 0])
 @pytest.mark.parametrize("ny,nx,npes,groups,threads", [
     (64, 48, 12, 1, 128), (200, 131, 12, 3, 128), (257, 33, 5, 4, 128),       # odd nx: row-by-row path
@@ -51,10 +51,11 @@ def run_gpu(grid, npes, iters, overlap, groups, threads):
 def test_jacobi_matches_oracle(ny, nx, npes, groups, threads, overlap, split, monkeypatch):
     """split: the persistent kernel with the strips cut by columns or by rows, or `sweeps`: the form the
     library picks by itself for threads = 0 and even nx (one tile per warp, two sweeps per launch where the
-    count allows), or the same with one sweep per launch."""
-    if split in ("sweeps", "single_sweeps"):
+    count allows, four columns per lane), the same with two columns per lane, or with one sweep per launch."""
+    if split in ("sweeps", "sweeps_two_columns_per_lane", "single_sweeps"):
         monkeypatch.delenv("ISHMEM_JACOBI_SPLIT", raising=False)
-        monkeypatch.setenv("ISHMEM_JACOBI_FUSE", "1" if split == "sweeps" else "0")
+        monkeypatch.setenv("ISHMEM_JACOBI_FUSE", "0" if split == "single_sweeps" else "1")
+        monkeypatch.setenv("ISHMEM_JACOBI_WIDE", "0" if split == "sweeps_two_columns_per_lane" else "1")
         threads = 0
     else:
         monkeypatch.setenv("ISHMEM_JACOBI_SPLIT", split)
