@@ -525,8 +525,9 @@ int ishmemx_rma_latency(int my_pe, void *dest, const void *src, size_t nbytes, i
  * halo, the interior never does.  Where the count allows, a launch does TWO sweeps (every element
  * read once, the second result written once; two halo rows each way, the second one parked in the
  * halo row of the buffer being written) -- an even number of such passes, then one to three
- * single-sweep launches, so that the result ends in the buffer named below; 455 us per sweep at
- * 16384^2 (single sweeps only, ISHMEM_JACOBI_FUSE=0: 652 us = the copy rate).  groups_per_pe is
+ * single-sweep launches, so that the result ends in the buffer named below; 428 us per sweep at
+ * 16384^2 (single sweeps only, ISHMEM_JACOBI_FUSE=0: 650 us = the copy rate; ISHMEM_JACOBI_WIDE=0:
+ * two instead of four columns per lane in the two-sweep launches).  groups_per_pe is
  * not used by this form and nothing needs to be co-resident.
  * threads > 0 (a multiple of 32 up to 1024): one persistent co-resident launch of
  * npes x groups_per_pe blocks of that size for all sweeps; the blocks of a PE take bands of rows,
