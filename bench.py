@@ -508,14 +508,14 @@ def run_profile_case(args) -> dict:
 
 
 def run_profile_jacobi(args) -> dict:
-    """Small Jacobi case for profiler captures: 8 PEs, 2048 x 16384 float64 (full-width rows as in config 5,
-    two buffers of 256 MiB: larger than L2), `--steps` launches of 4 sweeps each; with --jacobi-groups 17 or
-    fewer the library splits the strips by columns, as it does at full size."""
+    """Small Jacobi case for profiler captures: 8 PEs, 4096 x 16384 float64 (full-width rows as in config 5,
+    two buffers of 512 MiB: larger than L2, and enough blocks for the launch shape used at full size),
+    `--steps` calls of 4 sweeps each (two launches of two sweeps)."""
     import torch
     from paper_2409_20476_b200 import binding as B
     from paper_2409_20476_b200 import inputs
 
-    ny, nx, sweeps = 2048, 16384, 4
+    ny, nx, sweeps = 4096, 16384, 4
     rows = ny // NPES
     nbytes = (rows + 2) * nx * 8
     heap_bytes = 2 * nbytes + MiB
