@@ -191,7 +191,7 @@ ISHMEM_DECL_RMA(uint32, uint32_t)
 ISHMEM_DECL_RMA(uint64, uint64_t)
 #undef ISHMEM_DECL_RMA
 
-/* Strided put / get (OpenSHMEM iput / iget; Section 3.7.1, "blocked or strided"): element k of
+/* Strided put / get (OpenSHMEM iput / iget; the strided form that Section 3.7.1 lists): element k of
  * the source, taken every `sst` elements, becomes element k*dst of the destination, k = 0 ..
  * nelems-1.  Strides are in elements and at least 1; elem_size is 1, 2, 4, 8 or 16 bytes and both
  * addresses must be aligned to it.  Symmetric side and ordering as for ishmem_putmem /
@@ -462,7 +462,7 @@ ISHMEM_DECL_REDUCE_BITS(int32, int32_t)
 ISHMEM_DECL_REDUCE_BITS(int64, int64_t)
 ISHMEM_DECL_REDUCE_BITS(uint32, uint32_t)
 ISHMEM_DECL_REDUCE_BITS(uint64, uint64_t)
-/* "fixed-point datatypes from 8 to 64 bits" (Section 3.7.2): sum and product modulo 2^8 / 2^16 */
+/* Integer types of 8 to 64 bits (Section 3.7.2): sum and product modulo 2^8 / 2^16 */
 ISHMEM_DECL_REDUCE_ARITH(int8, int8_t)
 ISHMEM_DECL_REDUCE_ARITH(uint8, uint8_t)
 ISHMEM_DECL_REDUCE_ARITH(int16, int16_t)

@@ -21,9 +21,11 @@
  * fcollect / broadcast, numpy wrap-around sums (also for 8- and 16-bit elements), numpy strided
  * slices for iput / iget, np.concatenate for collect, a block transpose for alltoall (with its
  * involution property), conservation and chain checks
- * for atomics, Jacobi eigenmode decay and decomposition independence.
- * "parity unpinned": oracle_test (the comparison of wait_until) beyond its truth
- * table, and the root-writes-dest reading of broadcast (both readings offered).
+ * for atomics, hand-worked allocator offsets, the truth table of oracle_test,
+ * Jacobi eigenmode decay, decomposition independence and a hand case that fixes
+ * the association order of the update.
+ * "parity unpinned": the root-writes-dest reading of broadcast (the OpenSHMEM
+ * text is not at hand; both readings are offered and tested).
  *
  * Build: gcc -O2 -ffp-contract=off -fno-fast-math -shared -fPIC
  */
@@ -163,7 +165,7 @@ int oracle_getmem(oracle_t *o, int my_pe, void *dest, size_t src_off, size_t n, 
     return ORACLE_OK;
 }
 
-/* strided put (OpenSHMEM iput; "put ... that are blocked or strided", Section 3.7.1): element k
+/* strided put (OpenSHMEM iput; the strided form of put that Section 3.7.1 lists): element k
  * of the source, taken every `sst` elements from `src`, becomes element k*dst of the symmetric
  * object at `dest_off` on PE `pe`, k = 0..nelems-1.  Elements are `esize` bytes; strides are in
  * elements and at least 1. */
@@ -396,8 +398,8 @@ int oracle_fcollectmem(oracle_t *o, int t_start, int t_stride, int t_size, size_
     return ORACLE_OK;
 }
 
-/* collect: like fcollect with contributions of different sizes ("collect (which is like MPI
- * allgather)", Section 3.7.2) -- every member's dest is the concatenation, in team order, of
+/* collect: like fcollect with contributions of different sizes (Section 3.7.2 likens it to MPI's
+ * allgather) -- every member's dest is the concatenation, in team order, of
  * the members' sources; member i contributes nbytes[i] bytes. */
 int oracle_collectmem(oracle_t *o, int t_start, int t_stride, int t_size, size_t dest_off,
                       size_t src_off, const size_t *nbytes)
@@ -474,7 +476,7 @@ COMBINE_INT(int32_t, uint32_t)
 COMBINE_INT(int64_t, uint64_t)
 COMBINE_INT(uint32_t, uint32_t)
 COMBINE_INT(uint64_t, uint64_t)
-/* 8- and 16-bit elements ("fixed-point datatypes from 8 to 64 bits"): the unsigned type of the
+/* 8- and 16-bit elements (integer types of 8 to 64 bits, Section 3.7.2): the unsigned type of the
  * same width keeps sum and product modulo 2^8 / 2^16 */
 COMBINE_INT(int8_t, uint8_t)
 COMBINE_INT(uint8_t, uint8_t)

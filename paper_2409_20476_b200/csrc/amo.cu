@@ -1,5 +1,5 @@
 /* Remote atomic memory operations: host-initiated single operations and the device-initiated
- * batches ("one op per GPU thread").  All atomics go through the device API of
+ * batches (one operation per GPU thread).  All atomics go through the device API of
  * ishmem_device.cuh (address translation + .gpu-scope atomic). */
 #include "internal.h"
 

@@ -1,6 +1,6 @@
 /* Reverse offload (Section 3.4 of the paper, "Synchronization with Host"): GPU threads post
  * fixed-size requests into a lock-free ring in pinned host memory; one host thread serves them
- * "as though they had been host-initiated operations" (Section 3.7.1) -- here: it starts the
+ * the way it would serve operations started on the host (Section 3.7.1) -- here: it starts the
  * copy engine for device-initiated puts and gets above the cutover.
  *
  * Both directions use stores only.  GPU -> host: the message, then its sequence number with a

@@ -140,3 +140,42 @@ def test_blocked_grid_generator_windows():
     assert not full[0].any() and not full[-1].any() and not full[:, 0].any()
     win = inputs.jacobi_cell_init(4, ny, nx, 1000, 1100, 3, 30)
     assert np.array_equal(win, full[1000:1100, 3:30])
+
+
+GOLD_ASSOC = Path(__file__).parent / "golden" / "jacobi_3x3_association.txt"
+
+
+def read_gold_assoc():
+    out = {}
+    for line in GOLD_ASSOC.read_text().splitlines():
+        if not line or line.startswith("#"):
+            continue
+        k, *v = line.split()
+        out[k] = np.array([float(x) for x in v])
+    return out
+
+
+def test_association_order_of_the_update_is_pinned():
+    """(N+S)+(W+E), fixed by a case in which every other order of the three additions gives
+    a different float64 (0.0 against 0.25 or 0.5): full grid, PE program and cone form."""
+    g = read_gold_assoc()
+    init = g["init"].reshape(3, 3)
+    # the hand derivation's premises hold in this arithmetic
+    assert np.float64(1e16) + np.float64(1.0) == np.float64(1e16)
+    assert g["wrong_left_to_right"][0] == 0.25 * (((init[0, 1] + init[2, 1]) + init[1, 0]) + init[1, 2])
+    assert g["wrong_pair_by_axis_swapped"][0] == 0.25 * ((init[0, 1] + init[1, 0]) + (init[2, 1] + init[1, 2]))
+    u, r = orc.jacobi(init, 1)
+    assert u.tobytes() == g["sweep1"].reshape(3, 3).tobytes()
+    assert r == g["residual_sq1"][0]
+    for npes in (1, 3):   # 3 PEs: one row each, N and S arrive through the put_signal halos
+        strips, rs = run_strips(init, npes, 1)
+        assert strips.tobytes() == g["sweep1"].reshape(3, 3).tobytes()
+        assert rs == g["residual_sq1"][0]
+    assert orc.jacobi_cell(init, 0, 0, 3, 3, 1, 1, 1) == 0.0
+    # the same stencil embedded in a larger grid, so that the cone form takes its interior
+    # branch with a window that is not the whole grid
+    big = np.zeros((7, 8))
+    big[2:5, 3:6] = init
+    full, _ = orc.jacobi(big, 1)
+    assert full[3, 4] == 0.0
+    assert orc.jacobi_cell(big[2:5, 3:6], 2, 3, 7, 8, 1, 3, 4) == 0.0
