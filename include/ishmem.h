@@ -116,14 +116,43 @@ typedef int ishmem_team_t;
  * e.g. a torch tensor; cf. the external-heap registration of Section 3.5) and does
  * not clear it.  ISHMEM_ERR_ARG if already initialised.  ishmem_init(npes, 0) takes the heap
  * size per PE from the environment variable ISHMEM_SYMMETRIC_SIZE (bytes).  Other variables read
- * at initialisation: ISHMEM_CUTOVER_{PUT,BCAST,FCOLLECT,WORK_GROUP} (bytes, "never" or "always";
- * see ishmemx_set_cutover) and ISHMEM_WAIT_TIMEOUT_NS (see ishmemx_set_wait_limit_ns). */
+ * at initialisation: ISHMEM_CUTOVER_{PUT,PUT_UPTO,BCAST,FCOLLECT,WORK_GROUP} (bytes, "never" or "always";
+ * see ishmemx_set_cutover), ISHMEM_WAIT_TIMEOUT_NS (see ishmemx_set_wait_limit_ns) and the
+ * initial values of the launch-shape switches (ISHMEM_JACOBI_SPLIT, _JACOBI_FUSE, _JACOBI_WIDE,
+ * ISHMEM_REDUCE_BULK, ISHMEM_BULK_SMEM; see ishmemx_set_option).  No variable is read later. */
 int ishmem_init(int npes, size_t heap_bytes);
 int ishmemx_init_external(int npes, size_t heap_bytes, void *base);
 /* Waits for all streams, frees everything the library allocated. */
 int ishmem_finalize(void);
 int ishmem_n_pes(void);                /* 0 when not initialised */
 size_t ishmemx_heap_bytes(void);
+/* Launch-shape switches.  Each has a default that the library picks from measurement; a test or
+ * a size sweep selects another form through ishmemx_set_option, never through the process
+ * environment at call time.  The environment variable named beside an option is read ONCE, by
+ * ishmem_init / ishmemx_init_external, and only sets the option's initial value; a later
+ * ishmemx_set_option wins.  All options are reset by the next initialisation.
+ *   ISHMEMX_OPT_JACOBI_SPLIT (ISHMEM_JACOBI_SPLIT=rows|columns): 0 = the library's choice (for
+ *       threads = 0 and an even nx: launch-ordered sweeps; else the persistent kernel, strips cut
+ *       by rows), 1 = persistent kernel with the strips cut by rows, 2 = by ranges of column
+ *       tiles.
+ *   ISHMEMX_OPT_JACOBI_FUSE (ISHMEM_JACOBI_FUSE=0|1): sweeps per launch of the launch-ordered
+ *       form: 1 = two where the count allows (default), 0 = always one.
+ *   ISHMEMX_OPT_JACOBI_WIDE (ISHMEM_JACOBI_WIDE=0|1): columns per lane in the two-sweep launches:
+ *       -1 = by grid size (default), 0 = two, 1 = four.
+ *   ISHMEMX_OPT_REDUCE_BULK (ISHMEM_REDUCE_BULK=0|1): 1 = large split reductions go through the
+ *       shared-memory TMA fold ring instead of one tile per block (default 0).
+ *   ISHMEMX_OPT_BULK_SMEM (ISHMEM_BULK_SMEM=bytes): shared-memory staging per block of the
+ *       ISHMEMX_WORK_GROUP_BULK level (default 192 KiB + 128, capped by the device limit).
+ * ishmemx_set_option returns ISHMEM_ERR_ARG for an unknown option or a value outside its range;
+ * ishmemx_get_option returns the current value (0 for an unknown option). */
+#define ISHMEMX_OPT_JACOBI_SPLIT 0
+#define ISHMEMX_OPT_JACOBI_FUSE 1
+#define ISHMEMX_OPT_JACOBI_WIDE 2
+#define ISHMEMX_OPT_REDUCE_BULK 3
+#define ISHMEMX_OPT_BULK_SMEM 4
+#define ISHMEMX_OPT_COUNT 5
+int ishmemx_set_option(int option, long long value);
+long long ishmemx_get_option(int option);
 /* Device pointer to PE `pe`'s context (ishmem_ctx_t, see ishmem_device.cuh), to hand to
  * user kernels; the array of all contexts starts at ishmemx_ctx(0).  NULL on error. */
 void *ishmemx_ctx(int pe);
@@ -249,9 +278,13 @@ int ishmemx_putmem_spmd_copy_engine(void *dest, const void *src, size_t nbytes, 
 /* Cutover sizes in bytes (Section 4: tuned from measurement; for the collaborative calls
  * it depends on the number of threads).  which: 0 = host-initiated put/get, 1 = broadcast,
  * 2 = fcollect, 3 = device-initiated work-group put/get (takes effect while the host proxy of
- * ishmemx_proxy_start runs).  SIZE_MAX = never use the copy engine, 0 = always.  Defaults, from
- * the size sweep on B200: 4 MiB for which = 0, SIZE_MAX for the others (environment overrides:
- * ISHMEM_CUTOVER_PUT, _BCAST, _FCOLLECT, _WORK_GROUP).
+ * ishmemx_proxy_start runs).  SIZE_MAX = never use the copy engine, 0 = always.
+ * which = 5 is the upper end of the host-initiated band: ishmem_putmem / getmem (and _nbi) use
+ * the engine for cutover 0 <= nbytes < cutover 5 and the tiled kernel outside it (SIZE_MAX = no
+ * upper end).  Defaults, from the size sweep on B200: the engine wins from 4 MiB to 32 MiB and
+ * loses or ties from 64 MiB on, so which = 0 is 4 MiB and which = 5 is 64 MiB; SIZE_MAX for
+ * 1, 2 and 3 (environment overrides: ISHMEM_CUTOVER_PUT, _PUT_UPTO, _BCAST, _FCOLLECT,
+ * _WORK_GROUP).
  * which = 4 is not a threshold but the hybrid head: a blocking work-group put/get above cutover 3
  * gives the engine everything past the first `nbytes` bytes (rounded down to 256) and copies
  * that head itself meanwhile, hiding the engine's start-up; 0 (the default) = engine only. */
@@ -260,11 +293,14 @@ size_t ishmemx_get_cutover(int which);
 /* Picks the cutover from measurement on this device (Section 4: "tuned from measurement"), for
  * which = 0 (host-initiated put, PE 0 -> PE 1, CUDA events) or which = 3 (device-initiated put
  * by ONE work-group of `threads` threads, timed inside the kernel; needs a running proxy).
- * Times both paths at 4 KiB, 16 KiB, ... up to max_bytes (two temporary symmetric buffers of
- * max_bytes are allocated and freed: ISHMEM_ERR_OOM if the heap has no room) and sets the
- * cutover to the smallest size from which the copy engine is at least as fast at every larger
- * size tried, or SIZE_MAX when it never is.  The choice is also written to HOST *chosen (may
- * be NULL).  Blocks the host. */
+ * Times both paths at 4 KiB, 16 KiB, ... (which = 0: 4 KiB, 8 KiB, ...) up to max_bytes (two
+ * temporary symmetric buffers of max_bytes are allocated and freed: ISHMEM_ERR_OOM if the heap
+ * has no room).  which = 3: sets the cutover to the smallest size from which the copy engine is at
+ * least as fast at every larger size tried, or SIZE_MAX when it never is.  which = 0: gives the
+ * engine the longest run of consecutive sizes at which it is at least as fast -- cutover 0 becomes
+ * the first size of that run and cutover 5 the first size after it at which the kernel wins
+ * (SIZE_MAX when the run reaches max_bytes; both SIZE_MAX when the engine never wins).  The
+ * lower bound is also written to HOST *chosen (may be NULL).  Blocks the host. */
 int ishmemx_tune_cutover(int which, int threads, size_t max_bytes, size_t *chosen);
 
 /* ------------------------------------- reverse offload: GPU -> host requests (Section 3.4) --- */
@@ -283,7 +319,9 @@ int ishmemx_tune_cutover(int which, int threads, size_t max_bytes, size_t *chose
  * the proxy's copy, and the wait then ends only by its time limit (ISHMEM_ERR_TIMEOUT latched,
  * nothing hangs).  Either queue nothing behind such a kernel, or start the process with
  * CUDA_DEVICE_MAX_CONNECTIONS=32 (read when the CUDA context is created; measured on B200:
- * 32 launches queued back to back, no time-outs with 32 queues, sporadic ones with 8). */
+ * 32 launches queued back to back, no time-outs with 32 queues, sporadic ones with 8).
+ * ishmemx_proxy_start reads one environment variable, once: ISHMEM_PROXY_NO_STREAM_MEMOPS (set to
+ * anything) makes the replies 8-byte copies even where stream memory operations exist. */
 int ishmemx_proxy_start(void);
 int ishmemx_proxy_stop(void);
 /* Requests served and copies started since ishmemx_proxy_start (HOST pointers, may be NULL);
@@ -369,6 +407,9 @@ void ishmem_info_get_name(char *name);
     int ishmem_##NAME##_atomic_add(int my_pe, T *target, T value, int pe);                     \
     int ishmem_##NAME##_atomic_inc(int my_pe, T *target, int pe);                              \
     int ishmem_##NAME##_atomic_set(int my_pe, T *target, T value, int pe);                     \
+    int ishmem_##NAME##_atomic_and(int my_pe, T *target, T value, int pe);                     \
+    int ishmem_##NAME##_atomic_or(int my_pe, T *target, T value, int pe);                      \
+    int ishmem_##NAME##_atomic_xor(int my_pe, T *target, T value, int pe);                     \
     int ishmem_##NAME##_atomic_fetch(int my_pe, T *fetched_host, const T *target, int pe);     \
     int ishmem_##NAME##_atomic_fetch_add(int my_pe, T *fetched_host, T *target, T value, int pe); \
     int ishmem_##NAME##_atomic_fetch_inc(int my_pe, T *fetched_host, T *target, int pe);       \
@@ -526,14 +567,14 @@ int ishmemx_rma_latency(int my_pe, void *dest, const void *src, size_t nbytes, i
  * read once, the second result written once; two halo rows each way, the second one parked in the
  * halo row of the buffer being written) -- an even number of such passes, then one to three
  * single-sweep launches, so that the result ends in the buffer named below; 428 us per sweep at
- * 16384^2 (single sweeps only, ISHMEM_JACOBI_FUSE=0: 650 us = the copy rate; ISHMEM_JACOBI_WIDE=0:
- * two instead of four columns per lane in the two-sweep launches).  groups_per_pe is
+ * 16384^2 (single sweeps only, ISHMEMX_OPT_JACOBI_FUSE = 0: 650 us = the copy rate;
+ * ISHMEMX_OPT_JACOBI_WIDE = 0: two instead of four columns per lane in the two-sweep launches).  groups_per_pe is
  * not used by this form and nothing needs to be co-resident.
  * threads > 0 (a multiple of 32 up to 1024): one persistent co-resident launch of
  * npes x groups_per_pe blocks of that size for all sweeps; the blocks of a PE take bands of rows,
  * one of them sends each halo row, and neighbouring blocks hand over through flags.
- * ISHMEM_ERR_NOT_CORESIDENT when the blocks cannot all be resident at once.  The environment
- * variable ISHMEM_JACOBI_SPLIT=rows|columns selects the persistent kernel also for threads = 0,
+ * ISHMEM_ERR_NOT_CORESIDENT when the blocks cannot all be resident at once.  The option
+ * ISHMEMX_OPT_JACOBI_SPLIT = 1 (rows) | 2 (columns) selects the persistent kernel also for threads = 0,
  * with the strips cut by rows, or by ranges of column tiles (one warp per tile; every block then
  * sends its columns of the halo rows); groups_per_pe is clamped to the rows (tiles) of the
  * shortest strip.
@@ -553,7 +594,9 @@ int ishmemx_jacobi(double *buf0, double *buf1, uint64_t *sig, size_t ny, size_t 
  *     exceed 2048 blocks; larger launches are refused with ISHMEM_ERR_ARG and
  *     ishmemx_last_cuda_error() names the limit.
  *   - The first call on each device resolves the array's device address
- *     (cudaGetSymbolAddress); make that first call before any stream capture begins.
+ *     (cudaGetSymbolAddress); make that first call before any stream capture begins, and from
+ *     one host thread: the per-device address cache is filled without a lock (two threads
+ *     racing there would store the same value, but the call is not documented as re-entrant).
  *   - All calls share the one array.  It still holds the previous call's contents, so each
  *     call clears the part it uses first; two calls whose kernels overlap on the GPU (from
  *     two host threads, say) would race on it -- serialise them.

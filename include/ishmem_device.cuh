@@ -1002,7 +1002,9 @@ __device__ __forceinline__ int ishmemx_putmem_signal_work_group(
     __syncthreads();
     /* the release below is cumulative: it also covers the other threads' stores, which the
      * block barrier has ordered before it */
-    if (r && rs && ishmemi::block_tid() == 0) ishmemi::signal_update(rs, signal, sig_op);
+    /* no signal after a copy that gave up (rc is the same in every thread): the waiter must
+     * never acquire a signal whose payload is incomplete */
+    if (rc == 0 && ishmemi::block_tid() == 0) ishmemi::signal_update(rs, signal, sig_op);
     return rc;
 }
 __device__ __forceinline__ unsigned long long ishmem_signal_fetch(const ishmem_ctx_t *,
@@ -1165,6 +1167,19 @@ __device__ __forceinline__ void ishmem_atomic_add(const ishmem_ctx_t *ctx, T *ta
     T *r = ishmemi::translate(ctx, target, pe);
     if (r) (void)ishmemi::amo<T>::fetch_add(r, value); /* result unused: compiles to a reduction */
 }
+/* non-fetching bitwise forms: the result is unused, so each compiles to a reduction */
+#define ISHMEMI_AMO_NF(NAME)                                                                          \
+    template <typename T>                                                                             \
+    __device__ __forceinline__ void ishmem_atomic_##NAME(const ishmem_ctx_t *ctx, T *target, T value, \
+                                                         int pe)                                      \
+    {                                                                                                 \
+        T *r = ishmemi::translate(ctx, target, pe);                                                   \
+        if (r) (void)ishmemi::amo<T>::fetch_##NAME(r, value);                                         \
+    }
+ISHMEMI_AMO_NF(and)
+ISHMEMI_AMO_NF(or)
+ISHMEMI_AMO_NF(xor)
+#undef ISHMEMI_AMO_NF
 template <typename T>
 __device__ __forceinline__ T ishmem_atomic_fetch_inc(const ishmem_ctx_t *ctx, T *target, int pe)
 {

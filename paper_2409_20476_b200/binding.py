@@ -43,6 +43,8 @@ ISHMEM_CMP_EQ, ISHMEM_CMP_NE, ISHMEM_CMP_GT, ISHMEM_CMP_GE, ISHMEM_CMP_LT, ISHME
 (ISHMEM_T_INT32, ISHMEM_T_INT64, ISHMEM_T_FLOAT, ISHMEM_T_DOUBLE, ISHMEM_T_UINT32,
  ISHMEM_T_UINT64, ISHMEM_T_INT8, ISHMEM_T_UINT8, ISHMEM_T_INT16, ISHMEM_T_UINT16) = range(10)
 ISHMEMX_REDUCE_AUTO, ISHMEMX_REDUCE_DUPLICATED, ISHMEMX_REDUCE_SPLIT = range(3)
+(ISHMEMX_OPT_JACOBI_SPLIT, ISHMEMX_OPT_JACOBI_FUSE, ISHMEMX_OPT_JACOBI_WIDE, ISHMEMX_OPT_REDUCE_BULK,
+ ISHMEMX_OPT_BULK_SMEM) = range(5)
 SIZE_MAX = 2**64 - 1
 
 
@@ -101,6 +103,8 @@ def _signatures() -> dict[str, tuple[str, list[str]]]:
         "ishmemx_last_cuda_error": ("str", []),
         "ishmemx_status": ("int", ["i"]),
         "ishmemx_set_wait_limit_ns": ("status", ["u64"]),
+        "ishmemx_set_option": ("status", ["i", "i64"]),
+        "ishmemx_get_option": ("i64", ["i"]),
         "ishmemx_launch_count": ("u64", []),
         "ishmem_malloc": ("ptr", ["z"]),
         "ishmem_calloc": ("ptr", ["z", "z"]),
@@ -180,6 +184,8 @@ def _signatures() -> dict[str, tuple[str, list[str]]]:
         S[pre + "add"] = ("status", ["i", "p", t, "i"])
         S[pre + "inc"] = ("status", ["i", "p", "i"])
         S[pre + "set"] = ("status", ["i", "p", t, "i"])
+        for op in ("and", "or", "xor"):
+            S[pre + op] = ("status", ["i", "p", t, "i"])
         S[pre + "fetch"] = ("status", ["i", "p", "p", "i"])
         S[pre + "fetch_inc"] = ("status", ["i", "p", "p", "i"])
         for op in ("fetch_add", "swap", "fetch_and", "fetch_or", "fetch_xor"):
@@ -231,6 +237,8 @@ def lib() -> C.CDLL:
                 f.restype = C.c_size_t
             elif ret == "u64":
                 f.restype = C.c_uint64
+            elif ret == "i64":
+                f.restype = C.c_int64
             elif ret == "str":
                 f.restype = C.c_char_p
         _lib = L

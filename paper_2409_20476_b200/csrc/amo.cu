@@ -4,7 +4,7 @@
 #include "internal.h"
 
 enum { AMO_ADD, AMO_INC, AMO_SET, AMO_FETCH, AMO_FETCH_ADD, AMO_FETCH_INC, AMO_SWAP, AMO_CAS, AMO_FETCH_AND,
-       AMO_FETCH_OR, AMO_FETCH_XOR };
+       AMO_FETCH_OR, AMO_FETCH_XOR, AMO_AND, AMO_OR, AMO_XOR };
 
 template <typename T>
 __global__ void k_amo(const ishmem_ctx_t *ctxs, int my_pe, int op, T *target_local, T value, T cond, int pe,
@@ -16,6 +16,9 @@ __global__ void k_amo(const ishmem_ctx_t *ctxs, int my_pe, int op, T *target_loc
     case AMO_ADD: ishmem_atomic_add<T>(ctx, target_local, value, pe); break;
     case AMO_INC: ishmem_atomic_inc<T>(ctx, target_local, pe); break;
     case AMO_SET: ishmem_atomic_set<T>(ctx, target_local, value, pe); break;
+    case AMO_AND: ishmem_atomic_and<T>(ctx, target_local, value, pe); break;
+    case AMO_OR: ishmem_atomic_or<T>(ctx, target_local, value, pe); break;
+    case AMO_XOR: ishmem_atomic_xor<T>(ctx, target_local, value, pe); break;
     case AMO_FETCH: old = ishmem_atomic_fetch<T>(ctx, target_local, pe); break;
     case AMO_FETCH_ADD: old = ishmem_atomic_fetch_add<T>(ctx, target_local, value, pe); break;
     case AMO_FETCH_INC: old = ishmem_atomic_fetch_inc<T>(ctx, target_local, pe); break;
@@ -61,6 +64,18 @@ static int host_amo(int my_pe, int op, T *fetched_host, const T *target, T value
     extern "C" int ishmem_##NAME##_atomic_set(int my_pe, T *target, T value, int pe)                              \
     {                                                                                                             \
         return host_amo<T, D>(my_pe, AMO_SET, nullptr, target, value, 0, pe, false);                              \
+    }                                                                                                             \
+    extern "C" int ishmem_##NAME##_atomic_and(int my_pe, T *target, T value, int pe)                              \
+    {                                                                                                             \
+        return host_amo<T, D>(my_pe, AMO_AND, nullptr, target, value, 0, pe, false);                              \
+    }                                                                                                             \
+    extern "C" int ishmem_##NAME##_atomic_or(int my_pe, T *target, T value, int pe)                               \
+    {                                                                                                             \
+        return host_amo<T, D>(my_pe, AMO_OR, nullptr, target, value, 0, pe, false);                               \
+    }                                                                                                             \
+    extern "C" int ishmem_##NAME##_atomic_xor(int my_pe, T *target, T value, int pe)                              \
+    {                                                                                                             \
+        return host_amo<T, D>(my_pe, AMO_XOR, nullptr, target, value, 0, pe, false);                              \
     }                                                                                                             \
     extern "C" int ishmem_##NAME##_atomic_fetch(int my_pe, T *fetched_host, const T *target, int pe)              \
     {                                                                                                             \

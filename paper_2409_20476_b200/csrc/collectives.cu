@@ -632,11 +632,10 @@ extern "C" int ishmemx_reduce(ishmem_team_t team, void *dest, const void *src, s
             const size_t most = (size_t)0x7fffffff / (size_t)t.size;
             a.groups = (int)(blocks < 1 ? 1 : (blocks < most ? blocks : most));
         }
-        /* ISHMEM_REDUCE_BULK=1 selects the TMA fold ring instead (one resident block per SM, three
+        /* ISHMEMX_OPT_REDUCE_BULK selects the TMA fold ring instead (one resident block per SM, three
          * stages of P tiles in shared memory): 6.2 TB/s at 12 PEs x 256 MiB where the tiles above
          * reach 6.5. */
-        static const char *env_bulk = getenv("ISHMEM_REDUCE_BULK");
-        const bool use_bulk = env_bulk && atoi(env_bulk) != 0 && !a.duplicated;
+        const bool use_bulk = g.opt[ISHMEMX_OPT_REDUCE_BULK] != 0 && !a.duplicated;
         if (use_bulk && g.coll_groups == 0 && per_member >= (1u << 20) && t.size <= 48) {
             unsigned want = 192 * 1024 + 128;
             if (want > g.max_dyn_smem) want = (unsigned)g.max_dyn_smem;

@@ -49,8 +49,10 @@ struct ishmemi_state {
 
     ishmemi_team teams[ISHMEM_MAX_TEAMS] = {};
     size_t cutover[3] = {0, 0, 0};
+    size_t cutover_put_upto = (size_t)-1; /* host-initiated put/get use the engine for cutover[0] <= n < this */
     size_t wg_cutover = (size_t)-1; /* device-initiated work-group put/get: bytes from which the engine is used */
     size_t hybrid_head = 0;         /* ... and bytes of the head the group copies itself meanwhile */
+    long long opt[ISHMEMX_OPT_COUNT] = {}; /* ishmemx_set_option: launch-shape switches */
     int coll_groups = 0, coll_threads = 512;
     int bcast_root_dest = 1;
     unsigned long long wait_limit_ns = 2000000000ull;

@@ -229,12 +229,19 @@ extern "C" int ishmemx_tune_cutover(int which, int threads, size_t max_bytes, si
         return ISHMEM_ERR_OOM;
     }
     const int to = g.npes > 1 ? 1 : 0;
-    const size_t saved = ishmemx_get_cutover(which);
+    const size_t saved = ishmemx_get_cutover(which), saved_upto = ishmemx_get_cutover(5);
     int rc = 0;
-    /* sizes 4 KiB, 16 KiB, ... <= max_bytes; the engine "wins" a size when it is at least as
-     * fast there; the cutover is the start of the unbroken run of wins at the top */
-    size_t pick = (size_t)-1;
-    for (size_t n = 4096; n <= max_bytes && !rc; n *= 4) {
+    /* The engine "wins" a size when it is at least as fast there.
+     * which = 3: sizes 4 KiB, 16 KiB, ...; the cutover is the start of the unbroken run of wins at
+     * the top.
+     * which = 0: sizes 4 KiB, 8 KiB, ...; the engine gets the LONGEST run of consecutive wins,
+     * [pick, upto): on this GPU it wins a middle range and loses or ties above it, which one
+     * threshold cannot say. */
+    size_t pick = (size_t)-1, upto = (size_t)-1;
+    size_t run_lo = (size_t)-1, best_lo = (size_t)-1, best_hi = (size_t)-1;
+    int run_len = 0, best_len = 0;
+    if (which == 0) ishmemx_set_cutover(5, (size_t)-1);
+    for (size_t n = 4096; n <= max_bytes && !rc; n *= (which == 0 ? 2 : 4)) {
         double t_ldst = 0, t_engine = 0;
         const int reps = n <= (1u << 20) ? 50 : (n <= (16u << 20) ? 10 : 3);
         if (which == 0) {
@@ -249,9 +256,18 @@ extern "C" int ishmemx_tune_cutover(int which, int threads, size_t max_bytes, si
         }
         if (t_engine <= t_ldst) {
             if (pick == (size_t)-1) pick = n;
+            if (run_len++ == 0) run_lo = n;
+            if (run_len > best_len) best_len = run_len, best_lo = run_lo, best_hi = (size_t)-1;
         } else {
             pick = (size_t)-1;
+            if (run_len && run_len == best_len && best_hi == (size_t)-1) best_hi = n; /* first loss after the best run */
+            run_len = 0;
         }
+    }
+    if (which == 0) {
+        pick = best_lo;
+        upto = best_hi;
+        ishmemx_set_cutover(5, rc ? saved_upto : upto);
     }
     ishmemx_set_cutover(which, rc ? saved : pick);
     cudaDeviceSynchronize();
@@ -1016,12 +1032,12 @@ __global__ void __launch_bounds__(256, WIDE ? 2 : 3) k_jacobi_pass2(const ishmem
  * (threads == 0) and every block gets at least 16 column tiles, one warp each; by rows when the
  * caller gives the block size, or when the grid is too narrow to fill the blocks with tiles (a
  * block then walks all tiles of its band, and any block size keeps its warps busy).
- * ISHMEM_JACOBI_SPLIT=rows / columns overrides; read at every call. */
+ * ISHMEMX_OPT_JACOBI_SPLIT = 1 (rows) / 2 (columns) overrides. */
 static bool jacobi_by_columns(int threads, size_t nx, int groups_per_pe)
 {
-    const char *env = getenv("ISHMEM_JACOBI_SPLIT");
-    if (env && !strcmp(env, "rows")) return false;
-    if (env && !strcmp(env, "columns")) return true;
+    const long long split = g_ishmem.opt[ISHMEMX_OPT_JACOBI_SPLIT];
+    if (split == 1) return false;
+    if (split == 2) return true;
     return threads == 0 && (nx + 59) / 60 >= (size_t)groups_per_pe * 16;
 }
 
@@ -1115,11 +1131,10 @@ static size_t jacobi_sweep_blocks(size_t ny, size_t nx, unsigned *bands, unsigne
     *tile_groups = (unsigned)(((nx + tile_cols - 1) / tile_cols + 7) / 8);
     return (size_t)g.npes * *bands * *tile_groups;
 }
-/* ISHMEM_JACOBI_FUSE=0 keeps one sweep per launch */
+/* ISHMEMX_OPT_JACOBI_FUSE = 0 keeps one sweep per launch */
 static bool jacobi_fuse(size_t ny)
 {
-    const char *env = getenv("ISHMEM_JACOBI_FUSE");
-    if (env && atoi(env) == 0) return false;
+    if (g_ishmem.opt[ISHMEMX_OPT_JACOBI_FUSE] == 0) return false;
     return ny / (size_t)g_ishmem.npes >= 2; /* the second halo row must be a row of the neighbour's strip */
 }
 /* partial: room for jacobi_partial_slots() residual terms; *nterms: how many the last launch wrote */
@@ -1136,11 +1151,12 @@ static int jacobi_launch_sweeps(double *buf0, double *buf1, uint64_t *sig, size_
     unsigned bands, tile_groups, bands2, tile_groups2;
     const size_t tile_blocks = jacobi_sweep_blocks(ny, nx, &bands, &tile_groups);
     /* four columns per lane (120-column tiles, 118 registers, two blocks per SM): 428 against 454 us per
-     * 16384^2 sweep for two columns per lane (56-column tiles), which ISHMEM_JACOBI_WIDE=0 selects */
-    bool wide = !(getenv("ISHMEM_JACOBI_WIDE") && atoi(getenv("ISHMEM_JACOBI_WIDE")) == 0);
-    /* ... unless the grid is too small to give every SM a few of the larger blocks (the variable
+     * 16384^2 sweep for two columns per lane (56-column tiles), which ISHMEMX_OPT_JACOBI_WIDE = 0 selects */
+    const long long wide_opt = g.opt[ISHMEMX_OPT_JACOBI_WIDE];
+    bool wide = wide_opt != 0;
+    /* ... unless the grid is too small to give every SM a few of the larger blocks (the option
      * set to 1 keeps the wide form regardless) */
-    if (wide && !getenv("ISHMEM_JACOBI_WIDE") &&
+    if (wide && wide_opt < 0 &&
         jacobi_sweep_blocks(ny, nx, &bands2, &tile_groups2, 120) < (size_t)g.sm_count * 4)
         wide = false;
     const size_t tile_blocks2 = jacobi_sweep_blocks(ny, nx, &bands2, &tile_groups2, wide ? 120 : 56);
@@ -1198,10 +1214,10 @@ static int jacobi_launch_sweeps(double *buf0, double *buf1, uint64_t *sig, size_
 }
 
 /* The library shapes the launch itself (threads == 0) and the grid has an even number of columns:
- * one launch per sweep.  ISHMEM_JACOBI_SPLIT=rows / columns asks for the persistent kernel. */
+ * one launch per sweep.  ISHMEMX_OPT_JACOBI_SPLIT = rows / columns asks for the persistent kernel. */
 static bool jacobi_per_sweep(int threads, size_t nx)
 {
-    return threads == 0 && nx % 2 == 0 && !getenv("ISHMEM_JACOBI_SPLIT");
+    return threads == 0 && nx % 2 == 0 && g_ishmem.opt[ISHMEMX_OPT_JACOBI_SPLIT] == 0;
 }
 
 extern "C" int ishmemx_jacobi(double *buf0, double *buf1, uint64_t *sig, size_t ny, size_t nx, int iters,

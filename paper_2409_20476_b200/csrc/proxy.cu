@@ -96,10 +96,14 @@ static void proxy_main(int device)
                 rc = reply_in_stream(s, (unsigned long long *)(uintptr_t)r.sig_addr, r.sig_value, tail);
             }
             g_px.copies.fetch_add(1, std::memory_order_relaxed);
-            if (!rc) {
-                if (r.completion) rc = reply_in_stream(s, g_px.comp + ((r.completion - 1) & (PROXY_COMP_SLOTS - 1)), r.completion, tail);
-                else rc = reply_in_stream(s, g_px.nbi_done + pe, ++g_px.nbi_count[pe], tail);
-            }
+            /* A copy that could not be started never raises its signal (the waiter must not see a
+             * signal without its payload), but the request still completes, in stream order like
+             * every other reply of this PE, so that the requester's wait or quiet ends at once
+             * instead of by its time limit; the failure is kept for ishmemx_proxy_stop to report. */
+            const int rc_copy = rc;
+            rc = r.completion ? reply_in_stream(s, g_px.comp + ((r.completion - 1) & (PROXY_COMP_SLOTS - 1)), r.completion, tail)
+                              : reply_in_stream(s, g_px.nbi_done + pe, ++g_px.nbi_count[pe], tail);
+            if (rc_copy) rc = rc_copy;
         } else if (r.completion) {
             /* ISHMEMI_REQ_NOP: the reply is a plain store into the polled word */
             __atomic_store_n(&g_px.comp[(r.completion - 1) & (PROXY_COMP_SLOTS - 1)], r.completion, __ATOMIC_RELEASE);

@@ -161,16 +161,15 @@ __global__ void k_test(const ishmem_ctx_t *ctxs, int my_pe, const unsigned long 
 
 /* ---- launch helpers --------------------------------------------------------------------- */
 
-static unsigned g_bulk_smem = 0;
+static unsigned g_bulk_smem = 0; /* the size the kernel's attribute was last set for */
 
 static unsigned bulk_staging_bytes()
 {
-    /* ring of shared-memory stages: one block per SM with a deep ring measured best on B200 */
-    if (!g_bulk_smem) {
-        unsigned want = 192 * 1024 + 128;
-        const char *env = getenv("ISHMEM_BULK_SMEM");
-        if (env) want = (unsigned)strtoul(env, nullptr, 0);
-        if (want > g_ishmem.max_dyn_smem) want = (unsigned)g_ishmem.max_dyn_smem;
+    /* ring of shared-memory stages: one block per SM with a deep ring measured best on B200
+     * (ISHMEMX_OPT_BULK_SMEM holds the size) */
+    unsigned want = (unsigned)g_ishmem.opt[ISHMEMX_OPT_BULK_SMEM];
+    if (want > g_ishmem.max_dyn_smem) want = (unsigned)g_ishmem.max_dyn_smem;
+    if (g_bulk_smem != want) {
         cudaFuncSetAttribute(k_rma<ISHMEMX_WORK_GROUP_BULK>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)want);
         g_bulk_smem = want;
@@ -266,7 +265,7 @@ static int rma_common(int my_pe, void *dest, const void *src, size_t n, int pe, 
     if (rc) return rc;
     if (n == 0) return ISHMEM_OK;
     auto &g = g_ishmem;
-    if (n >= g.cutover[0]) {
+    if (n >= g.cutover[0] && n < g.cutover_put_upto) {
         /* copy-engine path: translate the remote side on the host */
         char *d = is_get ? dl : dl + ((long long)pe - my_pe) * (long long)g.heap_bytes;
         const char *s = is_get ? sl + ((long long)pe - my_pe) * (long long)g.heap_bytes : sl;

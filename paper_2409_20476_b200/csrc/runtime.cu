@@ -218,18 +218,38 @@ static int init_common(int npes, size_t heap_bytes, void *external)
     g.free_blocks[0] = heap_bytes;
     /* default cutovers, from the committed size sweep on B200 (ishmemx_tune_cutover re-measures):
      * a host-initiated put/get of one PE is faster on the copy engine from 4 to 32 MiB (5.9 against
-     * 6.2 us at 4 MiB, 9.3 against 12.3 us at 32 MiB, back-to-back calls) and within a few per cent
-     * of the tiled kernel above that, while leaving the SMs free; the push collectives and the
-     * device-initiated work-group calls never gain, so they stay on loads and stores */
+     * 6.2 us at 4 MiB, 9.3 against 12.3 us at 32 MiB, back-to-back calls), slower at 64 MiB (24.7
+     * against 20.6 us) and level with the tiled kernel above that: the engine's range is a band,
+     * [4 MiB, 64 MiB); the push collectives and the device-initiated work-group calls never gain,
+     * so they stay on loads and stores */
     g.cutover[0] = (size_t)4 << 20;
+    g.cutover_put_upto = (size_t)64 << 20;
     g.cutover[1] = g.cutover[2] = g.wg_cutover = (size_t)-1;
     env_size("ISHMEM_CUTOVER_PUT", &g.cutover[0]);
+    env_size("ISHMEM_CUTOVER_PUT_UPTO", &g.cutover_put_upto);
     env_size("ISHMEM_CUTOVER_BCAST", &g.cutover[1]);
     env_size("ISHMEM_CUTOVER_FCOLLECT", &g.cutover[2]);
     env_size("ISHMEM_CUTOVER_WORK_GROUP", &g.wg_cutover);
     {
         size_t ns = 0;
         if (env_size("ISHMEM_WAIT_TIMEOUT_NS", &ns) && ns && ns != (size_t)-1) g.wait_limit_ns = ns;
+    }
+    /* launch-shape switches: defaults, then the environment's initial values (read here only) */
+    g.opt[ISHMEMX_OPT_JACOBI_SPLIT] = 0;
+    g.opt[ISHMEMX_OPT_JACOBI_FUSE] = 1;
+    g.opt[ISHMEMX_OPT_JACOBI_WIDE] = -1;
+    g.opt[ISHMEMX_OPT_REDUCE_BULK] = 0;
+    g.opt[ISHMEMX_OPT_BULK_SMEM] = 192 * 1024 + 128;
+    if (const char *v = getenv("ISHMEM_JACOBI_SPLIT")) {
+        if (!strcmp(v, "rows")) g.opt[ISHMEMX_OPT_JACOBI_SPLIT] = 1;
+        else if (!strcmp(v, "columns")) g.opt[ISHMEMX_OPT_JACOBI_SPLIT] = 2;
+    }
+    if (const char *v = getenv("ISHMEM_JACOBI_FUSE")) g.opt[ISHMEMX_OPT_JACOBI_FUSE] = atoi(v) != 0;
+    if (const char *v = getenv("ISHMEM_JACOBI_WIDE")) g.opt[ISHMEMX_OPT_JACOBI_WIDE] = atoi(v) != 0;
+    if (const char *v = getenv("ISHMEM_REDUCE_BULK")) g.opt[ISHMEMX_OPT_REDUCE_BULK] = atoi(v) != 0;
+    {
+        size_t b = 0;
+        if (env_size("ISHMEM_BULK_SMEM", &b) && b >= 128 + 2048 && b != (size_t)-1) g.opt[ISHMEMX_OPT_BULK_SMEM] = (long long)b;
     }
     g.hybrid_head = 0;
     g.launches = 0;
@@ -393,12 +413,23 @@ extern "C" void *ishmem_calloc(size_t count, size_t size)
     void *p = sym_alloc(ISHMEMI_ALIGN, count * size);
     if (!p) return nullptr;
     size_t off = (size_t)((char *)p - g.base);
-    for (int pe = 0; pe < g.npes; ++pe) {
-        cudaStream_t s = ishmemi_pe_stream_for_op(pe);
-        if (cudaMemsetAsync(g.base + (size_t)pe * g.heap_bytes + off, 0, count * size, s) != cudaSuccess) {
-            ishmem_free(p);
-            return nullptr;
-        }
+    /* The zeroing is one world-team operation: it waits for every PE's earlier work and every PE
+     * stream orders its later work after it, so a put or atomic that some PE issues right after
+     * the call cannot be overtaken by another PE's clearing (OpenSHMEM's calloc ends with a
+     * barrier for the same reason). */
+    cudaStream_t s;
+    if (ishmemi_team_stream_begin(ISHMEM_TEAM_WORLD, &s)) {
+        ishmem_free(p);
+        return nullptr;
+    }
+    bool ok = true;
+    for (int pe = 0; pe < g.npes && ok; ++pe)
+        ok = cudaMemsetAsync(g.base + (size_t)pe * g.heap_bytes + off, 0, count * size, s) == cudaSuccess;
+    ishmemi_team_stream_end();
+    if (!ok) {
+        (void)cudaGetLastError();
+        ishmem_free(p);
+        return nullptr;
     }
     return p;
 }
@@ -568,7 +599,11 @@ extern "C" void ishmem_info_get_name(char *name)
 extern "C" int ishmemx_set_cutover(int which, size_t nbytes)
 {
     ISHMEMI_REQUIRE_INIT();
-    if (which < 0 || which > 4) return ISHMEM_ERR_ARG;
+    if (which < 0 || which > 5) return ISHMEM_ERR_ARG;
+    if (which == 5) {
+        g_ishmem.cutover_put_upto = nbytes;
+        return ISHMEM_OK;
+    }
     if (which >= 3) {
         if (which == 3) g_ishmem.wg_cutover = nbytes;
         else g_ishmem.hybrid_head = nbytes;
@@ -582,7 +617,34 @@ extern "C" size_t ishmemx_get_cutover(int which)
 {
     if (which == 3) return g_ishmem.wg_cutover;
     if (which == 4) return g_ishmem.hybrid_head;
+    if (which == 5) return g_ishmem.cutover_put_upto;
     return (which < 0 || which > 2) ? 0 : g_ishmem.cutover[which];
+}
+extern "C" int ishmemx_set_option(int option, long long value)
+{
+    ISHMEMI_REQUIRE_INIT();
+    switch (option) {
+    case ISHMEMX_OPT_JACOBI_SPLIT:
+        if (value < 0 || value > 2) return ISHMEM_ERR_ARG;
+        break;
+    case ISHMEMX_OPT_JACOBI_FUSE:
+    case ISHMEMX_OPT_REDUCE_BULK:
+        if (value < 0 || value > 1) return ISHMEM_ERR_ARG;
+        break;
+    case ISHMEMX_OPT_JACOBI_WIDE:
+        if (value < -1 || value > 1) return ISHMEM_ERR_ARG;
+        break;
+    case ISHMEMX_OPT_BULK_SMEM:
+        if (value < 128 + 2048 || value > (1 << 20)) return ISHMEM_ERR_ARG;
+        break;
+    default: return ISHMEM_ERR_ARG;
+    }
+    g_ishmem.opt[option] = value;
+    return ISHMEM_OK;
+}
+extern "C" long long ishmemx_get_option(int option)
+{
+    return (option < 0 || option >= ISHMEMX_OPT_COUNT) ? 0 : g_ishmem.opt[option];
 }
 extern "C" int ishmemx_set_bcast_root_dest(int enable)
 {

@@ -187,6 +187,7 @@ def sweep_c2(args, out):
     s0 = torch.cuda.Stream()
     B.ishmemx_set_stream(0, s0.cuda_stream)
     T0 = Timer(torch, s0)
+    B.ishmemx_set_cutover(5, B.SIZE_MAX)          # no upper end: cutover 0 alone selects the path
     for n in sizes:
         B.ishmemx_set_cutover(0, B.SIZE_MAX)
         us, it = T0(lambda i: B.ishmem_putmem(0, dst, src, n, 1))
@@ -486,7 +487,7 @@ def sweep_c5(args, out):
 
     load()
     import os
-    # (variant, ISHMEM_JACOBI_SPLIT, threads, groups): the library's own choice (one launch per sweep), the
+    # (variant, form selected through ishmemx_set_option, threads, groups): the library's own choice (one launch per sweep), the
     # persistent kernel with strips cut by column tiles, and the persistent kernel with caller-shaped blocks
     variants = [("launch_per_two_sweeps", None, 0, 1), ("launch_per_sweep", "single", 0, 1)]
     variants += [("persistent_columns", "columns", 0, g) for g in (6, 12)]
@@ -495,12 +496,8 @@ def sweep_c5(args, out):
         for variant, split, threads, groups in variants:
             if npes * groups * threads > 148 * 2048:
                 continue
-            os.environ.pop("ISHMEM_JACOBI_SPLIT", None)
-            os.environ.pop("ISHMEM_JACOBI_FUSE", None)
-            if split == "single":
-                os.environ["ISHMEM_JACOBI_FUSE"] = "0"
-            elif split is not None:
-                os.environ["ISHMEM_JACOBI_SPLIT"] = split
+            B.ishmemx_set_option(B.ISHMEMX_OPT_JACOBI_SPLIT, {"rows": 1, "columns": 2}.get(split, 0))
+            B.ishmemx_set_option(B.ISHMEMX_OPT_JACOBI_FUSE, 0 if split == "single" else 1)
             def reset_signals():
                 for p in range(npes):
                     for w in range(4):
@@ -527,8 +524,6 @@ def sweep_c5(args, out):
             out.add(config=5, op="jacobi", pattern=f"{n}x{n}", variant=f"{variant} overlap={overlap}", threads=threads,
                     groups=groups, npes=npes, dtype="f64", nbytes=n * n * 8, l2="cold", iters=iters, us_per_op=us,
                     alg_bytes=16 * n * n, note=f"per sweep; residual_sq {res[0]:.6e} (grid keeps evolving)")
-    os.environ.pop("ISHMEM_JACOBI_SPLIT", None)
-    os.environ.pop("ISHMEM_JACOBI_FUSE", None)
     assert B.ishmemx_status(1) == 0
     B.ishmem_finalize()
 
@@ -565,6 +560,24 @@ def _crossover(a, b):
     return pick
 
 
+def _band(a, b):
+    """longest run of consecutive common sizes at which b's time is <= a's: (first size of the
+    run, first size after it at which a wins or None when the run reaches the top), or None"""
+    best, run = None, []
+    sizes = sorted(set(a) & set(b))
+    for k, n in enumerate(sizes):
+        if b[n] <= a[n]:
+            run.append(n)
+            if best is None or len(run) > best[2]:
+                best = (run[0], sizes[k + 1] if k + 1 < len(sizes) else None, len(run))
+        else:
+            run = []
+    if best is None:
+        return None
+    lo, after, _ = best
+    return lo, (after if after is not None and b[after] > a[after] else None)
+
+
 def summarize(path) -> str:
     rows = list(csv.DictReader(open(path)))
     cfg = int(rows[0]["config"])
@@ -589,8 +602,11 @@ def summarize(path) -> str:
                     "work_group_bulk_256x37", "work_group_tiled_256"):
             c = _crossover(t(var), t("copy_engine"))
             out.append(f"- `{var}` vs host-started copy engine (ring, 8 PEs): " + (_fmt_size(c) if c else "never"))
-        c = _crossover(t("host_api_kernel", pat="one_pe"), t("host_api_copy_engine", pat="one_pe"))
-        out.append("- host API `ishmem_putmem`, one PE, kernel vs engine: " + (_fmt_size(c) if c else "never (mixed)"))
+        band = _band(t("host_api_kernel", pat="one_pe"), t("host_api_copy_engine", pat="one_pe"))
+        out.append("- host API `ishmem_putmem`, one PE, kernel vs engine: the engine is at least as fast from "
+                   + (f"{_fmt_size(band[0])} up to " + (f"(not including) {_fmt_size(band[1])}" if band[1] else "the largest size")
+                      if band else "no size")
+                   + " -- a band, not a threshold (table below; defaults of cutover 0 and 5)")
         for var in ("in_kernel_work_item", "in_kernel_sub_group", "in_kernel_work_group_16", "in_kernel_work_group_128",
                     "in_kernel_work_group_256", "in_kernel_work_group_1024", "in_kernel_work_group_bulk_256"):
             c = _crossover(t(var, pat="one_pe"), t("in_kernel_work_group_engine_64", pat="one_pe"))
@@ -599,6 +615,9 @@ def summarize(path) -> str:
         sel = [r for r in rows if r["pattern"] == "one_pe" and r["op"] == "put" and r["variant"].startswith("in_kernel")]
         out += ["", "### one collaboration unit, PE 0 -> PE 1, put + quiet timed inside the kernel: microseconds", "",
                 _table(sel, nb, lambda r: r["variant"][10:], us, _fmt_size), ""]
+        sel = [r for r in rows if r["pattern"] == "one_pe" and r["variant"].startswith("host_api")]
+        out += ["### host API `ishmem_putmem` on ONE PE (PE 0 -> PE 1), back-to-back calls: microseconds per call / GB/s", "",
+                _table(sel, nb, lambda r: r["variant"][9:], lambda r: f"{us(r)} / {gb(r)}", _fmt_size), ""]
         sel = [r for r in rows if r["pattern"] == "all_pairs"]
         out += ["### all-pairs (mean of the 7 permutation rounds): GB/s", "",
                 _table(sel, nb, lambda r: r["variant"], gb, _fmt_size), ""]

@@ -17,11 +17,14 @@ def test_host_initiated_atomics_all_ops():
         t = s.malloc(256)
         seq = [("fetch_add", 5), ("add", 7), ("fetch_inc", None), ("inc", None), ("fetch", None),
                ("set", 0b1100), ("fetch_and", 0b1010), ("fetch_or", 1), ("fetch_xor", 0b1111),
-               ("swap", 99), ("compare_swap", (98, 1)), ("compare_swap", (99, 1)), ("fetch_add", -3)]
+               ("swap", 99), ("compare_swap", (98, 1)), ("compare_swap", (99, 1)), ("fetch_add", -3),
+               ("or", 0b110000), ("and", 0b111100), ("xor", 0b101010), ("fetch", None)]
         omap = {"fetch_add": orc.A_FETCH_ADD, "add": orc.A_ADD, "fetch_inc": orc.A_FETCH_INC,
                 "inc": orc.A_INC, "fetch": orc.A_FETCH, "set": orc.A_SET, "fetch_and": orc.A_FETCH_AND,
                 "fetch_or": orc.A_FETCH_OR, "fetch_xor": orc.A_FETCH_XOR, "swap": orc.A_SWAP,
-                "compare_swap": orc.A_COMPARE_SWAP}
+                "compare_swap": orc.A_COMPARE_SWAP,
+                # the non-fetching bitwise forms change memory as the fetching ones do
+                "and": orc.A_FETCH_AND, "or": orc.A_FETCH_OR, "xor": orc.A_FETCH_XOR}
         for tname, npd, width in (("int64", np.int64, 8), ("uint64", np.uint64, 8), ("int32", np.int32, 4),
                                   ("uint32", np.uint32, 4)):
             addr, ooff = t.addr + 64, t.ooff + 64
@@ -32,7 +35,7 @@ def test_host_initiated_atomics_all_ops():
                     arg = arg % (1 << (8 * width))
                 f = getattr(B, f"ishmem_{tname}_atomic_{op}")
                 out = np.zeros(1, dtype=npd)
-                if op in ("add", "set"):
+                if op in ("add", "set", "and", "or", "xor"):
                     f(me, addr, arg, pe)
                     s.oracle.atomic(omap[op], width, ooff, arg, 0, pe)
                 elif op == "inc":

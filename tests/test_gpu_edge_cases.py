@@ -156,3 +156,34 @@ def test_two_dimensional_team_split():
         with pytest.raises(B.IshmemError):
             B.ishmem_team_split_2d(W, 0, 0, tx, ty)
         assert s.status() == 0
+
+
+def test_calloc_is_ordered_before_any_pes_next_operation():
+    """calloc clears every PE's copy as one team operation: a put or an atomic that another PE
+    issues right after it, with no barrier in between, lands on zeroed memory and stays.  The
+    region is large, dirty beforehand and the puts hit its far end, where a clearing that
+    another PE's stream still had in flight would wipe them out."""
+    npes, n = 4, 96 << 20
+    with Session(npes, n + (1 << 20), with_oracle=False) as s:
+        for rep in range(3):
+            s.heap.fill_(0xA5)
+            torch.cuda.synchronize()
+            p = B.ishmem_calloc(n // 8, 8)
+            assert p
+            tail = p + n - 4096
+            for me in range(npes):
+                t = (me + 1) % npes
+                B.ishmem_uint64_p(me, tail + 8 * me, 1000 + me, t)             # a scalar put into the neighbour
+                B.ishmem_uint64_atomic_add(me, tail + 2048, 1, (me + 2) % npes)  # and an atomic two PEs on
+            B.ishmem_barrier_all()
+            s.sync()
+            off = p - s.base
+            for q in range(npes):
+                got = s.heap[q * s.heap_bytes + off:q * s.heap_bytes + off + n].view(torch.int64)
+                exp_nonzero = {(n - 4096) // 8 + (q - 1) % npes: 1000 + (q - 1) % npes, (n - 4096 + 2048) // 8: 1}
+                nz = torch.nonzero(got).flatten().cpu().tolist()
+                assert sorted(nz) == sorted(exp_nonzero), (rep, q, nz)
+                for k, v in exp_nonzero.items():
+                    assert int(got[k]) == v, (rep, q, k)
+            B.ishmem_free(p)
+        assert s.status() == 0

@@ -15,7 +15,7 @@ import torch
 import oracle as orc
 from paper_2409_20476_b200 import binding as B
 from paper_2409_20476_b200 import inputs
-from tests.gpu_util import Session
+from tests.gpu_util import Session, heaps_equal
 
 pytestmark = pytest.mark.gpu
 MiB = 1 << 20
@@ -108,10 +108,11 @@ OPS = [(B.ISHMEM_OP_SUM, orc.R_SUM), (B.ISHMEM_OP_MAX, orc.R_MAX), (B.ISHMEM_OP_
        (B.ISHMEM_OP_PROD, orc.R_PROD)]
 
 
-@pytest.mark.parametrize("kind,nelems", [("f32", 4 ** 13), ("f64", 4 ** 12), ("i64", 4 ** 12)])
+@pytest.mark.parametrize("kind,nelems", [("f32", 4 ** 13), ("f64", 4 ** 13), ("i64", 4 ** 13)])
 def test_config3_reduce_large_12_pes(kind, nelems):
-    """Config 3 at large counts: 12 PEs, sum/max/min/prod.  Whole output: all PEs hold
-    identical results.  Windows: the PE-order fold of the oracle, bit for bit (0 ulp)."""
+    """Config 3 at its largest count (4^13 = 64 Mi elements; 12 x 1 GiB of heap for the 8-byte
+    types): 12 PEs, sum/max/min/prod.  Whole output: all PEs hold identical results.  Windows: the
+    PE-order fold of the oracle, bit for bit (0 ulp)."""
     npd, ldt, odt = KIND[kind]
     es, npes, W = np.dtype(npd).itemsize, 12, 1024
     rng = np.random.default_rng(8)
@@ -138,9 +139,9 @@ def test_config3_reduce_large_12_pes(kind, nelems):
 
 
 def test_config3_broadcast_fcollect_large_12_pes():
-    """Config 3: broadcast of 64 Mi float32 (256 MiB) from root 0 and fcollect of 16 Mi
-    float32 per PE (768 MiB gathered on every PE), 12 PEs."""
-    npes, nb, nf = 12, 4 * 4 ** 13, 4 * 4 ** 12
+    """Config 3 at its largest count: broadcast of 64 Mi float32 (256 MiB) from root 0 and
+    fcollect of 64 Mi float32 per PE (3 GiB gathered on every PE, 39 GiB of heap), 12 PEs."""
+    npes, nb, nf = 12, 4 * 4 ** 13, 4 * 4 ** 13
     rng = np.random.default_rng(9)
     with Session(npes, nb + npes * nf + MiB, with_oracle=False) as s:
         src, dst = s.malloc(nb), s.malloc(npes * nf)
@@ -178,47 +179,154 @@ def test_config3_broadcast_fcollect_large_12_pes():
         assert s.status() == 0
 
 
+_GRID = {}
+
+
+def config5_grid(ny, nx):
+    """the seeded config-5 grid (cached: the full one is 2 GiB and three tests use it)"""
+    if (ny, nx) not in _GRID:
+        grid = np.empty((ny, nx))
+        nblk = -(-ny // 1024)
+
+        def gen(b):
+            grid[b * 1024:min(ny, (b + 1) * 1024)] = inputs.jacobi_grid_block(inputs.SEED_C5, ny, nx, b)
+
+        list(POOL.map(gen, range(nblk)))
+        _GRID[(ny, nx)] = grid
+    return _GRID[(ny, nx)]
+
+
+class Strips:
+    """config 5's buffers in a session: scatter a grid over the PEs' strips, run, read back"""
+
+    def __init__(self, s, npes, ny, nx):
+        self.s, self.npes, self.ny, self.nx = s, npes, ny, nx
+        rows_max = -(-ny // npes)
+        nbytes = (rows_max + 2) * nx * 8
+        self.b0, self.b1, self.sig = s.malloc(nbytes), s.malloc(nbytes), s.malloc(64)
+        base, extra = divmod(ny, npes)
+        self.firsts = [p * base + min(p, extra) for p in range(npes + 1)]
+
+    def load(self, grid):
+        ny, nx = self.ny, self.nx
+        for p in range(self.npes):
+            lo, hi = self.firsts[p], self.firsts[p + 1]
+            self.b0.gpu(p).zero_()
+            self.b1.gpu(p).zero_()
+            self.b0.gpu(p)[nx * 8:(hi - lo + 1) * nx * 8].copy_(torch.from_numpy(grid[lo:hi].view(np.uint8).ravel()))
+            self.sig.gpu(p).zero_()
+        self.s.sync()
+
+    def run(self, iters, overlap=1):
+        res = np.zeros(1)
+        B.ishmemx_jacobi(self.b0.addr, self.b1.addr, self.sig.addr, self.ny, self.nx, iters, overlap, 12, 0, res)
+        assert self.s.status() == 0
+        self.fin = self.b0 if iters % 2 == 0 else self.b1
+        return res[0]
+
+    def strip(self, p):
+        """PE p's rows of the final grid, as a device tensor of bytes"""
+        lo, hi = self.firsts[p], self.firsts[p + 1]
+        return self.fin.gpu(p)[self.nx * 8:(hi - lo + 1) * self.nx * 8]
+
+    def assert_equals_grid(self, exp, what):
+        for p in range(self.npes):
+            lo, hi = self.firsts[p], self.firsts[p + 1]
+            got = self.strip(p).cpu().numpy().view(np.uint64)
+            want = exp[lo:hi].view(np.uint64).ravel()
+            if not np.array_equal(got, want):
+                bad = np.nonzero(got != want)[0]
+                r, c = divmod(int(bad[0]), self.nx)
+                raise AssertionError(f"{what}: PE {p} differs from the oracle in {bad.size} cells, first at "
+                                     f"global row {lo + r}, column {c}")
+
+    def cell(self, ci, cj):
+        p = max(q for q in range(self.npes) if self.firsts[q] <= ci)
+        r = ci - self.firsts[p] + 1
+        return self.fin.gpu(p)[(r * self.nx + cj) * 8:(r * self.nx + cj + 1) * 8].cpu().numpy().view(np.float64)[0]
+
+
+def test_config5_jacobi_16384_whole_grid_even_and_odd_sweep_counts():
+    """Config 5 at full size in the launch shape the library picks by itself (wide two-sweep
+    passes at this size), 12 PEs: the WHOLE final grid bit for bit against the oracle's plain
+    full-grid sweeps, and the residual at 1e-6 relative, for 8 sweeps (two-sweep passes only)
+    and 9 (passes, then single-sweep launches) -- every band and tile-group seam and all eleven
+    strip seams are compared.  The ninth oracle sweep continues from the eighth (a sweep has no
+    memory, which a CPU test pins)."""
+    npes, n = 12, 16384
+    grid = config5_grid(n, n)
+    u8, r8 = orc.jacobi(grid, 8)
+    u9, r9 = orc.jacobi(u8, 1)
+    rows_max = -(-n // npes)
+    with Session(npes, 2 * (rows_max + 2) * n * 8 + MiB, with_oracle=False) as s:
+        st = Strips(s, npes, n, n)
+        for iters, exp, exp_res in ((8, u8, r8), (9, u9, r9)):
+            st.load(grid)
+            res = st.run(iters)
+            st.assert_equals_grid(exp, f"{iters} sweeps")
+            assert abs(res - exp_res) <= 1e-6 * exp_res, (iters, res, exp_res)
+
+
+def test_config5_jacobi_full_width_200_sweeps_whole_grid_and_residual():
+    """200 sweeps on rows of config 5's full width (16384 columns x 768 rows, 12 strips of one
+    64-row band each): whole grid and residual against the oracle, in the wide two-sweep form that
+    the library uses at full size.  (The oracle needs about eight minutes for 200 sweeps of the
+    full 16384 x 16384 grid; there the checks are the two tests around this one.)"""
+    npes, ny, nx, iters = 12, 768, 16384, 200
+    grid = config5_grid(ny, nx)
+    exp, exp_res = orc.jacobi(grid, iters)
+    with Session(npes, 2 * (ny // npes + 2) * nx * 8 + MiB, with_oracle=False) as s:
+        B.ishmemx_set_option(B.ISHMEMX_OPT_JACOBI_WIDE, 1)
+        st = Strips(s, npes, ny, nx)
+        st.load(grid)
+        res = st.run(iters)
+        st.assert_equals_grid(exp, "200 sweeps, full-width rows")
+        assert abs(res - exp_res) <= 1e-6 * exp_res, (res, exp_res)
+
+
 def test_config5_jacobi_16384_200_iterations_sampled_cells():
     """Config 5 at full size: 16384 x 16384 float64, 12 row strips, 200 sweeps with in-kernel
-    put_signal halos.  Sampled cells -- corners, edges, strip boundaries, interior -- are
-    compared bit for bit with the oracle's dependency-cone evaluation from the initial grid."""
+    put_signal halos.  Sampled cells -- corners, edges, both sides of strip boundaries, of band
+    seams (every 16 and 64 rows of a strip) and of tile seams (every 56, 60, 120 and 960
+    columns), interior -- are compared bit for bit with the oracle's dependency-cone evaluation
+    from the initial grid.  Then the same 200 sweeps as single-sweep launches, which the
+    whole-grid tests pin to the oracle: every strip and the residual must agree with the
+    default form's."""
     npes, n, iters = 12, 16384, 200
+    grid = config5_grid(n, n)
     rows_max = -(-n // npes)
-    nbytes = (rows_max + 2) * n * 8
-    nblk = n // 1024
-    grid = np.empty((n, n))
-
-    def gen(b):
-        grid[b * 1024:(b + 1) * 1024] = inputs.jacobi_grid_block(inputs.SEED_C5, n, n, b)
-
-    list(POOL.map(gen, range(nblk)))
-    base, extra = divmod(n, npes)
-    firsts = [p * base + min(p, extra) for p in range(npes + 1)]
-    with Session(npes, 2 * nbytes + MiB, with_oracle=False) as s:
-        b0, b1, sig = s.malloc(nbytes), s.malloc(nbytes), s.malloc(64)
-        for p in range(npes):
-            rows = firsts[p + 1] - firsts[p]
-            b0.gpu(p)[n * 8:(rows + 1) * n * 8].copy_(torch.from_numpy(grid[firsts[p]:firsts[p + 1]].view(np.uint8).ravel()))
-        s.sync()
-        for p in range(npes):
-            sig.fill(p, np.zeros(64, np.uint8))
-        s.sync()
-        B.ishmemx_jacobi(b0.addr, b1.addr, sig.addr, n, n, iters, 1, 12, 0, None)
-        assert s.status() == 0
+    with Session(npes, 2 * (rows_max + 2) * n * 8 + MiB, with_oracle=False) as s:
+        st = Strips(s, npes, n, n)
+        firsts = st.firsts
+        st.load(grid)
+        res = st.run(iters)
         rng = np.random.default_rng(10)
         cells = [(1, 1), (n - 2, n - 2), (1, n // 2), (n // 2, 1), (0, 5), (7, n - 1)]
         for p in (1, 4, 5, 11):                     # both sides of strip boundaries
             cells += [(firsts[p] - 1, int(rng.integers(1, n - 1))), (firsts[p], int(rng.integers(1, n - 1)))]
+        for band, tile in ((64, 120), (64, 960), (16, 60), (64, 56), (16, 480), (64, 448)):
+            p, k, t = int(rng.integers(0, npes)), int(rng.integers(1, 1300 // band)), int(rng.integers(1, n // tile))
+            row = firsts[p] + band * k              # first row of band k of strip p
+            cells += [(row - 1, tile * t - 1), (row, tile * t), (row - 1, tile * t), (row, tile * t - 1)]
         cells += [(int(i), int(j)) for i, j in rng.integers(1, n - 1, size=(6, 2))]
-        fin = b0 if iters % 2 == 0 else b1
-        for ci, cj in cells:
+
+        def check(cell):
+            ci, cj = cell
             i0, i1 = max(0, ci - iters), min(n, ci + iters + 1)
             j0, j1 = max(0, cj - iters), min(n, cj + iters + 1)
-            exp = orc.jacobi_cell(grid[i0:i1, j0:j1], i0, j0, n, n, iters, ci, cj)
-            p = max(q for q in range(npes) if firsts[q] <= ci)
-            r = ci - firsts[p] + 1
-            got = fin.gpu(p)[(r * n + cj) * 8:(r * n + cj + 1) * 8].cpu().numpy().view(np.float64)[0]
+            return orc.jacobi_cell(grid[i0:i1, j0:j1], i0, j0, n, n, iters, ci, cj)
+
+        for (ci, cj), exp in zip(cells, POOL.map(check, cells)):
+            got = st.cell(ci, cj)
             assert np.float64(got).tobytes() == np.float64(exp).tobytes(), (ci, cj, got, exp)
+        # the same run as 200 single-sweep launches
+        fused = [st.strip(p).clone() for p in range(npes)]      # 2 GiB of torch memory beside the heap
+        B.ishmemx_set_option(B.ISHMEMX_OPT_JACOBI_FUSE, 0)
+        st.load(grid)
+        res1 = st.run(iters)
+        for p in range(npes):
+            assert torch.equal(st.strip(p), fused[p]), p
+        assert abs(res - res1) <= 1e-6 * res1, (res, res1)
 
 
 def test_large_alltoall_collect_and_narrow_reduce():
@@ -261,4 +369,24 @@ def test_large_alltoall_collect_and_narrow_reduce():
                     assert np.array_equal(dst.gpu(5)[off:off + 4096].cpu().numpy(), o.view(8192, 4096, 5)), (lop, off)
         finally:
             o.close()
+        assert s.status() == 0
+
+
+@pytest.mark.parametrize("level,n,threads", [(B.ISHMEMX_WORK_ITEM, 4 * MiB, 1), (B.ISHMEMX_SUB_GROUP, 64 * MiB, 32)])
+def test_config2_one_thread_and_one_warp_at_their_largest_sweep_sizes(level, n, threads):
+    """The largest messages the size sweep times for a single work-item (4 MiB) and a single
+    sub-group (64 MiB): ONE collaboration unit moves the whole message, put and get, with
+    unaligned ends; every byte of both heaps against the oracle."""
+    npes = 2
+    with Session(npes, 2 * n + MiB) as s:
+        src, dst = s.malloc(n), s.malloc(n)
+        for p in range(npes):
+            src.fill(p, inputs.byte_payload(inputs.SEED_C2, 40 + p, n))
+        m = n - 3                                        # ragged tail; head at offset 1: misaligned by one
+        B.ishmemx_putmem_on_device(0, dst.addr + 1, src.addr + 1, m - 1, 1, level, threads, 1)
+        s.oracle.putmem(0, dst.ooff + 1, s.oracle.ptr(src.ooff + 1, m - 1, 0), m - 1, 1)
+        B.ishmemx_getmem_on_device(0, dst.addr, src.addr, n, 1, level, threads, 1)       # PE 0 <- PE 1's src
+        s.oracle.getmem(0, s.oracle.ptr(dst.ooff, n, 0), src.ooff, n, 1)
+        B.ishmem_barrier_all()
+        heaps_equal(s, f"level {level}, {n} bytes")
         assert s.status() == 0

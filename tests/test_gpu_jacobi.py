@@ -12,11 +12,13 @@ from tests.gpu_util import Session
 pytestmark = pytest.mark.gpu
 
 
-def run_gpu(grid, npes, iters, overlap, groups, threads):
+def run_gpu(grid, npes, iters, overlap, groups, threads, options=()):
     ny, nx = grid.shape
     rows_max = -(-ny // npes)
     nbytes = (rows_max + 2) * nx * 8
     with Session(npes, 2 * nbytes + (1 << 16), with_oracle=False) as s:
+        for opt, value in options:
+            B.ishmemx_set_option(opt, value)
         b0, b1, sig = s.malloc(nbytes), s.malloc(nbytes), s.malloc(64)
         base, extra = divmod(ny, npes)
         first = 0
@@ -48,27 +50,27 @@ def run_gpu(grid, npes, iters, overlap, groups, threads):
     (600, 256, 12, 13, 128), (300, 4096, 4, 2, 1024), (97, 62, 3, 5, 1024),    # sliding window, 64 registers
     (120, 2880, 6, 6, 0), (90, 1442, 3, 2, 0), (60, 5000, 2, 4, 640),          # threads chosen by the library; 80 registers
     (36, 600, 12, 12, 32), (50, 121, 4, 3, 64)])                               # one tile per block; odd nx by columns
-def test_jacobi_matches_oracle(ny, nx, npes, groups, threads, overlap, split, monkeypatch):
+def test_jacobi_matches_oracle(ny, nx, npes, groups, threads, overlap, split):
     """split: the persistent kernel with the strips cut by columns or by rows, or `sweeps`: the form the
     library picks by itself for threads = 0 and even nx (one tile per warp, two sweeps per launch where the
     count allows, four columns per lane), the same with two columns per lane, or with one sweep per launch."""
     if split in ("sweeps", "sweeps_two_columns_per_lane", "single_sweeps"):
-        monkeypatch.delenv("ISHMEM_JACOBI_SPLIT", raising=False)
-        monkeypatch.setenv("ISHMEM_JACOBI_FUSE", "0" if split == "single_sweeps" else "1")
-        monkeypatch.setenv("ISHMEM_JACOBI_WIDE", "0" if split == "sweeps_two_columns_per_lane" else "1")
+        options = [(B.ISHMEMX_OPT_JACOBI_SPLIT, 0),
+                   (B.ISHMEMX_OPT_JACOBI_FUSE, 0 if split == "single_sweeps" else 1),
+                   (B.ISHMEMX_OPT_JACOBI_WIDE, 0 if split == "sweeps_two_columns_per_lane" else 1)]
         threads = 0
     else:
-        monkeypatch.setenv("ISHMEM_JACOBI_SPLIT", split)
+        options = [(B.ISHMEMX_OPT_JACOBI_SPLIT, {"rows": 1, "columns": 2}[split])]
     grid = inputs.jacobi_grid(inputs.SEED_C5, ny, nx)
     iters = 21
     exp, exp_res = orc.jacobi(grid, iters)
-    got, res = run_gpu(grid, npes, iters, overlap, groups, threads)
+    got, res = run_gpu(grid, npes, iters, overlap, groups, threads, options)
     assert got.tobytes() == exp.tobytes()
     assert abs(res - exp_res) <= 1e-6 * exp_res
 
 
 def test_jacobi_default_split_and_repeated_calls():
-    """Without ISHMEM_JACOBI_SPLIT: threads = 0 launches once per sweep, a given block size runs the persistent
+    """With the options at their defaults: threads = 0 launches once per sweep, a given block size runs the persistent
     kernel with the strips cut by rows; both give the oracle's grid."""
     grid = inputs.jacobi_grid(inputs.SEED_C5, 150, 2400)         # 40 column tiles
     exp, _ = orc.jacobi(grid, 9)

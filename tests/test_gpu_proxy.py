@@ -153,6 +153,10 @@ def test_cutover_tuned_from_measurement():
                 pick = int(chosen[0])
                 assert pick == B.SIZE_MAX or (4096 <= pick <= 16 << 20 and pick & (pick - 1) == 0)
                 assert B.ishmemx_get_cutover(which) == pick
+                if which == 0:      # the host band: its upper end is a larger size tried, or open
+                    upto = B.ishmemx_get_cutover(5)
+                    assert upto == B.SIZE_MAX or (pick < upto <= 16 << 20 and upto & (upto - 1) == 0)
+                    print(f"tuned host band up to {'the top' if upto == B.SIZE_MAX else upto}")
                 print(f"tuned cutover[{which}] = {'never' if pick == B.SIZE_MAX else pick}")
             with pytest.raises(B.IshmemError) as e:
                 B.ishmemx_tune_cutover(0, 0, 1 << 30, None)          # no room for the temporaries

@@ -241,6 +241,43 @@ def test_host_put_get_typed_nbi_cutover_and_copy_engine():
         assert s.status() == 0
 
 
+def test_host_cutover_is_a_band_between_two_sizes():
+    """The default host-initiated cutover follows the committed size sweep: the copy engine from
+    4 MiB up to (not including) 64 MiB, the tiled kernel below and above.  A kernel launch shows
+    in the library's launch counter, an engine copy does not; both paths are bit-exact."""
+    MiB = 1 << 20
+    npes, n_max = 2, 64 * MiB
+    with Session(npes, 2 * n_max + MiB) as s:
+        assert B.ishmemx_get_cutover(0) == 4 * MiB and B.ishmemx_get_cutover(5) == 64 * MiB
+        src, dst = s.malloc(n_max), s.malloc(n_max)
+        src.fill(0, inputs.byte_payload(12, 0, n_max))
+        for n, kernel in ((1 * MiB, True), (4 * MiB - 1, True), (4 * MiB, False), (16 * MiB, False),
+                          (64 * MiB - 1, False), (64 * MiB, True)):
+            before = B.ishmemx_launch_count()
+            B.ishmem_putmem(0, dst.addr, src.addr, n, 1)
+            assert (B.ishmemx_launch_count() - before == 1) == kernel, (n, kernel)
+            s.oracle.putmem(0, dst.ooff, s.oracle.ptr(src.ooff, n, 0), n, 1)
+            B.ishmem_quiet(0)
+            dst.assert_equal(f"put of {n} bytes")
+            before = B.ishmemx_launch_count()
+            B.ishmem_getmem(1, src.addr, dst.addr, n, 1 - 1)      # PE 1 reads PE 0's dst (zeros) into its src
+            assert (B.ishmemx_launch_count() - before == 1) == kernel, (n, kernel)
+            s.oracle.getmem(1, s.oracle.ptr(src.ooff, n, 1), dst.ooff, n, 0)
+        B.ishmem_barrier_all()
+        src.assert_equal("gets")
+        # the band can be moved and removed
+        B.ishmemx_set_cutover(5, B.SIZE_MAX)
+        before = B.ishmemx_launch_count()
+        B.ishmem_putmem(0, dst.addr, src.addr, 64 * MiB, 1)
+        assert B.ishmemx_launch_count() == before
+        B.ishmemx_set_cutover(5, 8 * MiB)
+        B.ishmem_putmem(0, dst.addr, src.addr, 8 * MiB, 1)
+        assert B.ishmemx_launch_count() == before + 1
+        B.ishmem_barrier_all()
+        dst.assert_equal("after moving the band")
+        assert s.status() == 0
+
+
 def test_scalar_p_g():
     with Session(3, 1 << 16) as s:
         buf = s.malloc(256)
@@ -325,8 +362,27 @@ def test_environment_variables_at_initialisation(monkeypatch):
     monkeypatch.setenv("ISHMEM_CUTOVER_PUT", "never")
     monkeypatch.setenv("ISHMEM_CUTOVER_BCAST", "always")
     monkeypatch.setenv("ISHMEM_CUTOVER_FCOLLECT", "0x10000")
+    monkeypatch.setenv("ISHMEM_CUTOVER_PUT_UPTO", str(1 << 20))
+    monkeypatch.setenv("ISHMEM_JACOBI_SPLIT", "columns")
+    monkeypatch.setenv("ISHMEM_JACOBI_FUSE", "0")
+    monkeypatch.setenv("ISHMEM_REDUCE_BULK", "1")
     B.ishmem_init(2, 0)
     try:
+        # launch-shape switches: initial values from the environment, then only set_option counts
+        assert B.ishmemx_get_cutover(5) == 1 << 20
+        assert B.ishmemx_get_option(B.ISHMEMX_OPT_JACOBI_SPLIT) == 2
+        assert B.ishmemx_get_option(B.ISHMEMX_OPT_JACOBI_FUSE) == 0
+        assert B.ishmemx_get_option(B.ISHMEMX_OPT_JACOBI_WIDE) == -1
+        assert B.ishmemx_get_option(B.ISHMEMX_OPT_REDUCE_BULK) == 1
+        monkeypatch.setenv("ISHMEM_JACOBI_SPLIT", "rows")            # not read again
+        assert B.ishmemx_get_option(B.ISHMEMX_OPT_JACOBI_SPLIT) == 2
+        B.ishmemx_set_option(B.ISHMEMX_OPT_JACOBI_SPLIT, 0)
+        assert B.ishmemx_get_option(B.ISHMEMX_OPT_JACOBI_SPLIT) == 0
+        for opt, bad in ((B.ISHMEMX_OPT_JACOBI_SPLIT, 3), (B.ISHMEMX_OPT_JACOBI_WIDE, -2), (99, 0),
+                         (B.ISHMEMX_OPT_BULK_SMEM, 100)):
+            with pytest.raises(B.IshmemError) as e:
+                B.ishmemx_set_option(opt, bad)
+            assert e.value.code == B.ISHMEM_ERR_ARG
         assert B.ishmemx_heap_bytes() == 3 << 20 and B.ishmem_n_pes() == 2
         assert B.ishmemx_get_cutover(0) == B.SIZE_MAX and B.ishmemx_get_cutover(1) == 0
         assert B.ishmemx_get_cutover(2) == 0x10000 and B.ishmemx_get_cutover(3) == B.SIZE_MAX

@@ -179,3 +179,16 @@ def test_association_order_of_the_update_is_pinned():
     full, _ = orc.jacobi(big, 1)
     assert full[3, 4] == 0.0
     assert orc.jacobi_cell(big[2:5, 3:6], 2, 3, 7, 8, 1, 3, 4) == 0.0
+
+
+def test_sweeps_compose():
+    """k sweeps followed by m sweeps of the result are k + m sweeps, bit for bit, and the
+    residual is that of the last sweep alone (the full-size GPU test continues the oracle's
+    eighth sweep into a ninth)."""
+    g = inputs.jacobi_grid(4, 37, 22)
+    u8, _ = orc.jacobi(g, 8)
+    u9, r9 = orc.jacobi(g, 9)
+    v9, s9 = orc.jacobi(u8, 1)
+    assert v9.tobytes() == u9.tobytes() and s9 == r9
+    w9, t9 = orc.jacobi(orc.jacobi(g, 4)[0], 5)
+    assert w9.tobytes() == u9.tobytes() and t9 == r9
