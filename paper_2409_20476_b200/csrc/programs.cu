@@ -1,6 +1,8 @@
 /* Device-initiated programs built on the device API: the put_signal / wait_until ping-pong
  * and the Jacobi overlap workload.  Both are co-resident (cooperative) launches in which
  * blocks of different PEs wait on one another with bounded waits. */
+#include <algorithm>
+#include <type_traits>
 #include <vector>
 
 #include "internal.h"
@@ -682,37 +684,32 @@ __global__ void __launch_bounds__(MAXT) k_jacobi(const ishmem_ctx_t *ctxs, jacob
 /* sender block b of a sweep: piece (b mod JACOBI_PIECES) of a PE's first or last row.  Out of line,
  * like the full-featured window below, so that the common path of k_jacobi_sweep keeps its
  * registers to itself. */
-static __device__ __noinline__ void jacobi_send_piece(const ishmem_ctx_t *ctxs, const double *cur0, double *nxt0,
-                                                      unsigned long long *sig0, size_t ny, size_t nx, unsigned b)
+static __device__ __noinline__ void jacobi_send_piece(const ishmem_ctx_t *ctxs, const double *cur0, unsigned long long *sig0,
+                                                      size_t ny, size_t nx, unsigned b)
 {
-    /* cur0, nxt0, sig0: PE 0's copies of the source buffer, of the other buffer (two-sweep passes
-     * only, else null) and of the signal words.  By value: a reference to the kernel's argument
-     * block would put it on every thread's stack.
-     * One sweep per launch: 2 x JACOBI_PIECES blocks per PE send its first row up and its last row
-     * down, into the halo rows of the neighbours' source buffers.  Two sweeps per launch: twice as
-     * many; the second set sends the second and the second-to-last row into the halo rows of the
-     * neighbours' OTHER buffer, which nothing else uses during the pass. */
+    /* cur0, sig0: PE 0's copies of the source buffer and of the signal words.  By value: a reference to
+     * the kernel's argument block would put it on every thread's stack.  2 x JACOBI_PIECES blocks per
+     * PE send its first row up and its last row down, into the halo rows of the neighbours' source
+     * buffers. */
     const int P = ctxs[0].npes;
-    const unsigned per_pe = (nxt0 ? 4u : 2u) * JACOBI_PIECES;
-    const int p = (int)(b / per_pe), down = (int)((b / JACOBI_PIECES) & 1u), second = (int)((b % per_pe) / (2u * JACOBI_PIECES));
+    const unsigned per_pe = 2u * JACOBI_PIECES;
+    const int p = (int)(b / per_pe), down = (int)((b / JACOBI_PIECES) & 1u);
     const unsigned piece = b % JACOBI_PIECES;
     const ishmem_ctx_t *ctx = ctxs + p;
     size_t first, rows, rows_above = 0, f2;
     strip_of(ny, P, p, &first, &rows);
     if (p > 0) strip_of(ny, P, p - 1, &f2, &rows_above);
     const double *cur = (const double *)local_of(ctxs, ctx, cur0);
-    /* the destination is named by the calling PE's copy of the buffer that receives it */
-    double *into = second ? (double *)local_of(ctxs, ctx, nxt0) : (double *)cur;
     unsigned long long *sig = (unsigned long long *)local_of(ctxs, ctx, sig0);
     const size_t per = ((nx + JACOBI_PIECES - 1) / JACOBI_PIECES + 1) & ~(size_t)1; /* even: 16-byte pieces */
     const size_t c_lo = per * piece < nx ? per * piece : nx, c_hi = c_lo + per < nx ? c_lo + per : nx;
-    if (!down && p > 0) /* my first (second) row -> bottom halo of the PE above */
-        ishmemx_putmem_signal_work_group(ctx, (void *)(into + (rows_above + 1) * nx + c_lo),
-                                         cur + (size_t)(second ? 2 : 1) * nx + c_lo, (c_hi - c_lo) * 8, sig + 1, 1,
-                                         ISHMEM_SIGNAL_ADD, p - 1);
-    if (down && p + 1 < P) /* my last (second-to-last) row -> top halo of the PE below */
-        ishmemx_putmem_signal_work_group(ctx, (void *)(into + c_lo), cur + (rows - (second ? 1 : 0)) * nx + c_lo,
-                                         (c_hi - c_lo) * 8, sig + 0, 1, ISHMEM_SIGNAL_ADD, p + 1);
+    /* the destination is named by the calling PE's copy of the buffer that receives it */
+    if (!down && p > 0) /* my first row -> bottom halo of the PE above */
+        ishmemx_putmem_signal_work_group(ctx, (void *)(cur + (rows_above + 1) * nx + c_lo), cur + nx + c_lo,
+                                         (c_hi - c_lo) * 8, sig + 1, 1, ISHMEM_SIGNAL_ADD, p - 1);
+    if (down && p + 1 < P) /* my last row -> top halo of the PE below */
+        ishmemx_putmem_signal_work_group(ctx, (void *)(cur + c_lo), cur + rows * nx + c_lo, (c_hi - c_lo) * 8, sig + 0, 1,
+                                         ISHMEM_SIGNAL_ADD, p + 1);
 }
 static __device__ __noinline__ double jacobi_march_one(const double *cur, double *nxt, unsigned ra, unsigned rb,
                                                        unsigned fixed0, unsigned fixed1, unsigned nx, bool want_res,
@@ -734,7 +731,7 @@ __global__ void __launch_bounds__(256, 4) k_jacobi_sweep(const ishmem_ctx_t *ctx
     const unsigned nsend = (unsigned)P * 2u * JACOBI_PIECES;
     unsigned b = blockIdx.x;
     if (b < nsend) {
-        jacobi_send_piece(ctxs, flip ? a.buf1 : a.buf0, nullptr, a.sig, a.ny, nx, b);
+        jacobi_send_piece(ctxs, flip ? a.buf1 : a.buf0, a.sig, a.ny, nx, b);
         return;
     }
     b -= nsend;
@@ -789,197 +786,285 @@ __global__ void __launch_bounds__(256, 4) k_jacobi_sweep(const ishmem_ctx_t *ctx
     }
 }
 
-/* ---- two sweeps per launch -------------------------------------------------------------------
- * Every element of the source is read once and the result of the SECOND sweep written once: half
- * the memory traffic per sweep.  A warp's window now carries two time levels.  It loads 64 columns
- * of rows ra-2 .. rb+1 of u(t); from each new row it forms the row above it of u(t+1) (valid in
- * lanes 1..30), keeps two rows of that level in registers as well, and from each new u(t+1) row
- * forms the row above of u(t+2) (valid in lanes 2..29: 56 output columns per tile), which is
- * stored.  The same expression, in the same order, gives every value, so the result is
- * bit-identical to two single sweeps; values in the shrinking border of a tile are recomputed by
- * the neighbouring tile.  Rows -1 and rows+2 (the second halo) are read from the halo rows of the
- * destination buffer, where this pass's senders put them. */
-template <int DEPTH>
-__device__ __forceinline__ double jacobi_march2(const double *cur, double *nxt, unsigned ra, unsigned rb, unsigned rows,
-                                                unsigned fixed0, unsigned fixed1, unsigned nx, bool want_res,
-                                                unsigned t_lo, unsigned t_hi)
+/* ---- K sweeps per launch ----------------------------------------------------------------------
+ * Every element of the source is read once and the result of the K-th sweep written once: 1/K of the
+ * memory traffic per sweep.  A warp's window carries K time levels.  Its lanes hold NC (2 or 4)
+ * neighbouring columns each, so a tile is 32 x NC loaded columns; the warp walks down the rows, and
+ * from each new row of u(t) it forms the row above it of u(t+1), from that the row above of u(t+2),
+ * and so on up to u(t+K), which is stored.  Per level two rows stay in registers (the one being
+ * formed replaces the older one, so nothing is moved: steps alternate between two unrolled copies of
+ * the code), and only a lane's outermost columns need their neighbours by shuffle.  Every value is
+ * the same expression, in the same order, as in a single sweep, so the result is bit-identical to K
+ * single sweeps.  Each level loses one column on either side of the tile; the lanes that still hold
+ * NC valid columns store (a tile stores (32 - 2 ceil(K / NC)) x NC columns), the rest is recomputed
+ * by the neighbouring tile.  A band of R rows reads R + 2K rows.
+ * Halo rows: K each way.  The first one goes where a single sweep puts it (the halo rows of the
+ * source buffer), the second one into the halo rows of the destination buffer, which nothing else
+ * uses during the pass, the third and fourth into four extra rows per PE that the library takes from
+ * the symmetric heap for the duration of the call. */
+#define JW_FULL 0xffffffffu
+
+template <int NC>
+__device__ __forceinline__ void jw_ld(const double *p, double (&v)[NC])
 {
-    double acc = 0.0;
-    if (rb <= ra) return acc;
-    const unsigned lane = threadIdx.x & 31u;
-    const unsigned full = 0xffffffffu;
-    const double2 zero = make_double2(0.0, 0.0);
-    const unsigned t = t_lo + (threadIdx.x >> 5);
-    if (t >= t_hi) return acc;
-    const int jl = (int)(t * 56u) - 4 + 2 * (int)lane; /* first column of this lane's pair */
-    const bool ld_ok = jl >= 0 && jl < (int)nx;
-    const bool st_ok = ld_ok && lane >= 2 && lane <= 29;
-    const unsigned j = ld_ok ? (unsigned)jl : 0u;
-    /* row r of u(t), r = -1 .. rows+2 (local numbering): the strip and its first halo rows in cur,
-     * the second halo rows in the halo rows of nxt */
-    int r_in = (int)ra - 2;
-    auto fetch = [&]() -> double2 {
-        const double *row = (r_in < 0)                 ? nxt
-                            : (r_in > (int)rows + 1)   ? nxt + (size_t)(rows + 1) * nx
-                                                       : cur + (size_t)r_in * nx;
-        ++r_in;
-        return ld_ok ? *(const double2 *)(row + j) : zero;
-    };
-    double2 a0 = fetch(), b0 = fetch(); /* u(t) rows ra-2, ra-1 */
-    double2 f[DEPTH];
+    if (NC == 4)
+        asm volatile("ld.global.v4.f64 {%0,%1,%2,%3}, [%4];"
+                     : "=d"(v[0]), "=d"(v[1]), "=d"(v[2 % NC]), "=d"(v[3 % NC])
+                     : "l"(p)
+                     : "memory");
+    else
+        asm volatile("ld.global.v2.f64 {%0,%1}, [%2];" : "=d"(v[0]), "=d"(v[1]) : "l"(p) : "memory");
+}
+template <int NC>
+__device__ __forceinline__ void jw_st(double *p, const double (&v)[NC])
+{
+    if (NC == 4)
+        asm volatile("st.global.v4.f64 [%0], {%1,%2,%3,%4};" ::"l"(p), "d"(v[0]), "d"(v[1]), "d"(v[2 % NC]), "d"(v[3 % NC])
+                     : "memory");
+    else
+        asm volatile("st.global.v2.f64 [%0], {%1,%2};" ::"l"(p), "d"(v[0]), "d"(v[1]) : "memory");
+}
+/* column pairs whose bit in `ok` is clear lie outside the grid: not touched, read as zero */
+template <int NC>
+__device__ __forceinline__ void jw_ld_edge(const double *p, double (&v)[NC], unsigned ok)
+{
 #pragma unroll
-    for (int s = 0; s < DEPTH; ++s) f[s] = (r_in <= (int)rb + 1) ? fetch() : zero;
-    double ml0 = __shfl_up_sync(full, b0.y, 1), mr0 = __shfl_down_sync(full, b0.x, 1);
-    double2 a1 = zero, b1 = zero; /* u(t+1) rows r-2, r-1 */
-    double ml1 = 0.0, mr1 = 0.0;
-    double *po = nxt + (size_t)ra * nx + j;
-    for (unsigned r = ra - 1; r <= rb; r += DEPTH) { /* r: the u(t+1) row formed in this step */
+    for (int h = 0; h < NC / 2; ++h) {
+        double2 a = make_double2(0.0, 0.0);
+        if (ok & (1u << h)) a = *(const double2 *)(p + 2 * h);
+        v[2 * h] = a.x, v[2 * h + 1] = a.y;
+    }
+}
+
+template <int K, int NC>
+struct jw_window {
+    double w[K][2][NC]; /* level l: the two rows above the one being formed; which is which alternates */
+};
+struct jw_edge {
+    unsigned fixcol;    /* bit i: the lane's column i is the grid's first or last column */
+    int fixed0, fixed1; /* local numbers of the grid's first / last row, or a value never reached */
+};
+template <int K, int NC>
+struct jw_geo {
+    static constexpr int SKIP = (K + NC - 1) / NC;    /* lanes without a full result on either side */
+    static constexpr int TILE = (32 - 2 * SKIP) * NC; /* columns a warp stores */
+};
+
+/* One step of the window: `c` comes in as row R of u(t) and leaves as row R-K of u(t+K).  P: parity of
+ * the step (selects which of a level's two rows is the older one).  FILL: index of the step while the
+ * window fills -- levels whose inputs are not there yet are skipped -- or -1 in the steady state.
+ * rmask: bit h = the lane's column pair h counts for the residual. */
+template <int K, int NC, int P, bool EDGE, bool RES, int FILL>
+__device__ __forceinline__ void jw_step(jw_window<K, NC> &W, double (&c)[NC], int R, const jw_edge &e, double &acc,
+                                        unsigned rmask)
+{
 #pragma unroll
-        for (int s = 0; s < DEPTH; ++s) {
-            const unsigned rr = r + s;
-            if (rr <= rb) { /* uniform over the warp */
-                const double2 c0 = f[s]; /* u(t) row rr + 1 */
-                if (r_in <= (int)rb + 1) f[s] = fetch();
-                double2 n1 = b0;
-                if (rr != fixed0 && rr != fixed1) {
-                    if (j != 0) n1.x = 0.25 * ((a0.x + c0.x) + (ml0 + b0.y));
-                    if (j + 2 != nx) n1.y = 0.25 * ((a0.y + c0.y) + (b0.x + mr0));
-                }
-                const double nl = __shfl_up_sync(full, n1.y, 1), nr = __shfl_down_sync(full, n1.x, 1);
-                if (rr >= ra + 1) { /* u(t+2) row rr - 1 from u(t+1) rows rr-2, rr-1, rr */
-                    double2 o = b1;
-                    if (rr - 1 != fixed0 && rr - 1 != fixed1) {
-                        if (j != 0) o.x = 0.25 * ((a1.x + n1.x) + (ml1 + b1.y));
-                        if (j + 2 != nx) o.y = 0.25 * ((a1.y + n1.y) + (b1.x + mr1));
-                        if (want_res && st_ok) {
-                            const double dx = o.x - b1.x, dy = o.y - b1.y;
-                            acc += dx * dx;
-                            acc += dy * dy;
-                        }
-                    }
-                    if (st_ok) *(double2 *)po = o;
-                    po += nx;
-                }
-                a1 = b1;
-                b1 = n1;
-                ml1 = nl;
-                mr1 = nr;
-                a0 = b0;
-                b0 = c0;
-                ml0 = __shfl_up_sync(full, c0.y, 1);
-                mr0 = __shfl_down_sync(full, c0.x, 1);
-            }
+    for (int l = 0; l < K; ++l) {
+        const bool compute = FILL < 0 || FILL >= 2 * l;
+        const bool keep = compute || FILL >= 2 * l - 2; /* the incoming row of level l is valid: keep it */
+        if (!keep) break;
+        double(&up)[NC] = W.w[l][P];
+        double(&mid)[NC] = W.w[l][P ^ 1];
+        if (!compute) {
+#pragma unroll
+            for (int i = 0; i < NC; ++i) up[i] = c[i];
+            break;
         }
+        /* the lane's outer neighbours in the middle row */
+        const double nl = __shfl_up_sync(JW_FULL, mid[NC - 1], 1), nr = __shfl_down_sync(JW_FULL, mid[0], 1);
+        double o[NC];
+#pragma unroll
+        for (int i = 0; i < NC; ++i) {
+            const double left = i > 0 ? mid[i > 0 ? i - 1 : 0] : nl;
+            const double right = i < NC - 1 ? mid[i < NC - 1 ? i + 1 : 0] : nr;
+            o[i] = 0.25 * ((up[i] + c[i]) + (left + right));
+        }
+        if (EDGE) {
+            const int q = R - 1 - l; /* the row of level l+1 formed here */
+            const bool fixed_row = q == e.fixed0 || q == e.fixed1;
+#pragma unroll
+            for (int i = 0; i < NC; ++i)
+                if (fixed_row || (e.fixcol & (1u << i))) o[i] = mid[i];
+        }
+        if (RES && l == K - 1) {
+#pragma unroll
+            for (int i = 0; i < NC; ++i)
+                if (rmask & (1u << (i >> 1))) {
+                    const double d = o[i] - mid[i];
+                    acc += d * d;
+                }
+        }
+#pragma unroll
+        for (int i = 0; i < NC; ++i) {
+            up[i] = c[i]; /* the older row is done with: the incoming one takes its place */
+            c[i] = o[i];
+        }
+    }
+}
+
+/* where the rows of u(t) around a strip live (see the section comment) */
+struct jw_rows {
+    const double *cur; /* local rows 0 .. rows+1 */
+    const double *nxt; /* its rows 0 and rows+1 hold local rows -1 and rows+2 during the pass */
+    const double *xh;  /* four rows: local rows -2, -3, rows+3, rows+4 */
+    int rows;
+    size_t nx;
+    __device__ __forceinline__ const double *at(int r) const
+    {
+        if (r < 0) return r == -1 ? nxt : xh + (size_t)(-r - 2) * nx;
+        if (r > rows + 1) return r == rows + 2 ? nxt + (size_t)(rows + 1) * nx : xh + (size_t)(r - rows - 1) * nx;
+        return cur + (size_t)r * nx;
+    }
+};
+
+/* Rows [ra, rb) of the strip, tile t, by one warp.  D rows are in flight per lane.  EDGE: the tile
+ * touches the grid's first or last column or a column outside it, or the band reads rows outside the
+ * source buffer, or forms one of the grid's fixed rows; without EDGE nothing of that is tested.
+ * Returns the lane's share of the squared last update when RES. */
+template <int K, int NC, int D, bool EDGE, bool RES>
+__device__ __forceinline__ double jw_march(const jw_rows &src, double *nxt, int ra, int rb, int t, int fixed0, int fixed1)
+{
+    static_assert(D == 2 || D == 4, "the unrolled loop keeps the step parity");
+    static_assert(K >= 2 && K <= 4, "window depth");
+    using G = jw_geo<K, NC>;
+    const int lane = threadIdx.x & 31;
+    const int nx = (int)src.nx;
+    const int jA = t * G::TILE - G::SKIP * NC + NC * lane;
+    unsigned ok = 0;
+#pragma unroll
+    for (int h = 0; h < NC / 2; ++h)
+        if (!EDGE || (jA + 2 * h >= 0 && jA + 2 * h < nx)) ok |= 1u << h;
+    const bool st_lane = lane >= G::SKIP && lane < 32 - G::SKIP;
+    jw_edge e;
+    e.fixcol = 0;
+#pragma unroll
+    for (int i = 0; i < NC; ++i)
+        if (EDGE && (jA + i == 0 || jA + i == nx - 1)) e.fixcol |= 1u << i;
+    e.fixed0 = fixed0, e.fixed1 = fixed1;
+    const unsigned rmask = st_lane ? ok : 0u;
+    const int n_steps = (rb - ra) + 2 * K - 2;
+    const size_t pitch = src.nx;
+    const int jbase = (ok & 1u) ? jA : 0;
+    jw_window<K, NC> W;
+#pragma unroll
+    for (int l = 1; l < K; ++l)
+#pragma unroll
+        for (int i = 0; i < NC; ++i) W.w[l][0][i] = W.w[l][1][i] = 0.0;
+    double acc = 0.0;
+    double f[D][NC]; /* rows in flight */
+    int r_next = ra - K;
+    const double *pin = src.cur + (size_t)r_next * pitch + jbase; /* without EDGE all rows are in the source buffer */
+    auto request = [&](double(&v)[NC]) {
+        if (EDGE) {
+            jw_ld_edge<NC>(src.at(r_next) + jbase, v, ok);
+        } else {
+            jw_ld<NC>(pin, v);
+            pin += pitch;
+        }
+        ++r_next;
+    };
+    /* everything the window starts from is requested before the first use */
+    request(W.w[0][0]);
+    request(W.w[0][1]);
+#pragma unroll
+    for (int s = 0; s < D; ++s) {
+        if (s < n_steps) request(f[s]);
+        else {
+#pragma unroll
+            for (int i = 0; i < NC; ++i) f[s][i] = 0.0;
+        }
+    }
+    double *po = nxt + (size_t)ra * pitch + jbase;
+    int s = 0;
+    auto one = [&](auto slot, auto parity, auto fill) {
+        constexpr int S = decltype(slot)::value, P = decltype(parity)::value, F = decltype(fill)::value;
+        double c[NC];
+#pragma unroll
+        for (int i = 0; i < NC; ++i) c[i] = f[S][i];
+        if (s + D < n_steps) request(f[S]);
+        jw_step<K, NC, P, EDGE, RES, F>(W, c, ra - K + 2 + s, e, acc, rmask);
+        if (F < 0) {
+            if (EDGE) {
+#pragma unroll
+                for (int h = 0; h < NC / 2; ++h)
+                    if (st_lane && (ok & (1u << h))) *(double2 *)(po + 2 * h) = make_double2(c[2 * h], c[2 * h + 1]);
+            } else if (st_lane) {
+                jw_st<NC>(po, c);
+            }
+            po += pitch;
+        }
+        ++s;
+    };
+    /* the window fills: steps 0 .. 2K-3, none of which stores */
+#define JW_FILL(I)                                                                                              \
+    if ((I) < 2 * K - 2 && s < n_steps)                                                                         \
+        one(std::integral_constant<int, (I) % D>{}, std::integral_constant<int, (I)&1>{},                       \
+            std::integral_constant<int, (I) < 2 * K - 2 ? (I) : -1>{});
+    JW_FILL(0) JW_FILL(1) JW_FILL(2) JW_FILL(3) JW_FILL(4) JW_FILL(5)
+#undef JW_FILL
+    /* steady state: D steps per trip, slots and parities known at compile time */
+    constexpr int S0 = (2 * K - 2) % D;
+    while (s < n_steps) {
+#define JW_STEP(U)                                                                                              \
+    if ((U) < D && s < n_steps)                                                                                 \
+        one(std::integral_constant<int, (S0 + (U)) % D>{}, std::integral_constant<int, (U)&1>{},                \
+            std::integral_constant<int, -1>{});
+        JW_STEP(0) JW_STEP(1) JW_STEP(2) JW_STEP(3)
+#undef JW_STEP
     }
     return acc;
 }
 
-/* The two-level window with FOUR columns per lane (two pairs, A and B): a tile is 128 loaded and 120
- * stored columns, the neighbours inside a lane cost nothing, and only the lane's outer neighbours
- * travel by shuffle -- half the shuffles per cell of jacobi_march2, and 6 % instead of 12 % of the
- * columns computed twice. */
-template <int DEPTH>
-__device__ __forceinline__ double jacobi_march2w(const double *cur, double *nxt, unsigned ra, unsigned rb, unsigned rows,
-                                                 unsigned fixed0, unsigned fixed1, unsigned nx, bool want_res,
-                                                 unsigned t_lo, unsigned t_hi)
+/* sender block b of a K-sweep pass: piece (b mod JACOBI_PIECES) of one of the K first or K last rows of
+ * a PE's strip, into the neighbour's row of the same depth (see jw_rows for where that is) */
+static __device__ __noinline__ void jacobi_send_piece_k(const ishmem_ctx_t *ctxs, const double *cur0, double *nxt0,
+                                                        double *xh0, unsigned long long *sig0, size_t ny, size_t nx,
+                                                        unsigned b, unsigned K)
 {
-    double acc = 0.0;
-    if (rb <= ra) return acc;
-    const unsigned lane = threadIdx.x & 31u;
-    const unsigned full = 0xffffffffu;
-    const double2 zero = make_double2(0.0, 0.0);
-    const unsigned t = t_lo + (threadIdx.x >> 5);
-    if (t >= t_hi) return acc;
-    const int jA = (int)(t * 120u) - 4 + 4 * (int)lane, jB = jA + 2; /* first columns of this lane's two pairs */
-    const bool okA = jA >= 0 && jA < (int)nx, okB = jB >= 0 && jB < (int)nx;
-    const bool stA = okA && lane >= 1 && lane <= 30, stB = okB && lane >= 1 && lane <= 30;
-    int r_in = (int)ra - 2;
-    auto fetch = [&](double2 &A, double2 &B) {
-        const double *row = (r_in < 0)               ? nxt
-                            : (r_in > (int)rows + 1) ? nxt + (size_t)(rows + 1) * nx
-                                                     : cur + (size_t)r_in * nx;
-        ++r_in;
-        A = okA ? *(const double2 *)(row + jA) : zero;
-        B = okB ? *(const double2 *)(row + jB) : zero;
-    };
-    double2 a0A, a0B, b0A, b0B;
-    fetch(a0A, a0B);
-    fetch(b0A, b0B);
-    double2 fA[DEPTH], fB[DEPTH];
-#pragma unroll
-    for (int s = 0; s < DEPTH; ++s) {
-        fA[s] = fB[s] = zero;
-        if (r_in <= (int)rb + 1) fetch(fA[s], fB[s]);
+    const int P = ctxs[0].npes;
+    const unsigned per_pe = 2u * K * JACOBI_PIECES;
+    const int p = (int)(b / per_pe), down = (int)((b / JACOBI_PIECES) & 1u);
+    const unsigned depth = (b % per_pe) / (2u * JACOBI_PIECES), piece = b % JACOBI_PIECES; /* depth 0: the edge row itself */
+    const ishmem_ctx_t *ctx = ctxs + p;
+    size_t first, rows, rows_above = 0, f2;
+    strip_of(ny, P, p, &first, &rows);
+    if (p > 0) strip_of(ny, P, p - 1, &f2, &rows_above);
+    const double *cur = (const double *)local_of(ctxs, ctx, cur0);
+    double *nxt = (double *)local_of(ctxs, ctx, nxt0), *xh = (double *)local_of(ctxs, ctx, xh0);
+    unsigned long long *sig = (unsigned long long *)local_of(ctxs, ctx, sig0);
+    const size_t per = ((nx + JACOBI_PIECES - 1) / JACOBI_PIECES + 1) & ~(size_t)1; /* even: 16-byte pieces */
+    const size_t c_lo = per * piece < nx ? per * piece : nx, c_hi = c_lo + per < nx ? c_lo + per : nx;
+    /* destinations are named by the calling PE's copy of the object that receives them */
+    if (!down && p > 0) { /* my row 1 + depth -> row rows_above + 1 + depth of the PE above */
+        double *into = depth == 0   ? (double *)cur + (rows_above + 1) * nx
+                       : depth == 1 ? nxt + (rows_above + 1) * nx
+                                    : xh + (size_t)(depth) * nx; /* its rows+3, rows+4: slots 2, 3 */
+        ishmemx_putmem_signal_work_group(ctx, (void *)(into + c_lo), cur + (size_t)(1 + depth) * nx + c_lo,
+                                         (c_hi - c_lo) * 8, sig + 1, 1, ISHMEM_SIGNAL_ADD, p - 1);
     }
-    double ml0 = __shfl_up_sync(full, b0B.y, 1), mr0 = __shfl_down_sync(full, b0A.x, 1);
-    double2 a1A = zero, a1B = zero, b1A = zero, b1B = zero;
-    double ml1 = 0.0, mr1 = 0.0;
-    double *po = nxt + (size_t)ra * nx + (okA ? jA : 0);
-    for (unsigned r = ra - 1; r <= rb; r += DEPTH) {
-#pragma unroll
-        for (int s = 0; s < DEPTH; ++s) {
-            const unsigned rr = r + s;
-            if (rr <= rb) {
-                const double2 c0A = fA[s], c0B = fB[s];
-                if (r_in <= (int)rb + 1) fetch(fA[s], fB[s]);
-                double2 n1A = b0A, n1B = b0B;
-                if (rr != fixed0 && rr != fixed1) {
-                    if (jA != 0) n1A.x = 0.25 * ((a0A.x + c0A.x) + (ml0 + b0A.y));
-                    if (jA + 2 != (int)nx) n1A.y = 0.25 * ((a0A.y + c0A.y) + (b0A.x + b0B.x));
-                    n1B.x = 0.25 * ((a0B.x + c0B.x) + (b0A.y + b0B.y));
-                    if (jB + 2 != (int)nx) n1B.y = 0.25 * ((a0B.y + c0B.y) + (b0B.x + mr0));
-                }
-                const double nl = __shfl_up_sync(full, n1B.y, 1), nr = __shfl_down_sync(full, n1A.x, 1);
-                if (rr >= ra + 1) {
-                    double2 oA = b1A, oB = b1B;
-                    if (rr - 1 != fixed0 && rr - 1 != fixed1) {
-                        if (jA != 0) oA.x = 0.25 * ((a1A.x + n1A.x) + (ml1 + b1A.y));
-                        if (jA + 2 != (int)nx) oA.y = 0.25 * ((a1A.y + n1A.y) + (b1A.x + b1B.x));
-                        oB.x = 0.25 * ((a1B.x + n1B.x) + (b1A.y + b1B.y));
-                        if (jB + 2 != (int)nx) oB.y = 0.25 * ((a1B.y + n1B.y) + (b1B.x + mr1));
-                        if (want_res) {
-                            if (stA) {
-                                const double dx = oA.x - b1A.x, dy = oA.y - b1A.y;
-                                acc += dx * dx;
-                                acc += dy * dy;
-                            }
-                            if (stB) {
-                                const double dx = oB.x - b1B.x, dy = oB.y - b1B.y;
-                                acc += dx * dx;
-                                acc += dy * dy;
-                            }
-                        }
-                    }
-                    if (stA) *(double2 *)po = oA;
-                    if (stB) *(double2 *)(po + 2) = oB;
-                    po += nx;
-                }
-                a1A = b1A, a1B = b1B;
-                b1A = n1A, b1B = n1B;
-                ml1 = nl, mr1 = nr;
-                a0A = b0A, a0B = b0B;
-                b0A = c0A, b0B = c0B;
-                ml0 = __shfl_up_sync(full, c0B.y, 1);
-                mr0 = __shfl_down_sync(full, c0A.x, 1);
-            }
-        }
+    if (down && p + 1 < P) { /* my row rows - depth -> row -depth of the PE below */
+        double *into = depth == 0 ? (double *)cur : depth == 1 ? nxt : xh + (size_t)(depth - 2) * nx; /* slots 0, 1 */
+        ishmemx_putmem_signal_work_group(ctx, (void *)(into + c_lo), cur + (rows - depth) * nx + c_lo,
+                                         (c_hi - c_lo) * 8, sig + 0, 1, ISHMEM_SIGNAL_ADD, p + 1);
     }
-    return acc;
 }
 
-/* one launch = two sweeps: sender blocks (two rows each way per PE), then one block per band of
- * `band_rows` rows x 8 tiles of 56 columns, in launch order as in k_jacobi_sweep */
-template <bool WIDE>
-__global__ void __launch_bounds__(256, WIDE ? 2 : 3) k_jacobi_pass2(const ishmem_ctx_t *ctxs, jacobi_args a, int flip,
-                                                          unsigned long long arrived, int last, unsigned band_rows,
-                                                          unsigned bands, unsigned tile_groups, int P, size_t heap_stride)
+/* one launch = K sweeps: sender blocks (K rows each way per PE), then one block per band of `band_rows`
+ * rows x (blockDim / 32) tiles, in launch order as in k_jacobi_sweep */
+#define JACOBI_PASS_THREADS 128
+template <int K, int NC>
+__global__ void __launch_bounds__(JACOBI_PASS_THREADS, 4) k_jacobi_pass(const ishmem_ctx_t *ctxs, jacobi_args a, double *xh0,
+                                                                        int flip, unsigned long long arrived, int last,
+                                                                        unsigned band_rows, unsigned bands,
+                                                                        unsigned tile_groups, int P, size_t heap_stride)
 {
+    using G = jw_geo<K, NC>;
     const unsigned tid = threadIdx.x;
     const size_t nx = a.nx;
-    const unsigned nsend = (unsigned)P * 4u * JACOBI_PIECES;
+    const unsigned nsend = (unsigned)P * 2u * K * JACOBI_PIECES;
     unsigned b = blockIdx.x;
     if (b < nsend) {
-        jacobi_send_piece(ctxs, flip ? a.buf1 : a.buf0, flip ? a.buf0 : a.buf1, a.sig, a.ny, nx, b);
+        jacobi_send_piece_k(ctxs, flip ? a.buf1 : a.buf0, flip ? a.buf0 : a.buf1, xh0, a.sig, a.ny, nx, b, K);
         return;
     }
     b -= nsend;
@@ -987,15 +1072,16 @@ __global__ void __launch_bounds__(256, WIDE ? 2 : 3) k_jacobi_pass2(const ishmem
     const unsigned band = (b / tile_groups) % bands, tg = b % tile_groups;
     const ishmem_ctx_t *ctx = ctxs + p;
     const unsigned base_rows = (unsigned)a.ny / (unsigned)P, extra = (unsigned)a.ny % (unsigned)P;
-    const unsigned rows = base_rows + ((unsigned)p < extra ? 1u : 0u);
+    const int rows = (int)(base_rows + ((unsigned)p < extra ? 1u : 0u));
     const unsigned first = (unsigned)p * base_rows + ((unsigned)p < extra ? (unsigned)p : extra);
-    const unsigned ra = 1u + band * band_rows;
-    const unsigned rb = (ra + band_rows < rows + 1u) ? ra + band_rows : rows + 1u;
+    const int ra = 1 + (int)(band * band_rows);
+    const int rb = (ra + (int)band_rows < rows + 1) ? ra + (int)band_rows : rows + 1;
     double acc = 0.0;
     __shared__ int give_up;
     if (ra < rb) {
-        /* the first band of a strip reads the two halo rows above it, the last one the two below */
-        const bool top = (band == 0 || !a.overlap) && p > 0, bottom = (rb == rows + 1u || !a.overlap) && p + 1 < P;
+        /* a band that reads rows above the strip needs the K halo rows from above, one that reads rows
+         * below it those from below (overlap = 0: every band waits for both: exchange, wait, compute) */
+        const bool top = (ra - K < 1 || !a.overlap) && p > 0, bottom = (rb - 1 + K > rows || !a.overlap) && p + 1 < P;
         if (top || bottom) {
             if (tid == 0) {
                 const unsigned long long *sig = (const unsigned long long *)local_of(ctxs, ctx, a.sig);
@@ -1006,17 +1092,34 @@ __global__ void __launch_bounds__(256, WIDE ? 2 : 3) k_jacobi_pass2(const ishmem
             __syncthreads();
             if (give_up) return;
         }
-        const double *cur = (const double *)((const char *)(flip ? a.buf1 : a.buf0) + (size_t)p * heap_stride);
+        jw_rows src;
+        src.cur = (const double *)((const char *)(flip ? a.buf1 : a.buf0) + (size_t)p * heap_stride);
         double *nxt = (double *)((char *)(flip ? a.buf0 : a.buf1) + (size_t)p * heap_stride);
-        const unsigned fixed0 = (first == 0) ? 1u : ~0u;
-        const unsigned fixed1 = (first + rows == (unsigned)a.ny) ? rows : ~0u;
-        const unsigned ntiles = (unsigned)((nx + (WIDE ? 119 : 55)) / (WIDE ? 120 : 56)), t_lo = tg * (blockDim.x >> 5);
-        const unsigned t_hi = t_lo + (blockDim.x >> 5) < ntiles ? t_lo + (blockDim.x >> 5) : ntiles;
-        acc = WIDE ? jacobi_march2w<2>(cur, nxt, ra, rb, rows, fixed0, fixed1, (unsigned)nx, last != 0, t_lo, t_hi)
-                   : jacobi_march2<3>(cur, nxt, ra, rb, rows, fixed0, fixed1, (unsigned)nx, last != 0, t_lo, t_hi);
+        src.nxt = nxt;
+        src.xh = (const double *)((const char *)xh0 + (size_t)p * heap_stride);
+        src.rows = rows;
+        src.nx = nx;
+        const int fixed0 = (first == 0) ? 1 : -100;
+        const int fixed1 = (first + (unsigned)rows == (unsigned)a.ny) ? rows : -100;
+        const int ntiles = (int)((nx + G::TILE - 1) / G::TILE);
+        const int t = (int)(tg * (blockDim.x >> 5) + (tid >> 5));
+        if (t < ntiles) {
+            const int j0 = t * G::TILE - G::SKIP * NC;
+            /* the plain form: all loaded columns inside the grid and none of them its first or last one,
+             * all rows read inside the source buffer, no fixed row among the rows formed */
+            const bool plain = j0 > 0 && j0 + 32 * NC < (int)nx && ra - K >= 0 && rb - 1 + K <= rows + 1 &&
+                               !(fixed0 >= ra - K + 1 && fixed0 <= rb + K - 2) &&
+                               !(fixed1 >= ra - K + 1 && fixed1 <= rb + K - 2);
+            if (last)
+                acc = jw_march<K, NC, 2, true, true>(src, nxt, ra, rb, t, fixed0, fixed1);
+            else if (plain)
+                jw_march<K, NC, 2, false, false>(src, nxt, ra, rb, t, fixed0, fixed1);
+            else
+                jw_march<K, NC, 2, true, false>(src, nxt, ra, rb, t, fixed0, fixed1);
+        }
     }
     if (last) {
-        __shared__ double red[8];
+        __shared__ double red[JACOBI_PASS_THREADS / 32];
         for (int o = 16; o > 0; o >>= 1) acc += __shfl_down_sync(0xffffffffu, acc, o);
         if ((tid & 31u) == 0) red[tid >> 5] = acc;
         __syncthreads();
@@ -1116,53 +1219,133 @@ static int jacobi_launch(double *buf0, double *buf1, uint64_t *sig, size_t ny, s
     return rc;
 }
 
-/* one launch per sweep (k_jacobi_sweep); `partial` receives one residual term per tile block */
+/* one launch per sweep (k_jacobi_sweep): bands of 16 rows x 8 tiles of 60 columns per block */
 #define JACOBI_BAND_ROWS 16u /* measured at 16384^2: 8 rows 687 us, 12: 663, 16: 652, 20: 652, 24: 659, 32: 666, 64: 680 */
-/* two sweeps per launch: a band pays four extra rows instead of two, and the pass is bound by
- * instructions rather than memory, so taller bands win (16384^2, per sweep: 16 rows 501 us, 32: 481,
- * 64: 469, 128: 461) */
-#define JACOBI_BAND_ROWS2 64u
-static size_t jacobi_sweep_blocks(size_t ny, size_t nx, unsigned *bands, unsigned *tile_groups, unsigned tile_cols = 60)
+/* K sweeps per launch (k_jacobi_pass): a band pays 2K extra rows, so it is taller; 64 and 128 rows
+ * measure the same at 16384^2 and 64 gives small grids more blocks */
+#define JACOBI_PASS_BAND_ROWS 64u
+
+/* The launches of one call.  Every launch moves the grid from one buffer to the other, and the result
+ * has to end where `iters` single sweeps would leave it (buf0 for an even count), so the number of
+ * launches has the parity of iters.  Within that the split is the cheapest one by the measured time of
+ * a launch of 1, 2, 3 and 4 sweeps at 16384^2 (650, 850, 820 and 900 us: a launch costs about the same
+ * whatever its depth, so deep launches win and a single sweep is the cheapest filler). */
+struct jacobi_plan {
+    std::vector<int> depth; /* sweeps of each launch, deepest first */
+    int nc;                 /* columns per lane of the multi-sweep launches */
+    unsigned bands1, groups1, bands_k;
+    unsigned groups_k[5];   /* tile groups per band of a launch of depth k */
+    size_t blocks_last;     /* tile blocks (= residual terms) of the last launch */
+    bool needs_xh;          /* some launch is deeper than two sweeps */
+};
+
+static void jacobi_split(int iters, int kmax, std::vector<int> *out)
+{
+    static const double cost[5] = {0, 650, 850, 820, 900};
+    out->clear();
+    int full = 0, r = iters;
+    while (r > 24) { /* far from the end only the deepest launch is ever right */
+        r -= kmax;
+        ++full;
+    }
+    const double inf = 1e30;
+    double best[25][2];
+    int pick[25][2];
+    best[0][0] = 0, best[0][1] = inf;
+    pick[0][0] = pick[0][1] = 0;
+    for (int n = 1; n <= r; ++n)
+        for (int par = 0; par < 2; ++par) {
+            best[n][par] = inf;
+            pick[n][par] = 0;
+            for (int k = 1; k <= kmax && k <= n; ++k)
+                if (cost[k] + best[n - k][par ^ 1] < best[n][par]) {
+                    best[n][par] = cost[k] + best[n - k][par ^ 1];
+                    pick[n][par] = k;
+                }
+        }
+    int par = (iters - full) & 1; /* launches still to come must have this parity */
+    for (int i = 0; i < full; ++i) out->push_back(kmax);
+    for (int n = r; n > 0;) {
+        const int k = pick[n][par];
+        if (k == 0) { /* no split of this parity (cannot happen for n >= 1 with k = 1 allowed and parity n) */
+            out->assign((size_t)iters, 1);
+            return;
+        }
+        out->push_back(k);
+        n -= k;
+        par ^= 1;
+    }
+    std::sort(out->begin(), out->end(), [](int x, int y) { return x > y; });
+}
+
+static unsigned jacobi_pass_groups(size_t nx, int k, int nc)
+{
+    const unsigned skip = (unsigned)((k + nc - 1) / nc), tile = (32u - 2u * skip) * (unsigned)nc;
+    const unsigned ntiles = (unsigned)((nx + tile - 1) / tile), warps = JACOBI_PASS_THREADS / 32;
+    return (ntiles + warps - 1) / warps;
+}
+
+/* kmax: the deepest launch allowed (the caller lowers it to 2 when the symmetric heap has no room for
+ * the extra halo rows) */
+static void jacobi_make_plan(size_t ny, size_t nx, int iters, int kmax, jacobi_plan *pl)
 {
     auto &g = g_ishmem;
-    const size_t rows_max = (ny + g.npes - 1) / g.npes;
-    const unsigned band_rows = tile_cols == 60 ? JACOBI_BAND_ROWS : JACOBI_BAND_ROWS2;
-    *bands = (unsigned)((rows_max + band_rows - 1) / band_rows);
-    *tile_groups = (unsigned)(((nx + tile_cols - 1) / tile_cols + 7) / 8);
-    return (size_t)g.npes * *bands * *tile_groups;
+    const size_t rows_min = ny / (size_t)g.npes, rows_max = (ny + g.npes - 1) / g.npes;
+    /* ISHMEMX_OPT_JACOBI_FUSE: 0 = single sweeps only, 1 = the library's choice, 2..4 = at most that deep */
+    const long long fuse = g.opt[ISHMEMX_OPT_JACOBI_FUSE];
+    if (fuse == 0) kmax = 1;
+    else if (fuse >= 2 && fuse < kmax) kmax = (int)fuse;
+    /* a strip sends its k first and k last rows: it must own that many */
+    if ((size_t)kmax > rows_min) kmax = rows_min < 1 ? 1 : (int)rows_min;
+    jacobi_split(iters, kmax, &pl->depth);
+    pl->bands1 = (unsigned)((rows_max + JACOBI_BAND_ROWS - 1) / JACOBI_BAND_ROWS);
+    pl->groups1 = (unsigned)(((nx + 59) / 60 + 7) / 8);
+    pl->bands_k = (unsigned)((rows_max + JACOBI_PASS_BAND_ROWS - 1) / JACOBI_PASS_BAND_ROWS);
+    /* four columns per lane (32-byte accesses: nx a multiple of 4) unless the grid is too small to give
+     * every SM its blocks that way; ISHMEMX_OPT_JACOBI_WIDE = 0 / 1 decides otherwise */
+    const long long wide = g.opt[ISHMEMX_OPT_JACOBI_WIDE];
+    pl->nc = 4;
+    if (nx % 4 != 0 || wide == 0) pl->nc = 2;
+    else if (wide < 0 && (size_t)g.npes * pl->bands_k * jacobi_pass_groups(nx, 4, 4) < (size_t)g.sm_count * 8) pl->nc = 2;
+    pl->needs_xh = false;
+    for (int k = 2; k <= 4; ++k) pl->groups_k[k] = jacobi_pass_groups(nx, k, pl->nc);
+    for (int k : pl->depth) pl->needs_xh |= k > 2;
+    const int k_last = pl->depth.empty() ? 1 : pl->depth.back();
+    pl->blocks_last = k_last == 1 ? (size_t)g.npes * pl->bands1 * pl->groups1
+                                  : (size_t)g.npes * pl->bands_k * pl->groups_k[k_last];
+    if (pl->depth.empty()) pl->blocks_last = 0;
 }
-/* ISHMEMX_OPT_JACOBI_FUSE = 0 keeps one sweep per launch */
-static bool jacobi_fuse(size_t ny)
+
+template <int NC>
+static void jacobi_launch_pass(int k, unsigned nblocks, cudaStream_t s, const jacobi_args &a, double *xh, int flip,
+                               unsigned long long arrived, int last, unsigned bands, unsigned groups)
 {
-    if (g_ishmem.opt[ISHMEMX_OPT_JACOBI_FUSE] == 0) return false;
-    return ny / (size_t)g_ishmem.npes >= 2; /* the second halo row must be a row of the neighbour's strip */
+    auto &g = g_ishmem;
+    switch (k) {
+    case 2:
+        k_jacobi_pass<2, NC><<<nblocks, JACOBI_PASS_THREADS, 0, s>>>(g.d_ctx, a, xh, flip, arrived, last, JACOBI_PASS_BAND_ROWS,
+                                                                    bands, groups, g.npes, g.heap_bytes);
+        break;
+    case 3:
+        k_jacobi_pass<3, NC><<<nblocks, JACOBI_PASS_THREADS, 0, s>>>(g.d_ctx, a, xh, flip, arrived, last, JACOBI_PASS_BAND_ROWS,
+                                                                    bands, groups, g.npes, g.heap_bytes);
+        break;
+    default:
+        k_jacobi_pass<4, NC><<<nblocks, JACOBI_PASS_THREADS, 0, s>>>(g.d_ctx, a, xh, flip, arrived, last, JACOBI_PASS_BAND_ROWS,
+                                                                    bands, groups, g.npes, g.heap_bytes);
+        break;
+    }
 }
-/* partial: room for jacobi_partial_slots() residual terms; *nterms: how many the last launch wrote */
-static size_t jacobi_partial_slots(size_t ny, size_t nx)
-{
-    unsigned b, t;
-    const size_t one = jacobi_sweep_blocks(ny, nx, &b, &t), two = jacobi_sweep_blocks(ny, nx, &b, &t, 56);
-    return one > two ? one : two;
-}
+
+/* partial: room for pl.blocks_last residual terms; xh: four symmetric rows (PE 0's copy) when pl.needs_xh */
 static int jacobi_launch_sweeps(double *buf0, double *buf1, uint64_t *sig, size_t ny, size_t nx, int iters, int overlap,
-                                double *partial, size_t *nterms)
+                                const jacobi_plan &pl, double *partial, double *xh)
 {
     auto &g = g_ishmem;
-    unsigned bands, tile_groups, bands2, tile_groups2;
-    const size_t tile_blocks = jacobi_sweep_blocks(ny, nx, &bands, &tile_groups);
-    /* four columns per lane (120-column tiles, 118 registers, two blocks per SM): 428 against 454 us per
-     * 16384^2 sweep for two columns per lane (56-column tiles), which ISHMEMX_OPT_JACOBI_WIDE = 0 selects */
-    const long long wide_opt = g.opt[ISHMEMX_OPT_JACOBI_WIDE];
-    bool wide = wide_opt != 0;
-    /* ... unless the grid is too small to give every SM a few of the larger blocks (the option
-     * set to 1 keeps the wide form regardless) */
-    if (wide && wide_opt < 0 &&
-        jacobi_sweep_blocks(ny, nx, &bands2, &tile_groups2, 120) < (size_t)g.sm_count * 4)
-        wide = false;
-    const size_t tile_blocks2 = jacobi_sweep_blocks(ny, nx, &bands2, &tile_groups2, wide ? 120 : 56);
-    const size_t nblocks = (size_t)g.npes * 2 * JACOBI_PIECES + tile_blocks;
-    const size_t nblocks2 = (size_t)g.npes * 4 * JACOBI_PIECES + tile_blocks2;
-    if (nblocks > 0x7fffffffu || nblocks2 > 0x7fffffffu) return ISHMEM_ERR_ARG;
+    for (int k = 1; k <= 4; ++k) {
+        const size_t tiles = k == 1 ? (size_t)g.npes * pl.bands1 * pl.groups1 : (size_t)g.npes * pl.bands_k * pl.groups_k[k];
+        if (tiles + (size_t)g.npes * 2 * k * JACOBI_PIECES > 0x7fffffffu) return ISHMEM_ERR_ARG;
+    }
     cudaStream_t s;
     int rc = ishmemi_team_stream_begin(ISHMEM_TEAM_WORLD, &s);
     if (rc) return rc;
@@ -1176,33 +1359,19 @@ static int jacobi_launch_sweeps(double *buf0, double *buf1, uint64_t *sig, size_
     a.overlap = overlap;
     a.partial = partial;
     a.sliding = 1;
-    /* Every launch moves the grid from one buffer to the other, and the result has to end up where
-     * `iters` single sweeps would leave it (buf0 for an even count): an even number of two-sweep
-     * passes, then one to three single sweeps. */
-    int fused = jacobi_fuse(ny) ? iters / 2 : 0;
-    if (fused & 1) --fused;
-    int flip = 0, done = 0;
-    unsigned long long arrived = 0;
-    *nterms = 0;
-    while (done < iters && !rc) {
-        *nterms = fused > 0 ? tile_blocks2 : tile_blocks;
-        if (fused > 0) {
-            arrived += 2 * JACOBI_PIECES;
-            if (wide)
-                k_jacobi_pass2<true><<<(unsigned)nblocks2, 256, 0, s>>>(g.d_ctx, a, flip, arrived, done + 2 == iters,
-                                                                        JACOBI_BAND_ROWS2, bands2, tile_groups2, g.npes,
-                                                                        g.heap_bytes);
-            else
-                k_jacobi_pass2<false><<<(unsigned)nblocks2, 256, 0, s>>>(g.d_ctx, a, flip, arrived, done + 2 == iters,
-                                                                         JACOBI_BAND_ROWS2, bands2, tile_groups2, g.npes,
-                                                                         g.heap_bytes);
-            --fused;
-            done += 2;
+    int flip = 0;
+    unsigned long long arrived = 0; /* pieces the halo words count once the launch's senders are through */
+    for (size_t i = 0; i < pl.depth.size() && !rc; ++i) {
+        const int k = pl.depth[i], last = i + 1 == pl.depth.size();
+        arrived += (unsigned long long)k * JACOBI_PIECES;
+        const unsigned nsend = (unsigned)g.npes * 2u * (unsigned)k * JACOBI_PIECES;
+        if (k == 1) {
+            k_jacobi_sweep<<<nsend + (unsigned)g.npes * pl.bands1 * pl.groups1, 256, 0, s>>>(
+                g.d_ctx, a, flip, arrived, last, JACOBI_BAND_ROWS, pl.bands1, pl.groups1, g.npes, g.heap_bytes);
         } else {
-            arrived += JACOBI_PIECES;
-            k_jacobi_sweep<<<(unsigned)nblocks, 256, 0, s>>>(g.d_ctx, a, flip, arrived, done + 1 == iters, JACOBI_BAND_ROWS,
-                                                             bands, tile_groups, g.npes, g.heap_bytes);
-            done += 1;
+            const unsigned nblocks = nsend + (unsigned)g.npes * pl.bands_k * pl.groups_k[k];
+            if (pl.nc == 4) jacobi_launch_pass<4>(k, nblocks, s, a, xh, flip, arrived, last, pl.bands_k, pl.groups_k[k]);
+            else jacobi_launch_pass<2>(k, nblocks, s, a, xh, flip, arrived, last, pl.bands_k, pl.groups_k[k]);
         }
         flip ^= 1;
         ishmemi_count_launch();
@@ -1229,20 +1398,29 @@ extern "C" int ishmemx_jacobi(double *buf0, double *buf1, uint64_t *sig, size_t 
     int rc = jacobi_check(buf0, buf1, sig, ny, nx, iters, &groups_per_pe, threads, &by_columns);
     if (rc) return rc;
     if (jacobi_per_sweep(threads, nx)) {
+        jacobi_plan pl;
+        jacobi_make_plan(ny, nx, iters, 4, &pl);
+        /* launches deeper than two sweeps park their third and fourth halo rows in four extra symmetric
+         * rows; without room for them in the heap the call stays at two sweeps per launch */
+        double *xh = nullptr;
+        if (pl.needs_xh) {
+            xh = (double *)ishmem_malloc(4 * nx * sizeof(double));
+            if (!xh) jacobi_make_plan(ny, nx, iters, 2, &pl);
+        }
         double *partial = nullptr;
-        size_t nterms = 0;
-        ISHMEMI_CUDA(cudaMalloc((void **)&partial, jacobi_partial_slots(ny, nx) * 8));
-        rc = jacobi_launch_sweeps(buf0, buf1, sig, ny, nx, iters, overlap, partial, &nterms);
+        rc = ishmemi_cuda(cudaMalloc((void **)&partial, (pl.blocks_last ? pl.blocks_last : 1) * 8), "cudaMalloc");
+        if (!rc) rc = jacobi_launch_sweeps(buf0, buf1, sig, ny, nx, iters, overlap, pl, partial, xh);
         if (!rc && residual_sq_host) {
             double sum = 0.0;
-            if (nterms) {
-                std::vector<double> part(nterms);
-                rc = ishmemi_cuda(cudaMemcpy(part.data(), partial, nterms * 8, cudaMemcpyDeviceToHost), "cudaMemcpy");
-                for (size_t i = 0; i < nterms; ++i) sum += part[i];
+            if (pl.blocks_last) {
+                std::vector<double> part(pl.blocks_last);
+                rc = ishmemi_cuda(cudaMemcpy(part.data(), partial, pl.blocks_last * 8, cudaMemcpyDeviceToHost), "cudaMemcpy");
+                for (size_t i = 0; i < pl.blocks_last; ++i) sum += part[i];
             }
             *residual_sq_host = sum;
         }
         cudaFree(partial);
+        if (xh) ishmem_free(xh);
         return rc;
     }
     const size_t nblocks = (size_t)g.npes * groups_per_pe;

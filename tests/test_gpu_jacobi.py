@@ -12,11 +12,13 @@ from tests.gpu_util import Session
 pytestmark = pytest.mark.gpu
 
 
-def run_gpu(grid, npes, iters, overlap, groups, threads, options=()):
+def run_gpu(grid, npes, iters, overlap, groups, threads, options=(), spare_rows=4):
+    """spare_rows: rows of symmetric heap left free beside the two buffers -- launches of three and
+    four sweeps park their deeper halo rows in four rows that the library allocates for the call"""
     ny, nx = grid.shape
     rows_max = -(-ny // npes)
     nbytes = (rows_max + 2) * nx * 8
-    with Session(npes, 2 * nbytes + (1 << 16), with_oracle=False) as s:
+    with Session(npes, 2 * nbytes + (1 << 12) + spare_rows * nx * 8, with_oracle=False) as s:
         for opt, value in options:
             B.ishmemx_set_option(opt, value)
         b0, b1, sig = s.malloc(nbytes), s.malloc(nbytes), s.malloc(64)
@@ -42,7 +44,12 @@ def run_gpu(grid, npes, iters, overlap, groups, threads, options=()):
         return out, res[0]
 
 
-@pytest.mark.parametrize("split", ["sweeps", "sweeps_two_columns_per_lane", "single_sweeps", "columns", "rows"])
+SWEEP_FORMS = {   # (sweeps per launch at most: 1 = the library's choice, up to four; four columns per lane)
+    "sweeps": (1, 1), "sweeps_two_columns_per_lane": (1, 0), "two_per_launch": (2, 1),
+    "three_per_launch_two_columns_per_lane": (3, 0), "single_sweeps": (0, 1)}
+
+
+@pytest.mark.parametrize("split", list(SWEEP_FORMS) + ["columns", "rows"])
 @pytest.mark.parametrize("overlap", [1, 0])
 @pytest.mark.parametrize("ny,nx,npes,groups,threads", [
     (64, 48, 12, 1, 128), (200, 131, 12, 3, 128), (257, 33, 5, 4, 128),       # odd nx: row-by-row path
@@ -51,13 +58,14 @@ def run_gpu(grid, npes, iters, overlap, groups, threads, options=()):
     (120, 2880, 6, 6, 0), (90, 1442, 3, 2, 0), (60, 5000, 2, 4, 640),          # threads chosen by the library; 80 registers
     (36, 600, 12, 12, 32), (50, 121, 4, 3, 64)])                               # one tile per block; odd nx by columns
 def test_jacobi_matches_oracle(ny, nx, npes, groups, threads, overlap, split):
-    """split: the persistent kernel with the strips cut by columns or by rows, or `sweeps`: the form the
-    library picks by itself for threads = 0 and even nx (one tile per warp, two sweeps per launch where the
-    count allows, four columns per lane), the same with two columns per lane, or with one sweep per launch."""
-    if split in ("sweeps", "sweeps_two_columns_per_lane", "single_sweeps"):
-        options = [(B.ISHMEMX_OPT_JACOBI_SPLIT, 0),
-                   (B.ISHMEMX_OPT_JACOBI_FUSE, 0 if split == "single_sweeps" else 1),
-                   (B.ISHMEMX_OPT_JACOBI_WIDE, 0 if split == "sweeps_two_columns_per_lane" else 1)]
+    """split: the persistent kernel with the strips cut by columns or by rows, or one of the launch-ordered
+    forms that the library uses for threads = 0 and even nx: `sweeps` = its own choice (one tile per warp, up
+    to four sweeps per launch, four columns per lane where nx is a multiple of 4), the same with two columns
+    per lane, with at most two or three sweeps per launch, or with one sweep per launch.  21 sweeps are
+    launches of 4, 4, 4, 4, 3, 1 and 1 sweeps in the first form."""
+    if split in SWEEP_FORMS:
+        options = [(B.ISHMEMX_OPT_JACOBI_SPLIT, 0), (B.ISHMEMX_OPT_JACOBI_FUSE, SWEEP_FORMS[split][0]),
+                   (B.ISHMEMX_OPT_JACOBI_WIDE, SWEEP_FORMS[split][1])]
         threads = 0
     else:
         options = [(B.ISHMEMX_OPT_JACOBI_SPLIT, {"rows": 1, "columns": 2}[split])]
@@ -80,21 +88,24 @@ def test_jacobi_default_split_and_repeated_calls():
 
 
 def test_jacobi_per_sweep_many_bands_and_residual():
-    """The launch-per-sweep form on strips of several bands and tile groups, with strips of unequal length and
-    iteration counts that end in a two-sweep pass or in one to three single sweeps; final grid bit-exact,
-    residual within 1e-6 relative."""
+    """The launch-ordered form on strips of several bands and tile groups, with strips of unequal length and
+    iteration counts whose last launch -- the one that forms the residual -- is one of 1, 3 or 4 sweeps, with
+    and without room in the heap for the deeper halo rows (without it launches stay at two sweeps); final
+    grid bit-exact, residual within 1e-6 relative."""
     grid = inputs.jacobi_grid(inputs.SEED_C5, 1000, 1100)
-    for npes, iters in ((7, 5), (3, 12), (1, 3), (5, 8), (12, 4), (2, 10)):     # 2, 6, 0, 4, 2, 4 two-sweep passes
+    for npes, iters, spare in ((7, 5, 4), (3, 12, 4), (1, 3, 4), (5, 8, 4), (12, 4, 4), (2, 10, 4), (6, 6, 4),
+                               (7, 8, 0), (3, 5, 0), (4, 22, 4), (4, 16, 0)):
         exp, exp_res = orc.jacobi(grid, iters)
-        got, res = run_gpu(grid, npes, iters, 1, 1, 0)
-        assert got.tobytes() == exp.tobytes(), (npes, iters)
+        got, res = run_gpu(grid, npes, iters, 1, 1, 0, spare_rows=spare)
+        assert got.tobytes() == exp.tobytes(), (npes, iters, spare)
         assert abs(res - exp_res) <= 1e-6 * exp_res
 
 
-def test_jacobi_two_sweep_passes_on_the_shortest_strips():
-    """Strips of two and three rows: the second halo row of a neighbour is its first or last row but one, and a
-    strip's single band is both its first and its last; 4 and 8 sweeps are all two-sweep passes."""
-    for ny, nx, npes in ((24, 120, 12), (31, 232, 10), (8, 64, 4)):
+def test_jacobi_multi_sweep_launches_on_the_shortest_strips():
+    """Strips of one to five rows: a launch is at most as deep as the shortest strip has rows (it sends that many
+    of its rows each way), the deeper halo rows of a neighbour are its rows next to the edge row, and a strip's
+    single band is both its first and its last."""
+    for ny, nx, npes in ((24, 120, 12), (31, 232, 10), (8, 64, 4), (12, 128, 12), (48, 240, 12), (50, 484, 10)):
         grid = inputs.jacobi_grid(inputs.SEED_C5, ny, nx)
         for iters in (4, 8, 9):
             exp, exp_res = orc.jacobi(grid, iters)
