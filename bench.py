@@ -272,8 +272,110 @@ def run_ours(args) -> dict:
     if rank == 0 and world == 1 and not args.no_cpu:
         out["cpu_baseline"] = cpu_baseline(args.cpu_scale, reps=5)
     B.ishmem_finalize()
+    del heap
+    torch.cuda.empty_cache()
+    if rank == 0 and not args.no_breakdown:
+        # the other two bandwidth configurations, outside the timed step (12 PEs each, own sessions)
+        out["config5_jacobi"] = config5_leg(B, torch, peaks)
+        out["config3_collectives"] = config3_leg(B, torch, peaks)
     replicas.finalize()
     return out if rank == 0 else {}
+
+
+def config5_leg(B, torch, peaks) -> dict:
+    """configs[4]: 12 PEs, 16384 x 16384 float64 Jacobi with in-kernel put_signal halos, in the launch
+    shape the library picks (four sweeps per launch).  40 sweeps timed after an untimed call.  The
+    fraction is taken at the bytes a launch has to move: 16 B per cell per LAUNCH."""
+    npes, n, sweeps = 12, 16384, 40
+    rows_max = -(-n // npes)
+    nbytes = (rows_max + 2) * n * 8
+    heap_bytes = 2 * nbytes + MiB
+    heap = torch.zeros(npes * heap_bytes, dtype=torch.uint8, device="cuda")
+    B.ishmemx_init_external(npes, heap_bytes, heap.data_ptr())
+    ts = torch.cuda.Stream()
+    B.ishmemx_set_stream(-1, ts.cuda_stream)
+    b0, b1, sig = B.ishmem_malloc(nbytes), B.ishmem_malloc(nbytes), B.ishmem_calloc(4, 8)
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(4)
+    base, extra = divmod(n, npes)
+    for p in range(npes):                              # uniform [0, 1) interior, zero ring (config 5's recipe)
+        rows = base + (1 if p < extra else 0)
+        strip = heap[p * heap_bytes + (b0 - heap.data_ptr()):][:nbytes].view(torch.float64).view(rows_max + 2, n)
+        strip[1:rows + 1].uniform_(0.0, 1.0, generator=gen)
+        strip[:, 0] = 0
+        strip[:, n - 1] = 0
+        if p == 0:
+            strip[1] = 0
+        if p == npes - 1:
+            strip[rows] = 0
+    torch.cuda.synchronize()
+    res = np.zeros(1)
+    out = {}
+    for name, fuse, per_launch in (("four_sweeps_per_launch", 1, 4), ("one_sweep_per_launch", 0, 1)):
+        B.ishmemx_set_option(B.ISHMEMX_OPT_JACOBI_FUSE, fuse)
+        best = 1e30
+        for rep in range(3):
+            for p in range(npes):
+                for w in range(4):
+                    B.ishmem_uint64_p(p, sig + 8 * w, 0, p)
+            torch.cuda.synchronize()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(ts)
+            B.ishmemx_jacobi(b0, b1, sig, n, n, sweeps, 1, 12, 0, res)
+            b.record(ts)
+            torch.cuda.synchronize()
+            if rep:                                    # the first call loads the kernels
+                best = min(best, a.elapsed_time(b))
+        us = best * 1e3 / sweeps
+        moved = 16.0 * n * n / per_launch / (us * 1e-6) / 1e9
+        out[name] = {"us_per_sweep": round(us, 2), "us_per_launch": round(us * per_launch, 1),
+                     "GB/s_at_16B_per_cell_per_sweep": round(16.0 * n * n / (us * 1e-6) / 1e9, 1),
+                     "GB/s_moved": round(moved, 1), "frac_of_copy_peak_at_bytes_moved": round(moved / peaks["hbm_gbs"], 4)}
+    out["workload"] = f"{npes} PEs, {n} x {n} float64, {sweeps} sweeps per call, best of 2 timed calls"
+    out["device_status"] = int(B.ishmemx_status(1))
+    B.ishmem_finalize()
+    del heap
+    torch.cuda.empty_cache()
+    return out
+
+
+def config3_leg(B, torch, peaks) -> dict:
+    """configs[2] at large counts: 12 PEs, float32 sum_reduce of 64 Mi elements, broadcast of 256 MiB from
+    root 0, fcollect of 16 Mi float32 per PE; algorithmic bytes (2 P n s; n + P n; P n + P^2 n) over the
+    best of 5 launches."""
+    npes, n_red, n_bc, n_fc = 12, 64 << 20, 256 * MiB, 64 * MiB
+    heap_bytes = n_bc + npes * n_fc + MiB
+    heap = torch.empty(npes * heap_bytes, dtype=torch.uint8, device="cuda")
+    heap.view(torch.float32).normal_(generator=torch.Generator(device="cuda").manual_seed(2))
+    B.ishmemx_init_external(npes, heap_bytes, heap.data_ptr())
+    ts = torch.cuda.Stream()
+    B.ishmemx_set_stream(-1, ts.cuda_stream)
+    src, dst = B.ishmem_malloc(n_bc), B.ishmem_malloc(npes * n_fc)
+    W = B.ISHMEM_TEAM_WORLD
+    ops = {"sum_reduce_f32": (lambda: B.ishmem_float_sum_reduce(W, dst, src, n_red), 2 * npes * 4 * n_red),
+           "broadcast": (lambda: B.ishmem_broadcastmem(W, dst, src, n_bc, 0), n_bc * (1 + npes)),
+           "fcollect": (lambda: B.ishmem_fcollectmem(W, dst, src, n_fc), n_fc * (npes + npes * npes))}
+    out = {}
+    for name, (fn, nbytes) in ops.items():
+        best = 1e30
+        for rep in range(6):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            a.record(ts)
+            fn()
+            b.record(ts)
+            torch.cuda.synchronize()
+            if rep:
+                best = min(best, a.elapsed_time(b))
+        g = nbytes / (best * 1e-3) / 1e9
+        out[name] = {"ms": round(best, 4), "GB/s": round(g, 1), "frac_of_copy_peak": round(g / peaks["hbm_gbs"], 4)}
+    out["workload"] = (f"{npes} PEs; sum_reduce {n_red} float32, broadcast {n_bc // MiB} MiB, "
+                       f"fcollect {n_fc // MiB} MiB per PE")
+    out["device_status"] = int(B.ishmemx_status(1))
+    B.ishmem_finalize()
+    del heap
+    torch.cuda.empty_cache()
+    return out
 
 
 # DRAM bytes per launch of the put kernel: ncu capture of the 8 x 32 MiB case (reads scale with the
@@ -358,10 +460,41 @@ def e2e(B, torch, replicas, dst, src, level, args, world) -> dict:
     local_ms = (time.perf_counter() - t0) * 1e3
     ok = bool(torch.equal(hdst[n:2 * n], hsrc[0:n]))          # PE 1 received PE 0's payload
     rate, ms = replicas.whole_job_rate(2 * n * NPES * steps, local_ms)
+    # what the bus alone gives for the same bytes: plain pinned copies of NPES * n bytes each way, both
+    # directions at once on two streams (the end-to-end call overlaps them between PEs), and each alone
+    dev_in = torch.empty(NPES * n, dtype=torch.uint8, device="cuda")
+    dev_out = torch.empty(NPES * n, dtype=torch.uint8, device="cuda")
+    s_in, s_out = torch.cuda.Stream(), torch.cuda.Stream()
+
+    def copies(h2d, d2h):
+        best = 1e30
+        for _ in range(3):
+            torch.cuda.synchronize()
+            t = time.perf_counter()
+            if h2d:
+                with torch.cuda.stream(s_in):
+                    dev_in.copy_(hsrc, non_blocking=True)
+            if d2h:
+                with torch.cuda.stream(s_out):
+                    hdst.copy_(dev_out, non_blocking=True)
+            torch.cuda.synchronize()
+            best = min(best, time.perf_counter() - t)
+        return best
+
+    t_both, t_in, t_out = copies(True, True), copies(True, False), copies(False, True)
+    bus = 2 * n * NPES / t_both / 1e9
     return {"value": round(rate / 1e9, 2), "unit": "GB/s", "h2d_bytes_per_step": NPES * n,
             "d2h_bytes_per_step": NPES * n, "ms_per_step": round(ms / steps, 3), "steps": steps,
             "call": "ishmemx_host_put_ring (pinned host buffers -> heap -> work-group put ring -> host)",
-            "verified": ok}
+            "verified": ok,
+            "pcie_copy_only": {"both_directions_GB/s": round(bus, 2), "h2d_alone_GB/s": round(n * NPES / t_in / 1e9, 2),
+                               "d2h_alone_GB/s": round(n * NPES / t_out / 1e9, 2),
+                               "note": "plain pinned cudaMemcpyAsync of the same bytes, no put, this rank"},
+            "frac_of_pcie_copy_only": round(local_rate_gbs(2 * n * NPES * steps, local_ms) / bus, 3)}
+
+
+def local_rate_gbs(nbytes, ms):
+    return nbytes / (ms * 1e-3) / 1e9
 
 
 def measured_peaks() -> dict:
@@ -430,14 +563,80 @@ def sample_bytes(scale: int) -> int:
     return sum(b.values())
 
 
+def cpu_model() -> str:
+    try:
+        for line in open("/proc/cpuinfo"):
+            if line.lower().startswith("model name"):
+                return line.split(":", 1)[1].strip()
+    except OSError:
+        pass
+    return "unknown"
+
+
+def oracle_threaded(O, scale: int, state: dict, pool, nthreads: int) -> tuple[float, int]:
+    """The bandwidth ops of the step on the unchanged oracle, called from `nthreads` host threads where
+    the op is trivially parallel (ctypes releases the interpreter lock inside the C calls): per-PE puts and
+    gets concurrently, reduce / broadcast / fcollect cut into element ranges, Jacobi sweeps cut into bands
+    of rows (each band one single-sweep call on its rows plus one row above and below, which the call
+    keeps fixed).  Results are those of the sequential calls by construction.  Returns (seconds, bytes)."""
+    import oracle as orc
+    S = sizes(scale)
+    o, src, dst = state["o"], state["src"], state["dst"]
+    b = step_bytes(S)
+    P = NPES
+
+    def ranges(n, unit):
+        per = -(-n // nthreads)
+        per = -(-per // unit) * unit
+        return [(lo, min(n, lo + per)) for lo in range(0, n, per)]
+
+    t0 = time.perf_counter()
+    list(pool.map(lambda p: o.putmem(p, dst, o.ptr(src, S["put"], p), S["put"], (p + 1) % P), range(P)))
+    list(pool.map(lambda p: o.getmem(p, o.ptr(dst, S["get"], p), src, S["get"], (p + 1) % P), range(P)))
+    list(pool.map(lambda p: o.putmem(p, dst, o.ptr(src, S["nbi"], p), S["nbi"], (p + 1) % P), range(P)))
+    list(pool.map(lambda r: o.broadcastmem(o.world, dst + r[0], src + r[0], r[1] - r[0], 0), ranges(S["bcast"], 64)))
+    # fcollect in element ranges would change the layout of dest: one call per source PE's block instead
+    list(pool.map(lambda i: [o.putmem(i, dst + i * S["fcollect"], o.ptr(src, S["fcollect"], i), S["fcollect"], q)
+                             for q in range(P)], range(P)))
+    list(pool.map(lambda r: o.reduce(o.world, dst + 4 * r[0], src + 4 * r[0], r[1] - r[0], orc.R_SUM, orc.T_FLOAT),
+                  ranges(S["reduce_f32"], 16)))
+    g = state["grid"]
+    ny = g.shape[0]
+    a = g.copy()
+    for _ in range(S["jacobi_sweeps"]):
+        nxt = a.copy()
+
+        def band(r, a=a, nxt=nxt):
+            lo, hi = max(r[0], 1), min(r[1], ny - 1)
+            if lo < hi:
+                nxt[lo:hi] = orc.jacobi(a[lo - 1:hi + 1], 1)[0][1:-1]
+        list(pool.map(band, ranges(ny, 1)))
+        a = nxt
+    dt = time.perf_counter() - t0
+    nbytes = b["put"] + b["get"] + b["nbi"] + b["broadcast"] + b["fcollect"] + b["reduce_f32"] + b["jacobi"]
+    return dt, nbytes
+
+
 def cpu_baseline(scale: int, reps: int) -> dict:
+    from concurrent.futures import ThreadPoolExecutor
     from oracle import Oracle
     state: dict = {}
     best = min(oracle_step(Oracle, scale, state) for _ in range(reps))
+    nproc = os.cpu_count() or 1
+    nthreads = min(nproc, 64)
+    with ThreadPoolExecutor(max_workers=nthreads) as pool:
+        runs = [oracle_threaded(Oracle, scale, state, pool, nthreads) for _ in range(3)]
+    t_thr, b_thr = min(runs)
     return {"value": round(sample_bytes(scale) / best / 1e9, 3), "unit": "GB/s", "cores": 1,
             "kind": "oracle", "seconds": round(best, 2),
             "sample": f"one step of the same op list at 1/{scale} of the sizes "
-                      f"({sample_bytes(scale) / 2**30:.2f} GiB algorithmic), sequential CPU oracle, best of {reps}"}
+                      f"({sample_bytes(scale) / 2**30:.2f} GiB algorithmic), sequential CPU oracle, best of {reps}",
+            "nproc": nproc, "cpu_model": cpu_model(),
+            "threaded": {"value": round(b_thr / t_thr / 1e9, 3), "unit": "GB/s", "cores": nthreads,
+                         "seconds": round(t_thr, 2),
+                         "sample": f"the bandwidth ops of the same step (put, get, nbi put, broadcast, fcollect, float32 "
+                                   f"sum_reduce, Jacobi: {b_thr / 2**30:.2f} GiB algorithmic) on the unchanged oracle "
+                                   f"called from {nthreads} host threads, best of 3"}}
 
 
 def run_reference(args) -> dict:
@@ -464,6 +663,18 @@ def run_reference(args) -> dict:
             "config": {"workload": "configs[1] (8 logical PEs, ring pattern), bounded CPU sample", "sample": sample},
             "cpu_baseline": {"value": val, "unit": "GB/s", "cores": 1, "kind": "oracle", "sample": sample},
             "e2e": {"value": val, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+
+
+def run_plumbing(args) -> dict:
+    """The multi-rank plumbing alone (no GPU work): rendezvous, barrier, sum and max over ranks on made-up
+    figures -- rank r 'processed' (r + 1) * 100 units in (r + 1) * 10 ms.  Runs on CPU over gloo."""
+    from paper_2409_20476_b200 import replicas
+    rank, _, world = replicas.init(backend="gloo")
+    replicas.barrier()
+    rate, ms = replicas.whole_job_rate((rank + 1) * 100.0, (rank + 1) * 10.0)
+    replicas.barrier()
+    replicas.finalize()
+    return {"impl": "plumbing", "n_gpus": world, "value": rate, "ms_per_step": ms} if rank == 0 else {}
 
 
 def run_profile_case(args) -> dict:
@@ -555,7 +766,9 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=300)
     ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference", "plumbing"],
+                    help="ours: the CUDA library; reference: the CPU oracle on a bounded sample; plumbing: the "
+                         "multi-rank rendezvous / barrier / max-over-ranks path alone, on CPU")
     ap.add_argument("--level", default="tiled", choices=["tiled", "bulk", "ldst"],
                     help="tiled: loads/stores, one tile per block (the library's own choice for large messages); "
                          "bulk / ldst: resident blocks (--groups per PE) with the TMA ring / loads and stores")
@@ -570,8 +783,17 @@ def main():
     args = ap.parse_args()
     if args.level == "tiled":
         args.groups = 0  # the library sizes the grid: one tile of threads x 128 bytes per block
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and not args.profile_case:
+        # started by hand (python bench.py --gpus N) rather than by torchrun: this process starts the N
+        # ranks itself, one replica per device, and passes on what rank 0 prints
+        from paper_2409_20476_b200 import replicas
+        text, rc = replicas.spawn(args.gpus, [sys.executable, str(Path(__file__).resolve())] + sys.argv[1:])
+        sys.stdout.write(text)
+        sys.exit(rc)
     if args.profile_case:
         out = run_profile_case(args)
+    elif args.impl == "plumbing":
+        out = run_plumbing(args)
     else:
         out = run_reference(args) if args.impl == "reference" else run_ours(args)
     if out:

@@ -1228,7 +1228,7 @@ static int jacobi_launch(double *buf0, double *buf1, uint64_t *sig, size_t ny, s
 /* The launches of one call.  Every launch moves the grid from one buffer to the other, and the result
  * has to end where `iters` single sweeps would leave it (buf0 for an even count), so the number of
  * launches has the parity of iters.  Within that the split is the cheapest one by the measured time of
- * a launch of 1, 2, 3 and 4 sweeps at 16384^2 (650, 850, 820 and 900 us: a launch costs about the same
+ * a launch of 1, 2, 3 and 4 sweeps at 16384^2 (650, 765, 845 and 930 us: a launch costs about the same
  * whatever its depth, so deep launches win and a single sweep is the cheapest filler). */
 struct jacobi_plan {
     std::vector<int> depth; /* sweeps of each launch, deepest first */
@@ -1241,7 +1241,7 @@ struct jacobi_plan {
 
 static void jacobi_split(int iters, int kmax, std::vector<int> *out)
 {
-    static const double cost[5] = {0, 650, 850, 820, 900};
+    static const double cost[5] = {0, 650, 765, 845, 930};
     out->clear();
     int full = 0, r = iters;
     while (r > 24) { /* far from the end only the deepest launch is ever right */

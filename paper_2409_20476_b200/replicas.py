@@ -7,6 +7,9 @@ is used only to line the ranks up (barrier) and to take the maximum of their dev
 from __future__ import annotations
 
 import os
+import socket
+import subprocess
+import sys
 
 import torch
 import torch.distributed as dist
@@ -61,6 +64,31 @@ def whole_job_rate(local_units: float, local_ms: float) -> tuple[float, float]:
     total = sum_over_ranks(local_units)
     ms = max_over_ranks(local_ms)
     return (total / (ms * 1e-3) if ms > 0 else 0.0), ms
+
+
+def spawn(world: int, argv: list[str], extra_env: dict | None = None, timeout: float | None = None):
+    """Starts `world` ranks of the command `argv` on this node, one per device (RANK, LOCAL_RANK,
+    WORLD_SIZE and the rendezvous address set the way torchrun sets them), waits for all of them and
+    returns (rank 0's standard output, the largest exit code).  The ranks' standard error goes to this
+    process's; the other ranks' standard output is dropped (rank 0 alone reports)."""
+    with socket.socket() as s:                      # a free port for the rendezvous
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    procs = []
+    for rank in range(world):
+        env = dict(os.environ, RANK=str(rank), LOCAL_RANK=str(rank), WORLD_SIZE=str(world),
+                   MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+        env.setdefault("NCCL_DEBUG", "INFO")        # the communicator's size and transport show in the log
+        env.update(extra_env or {})
+        procs.append(subprocess.Popen(argv, env=env, stdout=subprocess.PIPE if rank == 0 else subprocess.DEVNULL,
+                                      stderr=sys.stderr, text=True))
+    out, rc = "", 0
+    for rank, p in enumerate(procs):
+        o, _ = p.communicate(timeout=timeout)
+        if rank == 0:
+            out = o or ""
+        rc = max(rc, abs(p.returncode))
+    return out, rc
 
 
 def finalize() -> None:

@@ -486,18 +486,23 @@ def sweep_c5(args, out):
             first += rows
 
     load()
-    import os
-    # (variant, form selected through ishmemx_set_option, threads, groups): the library's own choice (one launch per sweep), the
-    # persistent kernel with strips cut by column tiles, and the persistent kernel with caller-shaped blocks
-    variants = [("launch_per_two_sweeps", None, 0, 1), ("launch_per_sweep", "single", 0, 1)]
+    # (variant, form selected through ishmemx_set_option, threads, groups): the launch-ordered forms (the library's own
+    # choice: four sweeps per launch; at most three, two, one), the persistent kernel with strips cut by column tiles,
+    # and the persistent kernel with caller-shaped blocks
+    variants = [("launch_per_four_sweeps", 1, 0, 1), ("launch_per_three_sweeps", 3, 0, 1), ("launch_per_two_sweeps", 2, 0, 1),
+                ("launch_per_sweep", 0, 0, 1)]
     variants += [("persistent_columns", "columns", 0, g) for g in (6, 12)]
     variants += [("persistent_rows", "rows", t, g) for g in (6, 12, 24) for t in (256, 512, 1024)]
+    if args.quick:
+        variants = variants[:5]
     for overlap in (1, 0):
         for variant, split, threads, groups in variants:
             if npes * groups * threads > 148 * 2048:
                 continue
             B.ishmemx_set_option(B.ISHMEMX_OPT_JACOBI_SPLIT, {"rows": 1, "columns": 2}.get(split, 0))
-            B.ishmemx_set_option(B.ISHMEMX_OPT_JACOBI_FUSE, 0 if split == "single" else 1)
+            B.ishmemx_set_option(B.ISHMEMX_OPT_JACOBI_FUSE, split if isinstance(split, int) else 1)
+            # sweeps per launch of the bulk of the call (200 sweeps: 50 x 4, 66 x 3 + 1 + 1, 100 x 2, 200 x 1)
+            depth = {1: 4, 3: 3, 2: 2}.get(split, 1) if isinstance(split, int) else 1
             def reset_signals():
                 for p in range(npes):
                     for w in range(4):
@@ -521,9 +526,10 @@ def sweep_c5(args, out):
             b.record(stream)
             torch.cuda.synchronize()
             us = a.elapsed_time(b) * 1e3 / iters
-            out.add(config=5, op="jacobi", pattern=f"{n}x{n}", variant=f"{variant} overlap={overlap}", threads=threads,
-                    groups=groups, npes=npes, dtype="f64", nbytes=n * n * 8, l2="cold", iters=iters, us_per_op=us,
-                    alg_bytes=16 * n * n, note=f"per sweep; residual_sq {res[0]:.6e} (grid keeps evolving)")
+            out.add(config=5, op="jacobi", pattern=f"{n}x{n}", variant=f"{variant} overlap={overlap}", level=depth,
+                    threads=threads, groups=groups, npes=npes, dtype="f64", nbytes=n * n * 8, l2="cold", iters=iters,
+                    us_per_op=us, alg_bytes=16 * n * n,
+                    note=f"per sweep; level = sweeps per launch; residual_sq {res[0]:.6e} (grid keeps evolving)")
     assert B.ishmemx_status(1) == 0
     B.ishmem_finalize()
 
@@ -666,15 +672,23 @@ def summarize(path) -> str:
                 _table(sel, nb, lambda r: f"{r['threads']} threads", us, _fmt_size), ""]
     elif cfg == 5:
         out += ["### Jacobi 16384 x 16384 float64, 12 PEs, 200 sweeps: per sweep", "",
-                "| form | overlap | threads | groups/PE | us/sweep | GB/s (16 B/cell) | of measured copy | of 8 TB/s |",
-                "|---|---|---:|---:|---:|---:|---:|---:|"]
+                "GB/s at 16 B per cell and sweep (the algorithmic figure of a single sweep); the last two columns count the "
+                "bytes the form has to move -- 16 B per cell and LAUNCH, i.e. 16 / K per sweep -- against the measured copy rate.", "",
+                "| form | overlap | threads | groups/PE | sweeps per launch K | us/sweep | us/launch | GB/s (16 B/cell/sweep) | "
+                "of measured copy | of 8 TB/s | GB/s moved (16/K B) | of measured copy |",
+                "|---|---|---:|---:|---:|---:|---:|---:|---:|---:|---:|---:|"]
         for r in rows:
             form, ov = r["variant"].rsplit(" overlap=", 1) if " overlap=" in r["variant"] else ("", r["variant"][-1])
-            shape = f"| {form} | {ov} | {r['threads'] if r['threads'] != '0' else 'library'} | {r['groups'] if not form.startswith('launch_per') else '-'} |"
+            k = int(r["level"] or 1)
+            shape = (f"| {form} | {ov} | {r['threads'] if r['threads'] != '0' else 'library'} | "
+                     f"{r['groups'] if not form.startswith('launch_per') else '-'} | {k} |")
             if r["us_per_op"]:
-                out.append(f"{shape} {us(r)} | {gb(r)} | {r['frac_hbm']} | {r['frac_8tbs']} |")
+                moved = float(r["gbps"]) / k
+                peak = float(r["gbps"]) / float(r["frac_hbm"])
+                out.append(f"{shape} {us(r)} | {float(r['us_per_op']) * k:.1f} | {gb(r)} | {r['frac_hbm']} | {r['frac_8tbs']} | "
+                           f"{moved:.0f} | {moved / peak:.3f} |")
             else:
-                out.append(f"{shape} refused: not co-resident | | | |")
+                out.append(f"{shape} refused: not co-resident | | | | | | |")
     elif cfg == 6:
         out += ["### reverse-offload ring (64-byte requests, one host proxy thread)", "",
                 "| measurement | blocks x threads | us | M requests/s |", "|---|---:|---:|---:|"]

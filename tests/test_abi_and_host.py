@@ -155,3 +155,25 @@ def test_replicas_world_size_2_gloo(tmp_path):
         assert r["world"] == 2
         assert r["ms"] == 20.0                       # max over ranks
         assert abs(r["rate"] - 300.0 / 0.020) < 1e-6  # all ranks' units / slowest rank's time
+
+
+def test_bench_gpus_2_starts_two_ranks_by_itself():
+    """`python bench.py --gpus 2` without a torchrun environment starts the two ranks itself: the
+    plumbing arm (rendezvous over gloo, barrier, sum and max over ranks) reports a world of 2 and the
+    whole-job figures, and the reference arm prints exactly one line, rank 0's, with n_gpus 2."""
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "LOCAL_RANK", "WORLD_SIZE", "MASTER_PORT")}
+    env["PYTHONPATH"] = str(ROOT)
+    out = subprocess.run([sys.executable, str(ROOT / "bench.py"), "--impl", "plumbing", "--gpus", "2"], check=True,
+                         capture_output=True, text=True, env=env, timeout=180).stdout
+    lines = [ln for ln in out.strip().splitlines() if ln.startswith("{")]
+    assert len(lines) == 1
+    line = json.loads(lines[0])
+    assert line["n_gpus"] == 2 and line["ms_per_step"] == 20.0          # the slowest rank's time
+    assert abs(line["value"] - 300.0 / 0.020) < 1e-6                     # all ranks' units over it
+    out = subprocess.run([sys.executable, str(ROOT / "bench.py"), "--impl", "reference", "--gpus", "2", "--steps", "1",
+                          "--warmup", "0", "--cpu-scale", "64"], check=True, capture_output=True, text=True, env=env,
+                         timeout=300).stdout
+    lines = [ln for ln in out.strip().splitlines() if ln.startswith("{")]
+    assert len(lines) == 1
+    line = json.loads(lines[0])
+    assert line["impl"] == "reference" and line["n_gpus"] == 2 and line["value"] > 0
