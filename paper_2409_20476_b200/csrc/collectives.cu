@@ -217,9 +217,13 @@ template <int WHICH, typename T, int OP>
 __global__ void __launch_bounds__(1024) k_collective_on_device(const ishmem_ctx_t *ctxs, coll_args a)
 {
     const ishmemi_team t = ctxs[0].teams[a.team];
+    /* the context in shared memory: the collectives below look PEs up many times, each after the
+     * acquire that ends a sync */
+    __shared__ ishmem_ctx_t ctx_copy;
     const ishmem_ctx_t *ctx = ctxs + (t.start + (int)blockIdx.x * t.stride);
     char *d = a.dest ? local_of(ctxs, ctx, a.dest) : nullptr;
     const char *s = a.src ? local_of(ctxs, ctx, a.src) : nullptr;
+    ctx = ishmemx_ctx_stage_work_group(&ctx_copy, ctx);
     for (int r = 0; r < a.repeat; ++r) {
         int rc;
         if (WHICH == 0) rc = ishmemx_broadcastmem_work_group(ctx, a.team, d, s, a.n, a.root);

@@ -24,6 +24,8 @@ __global__ void __launch_bounds__(1024) k_pingpong(const ishmem_ctx_t *ctxs, int
                                                    pingpong_out *out)
 {
     const bool is_a = (blockIdx.x == 0);
+    /* the context in shared memory: each round translates two addresses right after an acquire */
+    __shared__ ishmem_ctx_t ctx_copy;
     const ishmem_ctx_t *ctx = ctxs + (is_a ? pe_a : pe_b);
     const int other = is_a ? pe_b : pe_a;
     char *data = local_of(ctxs, ctx, data0);
@@ -34,6 +36,7 @@ __global__ void __launch_bounds__(1024) k_pingpong(const ishmem_ctx_t *ctxs, int
     volatile unsigned long long *w1 =
         (nbytes >= 16 && nbytes % 8 == 0) ? (volatile unsigned long long *)(data + nbytes - 8) : nullptr;
     unsigned long long bad = 0, t0 = 0;
+    ctx = ishmemx_ctx_stage_work_group(&ctx_copy, ctx);
     if (is_a && threadIdx.x == 0) t0 = ishmemi::globaltimer_ns();
     for (int r = 1; r <= rounds; ++r) {
         if (is_a) {
@@ -102,7 +105,8 @@ __global__ void __launch_bounds__(1024) k_rma_latency(const ishmem_ctx_t *ctxs, 
                                                       int iters, unsigned staging_bytes, unsigned long long *elapsed_ns)
 {
     extern __shared__ __align__(128) unsigned char dyn_smem[];
-    const ishmem_ctx_t *ctx = ctxs + my_pe;
+    __shared__ ishmem_ctx_t ctx_copy;
+    const ishmem_ctx_t *ctx = ishmemx_ctx_stage_work_group(&ctx_copy, ctxs + my_pe);
     ishmemx_staging_t st = {nullptr, 0};
     if (LEVEL == ISHMEMX_WORK_GROUP_BULK) {
         st.smem = dyn_smem;
@@ -516,6 +520,7 @@ __global__ void __launch_bounds__(MAXT) k_jacobi(const ishmem_ctx_t *ctxs, jacob
 {
     const int P = ctxs[0].npes, G = a.groups;
     const int p = (int)blockIdx.x / G, g = (int)blockIdx.x % G;
+    __shared__ ishmem_ctx_t ctx_copy; /* every sweep's put_signal and wait read the context after an acquire */
     const ishmem_ctx_t *ctx = ctxs + p;
     const unsigned tid = threadIdx.x, nthr = blockDim.x;
     size_t first, rows, rows_above = 0, f2;
@@ -546,7 +551,7 @@ __global__ void __launch_bounds__(MAXT) k_jacobi(const ishmem_ctx_t *ctxs, jacob
      * while it still waits for one of this sweep -- never of the sweep after that, which needs
      * this PE's own next halo -- so a word only ever counts sweeps up to the one waited for. */
     if (tid == 0) give_up = 0;
-    __syncthreads();
+    ctx = ishmemx_ctx_stage_work_group(&ctx_copy, ctx); /* ends with the block barrier */
 
     /* rows [ra, rb) of this block's columns */
     auto sweep_rows = [&](const double *cur, double *nxt, size_t ra, size_t rb, bool want_res) {

@@ -186,9 +186,9 @@ static int init_common(int npes, size_t heap_bytes, void *external)
         c.heap_bytes = heap_bytes;
         c.heap_base = g.base + (size_t)p * heap_bytes;
         for (int q = 0; q < npes; ++q) {
-            /* every PE is reachable by load/store; entry q+1 of the table names the slot of
-             * the offset array that holds heap_base[q] - heap_base[p] */
-            c.reach[q] = (unsigned char)(q + 1);
+            /* every PE is reachable by load/store (non-zero flag); the offset array holds
+             * heap_base[q] - heap_base[p] under the same index */
+            c.reach[q] = 1;
             c.heap_delta[q] = ((long long)q - (long long)p) * (long long)heap_bytes;
         }
         char *mine = g.d_internal + (size_t)p * ISHMEMI_INTERNAL_BYTES;
