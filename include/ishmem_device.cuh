@@ -331,18 +331,43 @@ __device__ __forceinline__ void copy_bytes(char *d, const char *s, size_t n, uns
  * `sst` elements from s, goes to element k*dst of d, k = tid, tid+nthr, ...  ES = element size in
  * bytes (1, 2, 4, 8 or 16); both addresses aligned to it. */
 template <int ES>
+struct strided_word;
+template <> struct strided_word<1> { typedef unsigned char type; };
+template <> struct strided_word<2> { typedef unsigned short type; };
+template <> struct strided_word<4> { typedef unsigned type; };
+template <> struct strided_word<8> { typedef unsigned long long type; };
+template <> struct strided_word<16> { typedef uint4 type; };
+template <int ES>
+__device__ __forceinline__ typename strided_word<ES>::type strided_ld(const char *p)
+{
+    return ldv<typename strided_word<ES>::type>(p);
+}
+template <>
+__device__ __forceinline__ uint4 strided_ld<16>(const char *p) { return ld16(p); }
+template <int ES>
+__device__ __forceinline__ void strided_st(char *p, typename strided_word<ES>::type v)
+{
+    stv<typename strided_word<ES>::type>(p, v);
+}
+template <>
+__device__ __forceinline__ void strided_st<16>(char *p, uint4 v) { st16(p, v); }
+
+/* elements tid, tid + nthr, ... of [0, nelems): four independent loads are in flight per thread
+ * before the first store */
+template <int ES>
 __device__ __forceinline__ void strided_copy(char *d, const char *s, size_t dst, size_t sst, size_t nelems,
                                              size_t tid, size_t nthr)
 {
-    for (size_t k = tid; k < nelems; k += nthr) {
-        char *pd = d + k * dst * ES;
-        const char *ps = s + k * sst * ES;
-        if (ES == 1) stv<unsigned char>(pd, ldv<unsigned char>(ps));
-        else if (ES == 2) stv<unsigned short>(pd, ldv<unsigned short>(ps));
-        else if (ES == 4) stv<unsigned>(pd, ldv<unsigned>(ps));
-        else if (ES == 8) stv<unsigned long long>(pd, ldv<unsigned long long>(ps));
-        else st16(pd, ld16(ps));
+    typedef typename strided_word<ES>::type W;
+    size_t k = tid;
+    for (; k + 3 * nthr < nelems; k += 4 * nthr) {
+        W v[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) v[u] = strided_ld<ES>(s + (k + u * nthr) * sst * ES);
+#pragma unroll
+        for (int u = 0; u < 4; ++u) strided_st<ES>(d + (k + u * nthr) * dst * ES, v[u]);
     }
+    for (; k < nelems; k += nthr) strided_st<ES>(d + k * dst * ES, strided_ld<ES>(s + k * sst * ES));
 }
 __device__ __forceinline__ void strided_copy_any(char *d, const char *s, size_t dst, size_t sst, size_t nelems,
                                                  unsigned es, size_t tid, size_t nthr)

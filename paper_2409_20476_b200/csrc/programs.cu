@@ -808,6 +808,7 @@ __global__ void __launch_bounds__(256, 4) k_jacobi_sweep(const ishmem_ctx_t *ctx
  * uses during the pass, the third and fourth into four extra rows per PE that the library takes from
  * the symmetric heap for the duration of the call. */
 #define JW_FULL 0xffffffffu
+#define JW_AHEAD 3 /* rows between a load and the L2 prefetch issued with it */
 
 template <int NC>
 __device__ __forceinline__ void jw_ld(const double *p, double (&v)[NC])
@@ -958,12 +959,21 @@ __device__ __forceinline__ double jw_march(const jw_rows &src, double *nxt, int 
     double acc = 0.0;
     double f[D][NC]; /* rows in flight */
     int r_next = ra - K;
+    const int r_last = rb - 1 + K; /* last row of u(t) the band reads */
     const double *pin = src.cur + (size_t)r_next * pitch + jbase; /* without EDGE all rows are in the source buffer */
+    /* Each request also asks L2 for the row JW_AHEAD further down.  The registers hold D rows in flight,
+     * which at 128 registers per thread is all a K-level window leaves room for; the prefetch puts the
+     * DRAM latency of the following rows behind them without holding anything (measured at 16384^2, four
+     * sweeps per launch: 880 -> 740 us per launch with 2 or 3 rows ahead, 745 with 4, 780 with 8, 900
+     * with 16: further ahead the prefetched rows of all resident warps no longer fit beside one another). */
     auto request = [&](double(&v)[NC]) {
         if (EDGE) {
             jw_ld_edge<NC>(src.at(r_next) + jbase, v, ok);
+            if ((ok & 1u) && r_next + JW_AHEAD <= r_last)
+                asm volatile("prefetch.global.L2 [%0];" ::"l"(src.at(r_next + JW_AHEAD) + jbase));
         } else {
             jw_ld<NC>(pin, v);
+            if (r_next + JW_AHEAD <= r_last) asm volatile("prefetch.global.L2 [%0];" ::"l"(pin + (size_t)JW_AHEAD * pitch));
             pin += pitch;
         }
         ++r_next;
@@ -1233,11 +1243,11 @@ static int jacobi_launch(double *buf0, double *buf1, uint64_t *sig, size_t ny, s
 /* The launches of one call.  Every launch moves the grid from one buffer to the other, and the result
  * has to end where `iters` single sweeps would leave it (buf0 for an even count), so the number of
  * launches has the parity of iters.  Within that the split is the cheapest one by the measured time of
- * a launch of 1, 2, 3 and 4 sweeps at 16384^2 (650, 765, 845 and 930 us: a launch costs about the same
+ * a launch of 1, 2, 3 and 4 sweeps at 16384^2 (650, 690, 740 and 800 us: a launch costs about the same
  * whatever its depth, so deep launches win and a single sweep is the cheapest filler). */
 struct jacobi_plan {
     std::vector<int> depth; /* sweeps of each launch, deepest first */
-    int nc;                 /* columns per lane of the multi-sweep launches */
+    int nc[5];              /* columns per lane of a launch of depth k */
     unsigned bands1, groups1, bands_k;
     unsigned groups_k[5];   /* tile groups per band of a launch of depth k */
     size_t blocks_last;     /* tile blocks (= residual terms) of the last launch */
@@ -1246,7 +1256,7 @@ struct jacobi_plan {
 
 static void jacobi_split(int iters, int kmax, std::vector<int> *out)
 {
-    static const double cost[5] = {0, 650, 765, 845, 930};
+    static const double cost[5] = {0, 650, 690, 740, 800};
     out->clear();
     int full = 0, r = iters;
     while (r > 24) { /* far from the end only the deepest launch is ever right */
@@ -1306,14 +1316,19 @@ static void jacobi_make_plan(size_t ny, size_t nx, int iters, int kmax, jacobi_p
     pl->bands1 = (unsigned)((rows_max + JACOBI_BAND_ROWS - 1) / JACOBI_BAND_ROWS);
     pl->groups1 = (unsigned)(((nx + 59) / 60 + 7) / 8);
     pl->bands_k = (unsigned)((rows_max + JACOBI_PASS_BAND_ROWS - 1) / JACOBI_PASS_BAND_ROWS);
-    /* four columns per lane (32-byte accesses: nx a multiple of 4) unless the grid is too small to give
-     * every SM its blocks that way; ISHMEMX_OPT_JACOBI_WIDE = 0 / 1 decides otherwise */
+    /* Columns per lane: four (32-byte accesses: nx a multiple of 4) unless the grid is too small to give
+     * every SM its blocks that way.  At 16384^2, per sweep, four against two columns per lane: 345 / 395 us
+     * with two sweeps per launch, 247 / 295 with three, 200 / 230 with four (whose four-column window
+     * spills a few values at 128 registers and still wins).  ISHMEMX_OPT_JACOBI_WIDE = 0 / 1 forces two /
+     * four. */
     const long long wide = g.opt[ISHMEMX_OPT_JACOBI_WIDE];
-    pl->nc = 4;
-    if (nx % 4 != 0 || wide == 0) pl->nc = 2;
-    else if (wide < 0 && (size_t)g.npes * pl->bands_k * jacobi_pass_groups(nx, 4, 4) < (size_t)g.sm_count * 8) pl->nc = 2;
+    for (int k = 2; k <= 4; ++k) {
+        pl->nc[k] = 4;
+        if (nx % 4 != 0 || wide == 0) pl->nc[k] = 2;
+        else if (wide < 0 && (size_t)g.npes * pl->bands_k * jacobi_pass_groups(nx, k, 4) < (size_t)g.sm_count * 8) pl->nc[k] = 2;
+    }
     pl->needs_xh = false;
-    for (int k = 2; k <= 4; ++k) pl->groups_k[k] = jacobi_pass_groups(nx, k, pl->nc);
+    for (int k = 2; k <= 4; ++k) pl->groups_k[k] = jacobi_pass_groups(nx, k, pl->nc[k]);
     for (int k : pl->depth) pl->needs_xh |= k > 2;
     const int k_last = pl->depth.empty() ? 1 : pl->depth.back();
     pl->blocks_last = k_last == 1 ? (size_t)g.npes * pl->bands1 * pl->groups1
@@ -1375,7 +1390,7 @@ static int jacobi_launch_sweeps(double *buf0, double *buf1, uint64_t *sig, size_
                 g.d_ctx, a, flip, arrived, last, JACOBI_BAND_ROWS, pl.bands1, pl.groups1, g.npes, g.heap_bytes);
         } else {
             const unsigned nblocks = nsend + (unsigned)g.npes * pl.bands_k * pl.groups_k[k];
-            if (pl.nc == 4) jacobi_launch_pass<4>(k, nblocks, s, a, xh, flip, arrived, last, pl.bands_k, pl.groups_k[k]);
+            if (pl.nc[k] == 4) jacobi_launch_pass<4>(k, nblocks, s, a, xh, flip, arrived, last, pl.bands_k, pl.groups_k[k]);
             else jacobi_launch_pass<2>(k, nblocks, s, a, xh, flip, arrived, last, pl.bands_k, pl.groups_k[k]);
         }
         flip ^= 1;

@@ -119,7 +119,12 @@ __global__ void k_wait_until(const ishmem_ctx_t *ctxs, int my_pe, const unsigned
     ishmem_uint64_wait_until(ctxs + my_pe, ivar, cmp, value);
 }
 
-/* strided put/get: the blocks of the launch share the elements, one element per thread and step */
+/* strided put/get: every block takes tiles of K_STRIDED_TILE consecutive elements (its threads share a
+ * tile: neighbouring threads take neighbouring elements, four per thread in flight); blocks start in
+ * index order, so the running blocks sweep one window of the source and of the destination together,
+ * as in the contiguous copies.  The grid covers the message with one tile per block up to the launch
+ * limit, beyond which a block moves on by the grid's width. */
+#define K_STRIDED_TILE 1024u
 __global__ void __launch_bounds__(256) k_strided(const ishmem_ctx_t *ctxs, int my_pe, char *dest, const char *src,
                                                  size_t dst, size_t sst, size_t nelems, unsigned es, int pe, int is_get)
 {
@@ -129,8 +134,10 @@ __global__ void __launch_bounds__(256) k_strided(const ishmem_ctx_t *ctxs, int m
     if (is_get) s = ishmem_ptr(ctx, src, pe);
     else d = ishmem_ptr(ctx, dest, pe);
     if (!d || !s) return;
-    ishmemi::strided_copy_any(d, s, dst, sst, nelems, es, (size_t)blockIdx.x * blockDim.x + threadIdx.x,
-                              (size_t)gridDim.x * blockDim.x);
+    for (size_t lo = (size_t)blockIdx.x * K_STRIDED_TILE; lo < nelems; lo += (size_t)gridDim.x * K_STRIDED_TILE) {
+        const size_t n = nelems - lo < K_STRIDED_TILE ? nelems - lo : K_STRIDED_TILE;
+        ishmemi::strided_copy_any(d + lo * dst * es, s + lo * sst * es, dst, sst, n, es, threadIdx.x, blockDim.x);
+    }
 }
 
 /* which: 0 all, 1 any, 2 some; results (index / count + indices) go to host-mapped memory */
@@ -393,8 +400,8 @@ static int strided(int my_pe, void *dest, const void *src, size_t dst, size_t ss
         return ISHMEM_ERR_NOT_SYMMETRIC;
     char *dl = ishmemi_localise(dest, dspan, my_pe);
     const char *sl = ishmemi_localise(src, sspan, my_pe);
-    size_t blocks = (nelems + 255) / 256, cap = (size_t)g_ishmem.sm_count * 8;
-    if (blocks > cap) blocks = cap;
+    size_t blocks = (nelems + K_STRIDED_TILE - 1) / K_STRIDED_TILE;
+    if (blocks > 0x7fffffffu) blocks = 0x7fffffffu;
     k_strided<<<(unsigned)blocks, 256, 0, ishmemi_pe_stream_for_op(my_pe)>>>(g_ishmem.d_ctx, my_pe, dl, sl, dst, sst,
                                                                              nelems, (unsigned)es, pe, is_get ? 1 : 0);
     ishmemi_count_launch();

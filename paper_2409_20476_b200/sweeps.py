@@ -198,6 +198,21 @@ def sweep_c2(args, out):
         out.add(config=2, op="put", pattern="one_pe", variant="host_api_copy_engine", npes=1, dtype="u8", nbytes=n,
                 l2="hot", iters=it, us_per_op=us, alg_bytes=2 * n)
     B.ishmemx_set_cutover(0, B.SIZE_MAX)
+    # strided put (iput) of one PE, PE 0 -> PE 1: element size, the two strides, element count
+    span = 256 * MiB
+    for es in (4, 8, 16):
+        for dstride, sstride in ((1, 1), (2, 1), (1, 2), (2, 2), (4, 4), (8, 8), (64, 64)):
+            for k in range(10, 26, 2):
+                ne = 1 << k
+                if ne * max(dstride, sstride) * es > span:
+                    continue
+                us, it = T0(lambda i: B.ishmemx_iputmem(0, dst, src, dstride, sstride, ne, es, 1))
+                touched = ne * (min(32, dstride * es) + min(32, sstride * es))
+                out.add(config=2, op="iput", pattern="strided", variant=f"es{es}_dst{dstride}_sst{sstride}", level=es,
+                        threads=dstride, groups=sstride, npes=1, dtype="u8", nbytes=ne * es, l2="hot" if ne * es * max(dstride, sstride) < 32 * MiB else "cold",
+                        iters=it, us_per_op=us, alg_bytes=2 * ne * es,
+                        note=f"level = element size, threads = dest stride, groups = source stride (elements); "
+                             f"sectors touched carry {touched} bytes")
     # device-timed latency of one collaboration unit (in-kernel loop, PE 0 -> PE 1)
     ns = np.zeros(1)
     for op, is_get in (("put", 0), ("get", 1)):
@@ -509,8 +524,9 @@ def sweep_c5(args, out):
                         B.ishmem_uint64_p(p, sig + 8 * w, 0, p)
             try:
                 # a short untimed call first: the first launch of a kernel in a process loads its code
+                # (24 sweeps: launches of every depth the timed call uses)
                 reset_signals()
-                B.ishmemx_jacobi(b0, b1, sig, n, n, 6, overlap, groups, threads, res)
+                B.ishmemx_jacobi(b0, b1, sig, n, n, 24, overlap, groups, threads, res)
             except B.IshmemError:
                 pass
             reset_signals()
@@ -621,6 +637,19 @@ def summarize(path) -> str:
         sel = [r for r in rows if r["pattern"] == "one_pe" and r["op"] == "put" and r["variant"].startswith("in_kernel")]
         out += ["", "### one collaboration unit, PE 0 -> PE 1, put + quiet timed inside the kernel: microseconds", "",
                 _table(sel, nb, lambda r: r["variant"][10:], us, _fmt_size), ""]
+        sel = [r for r in rows if r["pattern"] == "strided"]
+        if sel:
+            out += ["### strided put `ishmemx_iputmem`, one PE (PE 0 -> PE 1): GB/s of useful bytes (2 x elements x element size) / "
+                    "GB/s of the bytes in the 32-byte sectors it has to touch", "",
+                    "Column: element size, destination stride, source stride (in elements).  A stride of s elements of e bytes "
+                    "touches min(32, s e) bytes per element on that side, so the second figure is what the memory system "
+                    "moves; it is the one to hold against the copy rate.", ""]
+
+            def both(r):
+                touched = float(r["note"].rsplit("carry ", 1)[1].split()[0])
+                t = float(r["us_per_op"])
+                return f"{float(r['gbps']):.0f} / {touched / t / 1e3:.0f}"
+            out += [_table(sel, nb, lambda r: r["variant"], both, _fmt_size), ""]
         sel = [r for r in rows if r["pattern"] == "one_pe" and r["variant"].startswith("host_api")]
         out += ["### host API `ishmem_putmem` on ONE PE (PE 0 -> PE 1), back-to-back calls: microseconds per call / GB/s", "",
                 _table(sel, nb, lambda r: r["variant"][9:], lambda r: f"{us(r)} / {gb(r)}", _fmt_size), ""]
@@ -658,9 +687,23 @@ def summarize(path) -> str:
         if sel:
             out += ["### alltoall (block size per pair; P x P blocks move): GB/s (algorithmic 2 P^2 n) / microseconds", "",
                     _table(sel, nb, lambda r: f"P={r['npes']}", lambda r: f"{gb(r)} / {us(r)}", _fmt_size), ""]
-        sel = [r for r in rows if r["variant"] == "device_resident" and r["npes"] in ("2", "12") and r["threads"] in ("128", "1024")]
-        out += ["### device-resident forms (one work-group per PE, in-kernel push sync): microseconds", "",
-                _table(sel, nb, lambda r: f"{r['op']} P={r['npes']} T={r['threads']}", us, _fmt_size), ""]
+        dev = [r for r in rows if r["variant"] == "device_resident"]
+        for op in ("broadcast", "fcollect", "sum_reduce_f32", "sync"):
+            sel = [r for r in dev if r["op"] == op]
+            if not sel:
+                continue
+            out += [f"### device-resident {op} (one work-group of T work-items per PE, in-kernel push sync): microseconds", "",
+                    _table(sel, nb, lambda r: f"P={r['npes']} T={r['threads']}", us, _fmt_size), ""]
+            if op in ("broadcast", "fcollect"):
+                eng = [r for r in rows if r["op"] == op and r["dtype"] == "u8" and r["variant"] == "copy_engine"]
+                for P in ("2", "4", "8", "12"):
+                    b = {nb(r): float(r["us_per_op"]) for r in eng if r["npes"] == P}
+                    for T_ in ("128", "256", "1024"):
+                        a = {nb(r): float(r["us_per_op"]) for r in sel if r["npes"] == P and r["threads"] == T_}
+                        c = _crossover(a, b)
+                        out.append(f"- {op}, {P} PEs, one work-group of {T_} work-items per PE against the host-started copy "
+                                   f"engine: engine at least as fast from " + (_fmt_size(c) if c else "no size measured (<= 256 KiB)"))
+                out.append("")
     elif cfg == 4:
         out += ["### remote atomics, 16 PEs: Mops/s (one op per GPU thread)", "", "| op | index stream | variant | threads | Mops/s | us |",
                 "|---|---|---|---:|---:|---:|"]

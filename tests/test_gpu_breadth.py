@@ -12,6 +12,27 @@ from tests.gpu_util import Session, heaps_equal
 pytestmark = pytest.mark.gpu
 
 
+@pytest.mark.parametrize("es,dstr,sstr,n", [(8, 3, 2, 70_001), (4, 1, 5, 1024 * 9), (16, 2, 1, 4 * 1024 + 1), (1, 2, 2, 300_000)])
+def test_strided_messages_of_many_tiles(es, dstr, sstr, n):
+    """strided put and get whose elements span many 1024-element tiles of the launch and a ragged
+    last tile; whole heaps against the oracle"""
+    npes = 2
+    span = ((n - 1) * max(dstr, sstr) + 1) * es + 64
+    with Session(npes, 2 * span + (1 << 12)) as s:
+        src, dst = s.malloc(span), s.malloc(span)
+        for p in range(npes):
+            src.fill(p, inputs.byte_payload(inputs.SEED_C2, 60 + p, span))
+        B.ishmemx_iputmem(0, dst.addr + es, src.addr + 2 * es, dstr, sstr, n, es, 1)
+        s.oracle.iput(0, dst.ooff + es, s.oracle.ptr(src.ooff + 2 * es, ((n - 1) * sstr + 1) * es, 0), dstr, sstr, n, es, 1)
+        B.ishmem_barrier_all()
+        heaps_equal(s, "iput")
+        B.ishmemx_igetmem(1, src.addr, dst.addr + es, sstr, dstr, n, es, 0)      # PE 1 gathers from PE 0's dst
+        s.oracle.iget(1, s.oracle.ptr(src.ooff, ((n - 1) * sstr + 1) * es, 1), dst.ooff + es, sstr, dstr, n, es, 0)
+        B.ishmem_barrier_all()
+        heaps_equal(s, "iget")
+        assert s.status() == 0
+
+
 @pytest.mark.parametrize("es", [1, 2, 4, 8, 16])
 def test_strided_put_get_match_the_oracle(es):
     npes, heap = 3, 1 << 19
