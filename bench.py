@@ -191,7 +191,8 @@ def run_ours(args) -> dict:
         B.ishmemx_putmem_spmd(dst, src, S["work_item"], 1, B.ISHMEMX_WORK_ITEM, 64, 1)
         B.ishmemx_putmem_spmd(dst, src, S["sub_group"], 2, B.ISHMEMX_SUB_GROUP, 256, 4)
         B.ishmem_long_p(0, dst, k, 1)
-        B.ishmemx_set_cutover(0, 1 * MiB)              # above 1 MiB: copy engine
+        B.ishmemx_set_cutover(0, 1 * MiB)              # from 1 MiB on, with no upper end: copy engine
+        B.ishmemx_set_cutover(5, B.SIZE_MAX)
         for p in range(NPES):
             B.ishmem_putmem_nbi(p, dst, src, S["nbi"], (p + 1) % NPES)
         for p in range(NPES):
@@ -721,12 +722,12 @@ def run_profile_case(args) -> dict:
 def run_profile_jacobi(args) -> dict:
     """Small Jacobi case for profiler captures: 8 PEs, 4096 x 16384 float64 (full-width rows as in config 5,
     two buffers of 512 MiB: larger than L2, and enough blocks for the launch shape used at full size),
-    `--steps` calls of 4 sweeps each (two launches of two sweeps)."""
+    `--steps` calls of 8 sweeps each (two launches of four sweeps)."""
     import torch
     from paper_2409_20476_b200 import binding as B
     from paper_2409_20476_b200 import inputs
 
-    ny, nx, sweeps = 4096, 16384, 4
+    ny, nx, sweeps = 4096, 16384, 8
     rows = ny // NPES
     nbytes = (rows + 2) * nx * 8
     heap_bytes = 2 * nbytes + MiB
@@ -754,7 +755,7 @@ def run_profile_jacobi(args) -> dict:
         times.append(a.elapsed_time(b))
     status = B.ishmemx_status(1)
     B.ishmem_finalize()
-    return {"profile_case": "jacobi", "ny": ny, "nx": nx, "sweeps_per_launch": sweeps, "status": status,
+    return {"profile_case": "jacobi", "ny": ny, "nx": nx, "sweeps_per_call": sweeps, "status": status,
             "ms": [round(t, 4) for t in times[2:]]}
 
 
