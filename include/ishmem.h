@@ -135,10 +135,12 @@ size_t ishmemx_heap_bytes(void);
  *       threads = 0 and an even nx: launch-ordered sweeps; else the persistent kernel, strips cut
  *       by rows), 1 = persistent kernel with the strips cut by rows, 2 = by ranges of column
  *       tiles.
- *   ISHMEMX_OPT_JACOBI_FUSE (ISHMEM_JACOBI_FUSE=0|1): sweeps per launch of the launch-ordered
- *       form: 1 = two where the count allows (default), 0 = always one.
- *   ISHMEMX_OPT_JACOBI_WIDE (ISHMEM_JACOBI_WIDE=0|1): columns per lane in the two-sweep launches:
- *       -1 = by grid size (default), 0 = two, 1 = four.
+ *   ISHMEMX_OPT_JACOBI_FUSE (ISHMEM_JACOBI_FUSE=0..4): sweeps per launch of the launch-ordered
+ *       form: 1 = the library's choice, up to four (default), 0 = always one, 2, 3, 4 = at most
+ *       that many.
+ *   ISHMEMX_OPT_JACOBI_WIDE (ISHMEM_JACOBI_WIDE=0|1): columns per lane in the multi-sweep launches:
+ *       -1 = four where nx is a multiple of 4 and the grid gives every SM its blocks (default),
+ *       0 = two, 1 = four (nx a multiple of 4, else two).
  *   ISHMEMX_OPT_REDUCE_BULK (ISHMEM_REDUCE_BULK=0|1): 1 = large split reductions go through the
  *       shared-memory TMA fold ring instead of one tile per block (default 0).
  *   ISHMEMX_OPT_BULK_SMEM (ISHMEM_BULK_SMEM=bytes): shared-memory staging per block of the
@@ -541,6 +543,22 @@ int ishmemx_collective_on_device(int which, ishmem_team_t team, void *dest, cons
 int ishmemx_pingpong(int pe_a, int pe_b, void *data, uint64_t *sig, size_t nbytes, int rounds,
                      int threads, double *half_rtt_ns, uint64_t *mismatches);
 
+/* Where a half round trip of that exchange goes.  The same ping-pong with the put_signal written out
+ * phase by phase and the SM cycle counter read between the phases by the first thread of each side
+ * (`rounds` rounds, `threads` threads per side; sig: 4 symmetric words, zero on entry; staged != 0: the
+ * kernel reads its context from a copy in shared memory, as k_pingpong does, 0: from global memory).
+ * Writes 14 doubles to HOST `ns_out`, nanoseconds per round at the device's nominal SM clock:
+ *   [0..4]  side A: wait for the answer / address translation / copy / block barrier / release of the
+ *           signal word (fence + store); a phase includes the wait for the loads its first instruction
+ *           needs, so the five add up to A's round;
+ *   [5..9]  side B, the same;
+ *   [10]    one dependent relaxed load of a word in L2 (one trip), [11] a store followed by
+ *           st.release.gpu, [12] st.release.gpu with nothing pending;
+ *   [13]    half round trip by the global timer.
+ * Blocks the host.  Errors as ishmemx_pingpong. */
+int ishmemx_pingpong_phases(int pe_a, int pe_b, void *data, uint64_t *sig, size_t nbytes, int rounds,
+                            int threads, int staged, double *ns_out);
+
 /* Device-initiated latency of one collaboration level (the measurement method of Section 4:
  * many back-to-back operations inside one kernel, timed on the device).  ONE work-group of
  * `threads` threads runs as PE my_pe and issues `iters` puts (is_get = 0) or gets of `nbytes`
@@ -561,15 +579,22 @@ int ishmemx_rma_latency(int my_pe, void *dest, const void *src, size_t nbytes, i
  * interior-first ordering (exchange, wait, then compute).
  * threads = 0 (and an even nx): the library shapes the launches itself -- many short launches whose
  * first blocks send the halo rows (in-kernel work-group put_signal) and whose other blocks each
- * take a band of rows of 8 neighbouring column tiles, one warp per tile, numbered so that the
- * blocks sweep the grid in launch order; only the first and the last band of a strip wait for a
- * halo, the interior never does.  Where the count allows, a launch does TWO sweeps (every element
- * read once, the second result written once; two halo rows each way, the second one parked in the
- * halo row of the buffer being written) -- an even number of such passes, then one to three
- * single-sweep launches, so that the result ends in the buffer named below; 428 us per sweep at
- * 16384^2 (single sweeps only, ISHMEMX_OPT_JACOBI_FUSE = 0: 650 us = the copy rate;
- * ISHMEMX_OPT_JACOBI_WIDE = 0: two instead of four columns per lane in the two-sweep launches).  groups_per_pe is
- * not used by this form and nothing needs to be co-resident.
+ * take a band of rows of a few neighbouring column tiles, one warp per tile, numbered so that the
+ * blocks sweep the grid in launch order; only the bands at the two ends of a strip wait for a halo,
+ * the interior never does.  A launch does up to FOUR sweeps: a warp's register window carries that
+ * many time levels, every element is read once and the last level written once, and as many halo
+ * rows go each way as the launch does sweeps -- the first into the halo row of the buffer being
+ * read, the second into the halo row of the buffer being written, the third and fourth into four
+ * rows per PE that the call takes from the symmetric heap and gives back (4 * nx * 8 bytes; when
+ * the heap has no room the call stays at two sweeps per launch).  The result of every cell is the
+ * same expression in the same order as in single sweeps, bit for bit.  The sweeps are cut into
+ * launches of 4, 3, 2 and 1 so that the number of launches has the parity of iters (each launch
+ * moves the grid to the other buffer) at the least cost by a table of measured launch times;
+ * a strip must own as many rows as a launch does sweeps.  At 16384^2 on 12 PEs: 200 us per sweep
+ * with four sweeps per launch, 247 with three, 345 with two, 650 with one (the copy rate).
+ * ISHMEMX_OPT_JACOBI_FUSE caps the sweeps per launch (0 = always one), ISHMEMX_OPT_JACOBI_WIDE
+ * picks two or four columns per lane (ishmemx_set_option).  groups_per_pe is not used by this
+ * form and nothing needs to be co-resident.
  * threads > 0 (a multiple of 32 up to 1024): one persistent co-resident launch of
  * npes x groups_per_pe blocks of that size for all sweeps; the blocks of a PE take bands of rows,
  * one of them sends each halo row, and neighbouring blocks hand over through flags.

@@ -159,6 +159,7 @@ def _signatures() -> dict[str, tuple[str, list[str]]]:
         "ishmemx_set_collective_geometry": ("status", ["i", "i"]),
         "ishmemx_collective_on_device": ("status", ["i", "i", "p", "p", "z", "i", "i", "i", "i", "i"]),
         "ishmemx_pingpong": ("status", ["i", "i", "p", "p", "z", "i", "i", "p", "p"]),
+        "ishmemx_pingpong_phases": ("status", ["i", "i", "p", "p", "z", "i", "i", "i", "p"]),
         "ishmemx_proxy_start": ("status", []),
         "ishmemx_proxy_stop": ("status", []),
         "ishmemx_proxy_stats": ("status", ["p", "p", "p"]),

@@ -97,6 +97,131 @@ extern "C" int ishmemx_pingpong(int pe_a, int pe_b, void *data, uint64_t *sig, s
     return ISHMEM_OK;
 }
 
+/* ---- where a half round trip goes ------------------------------------------------------------
+ * The same exchange as k_pingpong with the put_signal written out phase by phase (address translation,
+ * copy, block barrier, release of the signal word, wait for the answer) and the SM's cycle counter
+ * read between the phases by thread 0 of each block.  A thread issues in order, so a phase's count
+ * includes the wait for whatever earlier load its first instruction needs: the counts say where the time
+ * goes, not what each instruction costs in isolation.  staged: the context is read from a copy in
+ * shared memory instead of from global memory.  The first block also times three primitives on its own
+ * signal word: a dependent chain of relaxed loads (one trip to L2 each), a store followed by
+ * st.release.gpu, and st.release.gpu with nothing pending. */
+struct pingpong_phases {
+    unsigned long long cycles[2][5]; /* per block: wait / translate / copy / barrier / release */
+    unsigned long long prim[3];      /* L2 trip, store + release, release alone: cycles per operation */
+    unsigned long long elapsed_ns;
+};
+
+__global__ void __launch_bounds__(1024) k_pingpong_phases(const ishmem_ctx_t *ctxs, int pe_a, int pe_b, char *data0,
+                                                          unsigned long long *sig0, size_t nbytes, int rounds, int staged,
+                                                          pingpong_phases *out)
+{
+    const bool is_a = (blockIdx.x == 0);
+    __shared__ ishmem_ctx_t ctx_copy;
+    const ishmem_ctx_t *ctx = ctxs + (is_a ? pe_a : pe_b);
+    const int other = is_a ? pe_b : pe_a;
+    char *data = local_of(ctxs, ctx, data0);
+    unsigned long long *sig = (unsigned long long *)local_of(ctxs, ctx, sig0);
+    if (staged) ctx = ishmemx_ctx_stage_work_group(&ctx_copy, ctx);
+    unsigned long long acc[5] = {0, 0, 0, 0, 0}, t_start = 0;
+    const unsigned tid = threadIdx.x;
+    if (is_a && tid == 0) t_start = ishmemi::globaltimer_ns();
+    __shared__ int give_up;
+    if (tid == 0) give_up = 0;
+    __syncthreads();
+    for (int r = 1; r <= rounds; ++r) {
+        long long c0 = clock64();
+        if (!is_a) { /* B answers: it waits first */
+            if (tid == 0 && ishmem_uint64_wait_until(ctx, sig, ISHMEM_CMP_GE, (unsigned long long)r)) give_up = 1;
+            __syncthreads();
+            if (give_up) break;
+        }
+        long long c1 = clock64();
+        char *rdst = ishmemi::translate(ctx, data, other);
+        unsigned long long *rs = ishmemi::translate(ctx, sig, other);
+        if (!rdst || !rs) break;
+        /* consume the translated addresses so that the wait for the context reads is counted here */
+        asm volatile("" ::"l"(rdst), "l"(rs) : "memory");
+        long long c2 = clock64();
+        ishmemi::copy_bytes(rdst, data, nbytes, tid, blockDim.x);
+        long long c3 = clock64();
+        __syncthreads();
+        long long c4 = clock64();
+        if (tid == 0) ishmemi::st_release(rs, (unsigned long long)r);
+        long long c5 = clock64();
+        if (is_a) {
+            if (tid == 0 && ishmem_uint64_wait_until(ctx, sig, ISHMEM_CMP_GE, (unsigned long long)r)) give_up = 1;
+            __syncthreads();
+            if (give_up) break;
+        }
+        long long c6 = clock64();
+        acc[0] += (unsigned long long)((c1 - c0) + (c6 - c5));
+        acc[1] += (unsigned long long)(c2 - c1);
+        acc[2] += (unsigned long long)(c3 - c2);
+        acc[3] += (unsigned long long)(c4 - c3);
+        acc[4] += (unsigned long long)(c5 - c4);
+    }
+    if (tid == 0) {
+        for (int i = 0; i < 5; ++i) out->cycles[blockIdx.x][i] = acc[i];
+        if (is_a) {
+            out->elapsed_ns = ishmemi::globaltimer_ns() - t_start;
+            /* primitives, on a word of this PE's own signal area that nobody else touches */
+            unsigned long long *w = sig + 2;
+            const int n = 256;
+            unsigned long long v = 0;
+            long long p0 = clock64();
+            for (int i = 0; i < n; ++i) v += ishmemi::ld_relaxed(w + (v & 1));
+            long long p1 = clock64();
+            for (int i = 0; i < n; ++i) {
+                *(volatile unsigned long long *)(w + 1) = v + (unsigned long long)i;
+                ishmemi::st_release(w, 0ull);
+            }
+            long long p2 = clock64();
+            for (int i = 0; i < n; ++i) ishmemi::st_release(w, 0ull);
+            long long p3 = clock64();
+            out->prim[0] = (unsigned long long)(p1 - p0) / n;
+            out->prim[1] = (unsigned long long)(p2 - p1) / n;
+            out->prim[2] = (unsigned long long)(p3 - p2) / n;
+            *(volatile unsigned long long *)(w + 1) = 0;
+        }
+    }
+}
+
+extern "C" int ishmemx_pingpong_phases(int pe_a, int pe_b, void *data, uint64_t *sig, size_t nbytes, int rounds,
+                                       int threads, int staged, double *ns_out)
+{
+    ISHMEMI_REQUIRE_INIT();
+    auto &g = g_ishmem;
+    if (ishmemi_check_pe(pe_a) || ishmemi_check_pe(pe_b) || pe_a == pe_b) return ISHMEM_ERR_INVALID_PE;
+    if (rounds < 1 || threads < 32 || threads > 1024 || !ns_out) return ISHMEM_ERR_ARG;
+    if ((uintptr_t)sig % 8 || (uintptr_t)data % 8) return ISHMEM_ERR_ALIGN;
+    if (ishmemi_sym_offset(data, nbytes) < 0 || ishmemi_sym_offset(sig, 32) < 0) return ISHMEM_ERR_NOT_SYMMETRIC;
+    cudaStream_t s;
+    int rc = ishmemi_team_stream_begin(ISHMEM_TEAM_WORLD, &s);
+    if (rc) return rc;
+    pingpong_phases *out = (pingpong_phases *)g.h_pinned;
+    memset(out, 0, sizeof(*out));
+    const ishmem_ctx_t *ctxs = g.d_ctx;
+    char *d0 = (char *)data;
+    unsigned long long *s0 = (unsigned long long *)sig;
+    void *params[] = {(void *)&ctxs, (void *)&pe_a,  (void *)&pe_b,   (void *)&d0, (void *)&s0,
+                      (void *)&nbytes, (void *)&rounds, (void *)&staged, (void *)&out};
+    rc = ishmemi_cuda(cudaLaunchCooperativeKernel((void *)k_pingpong_phases, dim3(2), dim3(threads), params, 0, s),
+                      "cudaLaunchCooperativeKernel(pingpong_phases)");
+    ishmemi_count_launch();
+    ishmemi_team_stream_end();
+    if (rc) return rc;
+    ISHMEMI_CUDA(cudaStreamSynchronize(s));
+    int khz = 0;
+    ISHMEMI_CUDA(cudaDeviceGetAttribute(&khz, cudaDevAttrClockRate, g.device));
+    const double ns_per_cycle = 1e6 / (double)khz;
+    for (int b = 0; b < 2; ++b)
+        for (int i = 0; i < 5; ++i) ns_out[b * 5 + i] = (double)out->cycles[b][i] * ns_per_cycle / rounds;
+    for (int i = 0; i < 3; ++i) ns_out[10 + i] = (double)out->prim[i] * ns_per_cycle;
+    ns_out[13] = (double)out->elapsed_ns / (2.0 * rounds);
+    return ISHMEM_OK;
+}
+
 /* ---- device-timed put/get latency --------------------------------------------------------- */
 
 template <int LEVEL>

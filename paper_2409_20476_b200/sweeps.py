@@ -397,7 +397,7 @@ def sweep_c3(args, out):
         # device-resident forms: one work-group per PE, push sync inside the kernel, `rep` calls per launch
         rep = 50
         for threads in (128, 256, 1024):
-            for n in [4 ** k for k in range(0, 10)]:
+            for n in [4 ** k for k in range(0, 12)]:
                 for which, opname, nb in ((0, "broadcast", n * (1 + P)), (1, "fcollect", n * (P + P * P)),
                                           (2, "sum_reduce_f32", 2 * P * n)):
                     if which == 2 and n < 4:
@@ -468,6 +468,23 @@ def sweep_c4(args, out):
                 out.add(config=4, op="put_signal_pingpong", pattern="pe0<->pe1", variant="in_kernel", threads=threads,
                         groups=1, npes=2, dtype="u8", nbytes=n, l2="hot", iters=rounds, us_per_op=float(rtt[0]) / 1e3,
                         alg_bytes=2 * n + 8, note=f"half round trip; stamp mismatches {int(bad[0])}")
+    # where a half round trip goes: the instrumented exchange, context in global memory and in shared memory
+    ph = np.zeros(14)
+    names = ("wait", "translate", "copy", "barrier", "release")
+    for staged in (0, 1):
+        for threads in (32, 256):
+            for n in (8, 256, 4096):
+                for rep in range(2):
+                    B.ishmem_uint64_p(0, sig, 0, 0)
+                    B.ishmem_uint64_p(1, sig, 0, 1)
+                    B.ishmemx_pingpong_phases(0, 1, data, sig, n, 2000, threads, staged, ph)
+                note = "; ".join(f"{side} " + " ".join(f"{nm} {ph[5 * k + i]:.0f}" for i, nm in enumerate(names))
+                                 for k, side in enumerate("AB"))
+                note += f"; L2 trip {ph[10]:.0f}; store+release {ph[11]:.0f}; release alone {ph[12]:.0f}"
+                out.add(config=4, op="pingpong_phases", pattern="pe0<->pe1",
+                        variant="context_in_shared_memory" if staged else "context_in_global_memory", threads=threads,
+                        groups=1, npes=2, dtype="u8", nbytes=n, l2="hot", iters=2000, us_per_op=float(ph[13]) / 1e3,
+                        note="ns per round: " + note)
     assert B.ishmemx_status(1) == 0
     B.ishmem_finalize()
 
@@ -649,7 +666,11 @@ def summarize(path) -> str:
                 touched = float(r["note"].rsplit("carry ", 1)[1].split()[0])
                 t = float(r["us_per_op"])
                 return f"{float(r['gbps']):.0f} / {touched / t / 1e3:.0f}"
-            out += [_table(sel, nb, lambda r: r["variant"], both, _fmt_size), ""]
+            for es in ("4", "8", "16"):
+                part = [r for r in sel if r["level"] == es]
+                out += [f"elements of {es} bytes (row: number of elements; column: destination stride, source stride):", "",
+                        _table(part, lambda r: nb(r) // int(es), lambda r: r["variant"].split("_", 1)[1].replace("_", " "), both,
+                               lambda n: f"2^{int(n).bit_length() - 1}"), ""]
         sel = [r for r in rows if r["pattern"] == "one_pe" and r["variant"].startswith("host_api")]
         out += ["### host API `ishmem_putmem` on ONE PE (PE 0 -> PE 1), back-to-back calls: microseconds per call / GB/s", "",
                 _table(sel, nb, lambda r: r["variant"][9:], lambda r: f"{us(r)} / {gb(r)}", _fmt_size), ""]
@@ -702,7 +723,7 @@ def summarize(path) -> str:
                         a = {nb(r): float(r["us_per_op"]) for r in sel if r["npes"] == P and r["threads"] == T_}
                         c = _crossover(a, b)
                         out.append(f"- {op}, {P} PEs, one work-group of {T_} work-items per PE against the host-started copy "
-                                   f"engine: engine at least as fast from " + (_fmt_size(c) if c else "no size measured (<= 256 KiB)"))
+                                   f"engine: engine at least as fast from " + (_fmt_size(c) if c else "no size measured (<= 4 MiB)"))
                 out.append("")
     elif cfg == 4:
         out += ["### remote atomics, 16 PEs: Mops/s (one op per GPU thread)", "", "| op | index stream | variant | threads | Mops/s | us |",
@@ -710,6 +731,19 @@ def summarize(path) -> str:
         for r in rows:
             if r["mops"]:
                 out.append(f"| {r['op']} | {r['pattern']} | {r['variant']} | {r['threads']} | {float(r['mops']):.0f} | {us(r)} |")
+        sel = [r for r in rows if r["op"] == "pingpong_phases"]
+        if sel:
+            out += ["", "### where a half round trip goes (`ishmemx_pingpong_phases`): nanoseconds per round and side", "",
+                    "Each side's five phases add up to its round (= two half round trips); `wait` on a side contains the other "
+                    "side's translate + copy + barrier + release.  Cycle counter of the SM, converted at the nominal clock.", "",
+                    "| context | threads | size | half rtt us | A: wait / translate / copy / barrier / release | "
+                    "B: wait / translate / copy / barrier / release | L2 trip | store + release | release alone |",
+                    "|---|---:|---:|---:|---|---|---:|---:|---:|"]
+            for r in sel:
+                f = r["note"].replace("ns per round: ", "").split("; ")
+                side = lambda t: " / ".join(t.split()[2::2])
+                out.append(f"| {r['variant'][11:].replace('_', ' ')} | {r['threads']} | {_fmt_size(r['nbytes'])} | {us(r)} | {side(f[0])} | "
+                           f"{side(f[1])} | {f[2].split()[-1]} | {f[3].split()[-1]} | {f[4].split()[-1]} |")
         sel = [r for r in rows if r["op"] == "put_signal_pingpong"]
         out += ["", "### put_signal / wait_until ping-pong, half round trip in microseconds (in-kernel)", "",
                 _table(sel, nb, lambda r: f"{r['threads']} threads", us, _fmt_size), ""]

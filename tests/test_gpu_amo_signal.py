@@ -207,3 +207,25 @@ def test_compare_swap_token_passing_is_linearisable(aggregate):
                 assert np.array_equal(won, np.arange(final[w] - won.size, final[w])), w
             assert (final > 0).all()
         assert s.status() == 0
+
+
+@pytest.mark.parametrize("staged", [0, 1])
+def test_pingpong_phase_breakdown_moves_the_data_and_adds_up(staged):
+    """The instrumented exchange: the payload arrives on both sides (bit-exact against the oracle's
+    put_signal), both signal words count the rounds, and each side's five phases add up to its round
+    (two half round trips by the global timer, within the clocks' disagreement)."""
+    with Session(2, 1 << 16) as s:
+        data, sig = s.malloc(4096), s.malloc(64)
+        n, rounds = 256, 500
+        data.fill(0, inputs.byte_payload(inputs.SEED_C4, 7, n))
+        ph = np.zeros(14)
+        B.ishmemx_pingpong_phases(0, 1, data.addr, sig.addr, n, rounds, 64, staged, ph)
+        assert s.status() == 0
+        s.oracle.putmem_signal(0, data.ooff, s.oracle.ptr(data.ooff, n, 0), n, sig.ooff, rounds, orc.SIG_SET, 1)
+        s.oracle.putmem_signal(1, data.ooff, s.oracle.ptr(data.ooff, n, 1), n, sig.ooff, rounds, orc.SIG_SET, 0)
+        heaps_equal(s, "instrumented ping-pong")
+        assert (ph[:10] >= 0).all() and ph[10] > 50 and ph[11] > ph[12] > 0 and ph[13] > 0
+        for side in (0, 1):
+            assert abs(ph[5 * side:5 * side + 5].sum() - 2 * ph[13]) < 0.25 * 2 * ph[13], (side, ph)
+        with pytest.raises(B.IshmemError):
+            B.ishmemx_pingpong_phases(0, 0, data.addr, sig.addr, n, rounds, 64, staged, ph)
