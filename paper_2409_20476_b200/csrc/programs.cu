@@ -1192,8 +1192,10 @@ static __device__ __noinline__ void jacobi_send_piece_k(const ishmem_ctx_t *ctxs
 /* one launch = K sweeps: sender blocks (K rows each way per PE), then one block per band of `band_rows`
  * rows x (blockDim / 32) tiles, in launch order as in k_jacobi_sweep */
 #define JACOBI_PASS_THREADS 128
+/* four blocks per SM (128 registers); the four-level window with four columns per lane would spill there
+ * and gets three (170 registers): 718 against 739 us per launch on a single strip */
 template <int K, int NC>
-__global__ void __launch_bounds__(JACOBI_PASS_THREADS, 4) k_jacobi_pass(const ishmem_ctx_t *ctxs, jacobi_args a, double *xh0,
+__global__ void __launch_bounds__(JACOBI_PASS_THREADS, (K == 4 && NC == 4) ? 3 : 4) k_jacobi_pass(const ishmem_ctx_t *ctxs, jacobi_args a, double *xh0,
                                                                         int flip, unsigned long long arrived, int last,
                                                                         unsigned band_rows, unsigned bands,
                                                                         unsigned tile_groups, int P, size_t heap_stride)
