@@ -119,7 +119,7 @@ typedef int ishmem_team_t;
  * at initialisation: ISHMEM_CUTOVER_{PUT,PUT_UPTO,BCAST,FCOLLECT,WORK_GROUP} (bytes, "never" or "always";
  * see ishmemx_set_cutover), ISHMEM_WAIT_TIMEOUT_NS (see ishmemx_set_wait_limit_ns) and the
  * initial values of the launch-shape switches (ISHMEM_JACOBI_SPLIT, _JACOBI_FUSE, _JACOBI_WIDE,
- * ISHMEM_REDUCE_BULK, ISHMEM_BULK_SMEM; see ishmemx_set_option).  No variable is read later. */
+ * ISHMEM_REDUCE_BULK, ISHMEM_BULK_SMEM, ISHMEM_PUSH_SHAPE; see ishmemx_set_option).  No variable is read later. */
 int ishmem_init(int npes, size_t heap_bytes);
 int ishmemx_init_external(int npes, size_t heap_bytes, void *base);
 /* Waits for all streams, frees everything the library allocated. */
@@ -145,6 +145,11 @@ size_t ishmemx_heap_bytes(void);
  *       shared-memory TMA fold ring instead of one tile per block (default 0).
  *   ISHMEMX_OPT_BULK_SMEM (ISHMEM_BULK_SMEM=bytes): shared-memory staging per block of the
  *       ISHMEMX_WORK_GROUP_BULK level (default 192 KiB + 128, capped by the device limit).
+ *   ISHMEMX_OPT_PUSH_SHAPE (ISHMEM_PUSH_SHAPE=0|1|2): launch shape of host-called broadcast and
+ *       fcollect by stores: 1 = fan-out tiles (a thread stores each vector it loads to every
+ *       destination), 2 = one block per (tile, source member, destination), each a plain copy,
+ *       0 = by measurement (default: the second for messages of at least 4 MiB on teams of up to
+ *       6 members, where it is up to 25 % faster; the first otherwise).
  * ishmemx_set_option returns ISHMEM_ERR_ARG for an unknown option or a value outside its range;
  * ishmemx_get_option returns the current value (0 for an unknown option). */
 #define ISHMEMX_OPT_JACOBI_SPLIT 0
@@ -152,7 +157,8 @@ size_t ishmemx_heap_bytes(void);
 #define ISHMEMX_OPT_JACOBI_WIDE 2
 #define ISHMEMX_OPT_REDUCE_BULK 3
 #define ISHMEMX_OPT_BULK_SMEM 4
-#define ISHMEMX_OPT_COUNT 5
+#define ISHMEMX_OPT_PUSH_SHAPE 5
+#define ISHMEMX_OPT_COUNT 6
 int ishmemx_set_option(int option, long long value);
 long long ishmemx_get_option(int option);
 /* Device pointer to PE `pe`'s context (ishmem_ctx_t, see ishmem_device.cuh), to hand to

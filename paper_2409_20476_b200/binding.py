@@ -44,7 +44,7 @@ ISHMEM_CMP_EQ, ISHMEM_CMP_NE, ISHMEM_CMP_GT, ISHMEM_CMP_GE, ISHMEM_CMP_LT, ISHME
  ISHMEM_T_UINT64, ISHMEM_T_INT8, ISHMEM_T_UINT8, ISHMEM_T_INT16, ISHMEM_T_UINT16) = range(10)
 ISHMEMX_REDUCE_AUTO, ISHMEMX_REDUCE_DUPLICATED, ISHMEMX_REDUCE_SPLIT = range(3)
 (ISHMEMX_OPT_JACOBI_SPLIT, ISHMEMX_OPT_JACOBI_FUSE, ISHMEMX_OPT_JACOBI_WIDE, ISHMEMX_OPT_REDUCE_BULK,
- ISHMEMX_OPT_BULK_SMEM) = range(5)
+ ISHMEMX_OPT_BULK_SMEM, ISHMEMX_OPT_PUSH_SHAPE) = range(6)
 SIZE_MAX = 2**64 - 1
 
 

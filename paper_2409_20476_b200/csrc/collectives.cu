@@ -62,6 +62,53 @@ __global__ void __launch_bounds__(1024) k_fcollect(const ishmem_ctx_t *ctxs, col
                      local_of(ctxs, ctx, a.src), a.n, st, g, (size_t)a.groups, a.push_tile);
 }
 
+/* ---- broadcast / fcollect of large messages as (tile, source member, destination) triples --------
+ * One block copies one 32 KiB tile of one member's source into one member's destination, like a tile
+ * of a put; the destination runs fastest, then the source member, then the tile, so the P blocks that
+ * read the same source tile start together (one of them brings it from DRAM, the others find it in
+ * L2) and the running blocks sweep one window of every source and destination in launch order.  The
+ * fan-out kernels above store each loaded vector P times from the same thread, which wins on large
+ * teams; on small teams the P separate copies move more bytes per second (single launches, broadcast of
+ * 256 MiB / fcollect of 64 MiB per PE, fan-out against triples: 4 PEs 5.1 / 4.9 against 6.2 / 6.1 TB/s,
+ * 8 PEs 6.2 / 6.0 against 6.0 / 6.0, 12 PEs 6.4 / 6.4 against 5.9 / 5.8).  members = 1: broadcast from
+ * `root`; members = team size: fcollect. */
+#define PUSH_PAIR_TILE 32768u
+__global__ void __launch_bounds__(256) k_push_pairs(const ishmem_ctx_t *ctxs, coll_args a, int members, int skip)
+{
+    const ishmemi_team t = ctxs[0].teams[a.team];
+    const size_t P = (size_t)t.size, per = (a.n + PUSH_PAIR_TILE - 1) / PUSH_PAIR_TILE;
+    const size_t total = per * (size_t)members * P;
+    for (size_t b = blockIdx.x; b < total; b += gridDim.x) {
+        const int q = (int)(b % P), i = (int)((b / P) % (size_t)members);
+        const size_t o = (b / (P * (size_t)members)) * PUSH_PAIR_TILE;
+        if (q == skip) continue;
+        const int from = members == 1 ? a.root : i;
+        const ishmem_ctx_t *ctx = ctxs + (t.start + from * t.stride);
+        /* the pushing PE names the destination by its own copy and translates it to member q */
+        char *d = ishmemi::translate(ctx, local_of(ctxs, ctx, a.dest), t.start + q * t.stride);
+        if (!d) return;
+        const size_t len = a.n - o < PUSH_PAIR_TILE ? a.n - o : PUSH_PAIR_TILE;
+        ishmemi::copy_bytes(d + (members == 1 ? 0 : (size_t)i * a.n) + o, local_of(ctxs, ctx, a.src) + o, len, threadIdx.x,
+                            blockDim.x);
+    }
+}
+/* ISHMEMX_OPT_PUSH_SHAPE: 1 = fan-out tiles, 2 = (tile, member, destination) triples, 0 = by measurement:
+ * triples for messages of at least 4 MiB on teams of up to 6 members */
+static bool push_as_pairs(size_t nbytes, int team_size)
+{
+    const long long shape = g_ishmem.opt[ISHMEMX_OPT_PUSH_SHAPE];
+    if (shape == 1) return false;
+    if (shape == 2) return true;
+    return g_ishmem.coll_groups == 0 && nbytes >= ((size_t)4 << 20) && team_size <= 6;
+}
+static int launch_push_pairs(cudaStream_t s, const coll_args &a, int members, int P, int skip)
+{
+    const size_t per = (a.n + PUSH_PAIR_TILE - 1) / PUSH_PAIR_TILE, total = per * (size_t)members * (size_t)P;
+    k_push_pairs<<<(unsigned)(total < 0x7fffffffu ? total : 0x7fffffffu), 256, 0, s>>>(g_ishmem.d_ctx, a, members, skip);
+    ishmemi_count_launch();
+    return ishmemi_check_launch("k_push_pairs");
+}
+
 /* ---- collect: fcollect with a size and an offset per member ------------------------------------ */
 struct collect_args {
     ishmem_team_t team;
@@ -406,12 +453,16 @@ extern "C" int ishmem_broadcastmem(ishmem_team_t team, void *dest, const void *s
         a.src = (const char *)src;
         a.n = nbytes;
         a.root = root;
-        const push_shape sh = push_geometry(nbytes, 1, t.size);
-        a.staging_bytes = sh.staging;
-        a.push_tile = sh.tile;
-        k_broadcast<<<sh.blocks_per_member, sh.threads, sh.staging, s>>>(g.d_ctx, a);
-        ishmemi_count_launch();
-        rc = ishmemi_check_launch("k_broadcast");
+        if (push_as_pairs(nbytes, t.size)) {
+            rc = launch_push_pairs(s, a, 1, t.size, g.bcast_root_dest ? -1 : root);
+        } else {
+            const push_shape sh = push_geometry(nbytes, 1, t.size);
+            a.staging_bytes = sh.staging;
+            a.push_tile = sh.tile;
+            k_broadcast<<<sh.blocks_per_member, sh.threads, sh.staging, s>>>(g.d_ctx, a);
+            ishmemi_count_launch();
+            rc = ishmemi_check_launch("k_broadcast");
+        }
     }
     ishmemi_team_stream_end();
     return rc;
@@ -448,13 +499,17 @@ extern "C" int ishmem_fcollectmem(ishmem_team_t team, void *dest, const void *sr
         a.dest = (char *)dest;
         a.src = (const char *)src;
         a.n = nbytes;
-        const push_shape sh = push_geometry(nbytes, t.size, t.size);
-        a.groups = sh.blocks_per_member;
-        a.staging_bytes = sh.staging;
-        a.push_tile = sh.tile;
-        k_fcollect<<<a.groups * t.size, sh.threads, sh.staging, s>>>(g.d_ctx, a);
-        ishmemi_count_launch();
-        rc = ishmemi_check_launch("k_fcollect");
+        if (push_as_pairs(nbytes, t.size)) {
+            rc = launch_push_pairs(s, a, t.size, t.size, -1);
+        } else {
+            const push_shape sh = push_geometry(nbytes, t.size, t.size);
+            a.groups = sh.blocks_per_member;
+            a.staging_bytes = sh.staging;
+            a.push_tile = sh.tile;
+            k_fcollect<<<a.groups * t.size, sh.threads, sh.staging, s>>>(g.d_ctx, a);
+            ishmemi_count_launch();
+            rc = ishmemi_check_launch("k_fcollect");
+        }
     }
     ishmemi_team_stream_end();
     return rc;

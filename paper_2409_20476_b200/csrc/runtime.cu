@@ -240,6 +240,11 @@ static int init_common(int npes, size_t heap_bytes, void *external)
     g.opt[ISHMEMX_OPT_JACOBI_WIDE] = -1;
     g.opt[ISHMEMX_OPT_REDUCE_BULK] = 0;
     g.opt[ISHMEMX_OPT_BULK_SMEM] = 192 * 1024 + 128;
+    g.opt[ISHMEMX_OPT_PUSH_SHAPE] = 0;
+    if (const char *v = getenv("ISHMEM_PUSH_SHAPE")) {
+        const int f = atoi(v);
+        if (f >= 0 && f <= 2) g.opt[ISHMEMX_OPT_PUSH_SHAPE] = f;
+    }
     if (const char *v = getenv("ISHMEM_JACOBI_SPLIT")) {
         if (!strcmp(v, "rows")) g.opt[ISHMEMX_OPT_JACOBI_SPLIT] = 1;
         else if (!strcmp(v, "columns")) g.opt[ISHMEMX_OPT_JACOBI_SPLIT] = 2;
@@ -628,6 +633,7 @@ extern "C" int ishmemx_set_option(int option, long long value)
     ISHMEMI_REQUIRE_INIT();
     switch (option) {
     case ISHMEMX_OPT_JACOBI_SPLIT:
+    case ISHMEMX_OPT_PUSH_SHAPE:
         if (value < 0 || value > 2) return ISHMEM_ERR_ARG;
         break;
     case ISHMEMX_OPT_JACOBI_FUSE:

@@ -191,3 +191,38 @@ def test_device_resident_collectives_with_push_sync(threads):
         # (64 PEs would still fit; the refusal path is exercised through the argument check)
         with pytest.raises(B.IshmemError):
             B.ishmemx_collective_on_device(2, W, dst.addr, dst.addr, 4, 0, 0, 0, threads, 1)  # overlap
+
+
+@pytest.mark.parametrize("shape", [1, 2])
+def test_push_shapes_of_broadcast_and_fcollect(shape):
+    """Both launch shapes of host-called broadcast / fcollect (fan-out tiles; one block per tile, source
+    member and destination) on sizes around and across the 32 KiB tile, odd offsets, a strided team, a
+    non-zero root and the reading in which the root does not write its own dest: whole heaps against the
+    oracle."""
+    npes, nmax = 6, 100_003
+    with Session(npes, 8 * nmax + (1 << 16)) as s:
+        B.ishmemx_set_option(B.ISHMEMX_OPT_PUSH_SHAPE, shape)
+        assert B.ishmemx_get_option(B.ISHMEMX_OPT_PUSH_SHAPE) == shape
+        src, dst = s.malloc(nmax), s.malloc(npes * nmax)
+        for p in range(npes):
+            src.fill(p, inputs.byte_payload(inputs.SEED_C3, 90 + p, nmax))
+        W, o = B.ISHMEM_TEAM_WORLD, s.oracle
+        for n, so, do, root in ((1, 0, 0, 0), (32768, 0, 0, 5), (32769, 1, 3, 2), (nmax - 7, 7, 0, 1), (65536, 16, 48, 3)):
+            B.ishmem_broadcastmem(W, dst.addr + do, src.addr + so, n, root)
+            o.broadcastmem(o.world, dst.ooff + do, src.ooff + so, n, root)
+            heaps_equal(s, f"broadcast {n} shape {shape}")
+            B.ishmem_fcollectmem(W, dst.addr + do, src.addr + so, n)
+            o.fcollectmem(o.world, dst.ooff + do, src.ooff + so, n)
+            heaps_equal(s, f"fcollect {n} shape {shape}")
+        B.ishmemx_set_bcast_root_dest(0)
+        B.ishmem_broadcastmem(W, dst.addr, src.addr + 2, 70_000, 4)
+        o.broadcastmem(o.world, dst.ooff, src.ooff + 2, 70_000, 4, root_writes_dest=False)
+        B.ishmemx_set_bcast_root_dest(1)
+        team = B.ishmem_team_split_strided(W, 1, 2, 3)           # PEs 1, 3, 5
+        B.ishmem_broadcastmem(team, dst.addr + 5, src.addr, 40_000, 2)
+        o.broadcastmem((1, 2, 3), dst.ooff + 5, src.ooff, 40_000, 2)
+        B.ishmem_fcollectmem(team, dst.addr + 9, src.addr + 1, 33_333)
+        o.fcollectmem((1, 2, 3), dst.ooff + 9, src.ooff + 1, 33_333)
+        B.ishmem_barrier_all()
+        heaps_equal(s, f"strided team shape {shape}")
+        assert s.status() == 0
