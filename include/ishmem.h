@@ -614,6 +614,13 @@ int ishmemx_rma_latency(int my_pe, void *dest, const void *src, size_t nbytes, i
 int ishmemx_jacobi(double *buf0, double *buf1, uint64_t *sig, size_t ny, size_t nx, int iters,
                    int overlap, int groups_per_pe, int threads, double *residual_sq_host);
 
+/* How ishmemx_jacobi cuts `iters` sweeps into launches when a launch may do up to max_depth (1..4)
+ * sweeps: writes the sweeps of each launch, deepest first, to HOST depths_out (room for `capacity`
+ * entries; may be NULL with capacity 0) and returns the number of launches, which always has the
+ * parity of iters (every launch moves the grid to the other buffer), or ISHMEM_ERR_ARG.  Pure host
+ * arithmetic: needs neither a device nor ishmem_init. */
+int ishmemx_jacobi_launch_depths(int iters, int max_depth, int *depths_out, int capacity);
+
 /* The same Jacobi program for callers that must not allocate device memory at the point of
  * the call -- a frozen memory pool, a loop where cudaMalloc's device-wide synchronisation is
  * not acceptable, an allocator that owns the whole GPU.  (The paper has no counterpart; this

@@ -166,6 +166,7 @@ def _signatures() -> dict[str, tuple[str, list[str]]]:
         "ishmemx_ring_benchmark": ("status", ["i", "i", "i", "i", "p", "p"]),
         "ishmemx_rma_latency": ("status", ["i", "p", "p", "z", "i", "i", "i", "i", "i", "p"]),
         "ishmemx_jacobi": ("status", ["p", "p", "p", "z", "z", "i", "i", "i", "i", "p"]),
+        "ishmemx_jacobi_launch_depths": ("int", ["i", "i", "p", "i"]),
         "ishmemx_jacobi_noalloc": ("status", ["p", "p", "p", "z", "z", "i", "i", "i", "i", "p"]),
         "ishmemx_host_put_ring": ("status", ["p", "p", "p", "p", "z", "i", "i", "i", "i"]),
     }

@@ -1420,6 +1420,17 @@ static void jacobi_split(int iters, int kmax, std::vector<int> *out)
     std::sort(out->begin(), out->end(), [](int x, int y) { return x > y; });
 }
 
+/* The split alone, for callers that want to know the launches of a call beforehand and for tests of
+ * the host logic: needs no device and no initialised library. */
+extern "C" int ishmemx_jacobi_launch_depths(int iters, int max_depth, int *depths_out, int capacity)
+{
+    if (iters < 0 || max_depth < 1 || max_depth > 4 || capacity < 0 || (capacity && !depths_out)) return ISHMEM_ERR_ARG;
+    std::vector<int> d;
+    jacobi_split(iters, max_depth, &d);
+    for (size_t i = 0; i < d.size() && i < (size_t)capacity; ++i) depths_out[i] = d[i];
+    return (int)d.size();
+}
+
 static unsigned jacobi_pass_groups(size_t nx, int k, int nc)
 {
     const unsigned skip = (unsigned)((k + nc - 1) / nc), tile = (32u - 2u * skip) * (unsigned)nc;

@@ -177,3 +177,26 @@ def test_bench_gpus_2_starts_two_ranks_by_itself():
     assert len(lines) == 1
     line = json.loads(lines[0])
     assert line["impl"] == "reference" and line["n_gpus"] == 2 and line["value"] > 0
+
+
+def test_jacobi_launch_split_host_logic():
+    """The launches of a Jacobi call: depths between 1 and the cap, deepest first, adding up to the sweep
+    count, and as many as the sweep count is even or odd (each launch flips the buffers; the result must
+    end where single sweeps leave it).  Long calls are all deepest launches but for a short tail."""
+    import numpy as np
+    from paper_2409_20476_b200 import binding as B
+    for cap in (1, 2, 3, 4):
+        for iters in list(range(0, 60)) + [199, 200, 201, 1000, 1001]:
+            out = np.zeros(iters + 1, dtype=np.int32)
+            n = B.ishmemx_jacobi_launch_depths(iters, cap, out, len(out))
+            d = out[:n].tolist()
+            assert sum(d) == iters and n % 2 == iters % 2, (cap, iters, d)
+            assert all(1 <= k <= cap for k in d) and d == sorted(d, reverse=True), (cap, iters, d)
+            if iters >= 40:
+                assert d.count(cap) >= (iters - 24) // cap, (cap, iters, d)
+    out = np.zeros(64, dtype=np.int32)
+    assert B.ishmemx_jacobi_launch_depths(200, 4, out, 64) == 50 and set(out[:50].tolist()) == {4}
+    assert B.ishmemx_jacobi_launch_depths(9, 4, out, 64) == 3 and out[:3].tolist() == [4, 4, 1]
+    assert B.ishmemx_jacobi_launch_depths(7, 4, None, 0) == 3          # count only
+    for bad in ((-1, 4), (5, 0), (5, 5)):
+        assert B.ishmemx_jacobi_launch_depths(bad[0], bad[1], out, 64) == B.ISHMEM_ERR_ARG
