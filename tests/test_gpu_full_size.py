@@ -249,9 +249,9 @@ class Strips:
 def test_config5_jacobi_16384_whole_grid_even_and_odd_sweep_counts():
     """Config 5 at full size in the launch shape the library picks by itself (wide two-sweep
     passes at this size), 12 PEs: the WHOLE final grid bit for bit against the oracle's plain
-    full-grid sweeps, and the residual at 1e-6 relative, for 8 sweeps (two-sweep passes only)
-    and 9 (passes, then single-sweep launches) -- every band and tile-group seam and all eleven
-    strip seams are compared.  The ninth oracle sweep continues from the eighth (a sweep has no
+    full-grid sweeps, and the residual at 1e-6 relative, for 8 sweeps (two launches of four)
+    and 9 (three launches of three) -- every band and tile-group seam and all eleven strip seams are
+    compared.  The ninth oracle sweep continues from the eighth (a sweep has no
     memory, which a CPU test pins)."""
     npes, n = 12, 16384
     grid = config5_grid(n, n)

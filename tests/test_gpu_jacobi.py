@@ -61,8 +61,8 @@ def test_jacobi_matches_oracle(ny, nx, npes, groups, threads, overlap, split):
     """split: the persistent kernel with the strips cut by columns or by rows, or one of the launch-ordered
     forms that the library uses for threads = 0 and even nx: `sweeps` = its own choice (one tile per warp, up
     to four sweeps per launch, four columns per lane where nx is a multiple of 4), the same with two columns
-    per lane, with at most two or three sweeps per launch, or with one sweep per launch.  21 sweeps are
-    launches of 4, 4, 4, 4, 3, 1 and 1 sweeps in the first form."""
+    per lane, with at most two or three sweeps per launch, or with one sweep per launch.  The 21 sweeps are
+    cut into launches by ishmemx_jacobi_launch_depths (an odd number of them, deepest first)."""
     if split in SWEEP_FORMS:
         options = [(B.ISHMEMX_OPT_JACOBI_SPLIT, 0), (B.ISHMEMX_OPT_JACOBI_FUSE, SWEEP_FORMS[split][0]),
                    (B.ISHMEMX_OPT_JACOBI_WIDE, SWEEP_FORMS[split][1])]
