@@ -198,7 +198,7 @@ def test_jacobi_launch_split_host_logic():
     assert B.ishmemx_jacobi_launch_depths(200, 4, out, 64) == 50 and set(out[:50].tolist()) == {4}
     assert B.ishmemx_jacobi_launch_depths(9, 4, out, 64) == 3 and out[:3].tolist() == [3, 3, 3]
     assert B.ishmemx_jacobi_launch_depths(8, 4, out, 64) == 2 and out[:2].tolist() == [4, 4]
-    assert B.ishmemx_jacobi_launch_depths(5, 4, out, 64) == 3 and out[:3].tolist() == [3, 1, 1]
+    assert B.ishmemx_jacobi_launch_depths(5, 4, out, 64) == 3 and out[:3].tolist() == [2, 2, 1]
     assert B.ishmemx_jacobi_launch_depths(7, 4, None, 0) == 3          # count only
     for bad in ((-1, 4), (5, 0), (5, 5)):
         assert B.ishmemx_jacobi_launch_depths(bad[0], bad[1], out, 64) == B.ISHMEM_ERR_ARG
