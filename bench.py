@@ -686,7 +686,7 @@ def run_profile_case(args) -> dict:
     from paper_2409_20476_b200 import binding as B
     from paper_2409_20476_b200 import inputs
 
-    if args.profile_case == "jacobi":
+    if args.profile_case in ("jacobi", "jacobi_persistent"):
         return run_profile_jacobi(args)
     n = args.msg_mib * MiB
     heap_bytes = 2 * n + (1 << 20) if args.profile_case != "fcollect" else (NPES + 1) * n + (1 << 20)
@@ -728,6 +728,7 @@ def run_profile_jacobi(args) -> dict:
     from paper_2409_20476_b200 import inputs
 
     ny, nx, sweeps = 4096, 16384, 8
+    persistent = args.profile_case == "jacobi_persistent"   # the resident kernel, strips cut by column tiles
     rows = ny // NPES
     nbytes = (rows + 2) * nx * 8
     heap_bytes = 2 * nbytes + MiB
@@ -742,6 +743,8 @@ def run_profile_jacobi(args) -> dict:
     ts = torch.cuda.Stream()
     B.ishmemx_set_stream(-1, ts.cuda_stream)
     res, times = np.zeros(1), []
+    if persistent:
+        B.ishmemx_set_option(B.ISHMEMX_OPT_JACOBI_SPLIT, 2)
     for _ in range(2 + args.steps):
         for p in range(NPES):
             for w in range(4):
@@ -755,13 +758,13 @@ def run_profile_jacobi(args) -> dict:
         times.append(a.elapsed_time(b))
     status = B.ishmemx_status(1)
     B.ishmem_finalize()
-    return {"profile_case": "jacobi", "ny": ny, "nx": nx, "sweeps_per_call": sweeps, "status": status,
+    return {"profile_case": args.profile_case, "ny": ny, "nx": nx, "sweeps_per_call": sweeps, "status": status,
             "ms": [round(t, 4) for t in times[2:]]}
 
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--profile-case", default=None, choices=["put", "get", "reduce", "broadcast", "fcollect", "jacobi"],
+    ap.add_argument("--profile-case", default=None, choices=["put", "get", "reduce", "broadcast", "fcollect", "jacobi", "jacobi_persistent"],
                     help="run only a few launches of one kernel on a small case (for ncu captures)")
     ap.add_argument("--msg-mib", type=int, default=32)
     ap.add_argument("--gpus", type=int, default=1)
