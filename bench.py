@@ -290,7 +290,7 @@ def config5_leg(B, torch, peaks) -> dict:
     npes, n, sweeps = 12, 16384, 40
     rows_max = -(-n // npes)
     nbytes = (rows_max + 2) * n * 8
-    heap_bytes = 2 * nbytes + MiB
+    heap_bytes = 2 * nbytes + 2 * MiB     # the buffers, the signals and the call's own halo rows
     heap = torch.zeros(npes * heap_bytes, dtype=torch.uint8, device="cuda")
     B.ishmemx_init_external(npes, heap_bytes, heap.data_ptr())
     ts = torch.cuda.Stream()
@@ -731,7 +731,7 @@ def run_profile_jacobi(args) -> dict:
     persistent = args.profile_case == "jacobi_persistent"   # the resident kernel, strips cut by column tiles
     rows = ny // NPES
     nbytes = (rows + 2) * nx * 8
-    heap_bytes = 2 * nbytes + MiB
+    heap_bytes = 2 * nbytes + 2 * MiB     # the buffers, the signals and the call's own halo rows
     heap = torch.zeros(NPES * heap_bytes, dtype=torch.uint8, device="cuda")
     B.ishmemx_init_external(NPES, heap_bytes, heap.data_ptr())
     b0, b1, sig = B.ishmem_malloc(nbytes), B.ishmem_malloc(nbytes), B.ishmem_calloc(4, 8)

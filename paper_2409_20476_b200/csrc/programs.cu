@@ -934,6 +934,7 @@ __global__ void __launch_bounds__(256, 4) k_jacobi_sweep(const ishmem_ctx_t *ctx
  * the symmetric heap for the duration of the call. */
 #define JW_FULL 0xffffffffu
 #define JW_AHEAD 3 /* rows between a load and the L2 prefetch issued with it */
+#define JW_MAX_DEPTH 6 /* sweeps per launch at most */
 
 template <int NC>
 __device__ __forceinline__ void jw_ld(const double *p, double (&v)[NC])
@@ -1037,26 +1038,28 @@ __device__ __forceinline__ void jw_step(jw_window<K, NC> &W, double (&c)[NC], in
 struct jw_rows {
     const double *cur; /* local rows 0 .. rows+1 */
     const double *nxt; /* its rows 0 and rows+1 hold local rows -1 and rows+2 during the pass */
-    const double *xh;  /* four rows: local rows -2, -3, rows+3, rows+4 */
-    int rows;
+    const double *xh;  /* 2 x xh_side extra rows: local rows -2, -3, ... then rows+3, rows+4, ... */
+    int rows, xh_side;
     size_t nx;
     __device__ __forceinline__ const double *at(int r) const
     {
         if (r < 0) return r == -1 ? nxt : xh + (size_t)(-r - 2) * nx;
-        if (r > rows + 1) return r == rows + 2 ? nxt + (size_t)(rows + 1) * nx : xh + (size_t)(r - rows - 1) * nx;
+        if (r > rows + 1)
+            return r == rows + 2 ? nxt + (size_t)(rows + 1) * nx : xh + (size_t)(xh_side + r - rows - 3) * nx;
         return cur + (size_t)r * nx;
     }
 };
 
 /* Rows [ra, rb) of the strip, tile t, by one warp.  D rows are in flight per lane.  EDGE: the tile
- * touches the grid's first or last column or a column outside it, or the band reads rows outside the
- * source buffer, or forms one of the grid's fixed rows; without EDGE nothing of that is tested.
- * Returns the lane's share of the squared last update when RES. */
-template <int K, int NC, int D, bool EDGE, bool RES>
+ * touches the grid's first or last column or a column outside it, or the band forms one of the grid's
+ * fixed rows; without EDGE nothing of that is tested.  HALO: the band reads rows outside the source
+ * buffer (EDGE implies it); without it the rows are one pitch apart.  Returns the lane's share of the
+ * squared last update when RES. */
+template <int K, int NC, int D, bool EDGE, bool HALO, bool RES>
 __device__ __forceinline__ double jw_march(const jw_rows &src, double *nxt, int ra, int rb, int t, int fixed0, int fixed1)
 {
     static_assert(D == 2 || D == 4, "the unrolled loop keeps the step parity");
-    static_assert(K >= 2 && K <= 4, "window depth");
+    static_assert(K >= 2 && K <= JW_MAX_DEPTH, "window depth");
     using G = jw_geo<K, NC>;
     const int lane = threadIdx.x & 31;
     const int nx = (int)src.nx;
@@ -1085,7 +1088,7 @@ __device__ __forceinline__ double jw_march(const jw_rows &src, double *nxt, int 
     double f[D][NC]; /* rows in flight */
     int r_next = ra - K;
     const int r_last = rb - 1 + K; /* last row of u(t) the band reads */
-    const double *pin = src.cur + (size_t)r_next * pitch + jbase; /* without EDGE all rows are in the source buffer */
+    const double *pin = src.cur + (size_t)r_next * pitch + jbase; /* the plain form: all rows are in the source buffer */
     /* Each request also asks L2 for the row JW_AHEAD further down.  The registers hold D rows in flight,
      * which at 128 registers per thread is all a K-level window leaves room for; the prefetch puts the
      * DRAM latency of the following rows behind them without holding anything (measured at 16384^2, four
@@ -1095,6 +1098,10 @@ __device__ __forceinline__ double jw_march(const jw_rows &src, double *nxt, int 
         if (EDGE) {
             jw_ld_edge<NC>(src.at(r_next) + jbase, v, ok);
             if ((ok & 1u) && r_next + JW_AHEAD <= r_last)
+                asm volatile("prefetch.global.L2 [%0];" ::"l"(src.at(r_next + JW_AHEAD) + jbase));
+        } else if (HALO) {
+            jw_ld<NC>(src.at(r_next) + jbase, v);
+            if (r_next + JW_AHEAD <= r_last)
                 asm volatile("prefetch.global.L2 [%0];" ::"l"(src.at(r_next + JW_AHEAD) + jbase));
         } else {
             jw_ld<NC>(pin, v);
@@ -1140,8 +1147,9 @@ __device__ __forceinline__ double jw_march(const jw_rows &src, double *nxt, int 
     if ((I) < 2 * K - 2 && s < n_steps)                                                                         \
         one(std::integral_constant<int, (I) % D>{}, std::integral_constant<int, (I)&1>{},                       \
             std::integral_constant<int, (I) < 2 * K - 2 ? (I) : -1>{});
-    JW_FILL(0) JW_FILL(1) JW_FILL(2) JW_FILL(3) JW_FILL(4) JW_FILL(5)
+    JW_FILL(0) JW_FILL(1) JW_FILL(2) JW_FILL(3) JW_FILL(4) JW_FILL(5) JW_FILL(6) JW_FILL(7) JW_FILL(8) JW_FILL(9)
 #undef JW_FILL
+    static_assert(2 * JW_MAX_DEPTH - 2 <= 10, "one JW_FILL per step of the filling window");
     /* steady state: D steps per trip, slots and parities known at compile time */
     constexpr int S0 = (2 * K - 2) % D;
     while (s < n_steps) {
@@ -1155,11 +1163,31 @@ __device__ __forceinline__ double jw_march(const jw_rows &src, double *nxt, int 
     return acc;
 }
 
+/* The other forms as functions of their own: inlined beside the plain form they share its register
+ * allocation, and at five and six levels that costs the plain form -- which does nearly all the work --
+ * up to a fifth of its speed (six sweeps per launch at 16384^2: 1040 us inlined, 850 us for the plain
+ * form alone).  Both also form the residual, which the caller drops unless the launch is the last one:
+ * a few instructions per row against two more copies of the march. */
+template <int K, int NC, bool EDGE>
+static __device__ __noinline__ double jw_march_other(const double *cur, const double *nxt_halo, const double *xh, int rows,
+                                                     int xh_side, size_t nx, double *nxt, int ra, int rb, int t, int fixed0,
+                                                     int fixed1)
+{
+    jw_rows src;
+    src.cur = cur;
+    src.nxt = nxt_halo;
+    src.xh = xh;
+    src.rows = rows;
+    src.xh_side = xh_side;
+    src.nx = nx;
+    return jw_march<K, NC, 2, EDGE, true, true>(src, nxt, ra, rb, t, fixed0, fixed1);
+}
+
 /* sender block b of a K-sweep pass: piece (b mod JACOBI_PIECES) of one of the K first or K last rows of
  * a PE's strip, into the neighbour's row of the same depth (see jw_rows for where that is) */
 static __device__ __noinline__ void jacobi_send_piece_k(const ishmem_ctx_t *ctxs, const double *cur0, double *nxt0,
-                                                        double *xh0, unsigned long long *sig0, size_t ny, size_t nx,
-                                                        unsigned b, unsigned K)
+                                                        double *xh0, unsigned xh_side, unsigned long long *sig0, size_t ny,
+                                                        size_t nx, unsigned b, unsigned K)
 {
     const int P = ctxs[0].npes;
     const unsigned per_pe = 2u * K * JACOBI_PIECES;
@@ -1178,12 +1206,12 @@ static __device__ __noinline__ void jacobi_send_piece_k(const ishmem_ctx_t *ctxs
     if (!down && p > 0) { /* my row 1 + depth -> row rows_above + 1 + depth of the PE above */
         double *into = depth == 0   ? (double *)cur + (rows_above + 1) * nx
                        : depth == 1 ? nxt + (rows_above + 1) * nx
-                                    : xh + (size_t)(depth) * nx; /* its rows+3, rows+4: slots 2, 3 */
+                                    : xh + (size_t)(xh_side + depth - 2) * nx; /* its rows+3, ...: the second half */
         ishmemx_putmem_signal_work_group(ctx, (void *)(into + c_lo), cur + (size_t)(1 + depth) * nx + c_lo,
                                          (c_hi - c_lo) * 8, sig + 1, 1, ISHMEM_SIGNAL_ADD, p - 1);
     }
     if (down && p + 1 < P) { /* my row rows - depth -> row -depth of the PE below */
-        double *into = depth == 0 ? (double *)cur : depth == 1 ? nxt : xh + (size_t)(depth - 2) * nx; /* slots 0, 1 */
+        double *into = depth == 0 ? (double *)cur : depth == 1 ? nxt : xh + (size_t)(depth - 2) * nx; /* the first half */
         ishmemx_putmem_signal_work_group(ctx, (void *)(into + c_lo), cur + (rows - depth) * nx + c_lo,
                                          (c_hi - c_lo) * 8, sig + 0, 1, ISHMEM_SIGNAL_ADD, p + 1);
     }
@@ -1192,13 +1220,13 @@ static __device__ __noinline__ void jacobi_send_piece_k(const ishmem_ctx_t *ctxs
 /* one launch = K sweeps: sender blocks (K rows each way per PE), then one block per band of `band_rows`
  * rows x (blockDim / 32) tiles, in launch order as in k_jacobi_sweep */
 #define JACOBI_PASS_THREADS 128
-/* four blocks per SM (128 registers); the four-level window with four columns per lane would spill there
- * and gets three (170 registers): 718 against 739 us per launch on a single strip */
+/* four blocks per SM (128 registers); windows of four and more levels with four columns per lane would
+ * spill there and get three (170 registers): K = 4: 718 against 739 us per launch on a single strip */
 template <int K, int NC>
-__global__ void __launch_bounds__(JACOBI_PASS_THREADS, (K == 4 && NC == 4) ? 3 : 4) k_jacobi_pass(const ishmem_ctx_t *ctxs, jacobi_args a, double *xh0,
-                                                                        int flip, unsigned long long arrived, int last,
+__global__ void __launch_bounds__(JACOBI_PASS_THREADS, (K >= 4 && NC == 4) ? 3 : 4) k_jacobi_pass(const ishmem_ctx_t *ctxs, jacobi_args a, double *xh0,
+                                                                        int xh_side, int flip, unsigned long long arrived, int last,
                                                                         unsigned band_rows, unsigned bands,
-                                                                        unsigned tile_groups, int P, size_t heap_stride)
+                                                                        unsigned tile_groups, unsigned lead_bands, int P, size_t heap_stride)
 {
     using G = jw_geo<K, NC>;
     const unsigned tid = threadIdx.x;
@@ -1206,12 +1234,32 @@ __global__ void __launch_bounds__(JACOBI_PASS_THREADS, (K == 4 && NC == 4) ? 3 :
     const unsigned nsend = (unsigned)P * 2u * K * JACOBI_PIECES;
     unsigned b = blockIdx.x;
     if (b < nsend) {
-        jacobi_send_piece_k(ctxs, flip ? a.buf1 : a.buf0, flip ? a.buf0 : a.buf1, xh0, a.sig, a.ny, nx, b, K);
+        jacobi_send_piece_k(ctxs, flip ? a.buf1 : a.buf0, flip ? a.buf0 : a.buf1, xh0, (unsigned)xh_side, a.sig, a.ny, nx, b, K);
         return;
     }
     b -= nsend;
-    const int p = (int)(b / (bands * tile_groups));
-    const unsigned band = (b / tile_groups) % bands, tg = b % tile_groups;
+    /* Blocks that hold the grid's first or last column, or its last row, take the slow form of the march
+     * (three times the instructions per row).  Started in their natural place the last of them would run
+     * on alone after everything else has finished (8192^2, six sweeps per launch: 320 us against 210 us
+     * for the plain blocks), so they come first: the first and last tile group of every band, then the
+     * last band of the last strip (`lead_bands` bands counted from the end, the empty ones included),
+     * then all the others in the order of their rows. */
+    const unsigned edge_groups = tile_groups < 2u ? tile_groups : 2u, inner_groups = tile_groups - edge_groups;
+    const unsigned n_edge = (unsigned)P * bands * edge_groups;
+    unsigned pb, tg;
+    if (b < n_edge) {
+        pb = b / edge_groups;
+        tg = (b % edge_groups) ? tile_groups - 1u : 0u;
+    } else {
+        const unsigned n_inner = (unsigned)P * bands * inner_groups, lead = lead_bands * inner_groups;
+        b -= n_edge;
+        b = b < lead ? n_inner - lead + b : b - lead;
+        pb = b / inner_groups;
+        tg = 1u + b % inner_groups;
+    }
+    const int p = (int)(pb / bands);
+    const unsigned band = pb % bands;
+    b = pb * tile_groups + tg; /* the block's number in the order of rows and tiles: its residual slot */
     const ishmem_ctx_t *ctx = ctxs + p;
     const unsigned base_rows = (unsigned)a.ny / (unsigned)P, extra = (unsigned)a.ny % (unsigned)P;
     const int rows = (int)(base_rows + ((unsigned)p < extra ? 1u : 0u));
@@ -1240,6 +1288,7 @@ __global__ void __launch_bounds__(JACOBI_PASS_THREADS, (K == 4 && NC == 4) ? 3 :
         src.nxt = nxt;
         src.xh = (const double *)((const char *)xh0 + (size_t)p * heap_stride);
         src.rows = rows;
+        src.xh_side = xh_side;
         src.nx = nx;
         const int fixed0 = (first == 0) ? 1 : -100;
         const int fixed1 = (first + (unsigned)rows == (unsigned)a.ny) ? rows : -100;
@@ -1247,17 +1296,18 @@ __global__ void __launch_bounds__(JACOBI_PASS_THREADS, (K == 4 && NC == 4) ? 3 :
         const int t = (int)(tg * (blockDim.x >> 5) + (tid >> 5));
         if (t < ntiles) {
             const int j0 = t * G::TILE - G::SKIP * NC;
-            /* the plain form: all loaded columns inside the grid and none of them its first or last one,
-             * all rows read inside the source buffer, no fixed row among the rows formed */
-            const bool plain = j0 > 0 && j0 + 32 * NC < (int)nx && ra - K >= 0 && rb - 1 + K <= rows + 1 &&
-                               !(fixed0 >= ra - K + 1 && fixed0 <= rb + K - 2) &&
-                               !(fixed1 >= ra - K + 1 && fixed1 <= rb + K - 2);
-            if (last)
-                acc = jw_march<K, NC, 2, true, true>(src, nxt, ra, rb, t, fixed0, fixed1);
-            else if (plain)
-                jw_march<K, NC, 2, false, false>(src, nxt, ra, rb, t, fixed0, fixed1);
+            /* no edge: all loaded columns inside the grid and none of them its first or last one, no fixed
+             * row among the rows formed; the plain form also reads all its rows from the source buffer and
+             * forms no residual */
+            const bool no_edge = j0 > 0 && j0 + 32 * NC < (int)nx && !(fixed0 >= ra - K + 1 && fixed0 <= rb + K - 2) &&
+                                 !(fixed1 >= ra - K + 1 && fixed1 <= rb + K - 2);
+            const bool rows_inside = ra - K >= 0 && rb - 1 + K <= rows + 1;
+            if (no_edge && rows_inside && !last)
+                jw_march<K, NC, 2, false, false, false>(src, nxt, ra, rb, t, fixed0, fixed1);
+            else if (no_edge)
+                acc = jw_march_other<K, NC, false>(src.cur, src.nxt, src.xh, rows, xh_side, nx, nxt, ra, rb, t, fixed0, fixed1);
             else
-                jw_march<K, NC, 2, true, false>(src, nxt, ra, rb, t, fixed0, fixed1);
+                acc = jw_march_other<K, NC, true>(src.cur, src.nxt, src.xh, rows, xh_side, nx, nxt, ra, rb, t, fixed0, fixed1);
         }
     }
     if (last) {
@@ -1363,27 +1413,31 @@ static int jacobi_launch(double *buf0, double *buf1, uint64_t *sig, size_t ny, s
 
 /* one launch per sweep (k_jacobi_sweep): bands of 16 rows x 8 tiles of 60 columns per block */
 #define JACOBI_BAND_ROWS 16u /* measured at 16384^2: 8 rows 687 us, 12: 663, 16: 652, 20: 652, 24: 659, 32: 666, 64: 680 */
-/* K sweeps per launch (k_jacobi_pass): a band pays 2K extra rows, so it is taller; 64 and 128 rows
- * measure the same at 16384^2 and 64 gives small grids more blocks */
-#define JACOBI_PASS_BAND_ROWS 64u
+/* K sweeps per launch (k_jacobi_pass): a band pays 2K extra rows, so it is taller.  Up to four sweeps 64
+ * and 128 rows measure the same at 16384^2 and 64 gives small grids more blocks; five and six sweeps
+ * per launch are 5 % faster with 128 */
+static unsigned jacobi_pass_band_rows(int k) { return k >= 5 ? 128u : 64u; }
 
 /* The launches of one call.  Every launch moves the grid from one buffer to the other, and the result
  * has to end where `iters` single sweeps would leave it (buf0 for an even count), so the number of
  * launches has the parity of iters.  Within that the split is the cheapest one by the measured time of
- * a launch of 1, 2, 3 and 4 sweeps at 16384^2 (650, 690, 740 and 800 us: a launch costs about the same
- * whatever its depth, so deep launches win and a single sweep is the cheapest filler). */
+ * a launch of 1 .. 6 sweeps at 16384^2 (JACOBI_LAUNCH_US: a launch costs little more the deeper it is,
+ * so deep launches win and a single sweep is the cheapest filler). */
+static const double JACOBI_LAUNCH_US[JW_MAX_DEPTH + 1] = {0, 650, 690, 740, 800, 860, 960};
+
 struct jacobi_plan {
-    std::vector<int> depth; /* sweeps of each launch, deepest first */
-    int nc[5];              /* columns per lane of a launch of depth k */
-    unsigned bands1, groups1, bands_k;
-    unsigned groups_k[5];   /* tile groups per band of a launch of depth k */
-    size_t blocks_last;     /* tile blocks (= residual terms) of the last launch */
-    bool needs_xh;          /* some launch is deeper than two sweeps */
+    std::vector<int> depth;            /* sweeps of each launch, deepest first */
+    int nc[JW_MAX_DEPTH + 1];          /* columns per lane of a launch of depth k */
+    unsigned bands1, groups1;
+    unsigned bands_k[JW_MAX_DEPTH + 1];  /* bands per strip of a launch of depth k */
+    unsigned groups_k[JW_MAX_DEPTH + 1]; /* tile groups per band of a launch of depth k */
+    size_t blocks_last;                /* tile blocks (= residual terms) of the last launch */
+    int xh_side;                       /* extra halo rows per side: the deepest launch's depth - 2 */
 };
 
 static void jacobi_split(int iters, int kmax, std::vector<int> *out)
 {
-    static const double cost[5] = {0, 650, 690, 740, 800};
+    const double *cost = JACOBI_LAUNCH_US;
     out->clear();
     int full = 0, r = iters;
     while (r > 24) { /* far from the end only the deepest launch is ever right */
@@ -1424,7 +1478,7 @@ static void jacobi_split(int iters, int kmax, std::vector<int> *out)
  * the host logic: needs no device and no initialised library. */
 extern "C" int ishmemx_jacobi_launch_depths(int iters, int max_depth, int *depths_out, int capacity)
 {
-    if (iters < 0 || max_depth < 1 || max_depth > 4 || capacity < 0 || (capacity && !depths_out)) return ISHMEM_ERR_ARG;
+    if (iters < 0 || max_depth < 1 || max_depth > JW_MAX_DEPTH || capacity < 0 || (capacity && !depths_out)) return ISHMEM_ERR_ARG;
     std::vector<int> d;
     jacobi_split(iters, max_depth, &d);
     for (size_t i = 0; i < d.size() && i < (size_t)capacity; ++i) depths_out[i] = d[i];
@@ -1438,13 +1492,13 @@ static unsigned jacobi_pass_groups(size_t nx, int k, int nc)
     return (ntiles + warps - 1) / warps;
 }
 
-/* kmax: the deepest launch allowed (the caller lowers it to 2 when the symmetric heap has no room for
- * the extra halo rows) */
+/* kmax: the deepest launch allowed (the caller lowers it when the symmetric heap has no room for the
+ * extra halo rows) */
 static void jacobi_make_plan(size_t ny, size_t nx, int iters, int kmax, jacobi_plan *pl)
 {
     auto &g = g_ishmem;
     const size_t rows_min = ny / (size_t)g.npes, rows_max = (ny + g.npes - 1) / g.npes;
-    /* ISHMEMX_OPT_JACOBI_FUSE: 0 = single sweeps only, 1 = the library's choice, 2..4 = at most that deep */
+    /* ISHMEMX_OPT_JACOBI_FUSE: 0 = single sweeps only, 1 = the library's choice, 2..6 = at most that deep */
     const long long fuse = g.opt[ISHMEMX_OPT_JACOBI_FUSE];
     if (fuse == 0) kmax = 1;
     else if (fuse >= 2 && fuse < kmax) kmax = (int)fuse;
@@ -1453,55 +1507,60 @@ static void jacobi_make_plan(size_t ny, size_t nx, int iters, int kmax, jacobi_p
     jacobi_split(iters, kmax, &pl->depth);
     pl->bands1 = (unsigned)((rows_max + JACOBI_BAND_ROWS - 1) / JACOBI_BAND_ROWS);
     pl->groups1 = (unsigned)(((nx + 59) / 60 + 7) / 8);
-    pl->bands_k = (unsigned)((rows_max + JACOBI_PASS_BAND_ROWS - 1) / JACOBI_PASS_BAND_ROWS);
+    for (int k = 2; k <= JW_MAX_DEPTH; ++k)
+        pl->bands_k[k] = (unsigned)((rows_max + jacobi_pass_band_rows(k) - 1) / jacobi_pass_band_rows(k));
     /* Columns per lane: four (32-byte accesses: nx a multiple of 4) unless the grid is too small to give
      * every SM its blocks that way.  At 16384^2, per sweep, four against two columns per lane: 345 / 395 us
-     * with two sweeps per launch, 247 / 295 with three, 200 / 230 with four (whose four-column window
-     * spills a few values at 128 registers and still wins).  ISHMEMX_OPT_JACOBI_WIDE = 0 / 1 forces two /
-     * four. */
+     * with two sweeps per launch, 247 / 295 with three, 200 / 230 with four.  ISHMEMX_OPT_JACOBI_WIDE =
+     * 0 / 1 forces two / four. */
     const long long wide = g.opt[ISHMEMX_OPT_JACOBI_WIDE];
-    for (int k = 2; k <= 4; ++k) {
+    for (int k = 2; k <= JW_MAX_DEPTH; ++k) {
         pl->nc[k] = 4;
         if (nx % 4 != 0 || wide == 0) pl->nc[k] = 2;
-        else if (wide < 0 && (size_t)g.npes * pl->bands_k * jacobi_pass_groups(nx, k, 4) < (size_t)g.sm_count * 8) pl->nc[k] = 2;
+        else if (wide < 0 && (size_t)g.npes * pl->bands_k[k] * jacobi_pass_groups(nx, k, 4) < (size_t)g.sm_count * 8) pl->nc[k] = 2;
     }
-    pl->needs_xh = false;
-    for (int k = 2; k <= 4; ++k) pl->groups_k[k] = jacobi_pass_groups(nx, k, pl->nc[k]);
-    for (int k : pl->depth) pl->needs_xh |= k > 2;
+    pl->xh_side = 0;
+    for (int k = 2; k <= JW_MAX_DEPTH; ++k) pl->groups_k[k] = jacobi_pass_groups(nx, k, pl->nc[k]);
+    for (int k : pl->depth) pl->xh_side = std::max(pl->xh_side, k - 2);
     const int k_last = pl->depth.empty() ? 1 : pl->depth.back();
     pl->blocks_last = k_last == 1 ? (size_t)g.npes * pl->bands1 * pl->groups1
-                                  : (size_t)g.npes * pl->bands_k * pl->groups_k[k_last];
+                                  : (size_t)g.npes * pl->bands_k[k_last] * pl->groups_k[k_last];
     if (pl->depth.empty()) pl->blocks_last = 0;
 }
 
 template <int NC>
-static void jacobi_launch_pass(int k, unsigned nblocks, cudaStream_t s, const jacobi_args &a, double *xh, int flip,
-                               unsigned long long arrived, int last, unsigned bands, unsigned groups)
+static void jacobi_launch_pass(int k, unsigned nblocks, cudaStream_t s, const jacobi_args &a, double *xh, int xh_side,
+                               int flip, unsigned long long arrived, int last, unsigned bands, unsigned groups)
 {
     auto &g = g_ishmem;
+    const unsigned band_rows = jacobi_pass_band_rows(k);
+    /* the bands from the last strip's last band with rows on (see the kernel) */
+    const unsigned rows_last = (unsigned)(a.ny / (size_t)g.npes);
+    const unsigned lead_bands = bands - (rows_last - 1) / band_rows;
+#define JACOBI_PASS_CASE(K)                                                                                          \
+    case K:                                                                                                          \
+        k_jacobi_pass<K, NC><<<nblocks, JACOBI_PASS_THREADS, 0, s>>>(g.d_ctx, a, xh, xh_side, flip, arrived, last,   \
+                                                                    band_rows, bands, groups, lead_bands, g.npes, g.heap_bytes); \
+        break;
     switch (k) {
-    case 2:
-        k_jacobi_pass<2, NC><<<nblocks, JACOBI_PASS_THREADS, 0, s>>>(g.d_ctx, a, xh, flip, arrived, last, JACOBI_PASS_BAND_ROWS,
-                                                                    bands, groups, g.npes, g.heap_bytes);
-        break;
-    case 3:
-        k_jacobi_pass<3, NC><<<nblocks, JACOBI_PASS_THREADS, 0, s>>>(g.d_ctx, a, xh, flip, arrived, last, JACOBI_PASS_BAND_ROWS,
-                                                                    bands, groups, g.npes, g.heap_bytes);
-        break;
-    default:
-        k_jacobi_pass<4, NC><<<nblocks, JACOBI_PASS_THREADS, 0, s>>>(g.d_ctx, a, xh, flip, arrived, last, JACOBI_PASS_BAND_ROWS,
-                                                                    bands, groups, g.npes, g.heap_bytes);
-        break;
+        JACOBI_PASS_CASE(2)
+        JACOBI_PASS_CASE(3)
+        JACOBI_PASS_CASE(4)
+        JACOBI_PASS_CASE(5)
+        JACOBI_PASS_CASE(6)
     }
+#undef JACOBI_PASS_CASE
+    static_assert(JW_MAX_DEPTH == 6, "one case per depth");
 }
 
-/* partial: room for pl.blocks_last residual terms; xh: four symmetric rows (PE 0's copy) when pl.needs_xh */
+/* partial: room for pl.blocks_last residual terms, or NULL when no residual is wanted (the last launch
+ * then runs like the others); xh: 2 x pl.xh_side symmetric rows (PE 0's copy) */
 static int jacobi_launch_sweeps(double *buf0, double *buf1, uint64_t *sig, size_t ny, size_t nx, int iters, int overlap,
                                 const jacobi_plan &pl, double *partial, double *xh)
 {
     auto &g = g_ishmem;
-    for (int k = 1; k <= 4; ++k) {
-        const size_t tiles = k == 1 ? (size_t)g.npes * pl.bands1 * pl.groups1 : (size_t)g.npes * pl.bands_k * pl.groups_k[k];
+    for (int k = 1; k <= JW_MAX_DEPTH; ++k) {
+        const size_t tiles = k == 1 ? (size_t)g.npes * pl.bands1 * pl.groups1 : (size_t)g.npes * pl.bands_k[k] * pl.groups_k[k];
         if (tiles + (size_t)g.npes * 2 * k * JACOBI_PIECES > 0x7fffffffu) return ISHMEM_ERR_ARG;
     }
     cudaStream_t s;
@@ -1520,16 +1579,16 @@ static int jacobi_launch_sweeps(double *buf0, double *buf1, uint64_t *sig, size_
     int flip = 0;
     unsigned long long arrived = 0; /* pieces the halo words count once the launch's senders are through */
     for (size_t i = 0; i < pl.depth.size() && !rc; ++i) {
-        const int k = pl.depth[i], last = i + 1 == pl.depth.size();
+        const int k = pl.depth[i], last = partial && i + 1 == pl.depth.size();
         arrived += (unsigned long long)k * JACOBI_PIECES;
         const unsigned nsend = (unsigned)g.npes * 2u * (unsigned)k * JACOBI_PIECES;
         if (k == 1) {
             k_jacobi_sweep<<<nsend + (unsigned)g.npes * pl.bands1 * pl.groups1, 256, 0, s>>>(
                 g.d_ctx, a, flip, arrived, last, JACOBI_BAND_ROWS, pl.bands1, pl.groups1, g.npes, g.heap_bytes);
         } else {
-            const unsigned nblocks = nsend + (unsigned)g.npes * pl.bands_k * pl.groups_k[k];
-            if (pl.nc[k] == 4) jacobi_launch_pass<4>(k, nblocks, s, a, xh, flip, arrived, last, pl.bands_k, pl.groups_k[k]);
-            else jacobi_launch_pass<2>(k, nblocks, s, a, xh, flip, arrived, last, pl.bands_k, pl.groups_k[k]);
+            const unsigned nblocks = nsend + (unsigned)g.npes * pl.bands_k[k] * pl.groups_k[k];
+            if (pl.nc[k] == 4) jacobi_launch_pass<4>(k, nblocks, s, a, xh, pl.xh_side, flip, arrived, last, pl.bands_k[k], pl.groups_k[k]);
+            else jacobi_launch_pass<2>(k, nblocks, s, a, xh, pl.xh_side, flip, arrived, last, pl.bands_k[k], pl.groups_k[k]);
         }
         flip ^= 1;
         ishmemi_count_launch();
@@ -1557,16 +1616,18 @@ extern "C" int ishmemx_jacobi(double *buf0, double *buf1, uint64_t *sig, size_t 
     if (rc) return rc;
     if (jacobi_per_sweep(threads, nx)) {
         jacobi_plan pl;
-        jacobi_make_plan(ny, nx, iters, 4, &pl);
-        /* launches deeper than two sweeps park their third and fourth halo rows in four extra symmetric
-         * rows; without room for them in the heap the call stays at two sweeps per launch */
+        /* a launch of k > 2 sweeps parks its third to k-th halo rows in 2 (k - 2) extra symmetric rows;
+         * without room for them in the heap the call falls back to shallower launches */
         double *xh = nullptr;
-        if (pl.needs_xh) {
-            xh = (double *)ishmem_malloc(4 * nx * sizeof(double));
-            if (!xh) jacobi_make_plan(ny, nx, iters, 2, &pl);
+        for (int kmax : {JW_MAX_DEPTH, 4, 2}) {
+            jacobi_make_plan(ny, nx, iters, kmax, &pl);
+            if (pl.xh_side == 0) break;
+            xh = (double *)ishmem_malloc(2 * (size_t)pl.xh_side * nx * sizeof(double));
+            if (xh) break;
         }
         double *partial = nullptr;
-        rc = ishmemi_cuda(cudaMalloc((void **)&partial, (pl.blocks_last ? pl.blocks_last : 1) * 8), "cudaMalloc");
+        if (residual_sq_host)
+            rc = ishmemi_cuda(cudaMalloc((void **)&partial, (pl.blocks_last ? pl.blocks_last : 1) * 8), "cudaMalloc");
         if (!rc) rc = jacobi_launch_sweeps(buf0, buf1, sig, ny, nx, iters, overlap, pl, partial, xh);
         if (!rc && residual_sq_host) {
             double sum = 0.0;

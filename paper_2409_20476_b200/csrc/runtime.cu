@@ -251,7 +251,7 @@ static int init_common(int npes, size_t heap_bytes, void *external)
     }
     if (const char *v = getenv("ISHMEM_JACOBI_FUSE")) {
         const int f = atoi(v);
-        if (f >= 0 && f <= 4) g.opt[ISHMEMX_OPT_JACOBI_FUSE] = f;
+        if (f >= 0 && f <= 6) g.opt[ISHMEMX_OPT_JACOBI_FUSE] = f;
     }
     if (const char *v = getenv("ISHMEM_JACOBI_WIDE")) g.opt[ISHMEMX_OPT_JACOBI_WIDE] = atoi(v) != 0;
     if (const char *v = getenv("ISHMEM_REDUCE_BULK")) g.opt[ISHMEMX_OPT_REDUCE_BULK] = atoi(v) != 0;
@@ -637,7 +637,7 @@ extern "C" int ishmemx_set_option(int option, long long value)
         if (value < 0 || value > 2) return ISHMEM_ERR_ARG;
         break;
     case ISHMEMX_OPT_JACOBI_FUSE:
-        if (value < 0 || value > 4) return ISHMEM_ERR_ARG;
+        if (value < 0 || value > 6) return ISHMEM_ERR_ARG;
         break;
     case ISHMEMX_OPT_REDUCE_BULK:
         if (value < 0 || value > 1) return ISHMEM_ERR_ARG;

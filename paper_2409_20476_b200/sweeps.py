@@ -501,7 +501,7 @@ def sweep_c5(args, out):
     npes, n, iters = 12, (16384 if not args.quick else 4096), 200
     rows_max = -(-n // npes)
     nbytes = (rows_max + 2) * n * 8
-    heap_bytes = 2 * nbytes + MiB
+    heap_bytes = 2 * nbytes + 2 * MiB     # the buffers, the signals and the call's own halo rows
     heap, stream = _session(torch, B, npes, heap_bytes)
     b0, b1, sig = B.ishmem_malloc(nbytes), B.ishmem_malloc(nbytes), B.ishmem_calloc(4, 8)
     base, extra = divmod(n, npes)

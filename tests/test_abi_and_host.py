@@ -185,7 +185,7 @@ def test_jacobi_launch_split_host_logic():
     end where single sweeps leave it).  Long calls are all deepest launches but for a short tail."""
     import numpy as np
     from paper_2409_20476_b200 import binding as B
-    for cap in (1, 2, 3, 4):
+    for cap in (1, 2, 3, 4, 5, 6):
         for iters in list(range(0, 60)) + [199, 200, 201, 1000, 1001]:
             out = np.zeros(iters + 1, dtype=np.int32)
             n = B.ishmemx_jacobi_launch_depths(iters, cap, out, len(out))
@@ -200,5 +200,7 @@ def test_jacobi_launch_split_host_logic():
     assert B.ishmemx_jacobi_launch_depths(8, 4, out, 64) == 2 and out[:2].tolist() == [4, 4]
     assert B.ishmemx_jacobi_launch_depths(5, 4, out, 64) == 3 and out[:3].tolist() == [2, 2, 1]
     assert B.ishmemx_jacobi_launch_depths(7, 4, None, 0) == 3          # count only
-    for bad in ((-1, 4), (5, 0), (5, 5)):
+    assert B.ishmemx_jacobi_launch_depths(200, 6, out, 64) == 34 and out[:34].tolist().count(6) >= 30
+    assert B.ishmemx_jacobi_launch_depths(12, 6, out, 64) == 2 and out[:2].tolist() == [6, 6]
+    for bad in ((-1, 4), (5, 0), (5, 7)):
         assert B.ishmemx_jacobi_launch_depths(bad[0], bad[1], out, 64) == B.ISHMEM_ERR_ARG

@@ -258,7 +258,7 @@ def test_config5_jacobi_16384_whole_grid_even_and_odd_sweep_counts():
     u8, r8 = orc.jacobi(grid, 8)
     u9, r9 = orc.jacobi(u8, 1)
     rows_max = -(-n // npes)
-    with Session(npes, 2 * (rows_max + 2) * n * 8 + MiB, with_oracle=False) as s:
+    with Session(npes, 2 * (rows_max + 2) * n * 8 + 2 * MiB, with_oracle=False) as s:
         st = Strips(s, npes, n, n)
         for iters, exp, exp_res in ((8, u8, r8), (9, u9, r9)):
             st.load(grid)
@@ -274,7 +274,7 @@ def test_config5_jacobi_full_width_200_sweeps_whole_grid_and_residual():
     npes, ny, nx, iters = 12, 768, 16384, 200
     grid = config5_grid(ny, nx)
     exp, exp_res = orc.jacobi(grid, iters)
-    with Session(npes, 2 * (ny // npes + 2) * nx * 8 + MiB, with_oracle=False) as s:
+    with Session(npes, 2 * (ny // npes + 2) * nx * 8 + 2 * MiB, with_oracle=False) as s:
         B.ishmemx_set_option(B.ISHMEMX_OPT_JACOBI_WIDE, 1)
         st = Strips(s, npes, ny, nx)
         st.load(grid)
@@ -294,7 +294,7 @@ def test_config5_jacobi_16384_200_iterations_sampled_cells():
     npes, n, iters = 12, 16384, 200
     grid = config5_grid(n, n)
     rows_max = -(-n // npes)
-    with Session(npes, 2 * (rows_max + 2) * n * 8 + MiB, with_oracle=False) as s:
+    with Session(npes, 2 * (rows_max + 2) * n * 8 + 2 * MiB, with_oracle=False) as s:
         st = Strips(s, npes, n, n)
         firsts = st.firsts
         st.load(grid)

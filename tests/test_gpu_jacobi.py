@@ -12,9 +12,9 @@ from tests.gpu_util import Session
 pytestmark = pytest.mark.gpu
 
 
-def run_gpu(grid, npes, iters, overlap, groups, threads, options=(), spare_rows=4):
-    """spare_rows: rows of symmetric heap left free beside the two buffers -- launches of three and
-    four sweeps park their deeper halo rows in four rows that the library allocates for the call"""
+def run_gpu(grid, npes, iters, overlap, groups, threads, options=(), spare_rows=8):
+    """spare_rows: rows of symmetric heap left free beside the two buffers -- launches of three to six
+    sweeps park their deeper halo rows in up to eight rows that the library allocates for the call"""
     ny, nx = grid.shape
     rows_max = -(-ny // npes)
     nbytes = (rows_max + 2) * nx * 8
@@ -44,9 +44,10 @@ def run_gpu(grid, npes, iters, overlap, groups, threads, options=(), spare_rows=
         return out, res[0]
 
 
-SWEEP_FORMS = {   # (sweeps per launch at most: 1 = the library's choice, up to four; four columns per lane)
+SWEEP_FORMS = {   # (sweeps per launch at most: 1 = the library's choice, up to six; four columns per lane)
     "sweeps": (1, 1), "sweeps_two_columns_per_lane": (1, 0), "two_per_launch": (2, 1),
-    "three_per_launch_two_columns_per_lane": (3, 0), "single_sweeps": (0, 1)}
+    "three_per_launch_two_columns_per_lane": (3, 0), "four_per_launch": (4, 1),
+    "five_per_launch_two_columns_per_lane": (5, 0), "five_per_launch": (5, 1), "single_sweeps": (0, 1)}
 
 
 @pytest.mark.parametrize("split", list(SWEEP_FORMS) + ["columns", "rows"])
@@ -60,8 +61,8 @@ SWEEP_FORMS = {   # (sweeps per launch at most: 1 = the library's choice, up to 
 def test_jacobi_matches_oracle(ny, nx, npes, groups, threads, overlap, split):
     """split: the persistent kernel with the strips cut by columns or by rows, or one of the launch-ordered
     forms that the library uses for threads = 0 and even nx: `sweeps` = its own choice (one tile per warp, up
-    to four sweeps per launch, four columns per lane where nx is a multiple of 4), the same with two columns
-    per lane, with at most two or three sweeps per launch, or with one sweep per launch.  The 21 sweeps are
+    to six sweeps per launch, four columns per lane where nx is a multiple of 4), the same with two columns
+    per lane, with at most two to five sweeps per launch, or with one sweep per launch.  The 21 sweeps are
     cut into launches by ishmemx_jacobi_launch_depths (an odd number of them, deepest first)."""
     if split in SWEEP_FORMS:
         options = [(B.ISHMEMX_OPT_JACOBI_SPLIT, 0), (B.ISHMEMX_OPT_JACOBI_FUSE, SWEEP_FORMS[split][0]),
@@ -89,12 +90,13 @@ def test_jacobi_default_split_and_repeated_calls():
 
 def test_jacobi_per_sweep_many_bands_and_residual():
     """The launch-ordered form on strips of several bands and tile groups, with strips of unequal length and
-    iteration counts whose last launch -- the one that forms the residual -- is one of 1, 3 or 4 sweeps, with
-    and without room in the heap for the deeper halo rows (without it launches stay at two sweeps); final
-    grid bit-exact, residual within 1e-6 relative."""
+    iteration counts whose last launch -- the one that forms the residual -- is one of 1 to 6 sweeps, with
+    room in the heap for all the deeper halo rows (8), for those of four sweeps per launch (4) and for none
+    (launches then stay at two sweeps); final grid bit-exact, residual within 1e-6 relative."""
     grid = inputs.jacobi_grid(inputs.SEED_C5, 1000, 1100)
-    for npes, iters, spare in ((7, 5, 4), (3, 12, 4), (1, 3, 4), (5, 8, 4), (12, 4, 4), (2, 10, 4), (6, 6, 4),
-                               (7, 8, 0), (3, 5, 0), (4, 22, 4), (4, 16, 0)):
+    for npes, iters, spare in ((7, 5, 8), (3, 12, 8), (1, 3, 8), (5, 8, 8), (12, 4, 8), (2, 10, 8), (6, 6, 8),
+                               (7, 8, 0), (3, 5, 0), (4, 22, 8), (4, 16, 0), (4, 22, 4), (3, 12, 4), (5, 18, 8),
+                               (2, 11, 8), (1, 6, 8), (3, 24, 5)):
         exp, exp_res = orc.jacobi(grid, iters)
         got, res = run_gpu(grid, npes, iters, 1, 1, 0, spare_rows=spare)
         assert got.tobytes() == exp.tobytes(), (npes, iters, spare)
@@ -102,12 +104,13 @@ def test_jacobi_per_sweep_many_bands_and_residual():
 
 
 def test_jacobi_multi_sweep_launches_on_the_shortest_strips():
-    """Strips of one to five rows: a launch is at most as deep as the shortest strip has rows (it sends that many
+    """Strips of one to seven rows: a launch is at most as deep as the shortest strip has rows (it sends that many
     of its rows each way), the deeper halo rows of a neighbour are its rows next to the edge row, and a strip's
     single band is both its first and its last."""
-    for ny, nx, npes in ((24, 120, 12), (31, 232, 10), (8, 64, 4), (12, 128, 12), (48, 240, 12), (50, 484, 10)):
+    for ny, nx, npes in ((24, 120, 12), (31, 232, 10), (8, 64, 4), (12, 128, 12), (48, 240, 12), (50, 484, 10),
+                         (72, 120, 12), (26, 232, 4), (6, 64, 1)):
         grid = inputs.jacobi_grid(inputs.SEED_C5, ny, nx)
-        for iters in (4, 8, 9):
+        for iters in (4, 8, 9, 12):
             exp, exp_res = orc.jacobi(grid, iters)
             got, res = run_gpu(grid, npes, iters, 1, 1, 0)
             assert got.tobytes() == exp.tobytes(), (ny, nx, npes, iters)
