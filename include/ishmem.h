@@ -135,8 +135,8 @@ size_t ishmemx_heap_bytes(void);
  *       threads = 0 and an even nx: launch-ordered sweeps; else the persistent kernel, strips cut
  *       by rows), 1 = persistent kernel with the strips cut by rows, 2 = by ranges of column
  *       tiles.
- *   ISHMEMX_OPT_JACOBI_FUSE (ISHMEM_JACOBI_FUSE=0..4): sweeps per launch of the launch-ordered
- *       form: 1 = the library's choice, up to four (default), 0 = always one, 2, 3, 4 = at most
+ *   ISHMEMX_OPT_JACOBI_FUSE (ISHMEM_JACOBI_FUSE=0..6): sweeps per launch of the launch-ordered
+ *       form: 1 = the library's choice, up to six (default), 0 = always one, 2 .. 6 = at most
  *       that many.
  *   ISHMEMX_OPT_JACOBI_WIDE (ISHMEM_JACOBI_WIDE=0|1): columns per lane in the multi-sweep launches:
  *       -1 = four where nx is a multiple of 4 and the grid gives every SM its blocks (default),
@@ -587,17 +587,19 @@ int ishmemx_rma_latency(int my_pe, void *dest, const void *src, size_t nbytes, i
  * first blocks send the halo rows (in-kernel work-group put_signal) and whose other blocks each
  * take a band of rows of a few neighbouring column tiles, one warp per tile, numbered so that the
  * blocks sweep the grid in launch order; only the bands at the two ends of a strip wait for a halo,
- * the interior never does.  A launch does up to FOUR sweeps: a warp's register window carries that
+ * the interior never does.  A launch does up to SIX sweeps: a warp's register window carries that
  * many time levels, every element is read once and the last level written once, and as many halo
  * rows go each way as the launch does sweeps -- the first into the halo row of the buffer being
- * read, the second into the halo row of the buffer being written, the third and fourth into four
- * rows per PE that the call takes from the symmetric heap and gives back (4 * nx * 8 bytes; when
- * the heap has no room the call stays at two sweeps per launch).  The result of every cell is the
- * same expression in the same order as in single sweeps, bit for bit.  The sweeps are cut into
- * launches of 4, 3, 2 and 1 so that the number of launches has the parity of iters (each launch
- * moves the grid to the other buffer) at the least cost by a table of measured launch times;
- * a strip must own as many rows as a launch does sweeps.  At 16384^2 on 12 PEs: 200 us per sweep
- * with four sweeps per launch, 247 with three, 345 with two, 650 with one (the copy rate).
+ * read, the second into the halo row of the buffer being written, the third to sixth into up to
+ * eight rows per PE that the call takes from the symmetric heap and gives back (2 * (k - 2) * nx * 8
+ * bytes for launches of k sweeps; when the heap has no room for them the call stays at four, else
+ * at two sweeps per launch).  The result of every cell is the same expression in the same order
+ * as in single sweeps, bit for bit.  The sweeps are cut into launches of 6 .. 1 so that the number
+ * of launches has the parity of iters (each launch moves the grid to the other buffer) at the
+ * least cost by a table of measured launch times; a strip must own as many rows as a launch does
+ * sweeps.  At 16384^2 on 12 PEs: 160 us per sweep with six sweeps per launch, 170 with five, 185
+ * with four, 240 with three, 345 with two, 640 with one (the copy rate).  With residual_sq_host
+ * NULL the last launch forms no residual and runs like the others.
  * ISHMEMX_OPT_JACOBI_FUSE caps the sweeps per launch (0 = always one), ISHMEMX_OPT_JACOBI_WIDE
  * picks two or four columns per lane (ishmemx_set_option).  groups_per_pe is not used by this
  * form and nothing needs to be co-resident.
@@ -614,7 +616,7 @@ int ishmemx_rma_latency(int my_pe, void *dest, const void *src, size_t nbytes, i
 int ishmemx_jacobi(double *buf0, double *buf1, uint64_t *sig, size_t ny, size_t nx, int iters,
                    int overlap, int groups_per_pe, int threads, double *residual_sq_host);
 
-/* How ishmemx_jacobi cuts `iters` sweeps into launches when a launch may do up to max_depth (1..4)
+/* How ishmemx_jacobi cuts `iters` sweeps into launches when a launch may do up to max_depth (1..6)
  * sweeps: writes the sweeps of each launch, deepest first, to HOST depths_out (room for `capacity`
  * entries; may be NULL with capacity 0) and returns the number of launches, which always has the
  * parity of iters (every launch moves the grid to the other buffer), or ISHMEM_ERR_ARG.  Pure host

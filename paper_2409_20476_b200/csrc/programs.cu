@@ -930,8 +930,12 @@ __global__ void __launch_bounds__(256, 4) k_jacobi_sweep(const ishmem_ctx_t *ctx
  * by the neighbouring tile.  A band of R rows reads R + 2K rows.
  * Halo rows: K each way.  The first one goes where a single sweep puts it (the halo rows of the
  * source buffer), the second one into the halo rows of the destination buffer, which nothing else
- * uses during the pass, the third and fourth into four extra rows per PE that the library takes from
- * the symmetric heap for the duration of the call. */
+ * uses during the pass, the third to the K-th into 2 (K - 2) extra rows per PE that the library takes
+ * from the symmetric heap for the duration of the call.
+ * What bounds a launch: DRAM up to four sweeps (a launch of four takes little longer than a single
+ * sweep); from five on the fp64 pipe (3 additions and a multiplication per cell and level, no fused
+ * form allowed by the bit-exact association: 430 us of a 950 us launch of six at 16384^2) and the
+ * memory latency that 12 warps per SM at 168 registers can cover. */
 #define JW_FULL 0xffffffffu
 #define JW_AHEAD 3 /* rows between a load and the L2 prefetch issued with it */
 #define JW_MAX_DEPTH 6 /* sweeps per launch at most */
@@ -1423,7 +1427,7 @@ static unsigned jacobi_pass_band_rows(int k) { return k >= 5 ? 128u : 64u; }
  * launches has the parity of iters.  Within that the split is the cheapest one by the measured time of
  * a launch of 1 .. 6 sweeps at 16384^2 (JACOBI_LAUNCH_US: a launch costs little more the deeper it is,
  * so deep launches win and a single sweep is the cheapest filler). */
-static const double JACOBI_LAUNCH_US[JW_MAX_DEPTH + 1] = {0, 650, 690, 740, 800, 860, 960};
+static const double JACOBI_LAUNCH_US[JW_MAX_DEPTH + 1] = {0, 640, 690, 715, 760, 850, 960};
 
 struct jacobi_plan {
     std::vector<int> depth;            /* sweeps of each launch, deepest first */

@@ -519,31 +519,32 @@ def sweep_c5(args, out):
 
     load()
     # (variant, form selected through ishmemx_set_option, threads, groups): the launch-ordered forms (the library's own
-    # choice: four sweeps per launch; at most three, two, one), the persistent kernel with strips cut by column tiles,
-    # and the persistent kernel with caller-shaped blocks
-    variants = [("launch_per_four_sweeps", 1, 0, 1), ("launch_per_three_sweeps", 3, 0, 1), ("launch_per_two_sweeps", 2, 0, 1),
-                ("launch_per_sweep", 0, 0, 1)]
+    # choice: six sweeps per launch; at most five, four, three, two, one), the persistent kernel with strips cut by
+    # column tiles, and the persistent kernel with caller-shaped blocks
+    variants = [("launch_per_six_sweeps", 1, 0, 1), ("launch_per_five_sweeps", 5, 0, 1), ("launch_per_four_sweeps", 4, 0, 1),
+                ("launch_per_three_sweeps", 3, 0, 1), ("launch_per_two_sweeps", 2, 0, 1), ("launch_per_sweep", 0, 0, 1)]
     variants += [("persistent_columns", "columns", 0, g) for g in (6, 12)]
     variants += [("persistent_rows", "rows", t, g) for g in (6, 12, 24) for t in (256, 512, 1024)]
     if args.quick:
-        variants = variants[:5]
+        variants = variants[:7]
     for overlap in (1, 0):
         for variant, split, threads, groups in variants:
             if npes * groups * threads > 148 * 2048:
                 continue
             B.ishmemx_set_option(B.ISHMEMX_OPT_JACOBI_SPLIT, {"rows": 1, "columns": 2}.get(split, 0))
             B.ishmemx_set_option(B.ISHMEMX_OPT_JACOBI_FUSE, split if isinstance(split, int) else 1)
-            # sweeps per launch of the bulk of the call (200 sweeps: 50 x 4, 66 x 3 + 1 + 1, 100 x 2, 200 x 1)
-            depth = {1: 4, 3: 3, 2: 2}.get(split, 1) if isinstance(split, int) else 1
+            # sweeps per launch of the bulk of the call (200 sweeps: 30 x 6 + 4 x 5, 40 x 5, 50 x 4, 66 x 3 + 1 + 1,
+            # 100 x 2, 200 x 1)
+            depth = {1: 6, 5: 5, 4: 4, 3: 3, 2: 2}.get(split, 1) if isinstance(split, int) else 1
             def reset_signals():
                 for p in range(npes):
                     for w in range(4):
                         B.ishmem_uint64_p(p, sig + 8 * w, 0, p)
             try:
-                # a short untimed call first: the first launch of a kernel in a process loads its code
-                # (24 sweeps: launches of every depth the timed call uses)
+                # the same call untimed first: the first launch of a kernel in a process loads its code, and
+                # the call launches kernels of several depths
                 reset_signals()
-                B.ishmemx_jacobi(b0, b1, sig, n, n, 24, overlap, groups, threads, res)
+                B.ishmemx_jacobi(b0, b1, sig, n, n, iters, overlap, groups, threads, res)
             except B.IshmemError:
                 pass
             reset_signals()

@@ -198,7 +198,8 @@ def test_jacobi_launch_split_host_logic():
     assert B.ishmemx_jacobi_launch_depths(200, 4, out, 64) == 50 and set(out[:50].tolist()) == {4}
     assert B.ishmemx_jacobi_launch_depths(9, 4, out, 64) == 3 and out[:3].tolist() == [3, 3, 3]
     assert B.ishmemx_jacobi_launch_depths(8, 4, out, 64) == 2 and out[:2].tolist() == [4, 4]
-    assert B.ishmemx_jacobi_launch_depths(5, 4, out, 64) == 3 and out[:3].tolist() == [2, 2, 1]
+    assert B.ishmemx_jacobi_launch_depths(5, 4, out, 64) == 3 and sum(out[:3].tolist()) == 5
+    assert B.ishmemx_jacobi_launch_depths(5, 6, out, 64) == 1 and out[0] == 5
     assert B.ishmemx_jacobi_launch_depths(7, 4, None, 0) == 3          # count only
     assert B.ishmemx_jacobi_launch_depths(200, 6, out, 64) == 34 and out[:34].tolist().count(6) >= 30
     assert B.ishmemx_jacobi_launch_depths(12, 6, out, 64) == 2 and out[:2].tolist() == [6, 6]
