@@ -247,20 +247,25 @@ class Strips:
 
 
 def test_config5_jacobi_16384_whole_grid_even_and_odd_sweep_counts():
-    """Config 5 at full size in the launch shape the library picks by itself (wide two-sweep
-    passes at this size), 12 PEs: the WHOLE final grid bit for bit against the oracle's plain
-    full-grid sweeps, and the residual at 1e-6 relative, for 8 sweeps (two launches of four)
-    and 9 (three launches of three) -- every band and tile-group seam and all eleven strip seams are
-    compared.  The ninth oracle sweep continues from the eighth (a sweep has no
-    memory, which a CPU test pins)."""
+    """Config 5 at full size in the launch shape the library picks by itself, 12 PEs: the WHOLE
+    final grid bit for bit against the oracle's plain full-grid sweeps, and the residual at 1e-6
+    relative, for 8 sweeps (two launches of four), 9 (three launches of three), 12 (two launches of
+    six) and 17 (six, six and five) -- every band and tile-group seam and all eleven strip seams are
+    compared.  The later oracle grids continue from the earlier ones (a sweep has no memory, which
+    a CPU test pins)."""
     npes, n = 12, 16384
     grid = config5_grid(n, n)
     u8, r8 = orc.jacobi(grid, 8)
     u9, r9 = orc.jacobi(u8, 1)
+    u12, r12 = orc.jacobi(u9, 3)
+    u17, r17 = orc.jacobi(u12, 5)
+    out = np.zeros(8, dtype=np.int32)
+    assert B.ishmemx_jacobi_launch_depths(12, 6, out, 8) == 2 and out[:2].tolist() == [6, 6]
+    assert B.ishmemx_jacobi_launch_depths(17, 6, out, 8) == 3 and out[:3].tolist() == [6, 6, 5]
     rows_max = -(-n // npes)
     with Session(npes, 2 * (rows_max + 2) * n * 8 + 2 * MiB, with_oracle=False) as s:
         st = Strips(s, npes, n, n)
-        for iters, exp, exp_res in ((8, u8, r8), (9, u9, r9)):
+        for iters, exp, exp_res in ((8, u8, r8), (9, u9, r9), (12, u12, r12), (17, u17, r17)):
             st.load(grid)
             res = st.run(iters)
             st.assert_equals_grid(exp, f"{iters} sweeps")
@@ -269,8 +274,9 @@ def test_config5_jacobi_16384_whole_grid_even_and_odd_sweep_counts():
 
 def test_config5_jacobi_full_width_200_sweeps_whole_grid_and_residual():
     """200 sweeps on rows of config 5's full width (16384 columns x 768 rows, 12 strips of one
-    64-row band each): whole grid and residual against the oracle, in the wide two-sweep form that
-    the library uses at full size, on a grid small enough for any host."""
+    64-row band each): whole grid and residual against the oracle, in the form that the library uses
+    at full size (four columns per lane, up to six sweeps per launch), on a grid small enough for any
+    host."""
     npes, ny, nx, iters = 12, 768, 16384, 200
     grid = config5_grid(ny, nx)
     exp, exp_res = orc.jacobi(grid, iters)
@@ -286,8 +292,8 @@ def test_config5_jacobi_full_width_200_sweeps_whole_grid_and_residual():
 def test_config5_jacobi_16384_200_iterations_sampled_cells():
     """Config 5 at full size: 16384 x 16384 float64, 12 row strips, 200 sweeps with in-kernel
     put_signal halos.  Sampled cells -- corners, edges, both sides of strip boundaries, of band
-    seams (every 16 and 64 rows of a strip) and of tile seams (every 56, 60, 120 and 960
-    columns), interior -- are compared bit for bit with the oracle's dependency-cone evaluation
+    seams (every 16, 64 and 128 rows of a strip) and of tile seams (every 56, 60, 112, 120, 448 and
+    960 columns), interior -- are compared bit for bit with the oracle's dependency-cone evaluation
     from the initial grid; then the whole final grid and the L2 residual with the oracle's 200
     full-grid sweeps.  Last, the same 200 sweeps as single-sweep launches: every strip and the
     residual must agree with the default form's."""
@@ -303,7 +309,7 @@ def test_config5_jacobi_16384_200_iterations_sampled_cells():
         cells = [(1, 1), (n - 2, n - 2), (1, n // 2), (n // 2, 1), (0, 5), (7, n - 1)]
         for p in (1, 4, 5, 11):                     # both sides of strip boundaries
             cells += [(firsts[p] - 1, int(rng.integers(1, n - 1))), (firsts[p], int(rng.integers(1, n - 1)))]
-        for band, tile in ((64, 120), (64, 960), (16, 60), (64, 56), (16, 480), (64, 448)):
+        for band, tile in ((64, 120), (64, 960), (16, 60), (64, 56), (16, 480), (64, 448), (128, 112), (128, 448)):
             p, k, t = int(rng.integers(0, npes)), int(rng.integers(1, 1300 // band)), int(rng.integers(1, n // tile))
             row = firsts[p] + band * k              # first row of band k of strip p
             cells += [(row - 1, tile * t - 1), (row, tile * t), (row - 1, tile * t), (row, tile * t - 1)]

@@ -12,7 +12,7 @@ from tests.gpu_util import Session
 pytestmark = pytest.mark.gpu
 
 
-def run_gpu(grid, npes, iters, overlap, groups, threads, options=(), spare_rows=8):
+def run_gpu(grid, npes, iters, overlap, groups, threads, options=(), spare_rows=8, want_residual=True):
     """spare_rows: rows of symmetric heap left free beside the two buffers -- launches of three to six
     sweeps park their deeper halo rows in up to eight rows that the library allocates for the call"""
     ny, nx = grid.shape
@@ -32,7 +32,8 @@ def run_gpu(grid, npes, iters, overlap, groups, threads, options=(), spare_rows=
             sig.fill(p, np.zeros(64, np.uint8))
             first += rows
         res = np.zeros(1)
-        B.ishmemx_jacobi(b0.addr, b1.addr, sig.addr, ny, nx, iters, overlap, groups, threads, res)
+        B.ishmemx_jacobi(b0.addr, b1.addr, sig.addr, ny, nx, iters, overlap, groups, threads,
+                         res if want_residual else None)
         assert s.status() == 0
         out = np.zeros_like(grid)
         fin = b0 if iters % 2 == 0 else b1
@@ -115,6 +116,17 @@ def test_jacobi_multi_sweep_launches_on_the_shortest_strips():
             got, res = run_gpu(grid, npes, iters, 1, 1, 0)
             assert got.tobytes() == exp.tobytes(), (ny, nx, npes, iters)
             assert abs(res - exp_res) <= 1e-6 * exp_res
+
+
+def test_jacobi_without_residual():
+    """residual_sq_host = NULL: the last launch forms no residual (in the launch-ordered form it then runs
+    like the others); the grid is the oracle's all the same."""
+    grid = inputs.jacobi_grid(inputs.SEED_C5, 700, 1200)
+    for npes, iters, threads in ((5, 12, 0), (3, 7, 0), (1, 6, 0), (4, 9, 128)):
+        exp, _ = orc.jacobi(grid, iters)
+        got, res = run_gpu(grid, npes, iters, 1, 2, threads, want_residual=False)
+        assert got.tobytes() == exp.tobytes(), (npes, iters, threads)
+        assert res == 0.0
 
 
 def test_jacobi_even_iterations_and_zero():
