@@ -399,12 +399,12 @@ def test_environment_variables_at_initialisation(monkeypatch):
     assert e.value.code == B.ISHMEM_ERR_ARG
 
 
-@pytest.mark.parametrize("pinned", [True, False])
-def test_host_put_ring_with_host_buffers(pinned):
+@pytest.mark.parametrize("pinned,npes,n", [(True, 5, 70_001), (False, 5, 70_001), (True, 3, (20 << 20) + 12_345)])
+def test_host_put_ring_with_host_buffers(pinned, npes, n):
     """The end-to-end entry point: host payloads in, ring put on the device, destinations back
-    on the host -- against the oracle's puts, with pinned and with pageable host memory."""
-    npes, n = 5, 70_001
-    with Session(npes, 1 << 19) as s:
+    on the host -- against the oracle's puts, with pinned and with pageable host memory, and with a
+    message of 20 MiB and an odd tail."""
+    with Session(npes, max(1 << 19, 2 * n + (1 << 16))) as s:
         src, dst = s.malloc(n), s.malloc(n)
         hsrc = torch.from_numpy(np.concatenate([inputs.byte_payload(inputs.SEED_C2, 500 + p, n) for p in range(npes)]))
         hdst = torch.zeros(npes * n, dtype=torch.uint8)
