@@ -298,7 +298,7 @@ int ishmemx_putmem_spmd_copy_engine(void *dest, const void *src, size_t nbytes, 
  * that head itself meanwhile, hiding the engine's start-up; 0 (the default) = engine only. */
 int ishmemx_set_cutover(int which, size_t nbytes);
 size_t ishmemx_get_cutover(int which);
-/* Picks the cutover from measurement on this device (Section 4: "tuned from measurement"), for
+/* Picks the cutover from measurement on this device (Section 4 leaves it to tuning), for
  * which = 0 (host-initiated put, PE 0 -> PE 1, CUDA events) or which = 3 (device-initiated put
  * by ONE work-group of `threads` threads, timed inside the kernel; needs a running proxy).
  * Times both paths at 4 KiB, 16 KiB, ... (which = 0: 4 KiB, 8 KiB, ...) up to max_bytes (two
@@ -433,7 +433,7 @@ ISHMEM_DECL_AMO(uint32, uint32_t)
 ISHMEM_DECL_AMO(uint64, uint64_t)
 #undef ISHMEM_DECL_AMO
 
-/* Device-initiated batches (one op per GPU thread, "issued from all threads"): op i is
+/* Device-initiated batches (one op per GPU thread, every thread of the launch issuing): op i is
  * issued by PE (i mod npes); word w of the table lives on PE (w mod npes) at
  * table + 8*(w div npes).  word_idx/inc/cond/value/fetched are device arrays of `nops`
  * entries (fetched may be NULL).  aggregate = 0: one atomic per op.  aggregate = 1: the lanes

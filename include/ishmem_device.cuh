@@ -344,7 +344,7 @@ __device__ __forceinline__ void copy_bytes(char *d, const char *s, size_t n, uns
     for (size_t i = body + tid; i < n; i += nthr) stv<unsigned char>(d + i, ldv<unsigned char>(s + i));
 }
 
-/* Strided element copy (iput / iget, Section 3.7.1 "blocked or strided"): element k, taken every
+/* Strided element copy (iput / iget, the strided forms of Section 3.7.1): element k, taken every
  * `sst` elements from s, goes to element k*dst of d, k = tid, tid+nthr, ...  ES = element size in
  * bytes (1, 2, 4, 8 or 16); both addresses aligned to it. */
 template <int ES>
