@@ -325,7 +325,7 @@ def test_config5_jacobi_16384_200_iterations_sampled_cells():
             got = st.cell(ci, cj)
             assert np.float64(got).tobytes() == np.float64(exp).tobytes(), (ci, cj, got, exp)
         # the oracle's 200 plain full-grid sweeps (5.4 x 10^10 cell updates on one host core: about
-        # a minute on the GPU machine's CPU): the whole final grid bit for bit, the residual at 1e-6
+        # a minute on a server CPU): the whole final grid bit for bit, the residual at 1e-6
         exp, exp_res = orc.jacobi(grid, iters)
         st.assert_equals_grid(exp, "200 sweeps")
         assert abs(res - exp_res) <= 1e-6 * exp_res, (res, exp_res)
