@@ -118,6 +118,30 @@ def test_jacobi_multi_sweep_launches_on_the_shortest_strips():
             assert abs(res - exp_res) <= 1e-6 * exp_res
 
 
+def test_jacobi_launch_ordered_forms_on_random_shapes():
+    """Seeded random shapes for the launch-ordered form: grids from a few cells to several bands and tile groups
+    (one, two and more tile groups per band; strips shorter than a launch is deep; strips of unequal length;
+    widths with and without a multiple of four), any cap on the sweeps per launch, both column widths, with and
+    without overlap, with and without a residual, with room in the heap for all, some or none of the deeper halo
+    rows.  Grid bit-exact, residual within 1e-6 relative."""
+    rng = np.random.default_rng(20240917)
+    for case in range(60):
+        npes = int(rng.integers(1, 13))
+        ny = int(rng.integers(max(3, npes), 700))
+        nx = 2 * int(rng.integers(2, 1100 if case % 3 else 160))
+        iters = int(rng.integers(1, 20))
+        fuse, wide = int(rng.integers(0, 7)), int(rng.integers(-1, 2))
+        overlap, want, spare = int(rng.integers(0, 2)), bool(rng.integers(0, 2)), int(rng.choice([0, 2, 4, 6, 8]))
+        grid = inputs.jacobi_grid(inputs.SEED_C5 + case, ny, nx)
+        exp, exp_res = orc.jacobi(grid, iters)
+        options = [(B.ISHMEMX_OPT_JACOBI_FUSE, fuse), (B.ISHMEMX_OPT_JACOBI_WIDE, wide)]
+        got, res = run_gpu(grid, npes, iters, overlap, 1, 0, options, spare_rows=spare, want_residual=want)
+        what = (case, npes, ny, nx, iters, fuse, wide, overlap, want, spare)
+        assert got.tobytes() == exp.tobytes(), what
+        if want:
+            assert abs(res - exp_res) <= 1e-6 * exp_res + 1e-300, what
+
+
 def test_jacobi_without_residual():
     """residual_sq_host = NULL: the last launch forms no residual (in the launch-ordered form it then runs
     like the others); the grid is the oracle's all the same."""
