@@ -1433,6 +1433,7 @@ struct jacobi_plan {
     std::vector<int> depth;            /* sweeps of each launch, deepest first */
     int nc[JW_MAX_DEPTH + 1];          /* columns per lane of a launch of depth k */
     unsigned bands1, groups1;
+    unsigned band_rows_k[JW_MAX_DEPTH + 1]; /* rows per band of a launch of depth k */
     unsigned bands_k[JW_MAX_DEPTH + 1];  /* bands per strip of a launch of depth k */
     unsigned groups_k[JW_MAX_DEPTH + 1]; /* tile groups per band of a launch of depth k */
     size_t blocks_last;                /* tile blocks (= residual terms) of the last launch */
@@ -1508,11 +1509,12 @@ static void jacobi_make_plan(size_t ny, size_t nx, int iters, int kmax, jacobi_p
     else if (fuse >= 2 && fuse < kmax) kmax = (int)fuse;
     /* a strip sends its k first and k last rows: it must own that many */
     if ((size_t)kmax > rows_min) kmax = rows_min < 1 ? 1 : (int)rows_min;
-    jacobi_split(iters, kmax, &pl->depth);
     pl->bands1 = (unsigned)((rows_max + JACOBI_BAND_ROWS - 1) / JACOBI_BAND_ROWS);
     pl->groups1 = (unsigned)(((nx + 59) / 60 + 7) / 8);
-    for (int k = 2; k <= JW_MAX_DEPTH; ++k)
-        pl->bands_k[k] = (unsigned)((rows_max + jacobi_pass_band_rows(k) - 1) / jacobi_pass_band_rows(k));
+    for (int k = 2; k <= JW_MAX_DEPTH; ++k) {
+        pl->band_rows_k[k] = jacobi_pass_band_rows(k);
+        pl->bands_k[k] = (unsigned)((rows_max + pl->band_rows_k[k] - 1) / pl->band_rows_k[k]);
+    }
     /* Columns per lane: four (32-byte accesses: nx a multiple of 4) unless the grid is too small to give
      * every SM its blocks that way.  At 16384^2, per sweep, four against two columns per lane: 345 / 395 us
      * with two sweeps per launch, 247 / 295 with three, 200 / 230 with four.  ISHMEMX_OPT_JACOBI_WIDE =
@@ -1525,7 +1527,19 @@ static void jacobi_make_plan(size_t ny, size_t nx, int iters, int kmax, jacobi_p
     }
     pl->xh_side = 0;
     for (int k = 2; k <= JW_MAX_DEPTH; ++k) pl->groups_k[k] = jacobi_pass_groups(nx, k, pl->nc[k]);
+    jacobi_split(iters, kmax, &pl->depth);
     for (int k : pl->depth) pl->xh_side = std::max(pl->xh_side, k - 2);
+    /* Small grids: lower bands, down to 16 rows, until every SM has a dozen blocks to draw from -- more
+     * rows read twice, but blocks for all SMs (four sweeps per launch, per sweep, bands of 64 / 32 / 16
+     * rows: 1024^2 on 8 PEs 8.3 / 5.4 / 4.3 us, 2048^2 9.7 / 7.5 / 7.3, 4096^2 on 12 PEs 20.2 / 18.6 / 19.4;
+     * at 8192^2 the bands of 64 stay: 51 / 54 / 58).  With that, six sweeps per launch are the fastest
+     * at every size measured (4096^2 on 8 PEs: 16.4 us per sweep against 18.7 with four; with their
+     * bands of 128 rows kept they took 20). */
+    for (int k = 2; k <= JW_MAX_DEPTH; ++k)
+        while (pl->band_rows_k[k] > 16 && (size_t)g.npes * pl->bands_k[k] * pl->groups_k[k] < (size_t)g.sm_count * 12) {
+            pl->band_rows_k[k] /= 2;
+            pl->bands_k[k] = (unsigned)((rows_max + pl->band_rows_k[k] - 1) / pl->band_rows_k[k]);
+        }
     const int k_last = pl->depth.empty() ? 1 : pl->depth.back();
     pl->blocks_last = k_last == 1 ? (size_t)g.npes * pl->bands1 * pl->groups1
                                   : (size_t)g.npes * pl->bands_k[k_last] * pl->groups_k[k_last];
@@ -1534,10 +1548,10 @@ static void jacobi_make_plan(size_t ny, size_t nx, int iters, int kmax, jacobi_p
 
 template <int NC>
 static void jacobi_launch_pass(int k, unsigned nblocks, cudaStream_t s, const jacobi_args &a, double *xh, int xh_side,
-                               int flip, unsigned long long arrived, int last, unsigned bands, unsigned groups)
+                               int flip, unsigned long long arrived, int last, unsigned band_rows, unsigned bands,
+                               unsigned groups)
 {
     auto &g = g_ishmem;
-    const unsigned band_rows = jacobi_pass_band_rows(k);
     /* the bands from the last strip's last band with rows on (see the kernel) */
     const unsigned rows_last = (unsigned)(a.ny / (size_t)g.npes);
     const unsigned lead_bands = bands - (rows_last - 1) / band_rows;
@@ -1591,8 +1605,12 @@ static int jacobi_launch_sweeps(double *buf0, double *buf1, uint64_t *sig, size_
                 g.d_ctx, a, flip, arrived, last, JACOBI_BAND_ROWS, pl.bands1, pl.groups1, g.npes, g.heap_bytes);
         } else {
             const unsigned nblocks = nsend + (unsigned)g.npes * pl.bands_k[k] * pl.groups_k[k];
-            if (pl.nc[k] == 4) jacobi_launch_pass<4>(k, nblocks, s, a, xh, pl.xh_side, flip, arrived, last, pl.bands_k[k], pl.groups_k[k]);
-            else jacobi_launch_pass<2>(k, nblocks, s, a, xh, pl.xh_side, flip, arrived, last, pl.bands_k[k], pl.groups_k[k]);
+            if (pl.nc[k] == 4)
+                jacobi_launch_pass<4>(k, nblocks, s, a, xh, pl.xh_side, flip, arrived, last, pl.band_rows_k[k], pl.bands_k[k],
+                                      pl.groups_k[k]);
+            else
+                jacobi_launch_pass<2>(k, nblocks, s, a, xh, pl.xh_side, flip, arrived, last, pl.band_rows_k[k], pl.bands_k[k],
+                                      pl.groups_k[k]);
         }
         flip ^= 1;
         ishmemi_count_launch();
