@@ -564,6 +564,28 @@ def sweep_c5(args, out):
                     threads=threads, groups=groups, npes=npes, dtype="f64", nbytes=n * n * 8, l2="cold", iters=iters,
                     us_per_op=us, alg_bytes=16 * n * n,
                     note=f"per sweep; level = sweeps per launch; residual_sq {res[0]:.6e} (grid keeps evolving)")
+    # smaller square grids in the same buffers (timing only: the cells keep whatever the runs above left): the
+    # library's own choice against a cap of four sweeps per launch and single sweeps
+    B.ishmemx_set_option(B.ISHMEMX_OPT_JACOBI_SPLIT, 0)
+    for m in ([512, 1024, 2048, 4096, 8192] if not args.quick else [512, 2048]):
+        for variant, fuse in (("library_choice", 1), ("at_most_four_sweeps_per_launch", 4), ("launch_per_sweep", 0)):
+            B.ishmemx_set_option(B.ISHMEMX_OPT_JACOBI_FUSE, fuse)
+            best = None
+            for rep in range(4):                     # the first call loads the kernels
+                for p in range(npes):
+                    for w in range(4):
+                        B.ishmem_uint64_p(p, sig + 8 * w, 0, p)
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                torch.cuda.synchronize()
+                a.record(stream)
+                B.ishmemx_jacobi(b0, b1, sig, m, m, 120, 1, 1, 0, None)
+                b.record(stream)
+                torch.cuda.synchronize()
+                if rep:
+                    best = min(best or 1e30, a.elapsed_time(b) * 1e3 / 120)
+            out.add(config=5, op="jacobi_sizes", pattern=f"{m}x{m}", variant=variant, npes=npes, dtype="f64",
+                    nbytes=m * m * 8, l2="resident" if 2 * m * m * 8 < 100 * MiB else "cold", iters=120, us_per_op=best,
+                    alg_bytes=16 * m * m, note="per sweep, 120 sweeps per call, best of 3 calls")
     assert B.ishmemx_status(1) == 0
     B.ishmem_finalize()
 
@@ -755,7 +777,7 @@ def summarize(path) -> str:
                 "| form | overlap | threads | groups/PE | sweeps per launch K | us/sweep | us/launch | GB/s (16 B/cell/sweep) | "
                 "of measured copy | of 8 TB/s | GB/s moved (16/K B) | of measured copy |",
                 "|---|---|---:|---:|---:|---:|---:|---:|---:|---:|---:|---:|"]
-        for r in rows:
+        for r in [r for r in rows if r["op"] == "jacobi"]:
             form, ov = r["variant"].rsplit(" overlap=", 1) if " overlap=" in r["variant"] else ("", r["variant"][-1])
             k = int(r["level"] or 1)
             shape = (f"| {form} | {ov} | {r['threads'] if r['threads'] != '0' else 'library'} | "
@@ -767,6 +789,19 @@ def summarize(path) -> str:
                            f"{moved:.0f} | {moved / peak:.3f} |")
             else:
                 out.append(f"{shape} refused: not co-resident | | | | | | |")
+        sel = [r for r in rows if r["op"] == "jacobi_sizes"]
+        if sel:
+            out += ["", "### Smaller square grids, 12 PEs, 120 sweeps per call: microseconds per sweep", "",
+                    "Bands are lowered from 128 / 64 rows down to 16 until a launch has a dozen blocks per SM; the last column is one "
+                    "pass over the grid (16 B per cell) at the measured copy rate, for scale -- grids up to 2048^2 stay in L2.", ""]
+            peak = float(sel[0]["gbps"]) / float(sel[0]["frac_hbm"])
+            tab = _table(sel, lambda r: r["pattern"], lambda r: r["variant"], us, str).splitlines()
+            tab[0] = tab[0].replace("| size |", "| grid |") + " one pass at the copy rate |"
+            tab[1] += "---:|"
+            for i, m in enumerate(dict.fromkeys(r["pattern"] for r in sel)):
+                n = int(m.split("x")[0])
+                tab[2 + i] += f" {16.0 * n * n / peak / 1e3:.1f} |"
+            out += tab
     elif cfg == 6:
         out += ["### reverse-offload ring (64-byte requests, one host proxy thread)", "",
                 "| measurement | blocks x threads | us | M requests/s |", "|---|---:|---:|---:|"]
